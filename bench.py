@@ -1,0 +1,398 @@
+"""Benchmark of the block-diffusion decode hot path on B200.
+
+One "step" decodes one section block for every rollout of the scene:
+    fdd_fork -> repeat { fdd_block_attn x layers ; fdd_unmask ; read n_left } until no
+    MASKED position is left -> fdd_kv_commit x layers -> fdd_average_rollouts.
+Metric: committed (value) tokens per second over all rollouts.  Inputs are seeded synthetic
+tensors shaped like the paper's driving workload (see paper_2605_23163_b200/synth.py).
+
+    python bench.py --gpus 1 --steps 10 --warmup 3            # this implementation
+    python bench.py --impl reference --steps 2 --warmup 1      # the CPU fp64 oracle, timed
+Under torchrun (N > 1) every rank decodes an independent scene replica (no data-path
+collective); the time is the max over ranks and the value the sum of all ranks' tokens.
+"""
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "committed tokens/s per denoise step (N forks, shared prefix)"
+UNIT = "tokens/s"
+PRE_STEPS = 6      # distinct per-step input sets kept resident; later steps cycle through them
+
+
+def _peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return dict(hbm_gbs=p["hbm_gbs"], bf16_tflops=p["bf16_tflops"],
+                    bf16_tflops_sustained=p.get("bf16_tflops_sustained", p["bf16_tflops"]), source="measured")
+    return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=1400.0, source="fallback")
+
+
+class ClockSampler(threading.Thread):
+    """Samples SM clock and throttle reasons through NVML (read-only) while the timed region runs."""
+
+    def __init__(self, index):
+        super().__init__(daemon=True)
+        self.index, self.samples, self.reasons, self.stop_flag = index, [], set(), False
+        self.max_mhz = None
+
+    def run(self):
+        try:
+            import pynvml as nv
+            nv.nvmlInit()
+            h = nv.nvmlDeviceGetHandleByIndex(self.index)
+            self.max_mhz = nv.nvmlDeviceGetMaxClockInfo(h, nv.NVML_CLOCK_SM)
+            names = {
+                getattr(nv, "nvmlClocksEventReasonHwSlowdown", 0x8): "hw_slowdown",
+                getattr(nv, "nvmlClocksEventReasonHwThermalSlowdown", 0x40): "hw_thermal_slowdown",
+                getattr(nv, "nvmlClocksEventReasonSwThermalSlowdown", 0x20): "sw_thermal_slowdown",
+                getattr(nv, "nvmlClocksEventReasonSwPowerCap", 0x4): "sw_power_cap",
+            }
+            while not self.stop_flag:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(h, nv.NVML_CLOCK_SM))
+                try:
+                    mask = nv.nvmlDeviceGetCurrentClocksEventReasons(h)
+                except Exception:
+                    mask = nv.nvmlDeviceGetCurrentClocksThrottleReasons(h)
+                for bit, name in names.items():
+                    if mask & bit:
+                        self.reasons.add(name)
+                time.sleep(0.05)
+        except Exception as exc:      # NVML unavailable: report that instead of clocks
+            self.reasons.add(f"nvml_unavailable:{type(exc).__name__}")
+
+    def summary(self):
+        med = float(np.median(self.samples)) if self.samples else None
+        return {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
+                "samples": len(self.samples)}
+
+
+def _gen_step_inputs(w, scene_idx, block, step, pool):
+    """numpy inputs of one denoising step: q/k/v bits and logits (value rows only)."""
+    from paper_2605_23163_b200 import synth
+    q, k, v = synth.make_qkv(w, scene_idx, 0, block, step)
+    sc = w.scenes[scene_idx]
+    dt = np.uint16 if w.logits_dtype == "bf16" else np.float32
+    logits = np.zeros((sc.n_forks, sc.block_len, w.vocab), dtype=dt)
+    frozen = set(synth.scaffold_positions(w, scene_idx, block).tolist())
+    jobs = [(f, i) for f in range(sc.n_forks) for i in range(sc.block_len) if i not in frozen]
+
+    def fill(job):
+        f, i = job
+        logits[f, i] = synth.make_logits_row(w, scene_idx, block, step, f, i)
+
+    list(pool.map(fill, jobs))
+    return q, k, v, logits
+
+
+def _attn_flops(w, sc, suffix_len):
+    return 4.0 * sc.n_forks * sc.block_len * w.n_q_heads * (sc.prefix_len + suffix_len + sc.block_len) * w.head_dim
+
+
+def run_ours(args):
+    import torch
+    from concurrent.futures import ThreadPoolExecutor
+    from paper_2605_23163_b200 import fdd, harness, synth
+
+    rank = int(os.environ.get("RANK", 0))
+    world = int(os.environ.get("WORLD_SIZE", 1))
+    local = int(os.environ.get("LOCAL_RANK", 0))
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    fdd.lib()
+    w = synth.workload(args.workload)
+    if world > 1:     # every rank decodes its own scene replica (different seed)
+        w = synth.Workload(**{**w.__dict__, "seed": w.seed + 100 * rank})
+    sc = w.scenes[0]
+    L = args.layers
+    ctx = harness.create_context(w, n_layers=L)
+    scene = harness.GpuScene(ctx, w, 0, n_layers=L, suffix_capacity=sc.block_len)
+    stream = torch.cuda.current_stream()
+    scale = 1.0 / np.sqrt(w.head_dim)
+    d, N = sc.block_len, sc.n_forks
+
+    pool = ThreadPoolExecutor(max_workers=max(1, len(os.sched_getaffinity(0))))
+    host_steps = [_gen_step_inputs(w, 0, 0, t, pool) for t in range(PRE_STEPS)]
+    pool.shutdown()
+    dev_steps = []
+    for q, k, v, lg in host_steps:
+        dev_steps.append(tuple([harness.bf16_tensor(q), harness.bf16_tensor(k), harness.bf16_tensor(v),
+                                harness.logits_tensor(w, lg)]))
+    tokens0, state0 = synth.make_block_template(w, 0, 0)
+    tokens0_d = torch.from_numpy(tokens0).cuda()
+    state0_d = torch.from_numpy(state0).cuda()
+    tokens = torch.empty_like(tokens0_d)
+    state = torch.empty_like(state0_d)
+    out = torch.empty_like(dev_steps[0][0])
+    n_comm = torch.zeros(N, dtype=torch.int32, device="cuda")
+    n_left = torch.zeros(N, dtype=torch.int32, device="cuda")
+    n_left_host = torch.zeros(N, dtype=torch.int32).pin_memory()
+    traj = torch.from_numpy(synth.tokens_to_trajectory(w, tokens0, state0)).cuda()
+    traj_out = torch.zeros((w.waypoints, 2), dtype=torch.float32, device="cuda")
+    value_tokens = int((state0 == synth.MASKED).sum())
+    all_tokens = int(state0.size)
+
+    attn_events = []
+
+    def decode_block(inputs, timed_attn):
+        """One step of the benchmark: the whole block loop for all rollouts.  `inputs(t)` returns
+        device tensors (q, k, v, logits) of denoising step t."""
+        fs = fdd.fdd_fork(ctx, scene.prefix_k, scene.prefix_v, scene.page_table, sc.prefix_len,
+                          scene.prefix_capacity, N, scene.seeds, scene.suffix_k, scene.suffix_v,
+                          scene.suffix_capacity)
+        tokens.copy_(tokens0_d, non_blocking=True)
+        state.copy_(state0_d, non_blocking=True)
+        t = 0
+        while True:
+            q, k, v, lg = inputs(t)
+            for layer in range(L):
+                if timed_attn:
+                    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    e0.record(stream)
+                fdd.fdd_block_attn(ctx, [fs], layer, q, k, v, out, [d], scale, 0)
+                if timed_attn:
+                    e1.record(stream)
+                    attn_events.append((e0, e1))
+            fdd.fdd_unmask(ctx, [fs], lg, tokens, state, [d], w.threshold, w.temperature, 0, t, n_comm, n_left)
+            n_left_host.copy_(n_left, non_blocking=True)
+            stream.synchronize()
+            t += 1
+            if int(n_left_host.sum()) == 0 or t >= d:
+                break
+        for layer in range(L):
+            fdd.fdd_kv_commit(ctx, [fs], layer, k, v, [d], 1 if layer == L - 1 else 0)
+        fdd.fdd_average_rollouts(ctx, traj, N, w.waypoints, traj_out)
+        fdd.fdd_forkset_free(ctx, fs)
+        return t
+
+    resident = lambda t: dev_steps[t % PRE_STEPS]
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        n_denoise = decode_block(resident, False)
+    barrier()
+    sampler = ClockSampler(local)
+    sampler.start()
+    launches0 = fdd.fdd_launch_count(ctx)
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev0.record(stream)
+    denoise_steps = 0
+    for _ in range(args.steps):
+        denoise_steps += decode_block(resident, True)
+    ev1.record(stream)
+    barrier()
+    launches = fdd.fdd_launch_count(ctx) - launches0
+    sampler.stop_flag = True
+    sampler.join(timeout=2)
+    ms = ev0.elapsed_time(ev1)
+    attn_ms = [a.elapsed_time(b) for a, b in attn_events]
+    if dist is not None:
+        t_ = torch.tensor([ms], device="cuda")
+        dist.all_reduce(t_, op=dist.ReduceOp.MAX)
+        ms = float(t_.item())
+    fdd.fdd_poll_status(ctx)
+
+    # end to end: every denoising step's inputs come from pinned host memory, results go back
+    e2e = None
+    if not args.no_e2e:
+        pinned = [tuple(torch.from_numpy(np.ascontiguousarray(a).view(np.int16) if a.dtype == np.uint16 else a).pin_memory()
+                        for a in hs) for hs in host_steps]
+        stage = [torch.empty_like(x) for x in dev_steps[0]]
+        tok_host = torch.zeros_like(tokens0_d, device="cpu").pin_memory()
+        traj_host = torch.zeros((w.waypoints, 2), dtype=torch.float32).pin_memory()
+        h2d = sum(x.numel() * x.element_size() for x in pinned[0])
+        d2h_step = n_left_host.numel() * 4
+
+        def from_host(t):
+            src = pinned[t % PRE_STEPS]
+            for dst, s in zip(stage, src):
+                dst.view(torch.int16).copy_(s, non_blocking=True) if dst.dtype == torch.bfloat16 else dst.copy_(s, non_blocking=True)
+            return tuple(stage)
+
+        e2e_steps = max(1, min(args.steps, args.e2e_steps))
+        decode_block(from_host, False)
+        barrier()
+        ee0, ee1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        ee0.record(stream)
+        e2e_denoise = 0
+        for _ in range(e2e_steps):
+            e2e_denoise += decode_block(from_host, False)
+            tok_host.copy_(tokens, non_blocking=True)
+            traj_host.copy_(traj_out, non_blocking=True)
+            stream.synchronize()
+        ee1.record(stream)
+        barrier()
+        e_ms = ee0.elapsed_time(ee1)
+        if dist is not None:
+            t_ = torch.tensor([e_ms], device="cuda")
+            dist.all_reduce(t_, op=dist.ReduceOp.MAX)
+            e_ms = float(t_.item())
+        per_block_denoise = e2e_denoise / e2e_steps
+        e2e = {"value": world * value_tokens * e2e_steps / (e_ms * 1e-3), "unit": UNIT,
+               "h2d_bytes_per_step": int(h2d * per_block_denoise),
+               "d2h_bytes_per_step": int(d2h_step * per_block_denoise + tok_host.numel() * 4 + traj_host.numel() * 4),
+               "steps": e2e_steps, "ms_per_step": e_ms / e2e_steps}
+
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+    peaks = _peaks()
+    flops = _attn_flops(w, sc, 0)
+    attn_avg_ms = float(np.mean(attn_ms)) if attn_ms else None
+    achieved = flops / (attn_avg_ms * 1e-3) / 1e12 if attn_avg_ms else None
+    line = {
+        "metric": METRIC, "value": world * value_tokens * args.steps / (ms * 1e-3), "unit": UNIT,
+        "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+        "data": "synthetic",
+        "config": {"workload": args.workload, "n_forks": N, "block_len": d, "prefix_len": sc.prefix_len,
+                   "heads": f"{w.n_q_heads}q/{w.n_kv_heads}kv", "head_dim": w.head_dim, "vocab": w.vocab,
+                   "layers": L, "threshold": w.threshold, "temperature": w.temperature,
+                   "denoise_steps_per_block": denoise_steps / args.steps,
+                   "value_tokens_per_block": value_tokens, "tokens_incl_scaffold_per_block": all_tokens,
+                   "l2": "per-step inputs (logits) larger than L2",
+                   "replicas": "independent scene per GPU, no collective"},
+        "clocks": sampler.summary(),
+        "e2e": e2e,
+        "gpu_launches": int(launches),
+        "roofline": {"kernel": "fdd_block_attn", "bound": "tensor", "achieved": achieved,
+                     "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s",
+                     "frac": (achieved / peaks["bf16_tflops_sustained"]) if achieved else None,
+                     "traffic": None, "peak_source": peaks["source"] + " (sustained bf16)",
+                     "flops_per_launch": flops, "avg_launch_ms": attn_avg_ms, "launches_timed": len(attn_ms)},
+        "tokens_per_s_incl_scaffold": world * all_tokens * args.steps / (ms * 1e-3),
+    }
+    if not args.no_cpu_baseline and world >= 1:
+        line["cpu_baseline"] = cpu_baseline(args.workload, budget_s=args.cpu_budget)
+    print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+# -------------------------------------------------------------------------------------------------
+# CPU oracle legs
+# -------------------------------------------------------------------------------------------------
+def _oracle_block(w, fork, max_steps=None):
+    """Decode one block for a single rollout with the CPU oracle; returns (seconds, committed
+    value tokens, denoising steps)."""
+    from oracle.cache import ForkSet
+    from oracle.decode import decode_block
+    from oracle.attention import bf16_bits_to_f64
+    from paper_2605_23163_b200 import synth
+    sc = w.scenes[0]
+    pk, pv = synth.make_prefix(w, 0)
+    seeds = synth.fork_seeds(w, 0)[fork:fork + 1]
+    fs = ForkSet([pk], [pv], 1, seeds)
+    tokens, state = synth.make_block_template(w, 0, 0)
+    tokens, state = tokens[fork:fork + 1], state[fork:fork + 1]
+    frozen = set(synth.scaffold_positions(w, 0, 0).tolist())
+    cache = {}
+
+    def inputs(t):
+        if t not in cache:
+            q, k, v = synth.make_qkv(w, 0, 0, 0, t)
+            lg = np.zeros((1, sc.block_len, w.vocab), dtype=np.float64)
+            for i in range(sc.block_len):
+                if i not in frozen:
+                    row = synth.make_logits_row(w, 0, 0, t, fork, i)
+                    lg[0, i] = bf16_bits_to_f64(row) if w.logits_dtype == "bf16" else row
+            cache[t] = dict(q=[q[fork:fork + 1]], k=[k[fork:fork + 1]], v=[v[fork:fork + 1]], logits=lg)
+        return cache[t]
+
+    for t in range(PRE_STEPS):       # inputs are made outside the timed region
+        inputs(t)
+    t0 = time.perf_counter()
+    r = decode_block(fs, lambda t: inputs(t % PRE_STEPS), tokens, state, w.threshold, w.temperature, 0,
+                     1.0 / np.sqrt(w.head_dim), max_steps=max_steps)
+    dt = time.perf_counter() - t0
+    return dt, int(sum(int(c.sum()) for c in r["committed_per_step"])), r["steps"]
+
+
+def cpu_baseline(workload_name, budget_s=20.0):
+    from paper_2605_23163_b200 import synth
+    w = synth.workload(workload_name)
+    cores = len(os.sched_getaffinity(0))
+    try:
+        from threadpoolctl import threadpool_info
+        blas = [p.get("num_threads") for p in threadpool_info() if p.get("user_api") == "blas"]
+        if blas:
+            cores = int(max(blas))
+    except Exception:
+        pass
+    n = w.scenes[0].n_forks
+    dt = toks = steps = used = 0
+    while used < n and (used == 0 or dt < 0.5 * budget_s):
+        a, b, c = _oracle_block(w, used)
+        dt, toks, steps, used = dt + a, toks + b, steps + c, used + 1
+    return {"value": toks / dt, "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": f"rollouts 0..{used - 1} of {n}, one after the other: whole block loop each "
+                      f"({steps} denoising steps, {toks} committed tokens in total) in {dt:.2f} s; rollouts "
+                      "are independent, so tokens/s of the full workload is the same figure"}
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", 0))
+    if rank != 0:
+        return
+    from paper_2605_23163_b200 import synth
+    w = synth.workload(args.workload)
+    sc = w.scenes[0]
+    for i in range(args.warmup):
+        _oracle_block(w, i % sc.n_forks)
+    total_t, total_tok = 0.0, 0
+    for i in range(args.steps):
+        dt, toks, _ = _oracle_block(w, (args.warmup + i) % sc.n_forks)
+        total_t += dt
+        total_tok += toks
+    cores = len(os.sched_getaffinity(0))
+    val = total_tok / total_t
+    line = {"impl": "reference", "metric": METRIC, "value": val, "unit": UNIT,
+            "n_gpus": int(os.environ.get("WORLD_SIZE", 1)), "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": 1e3 * total_t / args.steps, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": args.workload, "sample": "one rollout per step (whole block loop)"},
+            "cpu_baseline": {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle",
+                             "sample": "each step decodes one rollout's block with the CPU fp64 oracle"},
+            "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="long_prefix")
+    ap.add_argument("--layers", type=int, default=1)
+    ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--cpu-budget", type=float, default=20.0)
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

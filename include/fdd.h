@@ -1,0 +1,191 @@
+/*
+ * fdd.h -- C ABI of the block-diffusion decode hot path for NVIDIA B200 (sm_100a).
+ *
+ * One denoising step of section-wise block-diffusion decoding with N rollouts
+ * forked from a shared prefix KV cache:
+ *   fdd_fork             share one prefix cache between N rollouts      (Sec. 3.4, "Shared prefix")
+ *   fdd_block_attn       block-causal attention of the current block    (Sec. 3.1, "Block-Causal Diffusion")
+ *   fdd_unmask           confidence-threshold parallel unmasking        (Sec. 3.3, "Section Diffusion";
+ *                                                                        Sec. 3.2 scaffold; Sec. 3.1 "visible tokens fixed")
+ *   fdd_kv_commit        append the finished block to each private cache (Sec. 3.3 cache reuse; Sec. 3.4 fork)
+ *   fdd_average_rollouts equal-weight mean of N trajectories            (Sec. 3.4, trajectory averaging)
+ *
+ * Conventions
+ *   - Every tensor is caller-owned.  "device" pointers are CUDA device memory of the
+ *     current device, "host" pointers are ordinary host memory.  The library allocates
+ *     only small metadata and its own scratch (at fdd_create / fdd_fork).
+ *   - bf16 tensors are raw 16-bit bfloat16.  All tensors are dense, row-major in the
+ *     index order written, and must be 16-byte aligned.
+ *   - Calls enqueue work on `stream` (a cudaStream_t passed as void*; NULL = default
+ *     stream) and return without synchronising unless stated.  Argument errors are
+ *     detected on the host before anything is launched and returned synchronously.
+ *   - No call aborts, throws or prints.  A negative fdd_status is an error; the text
+ *     is available from fdd_last_error().
+ *   - A context and its fork sets must be used from one host thread at a time.
+ *
+ * Position state codes (uint8): 0 = MASKED (to be decoded), 1 = COMMITTED, 2 = SCAFFOLD
+ * (frozen structural token, Sec. 3.2).
+ */
+#ifndef FDD_H_
+#define FDD_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef int fdd_status;
+#define FDD_OK                   0
+#define FDD_ERR_INVALID_ARG     (-1)  /* NULL pointer, negative size, bad enum                */
+#define FDD_ERR_SHAPE           (-2)  /* sizes inconsistent with the context configuration   */
+#define FDD_ERR_CAPACITY        (-3)  /* private cache, fork count or block length exceeded  */
+#define FDD_ERR_STATE           (-4)  /* freed / foreign fork set                            */
+#define FDD_ERR_CUDA            (-5)  /* a CUDA runtime call failed (text has the reason)    */
+#define FDD_ERR_DEVICE_TIMEOUT  (-6)  /* a bounded device-side wait gave up                  */
+#define FDD_ERR_UNSUPPORTED     (-7)  /* configuration outside what the kernels implement    */
+
+#define FDD_MASKED    0
+#define FDD_COMMITTED 1
+#define FDD_SCAFFOLD  2
+
+#define FDD_LOGITS_F32  0
+#define FDD_LOGITS_BF16 1
+
+typedef struct fdd_ctx fdd_ctx;         /* opaque: configuration, scratch, device status word */
+typedef struct fdd_forkset fdd_forkset; /* opaque: N rollouts over one shared prefix cache     */
+
+typedef struct fdd_config {
+    int n_q_heads;    /* Hq                                                        */
+    int n_kv_heads;   /* Hkv, divides Hq; query head h reads KV head h / (Hq/Hkv)  */
+    int head_dim;     /* D: 64 or 128                                              */
+    int vocab;        /* V                                                         */
+    int n_layers;     /* L: number of per-layer caches a fork set carries          */
+    int page_tokens;  /* 0: contiguous prefix cache; else tokens per page (64)     */
+    int max_block;    /* largest block length d accepted (<= 128)                  */
+    int max_forks;    /* largest total number of rollouts in one call              */
+    int logits_dtype; /* FDD_LOGITS_F32 or FDD_LOGITS_BF16                         */
+} fdd_config;
+
+/* Create / destroy a context on the current CUDA device.  Allocates the device status
+ * word and the scratch buffers (split-KV partials, unmask partials), sized from cfg.
+ * Returns FDD_ERR_UNSUPPORTED for head_dim not in {64,128}, Hq % Hkv != 0, Hq/Hkv > 16,
+ * max_block > 128; FDD_ERR_CUDA if no usable device.  *out is NULL on failure. */
+fdd_status fdd_create(const fdd_config* cfg, fdd_ctx** out);
+void fdd_destroy(fdd_ctx* ctx);
+
+/* Text of the most recent error on this context ("" if none).  Valid until the next call. */
+const char* fdd_last_error(const fdd_ctx* ctx);
+
+/* Number of kernels this context has launched so far (for accounting). */
+uint64_t fdd_launch_count(const fdd_ctx* ctx);
+
+/*
+ * fdd_fork -- Sec. 3.4 "Shared prefix": the deterministic sections are decoded once and
+ * their KV cache is forked N times.  Nothing is copied: the N rollouts read the same
+ * prefix memory, and each gets an empty private suffix.
+ *
+ *   prefix_k, prefix_v  host arrays [L] of device pointers, one cache per layer, bf16.
+ *                       contiguous (cfg.page_tokens == 0): [Hkv][prefix_capacity][D]
+ *                       paged:                             [prefix_capacity pages][Hkv][page_tokens][D]
+ *                       Read-only for the library; must stay valid and unmodified while
+ *                       the fork set lives.
+ *   page_table          device int32 [ceil(prefix_len / page_tokens)] physical page of each
+ *                       logical page (paged layout), NULL for the contiguous layout.  Every
+ *                       entry must be in [0, prefix_capacity); entries are read on the device.
+ *   prefix_len          valid prefix tokens (>= 0).
+ *   prefix_capacity     tokens per head (contiguous) or number of physical pages (paged).
+ *   n_forks             N >= 1, <= cfg.max_forks.
+ *   seeds               host uint64 [N]: the noise key of each rollout (copied).
+ *   suffix_k, suffix_v  host arrays [L] of device pointers, bf16 [N][Hkv][suffix_capacity][D],
+ *                       caller-owned, written by fdd_kv_commit only.
+ *   suffix_capacity     tokens each rollout may append per layer.
+ */
+fdd_status fdd_fork(fdd_ctx* ctx, const void* const* prefix_k, const void* const* prefix_v,
+                    const int32_t* page_table, int prefix_len, int prefix_capacity,
+                    int n_forks, const uint64_t* seeds,
+                    void* const* suffix_k, void* const* suffix_v, int suffix_capacity,
+                    fdd_forkset** out);
+fdd_status fdd_forkset_free(fdd_ctx* ctx, fdd_forkset* set);
+/* Committed private tokens per rollout (same for every rollout of a set); < 0 on error. */
+int fdd_forkset_suffix_len(const fdd_forkset* set);
+/* Forget every committed block (suffix length back to 0); the memory is not cleared. */
+fdd_status fdd_forkset_reset(fdd_ctx* ctx, fdd_forkset* set);
+
+/*
+ * fdd_block_attn -- Sec. 3.1: the tokens of the current block attend bidirectionally to
+ * each other and causally to everything before the block.  For rollout f of a set the keys
+ * are the shared prefix, f's private suffix and all block_len keys of f's block:
+ *   out[f,i,h,:] = sum_j softmax_j(scale * q[f,i,h,:] . k_j[h/G,:]) v_j[h/G,:]
+ * computed with bf16 operands, fp32 accumulation, bf16 output.
+ *
+ *   sets, n_sets   host array of fork sets handled in this call (independent scenes).
+ *   layer          which per-layer cache to read, 0 <= layer < L.
+ *   q              device bf16, rollouts of all sets packed in set order:
+ *                  set s contributes [N_s][d_s][Hq][D]; k_blk, v_blk likewise [N_s][d_s][Hkv][D].
+ *   out            device bf16, same packing and shape as q.
+ *   block_len      host int32 [n_sets]: d_s, 1 <= d_s <= cfg.max_block.
+ *   scale          soft-max scale (1/sqrt(D) by convention).
+ *   causal_in_block 0: bidirectional inside the block (denoising pass);
+ *                  1: query i sees block keys 0..i only (the causal verifier pass of
+ *                  Scaffold Speculative Decoding, Sec. 3.3 step 3).
+ */
+fdd_status fdd_block_attn(fdd_ctx* ctx, fdd_forkset* const* sets, int n_sets, int layer,
+                          const void* q, const void* k_blk, const void* v_blk, void* out,
+                          const int32_t* block_len, float scale, int causal_in_block,
+                          void* stream);
+
+/*
+ * fdd_unmask -- one parallel unmasking step (Sec. 3.3 "iteratively unmasks value
+ * positions"; Sec. 3.1: visible tokens stay fixed; Sec. 3.2: scaffold never rewritten).
+ * For every rollout f and every position i with state MASKED:
+ *   tok  = argmax_v (logit[v] + temperature * g[v])            lowest v on ties
+ *   conf = softmax(logit)[tok]                                  noise-free probability
+ * where g[v] = -ln(-ln(u)), u = ((x >> 9) + 0.5) * 2^-23 and x is output word v % 4 of
+ * Philox4x32-10 with key = the rollout's seed (low, high word) and counter =
+ * (v / 4, i, step, block_idx); temperature == 0 uses no noise.  Positions with
+ * conf > threshold are committed (token written, state -> COMMITTED); if a rollout has
+ * MASKED positions and none passes, its single most confident one (lowest i on ties)
+ * is committed.  Nothing else is written; rollouts without MASKED positions are no-ops.
+ *
+ *   logits        device, packed like q: [N_s][d_s][V], fp32 or bf16 per cfg.logits_dtype.
+ *                 Only rows of MASKED positions are read.
+ *   tokens        device int32 [N_s][d_s], in/out.     state: device uint8, in/out.
+ *   n_committed   device int32 [sum N_s]: commits of this step per rollout (written).
+ *   n_left        device int32 [sum N_s]: MASKED positions remaining per rollout (written).
+ *   conf          device fp32 packed [N_s][d_s] or NULL: confidence of every position that
+ *                 was MASKED on entry, NaN elsewhere.
+ */
+fdd_status fdd_unmask(fdd_ctx* ctx, fdd_forkset* const* sets, int n_sets, const void* logits,
+                      int32_t* tokens, uint8_t* state, const int32_t* block_len,
+                      float threshold, float temperature, uint32_t block_idx, uint32_t step,
+                      int32_t* n_committed, int32_t* n_left, float* conf, void* stream);
+
+/*
+ * fdd_kv_commit -- Sec. 3.3 / 3.4: a finished block's K/V join the cache of the rollout
+ * that produced them and are reused, not recomputed, by later blocks.  Copies rollout f's
+ * rows of k_blk / v_blk ([N_s][d_s][Hkv][D], packed like fdd_block_attn) to positions
+ * [len, len + d_s) of f's private suffix of `layer`, bit for bit.  With advance != 0 the
+ * set's suffix length grows by d_s afterwards (pass it on the last layer).
+ * FDD_ERR_CAPACITY if len + d_s > suffix_capacity (nothing is launched).
+ */
+fdd_status fdd_kv_commit(fdd_ctx* ctx, fdd_forkset* const* sets, int n_sets, int layer,
+                         const void* k_blk, const void* v_blk, const int32_t* block_len,
+                         int advance, void* stream);
+
+/*
+ * fdd_average_rollouts -- Sec. 3.4: tau_out = (1/N) sum_i tau_i.
+ *   traj  device fp32 [n][w][2];  out  device fp32 [w][2];  n >= 1, w >= 1.
+ */
+fdd_status fdd_average_rollouts(fdd_ctx* ctx, const float* traj, int n, int w, float* out,
+                                void* stream);
+
+/* Synchronise `stream` and return the device status word: FDD_OK, or the first error a
+ * kernel recorded (FDD_ERR_DEVICE_TIMEOUT).  Reading clears it. */
+fdd_status fdd_poll_status(fdd_ctx* ctx, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FDD_H_ */

@@ -1,0 +1,333 @@
+// Host side of the C ABI: argument validation, fork-set metadata, kernel dispatch.
+#include "fdd_internal.h"
+
+#include <algorithm>
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <new>
+
+cudaError_t launch_attention_simple(const AttnProblem& p, int head_dim, cudaStream_t st);
+
+namespace {
+
+fdd_status fail(fdd_ctx* ctx, fdd_status code, const char* fmt, ...) {
+    if (ctx) {
+        char buf[512];
+        va_list ap;
+        va_start(ap, fmt);
+        vsnprintf(buf, sizeof(buf), fmt, ap);
+        va_end(ap);
+        ctx->last_error = buf;
+    }
+    return code;
+}
+
+fdd_status cuda_fail(fdd_ctx* ctx, cudaError_t e, const char* what) {
+    return fail(ctx, FDD_ERR_CUDA, "%s: %s", what, cudaGetErrorString(e));
+}
+
+bool set_alive(const fdd_ctx* ctx, const fdd_forkset* s) {
+    return s && std::find(ctx->live_sets.begin(), ctx->live_sets.end(), s) != ctx->live_sets.end();
+}
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// Common checks of a batched call; fills total rollouts and per-set row offsets.
+fdd_status check_sets(fdd_ctx* ctx, fdd_forkset* const* sets, int n_sets, const int32_t* block_len,
+                      int* total_forks) {
+    if (!sets || n_sets < 1 || !block_len) return fail(ctx, FDD_ERR_INVALID_ARG, "sets/block_len missing or n_sets < 1");
+    int total = 0;
+    for (int s = 0; s < n_sets; ++s) {
+        if (!set_alive(ctx, sets[s])) return fail(ctx, FDD_ERR_STATE, "fork set %d is not a live set of this context", s);
+        if (block_len[s] < 1 || block_len[s] > ctx->cfg.max_block)
+            return fail(ctx, FDD_ERR_CAPACITY, "block_len[%d] = %d outside [1, %d]", s, block_len[s], ctx->cfg.max_block);
+        total += sets[s]->n_forks;
+    }
+    if (total > ctx->cfg.max_forks)
+        return fail(ctx, FDD_ERR_CAPACITY, "%d rollouts in one call exceed max_forks = %d", total, ctx->cfg.max_forks);
+    *total_forks = total;
+    return FDD_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+fdd_status fdd_create(const fdd_config* cfg, fdd_ctx** out) {
+    if (!out) return FDD_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (!cfg) return FDD_ERR_INVALID_ARG;
+    if (cfg->n_q_heads < 1 || cfg->n_kv_heads < 1 || cfg->vocab < 1 || cfg->n_layers < 1 ||
+        cfg->max_block < 1 || cfg->max_forks < 1 || cfg->page_tokens < 0)
+        return FDD_ERR_INVALID_ARG;
+    if (cfg->logits_dtype != FDD_LOGITS_F32 && cfg->logits_dtype != FDD_LOGITS_BF16) return FDD_ERR_INVALID_ARG;
+    if (cfg->head_dim != 64 && cfg->head_dim != 128) return FDD_ERR_UNSUPPORTED;
+    if (cfg->n_q_heads % cfg->n_kv_heads != 0 || cfg->n_q_heads / cfg->n_kv_heads > 16) return FDD_ERR_UNSUPPORTED;
+    if (cfg->max_block > 128) return FDD_ERR_UNSUPPORTED;
+    if (cfg->page_tokens != 0 && cfg->page_tokens != 64) return FDD_ERR_UNSUPPORTED;
+
+    fdd_ctx* ctx = new (std::nothrow) fdd_ctx();
+    if (!ctx) return FDD_ERR_CUDA;
+    ctx->cfg = *cfg;
+    cudaError_t e = cudaGetDevice(&ctx->device);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&ctx->sm_count, cudaDevAttrMultiProcessorCount, ctx->device);
+    if (e == cudaSuccess) e = cudaMalloc(&ctx->d_status, sizeof(int));
+    if (e == cudaSuccess) e = cudaMemset(ctx->d_status, 0, sizeof(int));
+    if (e == cudaSuccess) e = cudaMallocHost(&ctx->h_status, sizeof(int));
+    if (e == cudaSuccess) {
+        ctx->ws_unmask_bytes = static_cast<size_t>(cfg->max_forks) * cfg->max_block * unmask_chunks(cfg->vocab) * sizeof(UnmaskPartial);
+        e = cudaMalloc(&ctx->ws_unmask, ctx->ws_unmask_bytes);
+    }
+    if (e != cudaSuccess) {
+        fdd_destroy(ctx);
+        return FDD_ERR_CUDA;
+    }
+    *out = ctx;
+    return FDD_OK;
+}
+
+void fdd_destroy(fdd_ctx* ctx) {
+    if (!ctx) return;
+    for (fdd_forkset* s : ctx->live_sets) {
+        if (s->d_seeds) cudaFree(s->d_seeds);
+        delete s;
+    }
+    if (ctx->d_status) cudaFree(ctx->d_status);
+    if (ctx->h_status) cudaFreeHost(ctx->h_status);
+    if (ctx->ws_unmask) cudaFree(ctx->ws_unmask);
+    if (ctx->ws_attn) cudaFree(ctx->ws_attn);
+    delete ctx;
+}
+
+const char* fdd_last_error(const fdd_ctx* ctx) { return ctx ? ctx->last_error.c_str() : "null context"; }
+
+uint64_t fdd_launch_count(const fdd_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+fdd_status fdd_fork(fdd_ctx* ctx, const void* const* prefix_k, const void* const* prefix_v,
+                    const int32_t* page_table, int prefix_len, int prefix_capacity,
+                    int n_forks, const uint64_t* seeds,
+                    void* const* suffix_k, void* const* suffix_v, int suffix_capacity,
+                    fdd_forkset** out) {
+    if (!ctx) return FDD_ERR_INVALID_ARG;
+    if (!out) return fail(ctx, FDD_ERR_INVALID_ARG, "out is NULL");
+    *out = nullptr;
+    if (!prefix_k || !prefix_v || !seeds || !suffix_k || !suffix_v)
+        return fail(ctx, FDD_ERR_INVALID_ARG, "a pointer array is NULL");
+    if (prefix_len < 0 || prefix_capacity < 0 || suffix_capacity < 0)
+        return fail(ctx, FDD_ERR_INVALID_ARG, "negative length or capacity");
+    if (n_forks < 1 || n_forks > ctx->cfg.max_forks)
+        return fail(ctx, FDD_ERR_CAPACITY, "n_forks = %d outside [1, %d]", n_forks, ctx->cfg.max_forks);
+    const int pt = ctx->cfg.page_tokens;
+    if (pt == 0) {
+        if (page_table) return fail(ctx, FDD_ERR_INVALID_ARG, "page_table given but the context is configured contiguous");
+        if (prefix_len > prefix_capacity)
+            return fail(ctx, FDD_ERR_CAPACITY, "prefix_len %d exceeds prefix_capacity %d", prefix_len, prefix_capacity);
+    } else {
+        if (!page_table && prefix_len > 0) return fail(ctx, FDD_ERR_INVALID_ARG, "paged context needs a page_table");
+        if ((prefix_len + pt - 1) / pt > prefix_capacity)
+            return fail(ctx, FDD_ERR_CAPACITY, "prefix_len %d needs more than %d pages", prefix_len, prefix_capacity);
+    }
+    for (int l = 0; l < ctx->cfg.n_layers; ++l) {
+        if ((prefix_len > 0 && (!prefix_k[l] || !prefix_v[l])) || (suffix_capacity > 0 && (!suffix_k[l] || !suffix_v[l])))
+            return fail(ctx, FDD_ERR_INVALID_ARG, "NULL cache pointer for layer %d", l);
+        if (!aligned16(prefix_k[l]) || !aligned16(prefix_v[l]) || !aligned16(suffix_k[l]) || !aligned16(suffix_v[l]))
+            return fail(ctx, FDD_ERR_INVALID_ARG, "cache pointer of layer %d is not 16-byte aligned", l);
+    }
+    fdd_forkset* s = new (std::nothrow) fdd_forkset();
+    if (!s) return fail(ctx, FDD_ERR_CUDA, "out of host memory");
+    s->ctx = ctx;
+    s->n_forks = n_forks;
+    s->prefix_len = prefix_len;
+    s->prefix_capacity = prefix_capacity;
+    s->page_table = page_table;
+    s->prefix_k.assign(prefix_k, prefix_k + ctx->cfg.n_layers);
+    s->prefix_v.assign(prefix_v, prefix_v + ctx->cfg.n_layers);
+    s->suffix_k.assign(suffix_k, suffix_k + ctx->cfg.n_layers);
+    s->suffix_v.assign(suffix_v, suffix_v + ctx->cfg.n_layers);
+    s->suffix_capacity = suffix_capacity;
+    s->suffix_len = 0;
+    cudaError_t e = cudaMalloc(&s->d_seeds, sizeof(uint64_t) * n_forks);
+    if (e == cudaSuccess) e = cudaMemcpy(s->d_seeds, seeds, sizeof(uint64_t) * n_forks, cudaMemcpyHostToDevice);
+    if (e != cudaSuccess) {
+        if (s->d_seeds) cudaFree(s->d_seeds);
+        delete s;
+        return cuda_fail(ctx, e, "fdd_fork seeds");
+    }
+    ctx->live_sets.push_back(s);
+    *out = s;
+    return FDD_OK;
+}
+
+fdd_status fdd_forkset_free(fdd_ctx* ctx, fdd_forkset* set) {
+    if (!ctx) return FDD_ERR_INVALID_ARG;
+    auto it = std::find(ctx->live_sets.begin(), ctx->live_sets.end(), set);
+    if (!set || it == ctx->live_sets.end()) return fail(ctx, FDD_ERR_STATE, "fork set is not live (double free?)");
+    ctx->live_sets.erase(it);
+    cudaFree(set->d_seeds);
+    delete set;
+    return FDD_OK;
+}
+
+int fdd_forkset_suffix_len(const fdd_forkset* set) { return set ? set->suffix_len : FDD_ERR_INVALID_ARG; }
+
+fdd_status fdd_forkset_reset(fdd_ctx* ctx, fdd_forkset* set) {
+    if (!ctx) return FDD_ERR_INVALID_ARG;
+    if (!set_alive(ctx, set)) return fail(ctx, FDD_ERR_STATE, "fork set is not live");
+    set->suffix_len = 0;
+    return FDD_OK;
+}
+
+fdd_status fdd_block_attn(fdd_ctx* ctx, fdd_forkset* const* sets, int n_sets, int layer,
+                          const void* q, const void* k_blk, const void* v_blk, void* out,
+                          const int32_t* block_len, float scale, int causal_in_block, void* stream) {
+    if (!ctx) return FDD_ERR_INVALID_ARG;
+    int total = 0;
+    fdd_status st = check_sets(ctx, sets, n_sets, block_len, &total);
+    if (st != FDD_OK) return st;
+    if (!q || !k_blk || !v_blk || !out) return fail(ctx, FDD_ERR_INVALID_ARG, "q/k_blk/v_blk/out is NULL");
+    if (!aligned16(q) || !aligned16(k_blk) || !aligned16(v_blk) || !aligned16(out))
+        return fail(ctx, FDD_ERR_INVALID_ARG, "q/k_blk/v_blk/out must be 16-byte aligned");
+    if (layer < 0 || layer >= ctx->cfg.n_layers) return fail(ctx, FDD_ERR_SHAPE, "layer %d outside [0, %d)", layer, ctx->cfg.n_layers);
+    if (!(scale > 0.0f)) return fail(ctx, FDD_ERR_INVALID_ARG, "scale must be positive");
+    const fdd_config& c = ctx->cfg;
+    size_t q_off = 0, kv_off = 0;
+    for (int s = 0; s < n_sets; ++s) {
+        const fdd_forkset* fs = sets[s];
+        AttnProblem p;
+        p.q = static_cast<const __nv_bfloat16*>(q) + q_off;
+        p.k_blk = static_cast<const __nv_bfloat16*>(k_blk) + kv_off;
+        p.v_blk = static_cast<const __nv_bfloat16*>(v_blk) + kv_off;
+        p.out = static_cast<__nv_bfloat16*>(out) + q_off;
+        p.prefix_k = static_cast<const __nv_bfloat16*>(fs->prefix_k[layer]);
+        p.prefix_v = static_cast<const __nv_bfloat16*>(fs->prefix_v[layer]);
+        p.page_table = fs->page_table;
+        p.suffix_k = static_cast<const __nv_bfloat16*>(fs->suffix_k[layer]);
+        p.suffix_v = static_cast<const __nv_bfloat16*>(fs->suffix_v[layer]);
+        p.n_forks = fs->n_forks;
+        p.d = block_len[s];
+        p.n_q_heads = c.n_q_heads;
+        p.n_kv_heads = c.n_kv_heads;
+        p.prefix_len = fs->prefix_len;
+        p.prefix_capacity = fs->prefix_capacity;
+        p.page_tokens = c.page_tokens;
+        p.suffix_len = fs->suffix_len;
+        p.suffix_capacity = fs->suffix_capacity;
+        p.causal_in_block = causal_in_block ? 1 : 0;
+        p.scale = scale;
+        int n_launches = 0;
+        cudaError_t e = launch_attention(ctx, p, c.head_dim, static_cast<cudaStream_t>(stream), &n_launches);
+        ctx->launches += n_launches;
+        if (e != cudaSuccess) return cuda_fail(ctx, e, "fdd_block_attn launch");
+        q_off += static_cast<size_t>(fs->n_forks) * p.d * c.n_q_heads * c.head_dim;
+        kv_off += static_cast<size_t>(fs->n_forks) * p.d * c.n_kv_heads * c.head_dim;
+    }
+    return FDD_OK;
+}
+
+fdd_status fdd_unmask(fdd_ctx* ctx, fdd_forkset* const* sets, int n_sets, const void* logits,
+                      int32_t* tokens, uint8_t* state, const int32_t* block_len,
+                      float threshold, float temperature, uint32_t block_idx, uint32_t step,
+                      int32_t* n_committed, int32_t* n_left, float* conf, void* stream) {
+    if (!ctx) return FDD_ERR_INVALID_ARG;
+    int total = 0;
+    fdd_status st = check_sets(ctx, sets, n_sets, block_len, &total);
+    if (st != FDD_OK) return st;
+    if (!logits || !tokens || !state || !n_committed || !n_left)
+        return fail(ctx, FDD_ERR_INVALID_ARG, "logits/tokens/state/n_committed/n_left is NULL");
+    if (!(temperature >= 0.0f)) return fail(ctx, FDD_ERR_INVALID_ARG, "temperature must be >= 0");
+    if (threshold != threshold) return fail(ctx, FDD_ERR_INVALID_ARG, "threshold is NaN");
+    const fdd_config& c = ctx->cfg;
+    const size_t esz = c.logits_dtype == FDD_LOGITS_BF16 ? 2 : 4;
+    size_t row_off = 0;
+    int fork_off = 0;
+    for (int s = 0; s < n_sets; ++s) {
+        const fdd_forkset* fs = sets[s];
+        UnmaskProblem p;
+        p.logits = static_cast<const char*>(logits) + row_off * c.vocab * esz;
+        p.tokens = tokens + row_off;
+        p.state = state + row_off;
+        p.seeds = fs->d_seeds;
+        p.n_committed = n_committed + fork_off;
+        p.n_left = n_left + fork_off;
+        p.conf = conf ? conf + row_off : nullptr;
+        p.n_forks = fs->n_forks;
+        p.d = block_len[s];
+        p.vocab = c.vocab;
+        p.logits_dtype = c.logits_dtype;
+        p.threshold = threshold;
+        p.temperature = temperature;
+        p.block_idx = block_idx;
+        p.step = step;
+        int n_launches = 0;
+        cudaError_t e = launch_unmask(ctx, p, static_cast<cudaStream_t>(stream), &n_launches);
+        ctx->launches += n_launches;
+        if (e != cudaSuccess) return cuda_fail(ctx, e, "fdd_unmask launch");
+        row_off += static_cast<size_t>(fs->n_forks) * p.d;
+        fork_off += fs->n_forks;
+    }
+    return FDD_OK;
+}
+
+fdd_status fdd_kv_commit(fdd_ctx* ctx, fdd_forkset* const* sets, int n_sets, int layer,
+                         const void* k_blk, const void* v_blk, const int32_t* block_len,
+                         int advance, void* stream) {
+    if (!ctx) return FDD_ERR_INVALID_ARG;
+    int total = 0;
+    fdd_status st = check_sets(ctx, sets, n_sets, block_len, &total);
+    if (st != FDD_OK) return st;
+    if (!k_blk || !v_blk) return fail(ctx, FDD_ERR_INVALID_ARG, "k_blk/v_blk is NULL");
+    if (!aligned16(k_blk) || !aligned16(v_blk)) return fail(ctx, FDD_ERR_INVALID_ARG, "k_blk/v_blk must be 16-byte aligned");
+    if (layer < 0 || layer >= ctx->cfg.n_layers) return fail(ctx, FDD_ERR_SHAPE, "layer %d outside [0, %d)", layer, ctx->cfg.n_layers);
+    for (int s = 0; s < n_sets; ++s)
+        if (sets[s]->suffix_len + block_len[s] > sets[s]->suffix_capacity)
+            return fail(ctx, FDD_ERR_CAPACITY, "set %d: suffix %d + block %d exceeds capacity %d", s,
+                        sets[s]->suffix_len, block_len[s], sets[s]->suffix_capacity);
+    const fdd_config& c = ctx->cfg;
+    size_t kv_off = 0;
+    for (int s = 0; s < n_sets; ++s) {
+        fdd_forkset* fs = sets[s];
+        cudaError_t e = launch_kv_commit(static_cast<const __nv_bfloat16*>(k_blk) + kv_off,
+                                         static_cast<const __nv_bfloat16*>(v_blk) + kv_off,
+                                         static_cast<__nv_bfloat16*>(fs->suffix_k[layer]),
+                                         static_cast<__nv_bfloat16*>(fs->suffix_v[layer]),
+                                         fs->n_forks, block_len[s], c.n_kv_heads, c.head_dim,
+                                         fs->suffix_len, fs->suffix_capacity, static_cast<cudaStream_t>(stream));
+        ctx->launches += 1;
+        if (e != cudaSuccess) return cuda_fail(ctx, e, "fdd_kv_commit launch");
+        kv_off += static_cast<size_t>(fs->n_forks) * block_len[s] * c.n_kv_heads * c.head_dim;
+    }
+    if (advance)
+        for (int s = 0; s < n_sets; ++s) sets[s]->suffix_len += block_len[s];
+    return FDD_OK;
+}
+
+fdd_status fdd_average_rollouts(fdd_ctx* ctx, const float* traj, int n, int w, float* out, void* stream) {
+    if (!ctx) return FDD_ERR_INVALID_ARG;
+    if (!traj || !out) return fail(ctx, FDD_ERR_INVALID_ARG, "traj/out is NULL");
+    if (n < 1 || w < 1) return fail(ctx, FDD_ERR_INVALID_ARG, "n and w must be >= 1");
+    cudaError_t e = launch_average(traj, n, w, out, static_cast<cudaStream_t>(stream));
+    ctx->launches += 1;
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "fdd_average_rollouts launch");
+    return FDD_OK;
+}
+
+fdd_status fdd_poll_status(fdd_ctx* ctx, void* stream) {
+    if (!ctx) return FDD_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    cudaError_t e = cudaMemcpyAsync(ctx->h_status, ctx->d_status, sizeof(int), cudaMemcpyDeviceToHost, st);
+    if (e == cudaSuccess) e = cudaMemsetAsync(ctx->d_status, 0, sizeof(int), st);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "fdd_poll_status");
+    const int code = *ctx->h_status;
+    if (code != FDD_OK) return fail(ctx, code, "a kernel recorded device status %d", code);
+    return FDD_OK;
+}
+
+}  // extern "C"
+
+cudaError_t launch_attention(fdd_ctx* ctx, const AttnProblem& p, int head_dim, cudaStream_t st, int* n_launches) {
+    (void)ctx;
+    *n_launches += 1;
+    return launch_attention_simple(p, head_dim, st);
+}

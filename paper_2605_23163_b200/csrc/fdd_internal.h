@@ -1,0 +1,89 @@
+// Internal declarations shared by the host API and the kernel files.
+#pragma once
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+#include <string>
+#include <vector>
+
+#include "fdd.h"
+
+struct fdd_ctx {
+    fdd_config cfg;
+    int device = 0;
+    int sm_count = 0;
+    int* d_status = nullptr;          // device status word (first error wins)
+    int* h_status = nullptr;          // pinned mirror
+    void* ws_unmask = nullptr;        // per (row, chunk) partial reductions
+    size_t ws_unmask_bytes = 0;
+    void* ws_attn = nullptr;          // split-KV partial outputs
+    size_t ws_attn_bytes = 0;
+    uint64_t launches = 0;
+    std::string last_error;
+    std::vector<fdd_forkset*> live_sets;
+};
+
+struct fdd_forkset {
+    fdd_ctx* ctx = nullptr;
+    int n_forks = 0;
+    int prefix_len = 0;
+    int prefix_capacity = 0;
+    const int32_t* page_table = nullptr;   // device
+    std::vector<const void*> prefix_k, prefix_v;
+    std::vector<void*> suffix_k, suffix_v;
+    int suffix_capacity = 0;
+    int suffix_len = 0;
+    uint64_t* d_seeds = nullptr;            // device [n_forks]
+};
+
+// One scene's slice of a batched call, as the kernels see it.
+struct AttnProblem {
+    const __nv_bfloat16* q;        // [N][d][Hq][D]
+    const __nv_bfloat16* k_blk;    // [N][d][Hkv][D]
+    const __nv_bfloat16* v_blk;
+    __nv_bfloat16* out;            // [N][d][Hq][D]
+    const __nv_bfloat16* prefix_k; // contiguous [Hkv][cap][D] or paged [pages][Hkv][pt][D]
+    const __nv_bfloat16* prefix_v;
+    const int32_t* page_table;     // device or nullptr
+    const __nv_bfloat16* suffix_k; // [N][Hkv][scap][D]
+    const __nv_bfloat16* suffix_v;
+    int n_forks, d, n_q_heads, n_kv_heads;
+    int prefix_len, prefix_capacity, page_tokens;
+    int suffix_len, suffix_capacity;
+    int causal_in_block;
+    float scale;
+};
+
+struct UnmaskProblem {
+    const void* logits;     // [rows][V]
+    int32_t* tokens;        // [rows]
+    uint8_t* state;         // [rows]
+    const uint64_t* seeds;  // device [n_forks]
+    int32_t* n_committed;   // [n_forks]
+    int32_t* n_left;        // [n_forks]
+    float* conf;            // [rows] or nullptr
+    int n_forks, d, vocab, logits_dtype;
+    float threshold, temperature;
+    uint32_t block_idx, step;
+};
+
+// Unmask scratch: one record per (row, chunk).
+struct UnmaskPartial {
+    float row_max;     // max logit of the chunk
+    float sum_exp;     // sum exp(logit - row_max)
+    float best_score;  // max of logit + T * gumbel
+    float best_logit;  // logit at the best score
+    int best_index;    // vocabulary id of the best score (lowest on ties)
+    int pad[3];
+};
+
+static constexpr int kUnmaskChunk = 8192;   // vocabulary entries per CTA
+static inline int unmask_chunks(int vocab) { return (vocab + kUnmaskChunk - 1) / kUnmaskChunk; }
+
+cudaError_t launch_attention(fdd_ctx* ctx, const AttnProblem& p, int head_dim, cudaStream_t st, int* n_launches);
+cudaError_t launch_unmask(fdd_ctx* ctx, const UnmaskProblem& p, cudaStream_t st, int* n_launches);
+cudaError_t launch_kv_commit(const __nv_bfloat16* k_blk, const __nv_bfloat16* v_blk,
+                             __nv_bfloat16* suffix_k, __nv_bfloat16* suffix_v,
+                             int n_forks, int d, int n_kv_heads, int head_dim,
+                             int suffix_len, int suffix_capacity, cudaStream_t st);
+cudaError_t launch_average(const float* traj, int n, int w, float* out, cudaStream_t st);

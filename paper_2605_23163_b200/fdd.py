@@ -1,0 +1,202 @@
+"""ctypes binding of the C-ABI library declared in include/fdd.h.
+
+Argument marshalling only: every function below has the name and the argument
+order of its C counterpart, takes torch CUDA tensors (or raw integer device
+pointers) where the C call takes device pointers, and raises `FddError` when the
+C call returns a negative status.  All arithmetic runs in the CUDA kernels of
+libfdd.so; there is no fallback, and a missing library is an error.
+"""
+import ctypes
+import os
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libfdd.so")
+
+FDD_OK = 0
+FDD_ERR_INVALID_ARG, FDD_ERR_SHAPE, FDD_ERR_CAPACITY, FDD_ERR_STATE = -1, -2, -3, -4
+FDD_ERR_CUDA, FDD_ERR_DEVICE_TIMEOUT, FDD_ERR_UNSUPPORTED = -5, -6, -7
+FDD_MASKED, FDD_COMMITTED, FDD_SCAFFOLD = 0, 1, 2
+FDD_LOGITS_F32, FDD_LOGITS_BF16 = 0, 1
+
+EXPORTS = (
+    "fdd_create", "fdd_destroy", "fdd_last_error", "fdd_launch_count", "fdd_fork",
+    "fdd_forkset_free", "fdd_forkset_suffix_len", "fdd_forkset_reset", "fdd_block_attn",
+    "fdd_unmask", "fdd_kv_commit", "fdd_average_rollouts", "fdd_poll_status",
+)
+
+
+class FddError(RuntimeError):
+    def __init__(self, status, text):
+        super().__init__(f"fdd status {status}: {text}")
+        self.status = status
+
+
+class fdd_config(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int) for n in (
+        "n_q_heads", "n_kv_heads", "head_dim", "vocab", "n_layers", "page_tokens",
+        "max_block", "max_forks", "logits_dtype")]
+
+
+_lib_handle = None
+
+
+def lib():
+    """The loaded shared library.  Raises if it has not been built."""
+    global _lib_handle
+    if _lib_handle is not None:
+        return _lib_handle
+    if not os.path.exists(LIB_PATH):
+        raise RuntimeError(
+            f"{LIB_PATH} is missing: build it with `python -m paper_2605_23163_b200.build` "
+            "(there is no CPU fallback)")
+    L = ctypes.CDLL(LIB_PATH)
+    vp, ip, i32, u32, u64, f32 = (ctypes.c_void_p, ctypes.POINTER(ctypes.c_int32), ctypes.c_int,
+                                  ctypes.c_uint32, ctypes.c_uint64, ctypes.c_float)
+    vpp = ctypes.POINTER(ctypes.c_void_p)
+    L.fdd_create.argtypes = [ctypes.POINTER(fdd_config), vpp]
+    L.fdd_create.restype = i32
+    L.fdd_destroy.argtypes = [vp]
+    L.fdd_destroy.restype = None
+    L.fdd_last_error.argtypes = [vp]
+    L.fdd_last_error.restype = ctypes.c_char_p
+    L.fdd_launch_count.argtypes = [vp]
+    L.fdd_launch_count.restype = u64
+    L.fdd_fork.argtypes = [vp, vpp, vpp, vp, i32, i32, i32, ctypes.POINTER(u64), vpp, vpp, i32, vpp]
+    L.fdd_fork.restype = i32
+    L.fdd_forkset_free.argtypes = [vp, vp]
+    L.fdd_forkset_free.restype = i32
+    L.fdd_forkset_suffix_len.argtypes = [vp]
+    L.fdd_forkset_suffix_len.restype = i32
+    L.fdd_forkset_reset.argtypes = [vp, vp]
+    L.fdd_forkset_reset.restype = i32
+    L.fdd_block_attn.argtypes = [vp, vpp, i32, i32, vp, vp, vp, vp, ip, f32, i32, vp]
+    L.fdd_block_attn.restype = i32
+    L.fdd_unmask.argtypes = [vp, vpp, i32, vp, vp, vp, ip, f32, f32, u32, u32, vp, vp, vp, vp]
+    L.fdd_unmask.restype = i32
+    L.fdd_kv_commit.argtypes = [vp, vpp, i32, i32, vp, vp, ip, i32, vp]
+    L.fdd_kv_commit.restype = i32
+    L.fdd_average_rollouts.argtypes = [vp, vp, i32, i32, vp, vp]
+    L.fdd_average_rollouts.restype = i32
+    L.fdd_poll_status.argtypes = [vp, vp]
+    L.fdd_poll_status.restype = i32
+    _lib_handle = L
+    return L
+
+
+def _ptr(t):
+    """Device address of a tensor (must be contiguous) or a raw integer pointer / None."""
+    if t is None:
+        return None
+    if isinstance(t, ctypes.c_void_p):
+        return t
+    if isinstance(t, int):
+        return ctypes.c_void_p(t)
+    if not t.is_contiguous():
+        raise ValueError("tensor must be contiguous")
+    return ctypes.c_void_p(t.data_ptr())
+
+
+def _stream(stream):
+    if stream is None:
+        import torch
+        return ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+    if isinstance(stream, int):
+        return ctypes.c_void_p(stream)
+    return ctypes.c_void_p(stream.cuda_stream)
+
+
+def _check(ctx, status):
+    if status < 0:
+        raise FddError(status, lib().fdd_last_error(ctx).decode() if ctx else "no context")
+    return status
+
+
+def _ptr_array(items):
+    arr = (ctypes.c_void_p * len(items))()
+    for i, t in enumerate(items):
+        p = _ptr(t)
+        arr[i] = p.value if p is not None else None
+    return arr
+
+
+def _i32_array(vals):
+    return (ctypes.c_int32 * len(vals))(*[int(v) for v in vals])
+
+
+def fdd_create(n_q_heads, n_kv_heads, head_dim, vocab, n_layers=1, page_tokens=0, max_block=64,
+               max_forks=32, logits_dtype=FDD_LOGITS_BF16):
+    cfg = fdd_config(n_q_heads, n_kv_heads, head_dim, vocab, n_layers, page_tokens, max_block,
+                     max_forks, logits_dtype)
+    out = ctypes.c_void_p()
+    st = lib().fdd_create(ctypes.byref(cfg), ctypes.byref(out))
+    if st < 0:
+        raise FddError(st, "fdd_create failed")
+    return out
+
+
+def fdd_destroy(ctx):
+    lib().fdd_destroy(ctx)
+
+
+def fdd_last_error(ctx):
+    return lib().fdd_last_error(ctx).decode()
+
+
+def fdd_launch_count(ctx):
+    return int(lib().fdd_launch_count(ctx))
+
+
+def fdd_fork(ctx, prefix_k, prefix_v, page_table, prefix_len, prefix_capacity, n_forks, seeds,
+             suffix_k, suffix_v, suffix_capacity):
+    """prefix_k/v, suffix_k/v: per-layer lists of CUDA tensors; seeds: iterable of N ints."""
+    seeds = [int(s) & 0xFFFFFFFFFFFFFFFF for s in seeds]
+    seed_arr = (ctypes.c_uint64 * len(seeds))(*seeds)
+    out = ctypes.c_void_p()
+    st = lib().fdd_fork(ctx, _ptr_array(prefix_k), _ptr_array(prefix_v), _ptr(page_table),
+                        int(prefix_len), int(prefix_capacity), int(n_forks), seed_arr,
+                        _ptr_array(suffix_k), _ptr_array(suffix_v), int(suffix_capacity),
+                        ctypes.byref(out))
+    _check(ctx, st)
+    return out
+
+
+def fdd_forkset_free(ctx, fs):
+    return _check(ctx, lib().fdd_forkset_free(ctx, fs))
+
+
+def fdd_forkset_suffix_len(fs):
+    return int(lib().fdd_forkset_suffix_len(fs))
+
+
+def fdd_forkset_reset(ctx, fs):
+    return _check(ctx, lib().fdd_forkset_reset(ctx, fs))
+
+
+def fdd_block_attn(ctx, sets, layer, q, k_blk, v_blk, out, block_len, scale, causal_in_block=0,
+                   stream=None):
+    return _check(ctx, lib().fdd_block_attn(
+        ctx, _ptr_array(sets), len(sets), int(layer), _ptr(q), _ptr(k_blk), _ptr(v_blk), _ptr(out),
+        _i32_array(block_len), float(scale), int(causal_in_block), _stream(stream)))
+
+
+def fdd_unmask(ctx, sets, logits, tokens, state, block_len, threshold, temperature, block_idx, step,
+               n_committed, n_left, conf=None, stream=None):
+    return _check(ctx, lib().fdd_unmask(
+        ctx, _ptr_array(sets), len(sets), _ptr(logits), _ptr(tokens), _ptr(state),
+        _i32_array(block_len), float(threshold), float(temperature), int(block_idx), int(step),
+        _ptr(n_committed), _ptr(n_left), _ptr(conf), _stream(stream)))
+
+
+def fdd_kv_commit(ctx, sets, layer, k_blk, v_blk, block_len, advance, stream=None):
+    return _check(ctx, lib().fdd_kv_commit(
+        ctx, _ptr_array(sets), len(sets), int(layer), _ptr(k_blk), _ptr(v_blk),
+        _i32_array(block_len), int(advance), _stream(stream)))
+
+
+def fdd_average_rollouts(ctx, traj, n, w, out, stream=None):
+    return _check(ctx, lib().fdd_average_rollouts(ctx, _ptr(traj), int(n), int(w), _ptr(out),
+                                                  _stream(stream)))
+
+
+def fdd_poll_status(ctx, stream=None):
+    return _check(ctx, lib().fdd_poll_status(ctx, _stream(stream)))

@@ -1,0 +1,379 @@
+"""GPU parity: every C-ABI call against the CPU fp64 oracle on the same seeded inputs."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import MASKED, COMMITTED, SCAFFOLD
+from oracle.average import average_rollouts
+from oracle.cache import ForkSet
+from oracle.unmask import unmask_step
+from paper_2605_23163_b200 import fdd, harness, synth
+
+import parity_utils as pu
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(autouse=True)
+def _need_cuda():
+    assert torch.cuda.is_available(), "these tests need a CUDA device"
+    fdd.lib()   # fail loudly if the CUDA library is missing
+
+
+def _suffix_from_oracle(fs, layer=0):
+    return (fs.suffix_k[layer], fs.suffix_v[layer])
+
+
+# ---------------------------------------------------------------------------------------------
+# attention
+# ---------------------------------------------------------------------------------------------
+def _attention_case(w, n_blocks_before=0, causal=False, forks_checked=None, layer=0):
+    ctx = harness.create_context(w)
+    try:
+        scene = harness.GpuScene(ctx, w, 0, suffix_capacity=w.scenes[0].block_len * (n_blocks_before + 1))
+        pk, pv = synth.make_prefix(w, 0)
+        ofs = ForkSet([pk], [pv], w.scenes[0].n_forks, scene.seeds)
+        for b in range(n_blocks_before):         # fill the private suffix with earlier blocks
+            _, kb, vb = synth.make_qkv(w, 0, 0, b, 0)
+            fdd.fdd_kv_commit(ctx, [scene.forkset], 0, harness.bf16_tensor(kb), harness.bf16_tensor(vb),
+                              [kb.shape[1]], 1)
+            ofs.kv_commit(0, kb, vb)
+        assert fdd.fdd_forkset_suffix_len(scene.forkset) == n_blocks_before * w.scenes[0].block_len
+        q, k, v = synth.make_qkv(w, 0, 0, n_blocks_before, 0)
+        got = pu.attention_gpu(ctx, scene, q, k, v, causal=causal)
+        forks = list(range(q.shape[0])) if forks_checked is None else forks_checked
+        ref = pu.attention_oracle(w, (pk, pv), _suffix_from_oracle(ofs), q, k, v, causal=causal, forks=forks)
+        return pu.assert_attention_close(got[forks], ref)
+    finally:
+        fdd.fdd_destroy(ctx)
+
+
+def test_attention_tiny():
+    _attention_case(synth.workload("tiny"))
+
+
+def test_attention_single_scene_with_suffix():
+    _attention_case(synth.workload("single_scene"), n_blocks_before=2)
+
+
+def test_attention_tts_all_forks():
+    _attention_case(synth.workload("tts"), n_blocks_before=1)
+
+
+def test_attention_tts_ragged_prefix_and_block():
+    # prefix not a multiple of any tile, block of 13 positions (ragged row tile), 3 rollouts
+    w = synth.workload("tts")
+    sc = synth.Scene(prefix_len=1000 + 37, n_forks=3, block_len=13, n_scaffold=4, n_blocks=3)
+    w = synth.Workload("ragged", w.n_q_heads, w.n_kv_heads, w.head_dim, 1024, "bf16", "peaked", 0.9, 1.0,
+                       (sc,), seed=11)
+    _attention_case(w, n_blocks_before=2)
+
+
+def test_attention_long_prefix_sampled_forks():
+    # full-size largest configuration; the oracle checks three of the 32 rollouts
+    _attention_case(synth.workload("long_prefix"), forks_checked=[0, 13, 31])
+
+
+def test_attention_no_prefix_and_single_position():
+    w = synth.workload("tiny")
+    sc = synth.Scene(prefix_len=0, n_forks=2, block_len=1, n_scaffold=0, n_blocks=2)
+    w = synth.Workload("degenerate", 4, 1, 64, 64, "f32", "normal_sigma2", 0.9, 0.0, (sc,), qkv_sigma=0.5, seed=12)
+    _attention_case(w, n_blocks_before=0)       # a single key: output == that value row
+    _attention_case(w, n_blocks_before=1)
+
+
+def test_attention_causal_in_block():
+    w = synth.small_variant(synth.workload("tts"), prefix_len=300, vocab=512, n_forks=2, n_blocks=2)
+    _attention_case(w, n_blocks_before=1, causal=True)
+
+
+def test_attention_paged_prefix():
+    w = synth.workload("serving_mix")
+    sc = synth.Scene(prefix_len=64 * 9 + 17, n_forks=4, block_len=16, n_scaffold=5, n_blocks=2)
+    w = synth.Workload("paged", w.n_q_heads, w.n_kv_heads, w.head_dim, 1024, "bf16", "peaked", 0.9, 1.0,
+                       (sc,), page_tokens=64, seed=13)
+    _attention_case(w, n_blocks_before=1)
+
+
+def test_prefix_is_never_written_and_forks_with_equal_inputs_agree():
+    w = synth.small_variant(synth.workload("tts"), prefix_len=512, vocab=512, n_forks=4, n_blocks=1)
+    ctx = harness.create_context(w)
+    try:
+        scene = harness.GpuScene(ctx, w, 0)
+        before = [t.clone() for t in scene.prefix_k + scene.prefix_v]
+        q, k, v = synth.make_qkv(w, 0, 0, 0, 0)
+        q, k, v = (np.repeat(x[:1], 4, axis=0) for x in (q, k, v))
+        got = pu.attention_gpu(ctx, scene, q, k, v)
+        for f in range(1, 4):
+            assert np.array_equal(got[f], got[0])
+        fdd.fdd_kv_commit(ctx, [scene.forkset], 0, harness.bf16_tensor(k), harness.bf16_tensor(v), [k.shape[1]], 1)
+        fdd.fdd_poll_status(ctx)
+        for a, b in zip(before, scene.prefix_k + scene.prefix_v):
+            assert torch.equal(a, b)
+    finally:
+        fdd.fdd_destroy(ctx)
+
+
+# ---------------------------------------------------------------------------------------------
+# kv commit
+# ---------------------------------------------------------------------------------------------
+def test_kv_commit_bytes_and_capacity():
+    w = synth.small_variant(synth.workload("tts"), prefix_len=64, vocab=512, n_forks=3, n_blocks=2)
+    ctx = harness.create_context(w)
+    try:
+        scene = harness.GpuScene(ctx, w, 0, suffix_capacity=2 * w.scenes[0].block_len)
+        d = w.scenes[0].block_len
+        blocks = [synth.make_qkv(w, 0, 0, b, 0)[1:] for b in range(2)]
+        for b, (kb, vb) in enumerate(blocks):
+            fdd.fdd_kv_commit(ctx, [scene.forkset], 0, harness.bf16_tensor(kb), harness.bf16_tensor(vb), [d], 1)
+        fdd.fdd_poll_status(ctx)
+        sk = scene.suffix_k[0].view(torch.int16).cpu().numpy().view(np.uint16)    # [N,Hkv,cap,D]
+        sv = scene.suffix_v[0].view(torch.int16).cpu().numpy().view(np.uint16)
+        for b, (kb, vb) in enumerate(blocks):
+            assert np.array_equal(sk[:, :, b * d:(b + 1) * d], kb.transpose(0, 2, 1, 3))
+            assert np.array_equal(sv[:, :, b * d:(b + 1) * d], vb.transpose(0, 2, 1, 3))
+        with pytest.raises(fdd.FddError) as ei:
+            fdd.fdd_kv_commit(ctx, [scene.forkset], 0, harness.bf16_tensor(blocks[0][0]),
+                              harness.bf16_tensor(blocks[0][1]), [d], 1)
+        assert ei.value.status == fdd.FDD_ERR_CAPACITY
+        fdd.fdd_forkset_reset(ctx, scene.forkset)
+        assert fdd.fdd_forkset_suffix_len(scene.forkset) == 0
+    finally:
+        fdd.fdd_destroy(ctx)
+
+
+# ---------------------------------------------------------------------------------------------
+# unmask
+# ---------------------------------------------------------------------------------------------
+def _unmask_step_case(w, block=0, step=0, threshold=None, temperature=None, state_override=None):
+    ctx = harness.create_context(w)
+    try:
+        scene = harness.GpuScene(ctx, w, 0)
+        tokens, state = synth.make_block_template(w, 0, block)
+        if state_override is not None:
+            tokens, state = state_override(tokens, state)
+        logits = synth.make_logits(w, 0, block, step, rows="all")
+        th = w.threshold if threshold is None else threshold
+        te = w.temperature if temperature is None else temperature
+        got = pu.unmask_gpu(ctx, scene, logits, tokens, state, th, te, block, step)
+        ref = unmask_step(pu.widen_logits(w, logits), tokens, state, scene.seeds, th, te, block, step)
+        return pu.compare_unmask(got, ref, tokens, state, th), got, ref
+    finally:
+        fdd.fdd_destroy(ctx)
+
+
+def test_unmask_tiny_fallback_every_step():
+    w = synth.workload("tiny")
+    ctx = harness.create_context(w)
+    try:
+        scene = harness.GpuScene(ctx, w, 0)
+        tokens, state = synth.make_block_template(w, 0, 0)
+        steps = 0
+        while np.any(state == MASKED):
+            logits = synth.make_logits(w, 0, 0, steps, rows="all")
+            got = pu.unmask_gpu(ctx, scene, logits, tokens, state, w.threshold, 0.0, 0, steps)
+            ref = unmask_step(logits, tokens, state, scene.seeds, w.threshold, 0.0, 0, steps)
+            info = pu.compare_unmask(got, ref, tokens, state, w.threshold)
+            assert not info["ambiguous_forks"]
+            assert got["n_committed"][0] == 1
+            tokens, state = got["tokens"], got["state"]
+            steps += 1
+            assert steps <= 16
+        assert steps == 12
+    finally:
+        fdd.fdd_destroy(ctx)
+
+
+@pytest.mark.parametrize("temperature", [0.0, 1.0])
+def test_unmask_full_vocab_bf16(temperature):
+    w = synth.small_variant(synth.workload("tts"), prefix_len=64, n_forks=4, n_blocks=1)
+    info, got, ref = _unmask_step_case(w, temperature=temperature)
+    assert info["rows"] == 4 * 22
+    assert len(info["ambiguous_forks"]) <= 1
+    assert got["n_committed"].sum() >= 4
+
+
+def test_unmask_odd_vocab_and_partial_state():
+    # vocabulary not a multiple of the vector width, several chunks with a ragged tail, rows in
+    # every state, one rollout already finished
+    sc = synth.Scene(prefix_len=16, n_forks=3, block_len=9, n_scaffold=2, n_blocks=1)
+    w = synth.Workload("odd", 4, 1, 64, 8192 * 2 + 1237, "f32", "peaked", 0.7, 0.8, (sc,), seed=21)
+
+    def override(tokens, state):
+        state = state.copy()
+        tokens = tokens.copy()
+        state[1][state[1] == MASKED] = COMMITTED          # rollout 1 is done
+        tokens[1] = 5
+        first = np.nonzero(state[2] == MASKED)[0][0]
+        state[2, first] = COMMITTED
+        tokens[2, first] = 77
+        return tokens, state
+
+    info, got, ref = _unmask_step_case(w, state_override=override)
+    assert got["n_committed"][1] == 0 and got["n_left"][1] == 0
+    assert not info["ambiguous_forks"]
+    w2 = synth.Workload("odd_bf16", 4, 1, 64, 8192 + 3, "bf16", "peaked", 0.7, 1.3, (sc,), seed=22)
+    info, _, _ = _unmask_step_case(w2)
+    assert not info["ambiguous_forks"]
+
+
+def test_unmask_threshold_extremes():
+    w = synth.small_variant(synth.workload("tts"), prefix_len=64, vocab=4096, n_forks=2, n_blocks=1)
+    info, got, ref = _unmask_step_case(w, threshold=1.5)          # nothing passes: one commit each
+    assert list(got["n_committed"]) == [1, 1]
+    info, got, ref = _unmask_step_case(w, threshold=-1.0)         # everything commits
+    assert np.all(got["state"] != MASKED) and list(got["n_left"]) == [0, 0]
+
+
+def test_unmask_identical_seeds_give_identical_forks():
+    w = synth.small_variant(synth.workload("tts"), prefix_len=64, vocab=4096, n_forks=3, n_blocks=1)
+    ctx = harness.create_context(w)
+    try:
+        scene = harness.GpuScene(ctx, w, 0, identical_seeds=True)
+        tokens, state = synth.make_block_template(w, 0, 0)
+        logits = np.repeat(synth.make_logits(w, 0, 0, 0, rows="all")[:1], 3, axis=0)
+        got = pu.unmask_gpu(ctx, scene, logits, tokens, state, w.threshold, 1.0, 0, 0)
+        for f in (1, 2):
+            assert np.array_equal(got["tokens"][f], got["tokens"][0])
+            assert np.array_equal(got["state"][f], got["state"][0])
+    finally:
+        fdd.fdd_destroy(ctx)
+
+
+def test_unmask_long_prefix_full_size_step0():
+    # the largest configuration at full size: all 2048 rows on the GPU; the oracle checks every
+    # row of four sampled rollouts (1216 vocabulary-wide rows would take minutes on the CPU)
+    w = synth.workload("long_prefix")
+    ctx = harness.create_context(w)
+    try:
+        scene = harness.GpuScene(ctx, w, 0)
+        tokens, state = synth.make_block_template(w, 0, 0)
+        sample = [0, 7, 19, 31]
+        logits = np.zeros((32, 64, w.vocab), dtype=np.uint16)
+        frozen = set(synth.scaffold_positions(w, 0, 0).tolist())
+        for f in sample:
+            for i in range(64):
+                if i not in frozen:
+                    logits[f, i] = synth.make_logits_row(w, 0, 0, 0, f, i)
+        for f in range(32):      # rollouts outside the sample reuse rollout 0's rows (less host time)
+            if f not in sample:
+                logits[f] = logits[0]
+        got = pu.unmask_gpu(ctx, scene, logits, tokens, state, w.threshold, w.temperature, 0, 0)
+        ref = unmask_step(pu.widen_logits(w, logits[sample]), tokens[sample], state[sample],
+                          scene.seeds[sample], w.threshold, w.temperature, 0, 0)
+        sub = {k: (v[sample] if v is not None else None) for k, v in got.items()}
+        info = pu.compare_unmask(sub, ref, tokens[sample], state[sample], w.threshold)
+        assert info["rows"] == 4 * 38
+        assert len(info["ambiguous_forks"]) <= 1
+        assert np.all(got["n_committed"] >= 1)
+        assert np.all(got["n_left"] + got["n_committed"] == 38)
+    finally:
+        fdd.fdd_destroy(ctx)
+
+
+# ---------------------------------------------------------------------------------------------
+# whole block loop, averaging
+# ---------------------------------------------------------------------------------------------
+def test_block_loop_matches_oracle_and_averages():
+    w = synth.small_variant(synth.workload("tts"), prefix_len=200, vocab=2048, n_forks=4, n_blocks=2)
+    sc = w.scenes[0]
+    ctx = harness.create_context(w)
+    try:
+        scene = harness.GpuScene(ctx, w, 0)
+        pk, pv = synth.make_prefix(w, 0)
+        ofs = ForkSet([pk], [pv], sc.n_forks, scene.seeds)
+        scale = 1.0 / np.sqrt(w.head_dim)
+        all_tokens, all_state = [], []
+        diverged = set()
+        for block in range(sc.n_blocks):
+            tokens, state = synth.make_block_template(w, 0, block)
+            step = 0
+            while np.any(state == MASKED):
+                q, k, v = synth.make_qkv(w, 0, 0, block, step)
+                got_attn = pu.attention_gpu(ctx, scene, q, k, v)
+                ref_attn = pu.attention_oracle(w, (pk, pv), _suffix_from_oracle(ofs), q, k, v)
+                pu.assert_attention_close(got_attn, ref_attn)
+                logits = synth.make_logits(w, 0, block, step, rows="all")
+                got = pu.unmask_gpu(ctx, scene, logits, tokens, state, w.threshold, w.temperature, block, step)
+                ref = unmask_step(pu.widen_logits(w, logits), tokens, state, scene.seeds, w.threshold,
+                                  w.temperature, block, step)
+                info = pu.compare_unmask(got, ref, tokens, state, w.threshold)
+                diverged |= info["ambiguous_forks"]
+                tokens, state = got["tokens"], got["state"]
+                step += 1
+                assert step <= sc.block_len
+            fdd.fdd_kv_commit(ctx, [scene.forkset], 0, harness.bf16_tensor(k), harness.bf16_tensor(v), [sc.block_len], 1)
+            ofs.kv_commit(0, k, v)
+            all_tokens.append(tokens)
+            all_state.append(state)
+        assert len(diverged) <= 1
+        toks, sts = np.concatenate(all_tokens, axis=1), np.concatenate(all_state, axis=1)
+        traj = synth.tokens_to_trajectory(w, toks, sts)
+        t_dev = torch.from_numpy(traj).cuda()
+        out = torch.zeros((w.waypoints, 2), dtype=torch.float32, device="cuda")
+        fdd.fdd_average_rollouts(ctx, t_dev, sc.n_forks, w.waypoints, out)
+        fdd.fdd_poll_status(ctx)
+        ref = average_rollouts(traj)
+        got = out.cpu().numpy().astype(np.float64)
+        assert np.all(np.abs(got - ref) <= 1e-5 * np.maximum(np.abs(ref), 1e-30) + 1e-30)
+    finally:
+        fdd.fdd_destroy(ctx)
+
+
+def test_average_cancellation_and_single_rollout():
+    ctx = fdd.fdd_create(4, 1, 64, 64)
+    try:
+        g = np.random.default_rng(5)
+        traj = (g.standard_normal((32, 10, 2)) * 100).astype(np.float32)
+        traj[1::2] = -traj[::2] + np.float32(1e-3)        # heavy cancellation
+        out = torch.zeros((10, 2), dtype=torch.float32, device="cuda")
+        fdd.fdd_average_rollouts(ctx, torch.from_numpy(traj).cuda(), 32, 10, out)
+        ref = average_rollouts(traj)
+        got = out.cpu().numpy().astype(np.float64)
+        assert np.all(np.abs(got - ref) <= 1e-5 * np.abs(ref))
+        fdd.fdd_average_rollouts(ctx, torch.from_numpy(traj[:1].copy()).cuda(), 1, 10, out)
+        assert np.array_equal(out.cpu().numpy(), traj[0])
+    finally:
+        fdd.fdd_destroy(ctx)
+
+
+# ---------------------------------------------------------------------------------------------
+# host-side error paths (nothing is launched)
+# ---------------------------------------------------------------------------------------------
+def test_error_paths():
+    with pytest.raises(fdd.FddError) as ei:
+        fdd.fdd_create(16, 2, 96, 1000)
+    assert ei.value.status == fdd.FDD_ERR_UNSUPPORTED
+    with pytest.raises(fdd.FddError):
+        fdd.fdd_create(16, 3, 128, 1000)
+    w = synth.small_variant(synth.workload("tts"), prefix_len=64, vocab=512, n_forks=2, n_blocks=1)
+    ctx = harness.create_context(w)
+    try:
+        scene = harness.GpuScene(ctx, w, 0)
+        q, k, v = (harness.bf16_tensor(x) for x in synth.make_qkv(w, 0, 0, 0, 0))
+        out = torch.empty_like(q)
+        with pytest.raises(fdd.FddError) as ei:
+            fdd.fdd_block_attn(ctx, [scene.forkset], 0, q, k, v, out, [w.scenes[0].block_len + 100], 0.1)
+        assert ei.value.status == fdd.FDD_ERR_CAPACITY
+        with pytest.raises(fdd.FddError) as ei:
+            fdd.fdd_block_attn(ctx, [scene.forkset], 3, q, k, v, out, [32], 0.1)
+        assert ei.value.status == fdd.FDD_ERR_SHAPE
+        with pytest.raises(fdd.FddError) as ei:
+            fdd.fdd_block_attn(ctx, [scene.forkset], 0, None, k, v, out, [32], 0.1)
+        assert ei.value.status == fdd.FDD_ERR_INVALID_ARG
+        with pytest.raises(fdd.FddError) as ei:
+            fdd.fdd_fork(ctx, scene.prefix_k, scene.prefix_v, None, 64, 64, 999, [1] * 999,
+                         scene.suffix_k, scene.suffix_v, 32)
+        assert ei.value.status == fdd.FDD_ERR_CAPACITY
+        fs = scene.forkset
+        scene.free()
+        with pytest.raises(fdd.FddError) as ei:           # freed handle
+            fdd.fdd_block_attn(ctx, [fs], 0, q, k, v, out, [32], 0.1)
+        assert ei.value.status == fdd.FDD_ERR_STATE
+        with pytest.raises(fdd.FddError) as ei:           # double free
+            fdd.fdd_forkset_free(ctx, fs)
+        assert ei.value.status == fdd.FDD_ERR_STATE
+        assert "not live" in fdd.fdd_last_error(ctx)
+        assert fdd.fdd_poll_status(ctx) == fdd.FDD_OK
+    finally:
+        fdd.fdd_destroy(ctx)
