@@ -181,6 +181,43 @@ fdd_status fdd_kv_commit(fdd_ctx* ctx, fdd_forkset* const* sets, int n_sets, int
 fdd_status fdd_average_rollouts(fdd_ctx* ctx, const float* traj, int n, int w, float* out,
                                 void* stream);
 
+/*
+ * fdd_unmask_static -- the unmasking step of fdd_unmask for callers that cannot allocate device
+ * memory.  (The paper has no counterpart; this is a deployment variant of fdd_unmask.)
+ *
+ * Who needs it: code that runs after the vehicle stack has finished initialising and is then
+ * forbidden to allocate (a real-time planning loop with a fixed memory budget, a plugin that is
+ * handed pre-allocated buffers only, a process whose allocator is locked after start-up).
+ * cudaMalloc may block on the whole device, take unbounded time or fail late, so fdd_create and
+ * fdd_fork (which allocate scratch and seed storage) are not available to such callers.  This
+ * call needs neither a context nor a fork set and performs no allocation of any kind: its scratch
+ * is a fixed array inside the library image (FDD_UNMASK_STATIC_MAX_RECORDS records of 32 bytes =
+ * 2 MiB, resident on every GPU that loads the library until the process exits).
+ *
+ * It computes exactly what fdd_unmask computes for one set (same kernels, same rule, same noise).
+ *   logits        device [n_forks][block_len][vocab], fp32 or bf16 per logits_dtype
+ *   tokens, state device, in/out, [n_forks][block_len]
+ *   seeds         device uint64 [n_forks] (the caller keeps them on the device)
+ *   n_committed, n_left  device int32 [n_forks] (written);  conf: device fp32 [n_forks][block_len] or NULL
+ *   err, err_len  optional host buffer that receives the error text (may be NULL / 0)
+ * Limits: block_len <= 128 and n_forks * block_len * ceil(vocab / 8192) <= FDD_UNMASK_STATIC_MAX_RECORDS;
+ * anything larger is rejected with FDD_ERR_CAPACITY before any launch (e.g. vocab 151936 has 19
+ * chunks, so up to 3449 rows: 32 rollouts x 64 positions fit).
+ * Set-up: the first call on each device (with that device current) asks the runtime for the
+ * device address of the array (cudaGetSymbolAddress) and caches it; make that first call before
+ * any stream capture begins.  Later calls do no set-up.
+ * Sharing: all calls on a device use the same array, which keeps whatever the previous call
+ * left in it.  Nothing in it has to start at zero: every record that is read was written earlier
+ * in the same call.  Two calls whose kernels can overlap on the GPU (different streams without
+ * ordering) race on it; order them.  The host side is not thread-safe for the first call per device.
+ */
+#define FDD_UNMASK_STATIC_MAX_RECORDS 65536
+fdd_status fdd_unmask_static(const void* logits, int logits_dtype, int n_forks, int block_len,
+                             int vocab, int32_t* tokens, uint8_t* state, const uint64_t* seeds,
+                             float threshold, float temperature, uint32_t block_idx, uint32_t step,
+                             int32_t* n_committed, int32_t* n_left, float* conf, void* stream,
+                             char* err, size_t err_len);
+
 /* Synchronise `stream` and return the device status word: FDD_OK, or the first error a
  * kernel recorded (FDD_ERR_DEVICE_TIMEOUT).  Reading clears it. */
 fdd_status fdd_poll_status(fdd_ctx* ctx, void* stream);

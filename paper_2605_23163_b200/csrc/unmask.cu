@@ -276,3 +276,103 @@ cudaError_t launch_unmask(fdd_ctx* ctx, const UnmaskProblem& p, cudaStream_t st,
     *n_launches += 2;
     return cudaGetLastError();
 }
+
+// -------------------------------------------------------------------------------------------------
+// fdd_unmask_static: the same unmasking step for callers that must not allocate.
+//
+// Its scratch (the per (row, chunk) records) lives in a fixed device array that is part of the
+// loaded library image, so the call needs no context, no fork set and no allocation of any kind.
+// -------------------------------------------------------------------------------------------------
+namespace {
+
+constexpr int kStaticMaxRecords = FDD_UNMASK_STATIC_MAX_RECORDS;
+constexpr int kStaticMaxDevices = 64;
+
+// Held by every GPU that loads the library until the process exits (2 MiB).
+static __device__ __align__(256) UnmaskPartial g_static_partials[kStaticMaxRecords];
+
+// Device address of g_static_partials per device ordinal, resolved on first use.  In host code the
+// array's name is only a handle for the runtime; the address a kernel can use must be asked for.
+UnmaskPartial* g_static_ptr[kStaticMaxDevices];
+bool g_static_ready[kStaticMaxDevices];
+
+void put_error(char* err, size_t err_len, const char* text) {
+    if (err && err_len) snprintf(err, err_len, "%s", text);
+}
+
+}  // namespace
+
+extern "C" fdd_status fdd_unmask_static(const void* logits, int logits_dtype, int n_forks, int block_len,
+                                        int vocab, int32_t* tokens, uint8_t* state, const uint64_t* seeds,
+                                        float threshold, float temperature, uint32_t block_idx,
+                                        uint32_t step, int32_t* n_committed, int32_t* n_left, float* conf,
+                                        void* stream, char* err, size_t err_len) {
+    if (!logits || !tokens || !state || !seeds || !n_committed || !n_left) {
+        put_error(err, err_len, "fdd_unmask_static: a required pointer is NULL");
+        return FDD_ERR_INVALID_ARG;
+    }
+    if (logits_dtype != FDD_LOGITS_F32 && logits_dtype != FDD_LOGITS_BF16) {
+        put_error(err, err_len, "fdd_unmask_static: logits_dtype must be FDD_LOGITS_F32 or FDD_LOGITS_BF16");
+        return FDD_ERR_INVALID_ARG;
+    }
+    if (n_forks < 1 || block_len < 1 || vocab < 1 || !(temperature >= 0.0f) || threshold != threshold) {
+        put_error(err, err_len, "fdd_unmask_static: sizes must be >= 1, temperature >= 0, threshold not NaN");
+        return FDD_ERR_INVALID_ARG;
+    }
+    if (block_len > 128) {
+        put_error(err, err_len, "fdd_unmask_static: block_len above 128 is not supported");
+        return FDD_ERR_UNSUPPORTED;
+    }
+    const long long records = static_cast<long long>(n_forks) * block_len * unmask_chunks(vocab);
+    if (records > kStaticMaxRecords) {
+        if (err && err_len)
+            snprintf(err, err_len,
+                     "fdd_unmask_static: n_forks * block_len * ceil(vocab / %d) = %lld exceeds the fixed scratch of %d records",
+                     kUnmaskChunk, records, kStaticMaxRecords);
+        return FDD_ERR_CAPACITY;
+    }
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess || dev < 0 || dev >= kStaticMaxDevices) {
+        put_error(err, err_len, "fdd_unmask_static: no usable current CUDA device");
+        return FDD_ERR_CUDA;
+    }
+    if (!g_static_ready[dev]) {
+        // once per device, with that device current: resolve the array's device address
+        void* p = nullptr;
+        e = cudaGetSymbolAddress(&p, g_static_partials);
+        if (e != cudaSuccess || !p) {
+            if (err && err_len) snprintf(err, err_len, "fdd_unmask_static: cudaGetSymbolAddress failed: %s", cudaGetErrorString(e));
+            return FDD_ERR_CUDA;
+        }
+        g_static_ptr[dev] = static_cast<UnmaskPartial*>(p);
+        g_static_ready[dev] = true;
+    }
+    UnmaskPartial* partial = g_static_ptr[dev];
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const int rows = n_forks * block_len;
+    const int n_chunks = unmask_chunks(vocab);
+    const dim3 grid(static_cast<unsigned>(n_chunks) * static_cast<unsigned>(rows));
+    if (logits_dtype == FDD_LOGITS_BF16) {
+        const int vec_ok = (vocab % 8 == 0) && (reinterpret_cast<uintptr_t>(logits) % 16 == 0);
+        unmask_partial_kernel<__nv_bfloat16><<<grid, kThreads, 0, st>>>(
+            static_cast<const __nv_bfloat16*>(logits), state, seeds, partial, block_len, vocab, n_chunks,
+            temperature, block_idx, step, vec_ok);
+    } else {
+        const int vec_ok = (vocab % 4 == 0) && (reinterpret_cast<uintptr_t>(logits) % 16 == 0);
+        unmask_partial_kernel<float><<<grid, kThreads, 0, st>>>(
+            static_cast<const float*>(logits), state, seeds, partial, block_len, vocab, n_chunks,
+            temperature, block_idx, step, vec_ok);
+    }
+    e = cudaGetLastError();
+    if (e == cudaSuccess) {
+        unmask_finalize_kernel<<<n_forks, 128, 0, st>>>(partial, tokens, state, n_committed, n_left, conf,
+                                                       block_len, n_chunks, threshold);
+        e = cudaGetLastError();
+    }
+    if (e != cudaSuccess) {
+        if (err && err_len) snprintf(err, err_len, "fdd_unmask_static: launch failed: %s", cudaGetErrorString(e));
+        return FDD_ERR_CUDA;
+    }
+    return FDD_OK;
+}

@@ -21,8 +21,9 @@ FDD_LOGITS_F32, FDD_LOGITS_BF16 = 0, 1
 EXPORTS = (
     "fdd_create", "fdd_destroy", "fdd_last_error", "fdd_launch_count", "fdd_fork",
     "fdd_forkset_free", "fdd_forkset_suffix_len", "fdd_forkset_reset", "fdd_block_attn",
-    "fdd_unmask", "fdd_kv_commit", "fdd_average_rollouts", "fdd_poll_status",
+    "fdd_unmask", "fdd_kv_commit", "fdd_average_rollouts", "fdd_poll_status", "fdd_unmask_static",
 )
+FDD_UNMASK_STATIC_MAX_RECORDS = 65536
 
 
 class FddError(RuntimeError):
@@ -79,6 +80,9 @@ def lib():
     L.fdd_average_rollouts.restype = i32
     L.fdd_poll_status.argtypes = [vp, vp]
     L.fdd_poll_status.restype = i32
+    L.fdd_unmask_static.argtypes = [vp, i32, i32, i32, i32, vp, vp, vp, f32, f32, u32, u32, vp, vp, vp, vp,
+                                    ctypes.c_char_p, ctypes.c_size_t]
+    L.fdd_unmask_static.restype = i32
     _lib_handle = L
     return L
 
@@ -200,3 +204,17 @@ def fdd_average_rollouts(ctx, traj, n, w, out, stream=None):
 
 def fdd_poll_status(ctx, stream=None):
     return _check(ctx, lib().fdd_poll_status(ctx, _stream(stream)))
+
+
+def fdd_unmask_static(logits, logits_dtype, n_forks, block_len, vocab, tokens, state, seeds, threshold,
+                      temperature, block_idx, step, n_committed, n_left, conf=None, stream=None):
+    """The allocation-free unmasking step: no context, no fork set; `seeds` is a device uint64/int64
+    tensor [n_forks].  Raises FddError with the library's message on a negative status."""
+    buf = ctypes.create_string_buffer(256)
+    st = lib().fdd_unmask_static(_ptr(logits), int(logits_dtype), int(n_forks), int(block_len), int(vocab),
+                                 _ptr(tokens), _ptr(state), _ptr(seeds), float(threshold), float(temperature),
+                                 int(block_idx), int(step), _ptr(n_committed), _ptr(n_left), _ptr(conf),
+                                 _stream(stream), buf, len(buf))
+    if st < 0:
+        raise FddError(st, buf.value.decode())
+    return st
