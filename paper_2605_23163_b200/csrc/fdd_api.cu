@@ -8,6 +8,9 @@
 #include <new>
 
 cudaError_t launch_attention_simple(const AttnProblem& p, int head_dim, cudaStream_t st);
+cudaError_t launch_attention_tc(fdd_ctx* ctx, const AttnProblem& a, int head_dim, cudaStream_t st, int* n_launches);
+bool attention_tc_supported(const AttnProblem& a, int head_dim);
+size_t attention_tc_workspace_bytes(int head_dim, int sm_count);
 
 namespace {
 
@@ -78,6 +81,10 @@ fdd_status fdd_create(const fdd_config* cfg, fdd_ctx** out) {
     if (e == cudaSuccess) {
         ctx->ws_unmask_bytes = static_cast<size_t>(cfg->max_forks) * cfg->max_block * unmask_chunks(cfg->vocab) * sizeof(UnmaskPartial);
         e = cudaMalloc(&ctx->ws_unmask, ctx->ws_unmask_bytes);
+    }
+    if (e == cudaSuccess) {
+        ctx->ws_attn_bytes = attention_tc_workspace_bytes(cfg->head_dim, ctx->sm_count);
+        e = cudaMalloc(&ctx->ws_attn, ctx->ws_attn_bytes);
     }
     if (e != cudaSuccess) {
         fdd_destroy(ctx);
@@ -327,7 +334,8 @@ fdd_status fdd_poll_status(fdd_ctx* ctx, void* stream) {
 }  // extern "C"
 
 cudaError_t launch_attention(fdd_ctx* ctx, const AttnProblem& p, int head_dim, cudaStream_t st, int* n_launches) {
-    (void)ctx;
+    // The tensor-core kernel covers power-of-two GQA groups; the CUDA-core kernel the rest.
+    if (attention_tc_supported(p, head_dim)) return launch_attention_tc(ctx, p, head_dim, st, n_launches);
     *n_launches += 1;
     return launch_attention_simple(p, head_dim, st);
 }
