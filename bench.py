@@ -26,7 +26,7 @@ if ROOT not in sys.path:
 
 METRIC = "committed tokens/s per denoise step (N forks, shared prefix)"
 UNIT = "tokens/s"
-PRE_STEPS = 6      # distinct per-step input sets kept resident; later steps cycle through them
+PRE_STEPS = 6      # distinct per-step input sets kept resident; later steps cycle through them (--pre-steps)
 
 
 def _peaks():
@@ -67,7 +67,7 @@ class ClockSampler(threading.Thread):
                 for bit, name in names.items():
                     if mask & bit:
                         self.reasons.add(name)
-                time.sleep(0.05)
+                time.sleep(0.004)
         except Exception as exc:      # NVML unavailable: report that instead of clocks
             self.reasons.add(f"nvml_unavailable:{type(exc).__name__}")
 
@@ -376,6 +376,7 @@ def run_reference(args):
 
 
 def main():
+    global PRE_STEPS
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=10)
@@ -384,10 +385,13 @@ def main():
     ap.add_argument("--workload", default="long_prefix")
     ap.add_argument("--layers", type=int, default=1)
     ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--pre-steps", type=int, default=PRE_STEPS,
+                    help="distinct per-step input sets kept resident on the device")
     ap.add_argument("--cpu-budget", type=float, default=20.0)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
+    PRE_STEPS = max(1, args.pre_steps)
     if args.impl == "reference":
         run_reference(args)
     else:
