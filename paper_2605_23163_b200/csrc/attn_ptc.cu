@@ -1,0 +1,798 @@
+// Block-causal decode attention on the 5th-generation tensor cores (tcgen05 + TMEM + TMA),
+// persistent version: one CTA per SM, balanced ranges of key-tile steps, many scenes per launch.
+//
+// Work unit: one (scene, KV head, pair of 128-row query tiles, rollout).  Query row r = i * G + g
+// stacks block position i and the g-th query head of the GQA group, so 2 x 128 rows share every
+// staged K/V tile.  Keys come in tiles of 128 from three segments: the shared prefix (contiguous
+// or paged), the rollout's private suffix, the block itself.  A unit therefore is a run of
+// "tile steps"; all units of all scenes of a call, laid end to end, form one global sequence of
+// tile steps that is cut into equal contiguous ranges, one per CTA.  A CTA walks its range item
+// by item (item = the part of one unit inside the range).  A unit that lies inside one range is
+// written directly; a unit cut by a range border leaves normalised fp32 partials plus their
+// log-sum-exp in scratch, and whichever CTA finishes its piece last (an atomic counter per unit,
+// nobody waits) merges the pieces and writes the bf16 rows.
+//
+// Warp roles (384 threads): warps 0-3 and 4-7 are the two soft-max groups (thread = one query
+// row = one TMEM lane), warp 8 lane 0 drives TMA, warp 9 lane 0 issues every tcgen05.mma, warps
+// 10-11 only donate their registers.
+// TMEM (512 columns): S0 | S1 | O0 | O1; the bf16 probabilities P overwrite the first half of
+// their S tile and feed the PV product straight from TMEM.  Per key tile and query tile:
+//   S = Q K^T (smem x smem)  ->  soft-max warps: running max (rescaling O only when the max moved
+//   by more than 2^8), P = exp2(S * c - m) -> TMEM  ->  O += P V (TMEM x smem, V keys-major).
+// The two query tiles ping-pong, so one tile's soft-max overlaps the other tile's MMAs.  The
+// exponentials of a tile are split between the special-function unit (ex2.approx) and a cubic
+// polynomial on the FMA pipe, because one ex2 per score needs as many cycles as the MMAs.
+// Every mbarrier wait is bounded; on a timeout the CTA records FDD_ERR_DEVICE_TIMEOUT, drains
+// and returns (TMEM is always freed).
+#include "fdd_internal.h"
+#include "tc_ptx.cuh"
+#include "tmap.h"
+
+#include <math_constants.h>
+
+#include <cstdlib>
+
+namespace {
+
+constexpr int kTcThreads = 384;
+constexpr int kKeysPerTile = 128;
+constexpr long long kWaitLimit = 4000000000LL;   // about two seconds of SM clocks
+constexpr int kMinTilesPerCta = 4;               // do not cut the work finer than this
+// Registers per thread after the hand-over.  The CTA starts with 384 x 168; 8 soft-max warps x
+// kRegsSoftmax + 4 other warps x kRegsOther must not exceed that (2 * 208 + 88 = 3 * 168).
+constexpr int kRegsSoftmax = 208;
+constexpr int kRegsOther = 88;
+static_assert(2 * kRegsSoftmax + kRegsOther <= 3 * 168, "register hand-over exceeds the CTA's pool");
+
+struct SetParams {
+    __nv_bfloat16* out;
+    const int32_t* page_table;
+    long long step_base;       // first global tile step of this scene
+    int unit_base;             // first global unit id of this scene
+    int units;                 // Hkv * row_pairs * n_forks
+    int n_forks, d, n_q_heads, G, R;
+    int prefix_len, page_tokens, n_phys_pages, suffix_len;
+    int tiles_prefix, tiles_suffix, tiles_total;
+    int row_pairs;
+    int causal;
+};
+
+template <int MAXSETS>
+struct TcArgs {
+    TcSetMaps maps[MAXSETS];
+    SetParams sets[MAXSETS];
+    float* part_o;             // [2 * ctas][256][D] normalised partial outputs
+    float* part_lse;           // [2 * ctas][256] log2-domain log-sum-exp of the partial
+    int* unit_count;           // pieces finished per unit (self-resetting)
+    int* status;
+    long long total_steps;
+    int n_sets;
+    float scale_log2;
+};
+
+struct TileInfo {
+    int segment;   // 0 prefix, 1 suffix, 2 block
+    int index;     // tile index inside the segment
+    int nvalid;    // valid keys in the tile (1..128)
+};
+
+__device__ __forceinline__ TileInfo tile_info(const SetParams& p, int g) {
+    TileInfo t;
+    if (g < p.tiles_prefix) {
+        t.segment = 0; t.index = g;
+        t.nvalid = min(kKeysPerTile, p.prefix_len - g * kKeysPerTile);
+    } else if (g < p.tiles_prefix + p.tiles_suffix) {
+        t.segment = 1; t.index = g - p.tiles_prefix;
+        t.nvalid = min(kKeysPerTile, p.suffix_len - t.index * kKeysPerTile);
+    } else {
+        t.segment = 2; t.index = g - p.tiles_prefix - p.tiles_suffix;
+        t.nvalid = min(kKeysPerTile, p.d - t.index * kKeysPerTile);
+    }
+    return t;
+}
+
+template <int D>
+struct TcShape {
+    static constexpr int kTileBytes = 128 * D * 2;      // one 128-row operand tile
+    static constexpr int kChunks = D / 64;               // 64-element (128-byte) column chunks
+    static constexpr int kChunkBytes = 128 * 128;        // 128 rows x 128 bytes
+    static constexpr int kStages = D == 128 ? 2 : 4;     // K/V ring depth
+    // Q (two tiles) + K ring + V ring + alignment slack; always more than half an SM's shared
+    // memory, so two CTAs (each wanting all 512 TMEM columns) never share an SM.
+    static constexpr int kSmemBytes = 2 * kTileBytes + 2 * kStages * kTileBytes + 1024;
+};
+
+// Issue the TMA loads of one 128-key tile of K or V into `dst` (layout [chunk][128 rows][128 B]).
+template <int D>
+__device__ __forceinline__ void load_kv_tile(const SetParams& p, const CUtensorMap* seg_map, const CUtensorMap* tail_map,
+                                             const TileInfo& t, uint32_t dst, uint32_t bar, int h, int f) {
+    constexpr int kChunks = TcShape<D>::kChunks;
+#pragma unroll
+    for (int rh = 0; rh < 2; ++rh) {
+        const int row0 = t.index * kKeysPerTile + rh * 64;
+#pragma unroll
+        for (int ch = 0; ch < kChunks; ++ch) {
+            const uint32_t d_addr = dst + ch * TcShape<D>::kChunkBytes + rh * 8192;
+            if (t.segment == 0) {
+                if (p.page_tokens == 0) {
+                    tc::tma_load_3d(d_addr, seg_map, bar, ch * 64, row0, h);
+                } else {
+                    const int lp = row0 / 64;
+                    const int n_pages = (p.prefix_len + 63) / 64;
+                    if (lp < n_pages) {
+                        const int page = p.page_table[lp];
+                        const bool tail = (lp == n_pages - 1) && (p.prefix_len % 64 != 0);
+                        tc::tma_load_4d(d_addr, tail ? tail_map : seg_map, bar, ch * 64, 0, h, page);
+                    } else {
+                        tc::tma_load_4d(d_addr, seg_map, bar, ch * 64, 0, h, p.n_phys_pages);   // past the end: zeros
+                    }
+                }
+            } else if (t.segment == 1) {
+                tc::tma_load_4d(d_addr, seg_map, bar, ch * 64, row0, h, f);
+            } else {
+                tc::tma_load_4d(d_addr, seg_map, bar, ch * 64, h, row0, f);
+            }
+        }
+    }
+}
+
+// One item of a CTA's range: tiles [t0, t1) of unit `unit` of scene `s`.
+struct Item {
+    int s, unit, t0, t1;
+    long long unit_begin;      // global tile step of the unit's tile 0
+};
+
+template <int MAXSETS>
+__device__ __forceinline__ Item locate(const TcArgs<MAXSETS>& a, long long pos, long long end) {
+    Item it;
+    int s = 0;
+    while (s + 1 < a.n_sets && pos >= a.sets[s + 1].step_base) ++s;
+    const SetParams& p = a.sets[s];
+    const long long rel = pos - p.step_base;
+    it.s = s;
+    it.unit = static_cast<int>(rel / p.tiles_total);
+    it.t0 = static_cast<int>(rel - static_cast<long long>(it.unit) * p.tiles_total);
+    it.unit_begin = pos - it.t0;
+    const long long left = end - pos;
+    it.t1 = static_cast<int>(min(static_cast<long long>(p.tiles_total), it.t0 + left));
+    return it;
+}
+
+// Cubic 2^f on [-0.5, 0.5] (relative error 7.5e-5, far below the bf16 rounding of P), with the
+// factor 2^-112 of the range shift folded into the coefficients.
+constexpr float kExpShift = 112.0f;
+constexpr float kPolyScale = 1.92592994438723585e-34f;        // 2^-112
+constexpr float kPoly0 = 0.9999281167984009f * kPolyScale;
+constexpr float kPoly1 = 0.6932609677314758f * kPolyScale;
+constexpr float kPoly2 = 0.2426108568906784f * kPolyScale;
+constexpr float kPoly3 = 0.055171459913253784f * kPolyScale;
+constexpr float kRoundMagic = 12582912.0f;                    // 1.5 * 2^23: adding it rounds to an integer
+
+template <int D, int MAXSETS, int EMU>
+__global__ void __launch_bounds__(kTcThreads, 1)
+attn_ptc_kernel(const __grid_constant__ TcArgs<MAXSETS> a) {
+    using Shape = TcShape<D>;
+    constexpr int kStages = Shape::kStages;
+    static_assert(EMU % 8 == 0 && EMU >= 0 && EMU <= 128, "EMU: emulated exponentials per 128-key tile");
+    extern __shared__ __align__(1024) unsigned char smem_raw[];
+    unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    const uint32_t q_s = tc::smem_u32(smem);
+    const uint32_t k_s = q_s + 2 * Shape::kTileBytes;
+    const uint32_t v_s = k_s + kStages * Shape::kTileBytes;
+
+    __shared__ __align__(8) unsigned long long bar_q_full, bar_k_full[kStages], bar_k_empty[kStages],
+        bar_v_full[kStages], bar_v_empty[kStages], bar_s_full[2], bar_p_full[2], bar_o_done[2];
+    __shared__ uint32_t tmem_base_s;
+    __shared__ int abort_s, last_s;
+    volatile int* abort_flag = &abort_s;
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+
+    const long long T = a.total_steps;
+    const long long C = gridDim.x;
+    const long long range_begin = T * blockIdx.x / C;
+    const long long range_end = T * (blockIdx.x + 1) / C;
+
+    if (tid == 0) {
+        abort_s = 0;
+        last_s = 0;
+        tc::mbar_init(tc::smem_u32(&bar_q_full), 1);
+        for (int s = 0; s < kStages; ++s) {
+            tc::mbar_init(tc::smem_u32(&bar_k_full[s]), 1);
+            tc::mbar_init(tc::smem_u32(&bar_k_empty[s]), 1);
+            tc::mbar_init(tc::smem_u32(&bar_v_full[s]), 1);
+            tc::mbar_init(tc::smem_u32(&bar_v_empty[s]), 1);
+        }
+        for (int q = 0; q < 2; ++q) {
+            tc::mbar_init(tc::smem_u32(&bar_s_full[q]), 1);
+            tc::mbar_init(tc::smem_u32(&bar_p_full[q]), 128);
+            tc::mbar_init(tc::smem_u32(&bar_o_done[q]), 1);
+        }
+        tc::fence_barrier_init();
+    }
+    if (warp == 9) {
+        tc::tmem_alloc(tc::smem_u32(&tmem_base_s), 512);
+        tc::tmem_relinquish();
+    }
+    tc::fence_before_sync();
+    __syncthreads();
+    tc::fence_after_sync();
+    const uint32_t tmem = tmem_base_s;
+    const uint32_t tm_s[2] = {tmem, tmem + 128};
+    const uint32_t tm_o[2] = {tmem + 256, tmem + 256 + D};
+
+    // Each role runs its own copy of the item loop; all of them meet at the end of every item.
+    struct ItemView {
+        Item it;
+        int f, rp, h, nt, rows_here, NQ;
+    };
+    auto view_item = [&](long long pos) {
+        ItemView v;
+        v.it = locate(a, pos, range_end);
+        const SetParams& p = a.sets[v.it.s];
+        int idx = v.it.unit;
+        v.f = idx % p.n_forks; idx /= p.n_forks;
+        v.rp = idx % p.row_pairs; idx /= p.row_pairs;
+        v.h = idx;
+        v.nt = v.it.t1 - v.it.t0;
+        v.rows_here = min(256, p.R - v.rp * 256);
+        v.NQ = v.rows_here > 128 ? 2 : 1;
+        return v;
+    };
+    // End of an item: every MMA of the item has completed (the soft-max groups waited for the
+    // last PV), O has been read out, Q may be overwritten.  Returns false after an abort.
+    auto end_of_item = [&]() {
+        tc::fence_before_sync();
+        tc::named_barrier(2, kTcThreads);
+        tc::fence_after_sync();
+        return *abort_flag == 0;
+    };
+
+    if (warp >= 8) {
+        // The soft-max warps hold a 128-wide score row in registers; this warpgroup gives most of
+        // its registers up for them.
+        tc::reg_dealloc<kRegsOther>();
+        if (warp == 8) {
+            // ------------------------------------------------------------------ TMA producer
+            uint32_t kv_cnt = 0;            // K/V tiles staged so far: ring stage and phase carry over between items
+            for (long long pos = range_begin; pos < range_end;) {
+                const ItemView v = view_item(pos);
+                if (lane == 0) {
+                    const SetParams& p = a.sets[v.it.s];
+                    const TcSetMaps& maps = a.maps[v.it.s];
+                    tc::prefetch_tmap(&maps.q);
+                    const uint32_t bq = tc::smem_u32(&bar_q_full);
+                    tc::mbar_arrive_expect_tx(bq, v.NQ * Shape::kTileBytes);
+                    for (int q = 0; q < v.NQ; ++q)
+                        for (int ch = 0; ch < Shape::kChunks; ++ch)
+                            tc::tma_load_4d(q_s + q * Shape::kTileBytes + ch * Shape::kChunkBytes, &maps.q, bq, ch * 64,
+                                            v.h * p.G, (v.rp * 2 + q) * (128 / p.G), v.f);
+                    bool ok = true;
+                    for (int jl = 0; jl < v.nt && ok; ++jl) {
+                        const TileInfo t = tile_info(p, v.it.t0 + jl);
+                        const uint32_t n = kv_cnt + jl;
+                        const int s = n % kStages;
+                        const uint32_t ph = (n / kStages) & 1;
+                        const CUtensorMap* mk = t.segment == 0 ? &maps.pk : (t.segment == 1 ? &maps.sk : &maps.bk);
+                        const CUtensorMap* mv = t.segment == 0 ? &maps.pv : (t.segment == 1 ? &maps.sv : &maps.bv);
+                        ok = tc::mbar_wait(tc::smem_u32(&bar_k_empty[s]), ph ^ 1, abort_flag, kWaitLimit);
+                        if (!ok) break;
+                        tc::mbar_arrive_expect_tx(tc::smem_u32(&bar_k_full[s]), Shape::kTileBytes);
+                        load_kv_tile<D>(p, mk, &maps.pk_tail, t, k_s + s * Shape::kTileBytes, tc::smem_u32(&bar_k_full[s]), v.h, v.f);
+                        ok = tc::mbar_wait(tc::smem_u32(&bar_v_empty[s]), ph ^ 1, abort_flag, kWaitLimit);
+                        if (!ok) break;
+                        tc::mbar_arrive_expect_tx(tc::smem_u32(&bar_v_full[s]), Shape::kTileBytes);
+                        load_kv_tile<D>(p, mv, &maps.pv_tail, t, v_s + s * Shape::kTileBytes, tc::smem_u32(&bar_v_full[s]), v.h, v.f);
+                    }
+                    if (!ok) {
+                        if (*abort_flag == 0) atomicCAS(a.status, 0, FDD_ERR_DEVICE_TIMEOUT);
+                        *abort_flag = 1;
+                        const long long t0 = clock64();          // let copies already in flight land
+                        while (clock64() - t0 < 2000000) {}
+                    }
+                }
+                __syncwarp();
+                kv_cnt += v.nt;
+                pos += v.nt;
+                if (!end_of_item()) break;
+            }
+        } else if (warp == 9) {
+            // ------------------------------------------------------------------ MMA issuer
+            uint32_t kv_cnt = 0, item_cnt = 0;
+            uint32_t sp_cnt[2] = {0, 0};    // key tiles handled so far per query tile
+            for (long long pos = range_begin; pos < range_end;) {
+                const ItemView v = view_item(pos);
+                const int nt = v.nt, NQ = v.NQ;
+                if (lane == 0) {
+                    constexpr uint32_t kIdescQK = tc::idesc_bf16(128, 128, 0);
+                    constexpr uint32_t kIdescPV = tc::idesc_bf16(128, D, 1);
+                    auto issue_qk = [&](int q, int s) {
+#pragma unroll
+                        for (int k = 0; k < D / 16; ++k) {
+                            const uint32_t off = (k >> 2) * Shape::kChunkBytes + (k & 3) * 32;
+                            tc::mma_ss(tm_s[q], tc::smem_desc_sw128(q_s + q * Shape::kTileBytes + off, 0, 1024),
+                                       tc::smem_desc_sw128(k_s + s * Shape::kTileBytes + off, 0, 1024), kIdescQK, k > 0);
+                        }
+                    };
+                    auto issue_pv = [&](int q, int s, int accumulate) {
+#pragma unroll
+                        for (int j = 0; j < kKeysPerTile / 16; ++j)
+                            tc::mma_ts(tm_o[q], tm_s[q] + j * 8,
+                                       tc::smem_desc_sw128(v_s + s * Shape::kTileBytes + j * 2048, Shape::kChunkBytes, 1024),
+                                       kIdescPV, (accumulate || j > 0) ? 1u : 0u);
+                    };
+                    const int s0 = kv_cnt % kStages;
+                    bool ok = tc::mbar_wait(tc::smem_u32(&bar_q_full), item_cnt & 1, abort_flag, kWaitLimit);
+                    ok = ok && tc::mbar_wait(tc::smem_u32(&bar_k_full[s0]), (kv_cnt / kStages) & 1, abort_flag, kWaitLimit);
+                    if (ok) {
+                        tc::fence_after_sync();
+                        for (int q = 0; q < NQ; ++q) {
+                            issue_qk(q, s0);
+                            tc::mma_commit(tc::smem_u32(&bar_s_full[q]));
+                        }
+                        tc::mma_commit(tc::smem_u32(&bar_k_empty[s0]));
+                    }
+                    for (int jl = 0; jl < nt && ok; ++jl) {
+                        const uint32_t n = kv_cnt + jl;
+                        const int s = n % kStages;
+                        const uint32_t ph = (n / kStages) & 1;
+                        const int jn = jl + 1;
+                        const int sn = (n + 1) % kStages;
+                        const uint32_t phn = ((n + 1) / kStages) & 1;
+                        ok = tc::mbar_wait(tc::smem_u32(&bar_v_full[s]), ph, abort_flag, kWaitLimit);
+                        for (int q = 0; q < NQ && ok; ++q) {
+                            ok = tc::mbar_wait(tc::smem_u32(&bar_p_full[q]), (sp_cnt[q] + jl) & 1, abort_flag, kWaitLimit);
+                            if (!ok) break;
+                            tc::fence_after_sync();
+                            issue_pv(q, s, jl > 0);
+                            tc::mma_commit(tc::smem_u32(&bar_o_done[q]));
+                            if (jn < nt) {
+                                if (q == 0) {
+                                    ok = tc::mbar_wait(tc::smem_u32(&bar_k_full[sn]), phn, abort_flag, kWaitLimit);
+                                    if (!ok) break;
+                                    tc::fence_after_sync();
+                                }
+                                issue_qk(q, sn);
+                                tc::mma_commit(tc::smem_u32(&bar_s_full[q]));
+                            }
+                        }
+                        if (!ok) break;
+                        tc::mma_commit(tc::smem_u32(&bar_v_empty[s]));
+                        if (jn < nt) tc::mma_commit(tc::smem_u32(&bar_k_empty[sn]));
+                    }
+                    if (!ok) {
+                        if (*abort_flag == 0) atomicCAS(a.status, 0, FDD_ERR_DEVICE_TIMEOUT);
+                        *abort_flag = 1;
+                    }
+                }
+                __syncwarp();
+                kv_cnt += nt;
+                for (int q = 0; q < NQ; ++q) sp_cnt[q] += nt;
+                ++item_cnt;
+                pos += nt;
+                if (!end_of_item()) break;
+            }
+        } else {
+            // idle warps of the donor warpgroup: only keep the item barriers company
+            for (long long pos = range_begin; pos < range_end;) {
+                const ItemView v = view_item(pos);
+                pos += v.nt;
+                if (!end_of_item()) break;
+            }
+        }
+    } else {
+        tc::reg_alloc<kRegsSoftmax>();
+        // ---------------------------------------------------------------------- soft-max groups
+        const int q = warp >> 2;
+        const int row_local = tid & 127;
+        const uint32_t lane_base = (static_cast<uint32_t>(warp & 3) * 32u) << 16;
+        const uint32_t bs = tc::smem_u32(&bar_s_full[q]), bp = tc::smem_u32(&bar_p_full[q]), bo = tc::smem_u32(&bar_o_done[q]);
+        uint32_t sp0 = 0;                   // key tiles this group has handled so far
+        for (long long pos = range_begin; pos < range_end;) {
+            const ItemView v = view_item(pos);
+            const Item& it = v.it;
+            const SetParams& p = a.sets[it.s];
+            const int f = v.f, rp = v.rp, h = v.h, nt = v.nt, rows_here = v.rows_here;
+            const bool active = q < v.NQ;
+            const int r = rp * 256 + q * 128 + row_local;       // row inside the unit
+            const bool row_ok = r < p.R;
+            const int qi = row_ok ? r / p.G : 0;
+            const int qg = row_ok ? r - qi * p.G : 0;
+            float m_used = -CUDART_INF_F, l = 0.0f;
+            bool ok = true;
+            if (active) {
+                const float c = a.scale_log2;
+                const uint64_t c2 = tc::pack2(c, c);
+                const float c_emu = c * (1.0f / 128.0f);
+                for (int jl = 0; jl < nt; ++jl) {
+                    const TileInfo t = tile_info(p, it.t0 + jl);
+                    ok = tc::mbar_wait(bs, (sp0 + jl) & 1, abort_flag, kWaitLimit);
+                    if (!ok) break;
+                    tc::fence_after_sync();
+                    uint32_t sr[128];
+#pragma unroll
+                    for (int cc = 0; cc < 4; ++cc) tc::tmem_ld32(tm_s[q] + lane_base + cc * 32, sr + cc * 32);
+                    tc::wait_ld();
+                    int limit = t.nvalid;                               // keys [0, limit) are visible
+                    if (p.causal && t.segment == 2) limit = min(limit, qi - t.index * kKeysPerTile + 1);
+                    if (limit < kKeysPerTile) {
+#pragma unroll
+                        for (int i = 0; i < 128; ++i)
+                            if (i >= limit) sr[i] = 0xFF800000u;        // -inf
+                    }
+                    float mx[4] = {-CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F};
+#pragma unroll
+                    for (int i = 0; i < 128; i += 8) {
+#pragma unroll
+                        for (int u = 0; u < 4; ++u)
+                            mx[u] = tc::max3(mx[u], __uint_as_float(sr[i + 2 * u]), __uint_as_float(sr[i + 2 * u + 1]));
+                    }
+                    const float tmax = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
+                    float m_tile = tmax * c;
+                    if (!(m_tile > -CUDART_INF_F)) m_tile = m_used > -CUDART_INF_F ? m_used : 0.0f;
+                    if (jl == 0) {
+                        m_used = m_tile;
+                    } else {
+                        const bool need = m_tile > m_used + 8.0f;
+                        if (__any_sync(0xFFFFFFFFu, need)) {
+                            ok = tc::mbar_wait(bo, (sp0 + jl - 1) & 1, abort_flag, kWaitLimit);
+                            if (!ok) break;
+                            tc::fence_after_sync();
+                            const float alpha = need ? exp2f(m_used - m_tile) : 1.0f;
+#pragma unroll
+                            for (int cc = 0; cc < D / 32; ++cc) {
+                                uint32_t o[32];
+                                tc::tmem_ld32(tm_o[q] + lane_base + cc * 32, o);
+                                tc::wait_ld();
+#pragma unroll
+                                for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
+                                tc::tmem_st32(tm_o[q] + lane_base + cc * 32, o);
+                            }
+                            tc::wait_st();
+                            l *= alpha;
+                            if (need) m_used = m_tile;
+                        }
+                    }
+                    // P = 2^(S * c - m): the first 128 - EMU scores through ex2.approx, the rest
+                    // through the polynomial; row sums in four packed accumulators.
+                    uint64_t acc[4] = {0ull, 0ull, 0ull, 0ull};
+                    uint32_t packed[64];
+                    const uint64_t nm2 = tc::pack2(-m_used, -m_used);
+#pragma unroll
+                    for (int i = 0; i < (128 - EMU) / 2; ++i) {
+                        const uint64_t x2 = tc::fma2(tc::pack2(__uint_as_float(sr[2 * i]), __uint_as_float(sr[2 * i + 1])), c2, nm2);
+                        float x0, x1;
+                        tc::unpack2(x2, x0, x1);
+                        const float e0 = tc::ex2(x0), e1 = tc::ex2(x1);
+                        acc[i & 3] = tc::add2(acc[i & 3], tc::pack2(e0, e1));
+                        const __nv_bfloat162 pk = __floats2bfloat162_rn(e0, e1);
+                        packed[i] = *reinterpret_cast<const uint32_t*>(&pk);
+                    }
+                    if (EMU > 0) {
+                        // y = (S * c - m + 112) / 128 clamped to [0, 1]; 2^(128 y - 112) = 2^n * 2^f with
+                        // n = round(128 y), f = 128 y - n; 2^n enters through the exponent bits.
+                        const float k_emu = (kExpShift - m_used) * (1.0f / 128.0f);
+                        const uint64_t magic2 = tc::pack2(kRoundMagic, kRoundMagic);
+                        const uint64_t m1_2 = tc::pack2(-1.0f, -1.0f);
+                        const uint64_t s128_2 = tc::pack2(128.0f, 128.0f);
+                        const uint64_t p0_2 = tc::pack2(kPoly0, kPoly0), p1_2 = tc::pack2(kPoly1, kPoly1);
+                        const uint64_t p2_2 = tc::pack2(kPoly2, kPoly2), p3_2 = tc::pack2(kPoly3, kPoly3);
+#pragma unroll
+                        for (int i = (128 - EMU) / 2; i < 64; ++i) {
+                            const float y0 = tc::fma_sat(__uint_as_float(sr[2 * i]), c_emu, k_emu);
+                            const float y1 = tc::fma_sat(__uint_as_float(sr[2 * i + 1]), c_emu, k_emu);
+                            const uint64_t y2 = tc::pack2(y0, y1);
+                            const uint64_t t2 = tc::fma2(y2, s128_2, magic2);     // 128 y rounded to an integer (+ magic)
+                            const uint64_t nn2 = tc::fma2(t2, m1_2, magic2);      // -n
+                            const uint64_t f2 = tc::fma2(y2, s128_2, nn2);        // f in [-0.5, 0.5]
+                            uint64_t pl = tc::fma2(f2, p3_2, p2_2);
+                            pl = tc::fma2(pl, f2, p1_2);
+                            pl = tc::fma2(pl, f2, p0_2);
+                            float pa, pb, ta, tb;
+                            tc::unpack2(pl, pa, pb);
+                            tc::unpack2(t2, ta, tb);
+                            const float e0 = __uint_as_float(__float_as_uint(pa) + (__float_as_uint(ta) << 23));
+                            const float e1 = __uint_as_float(__float_as_uint(pb) + (__float_as_uint(tb) << 23));
+                            acc[i & 3] = tc::add2(acc[i & 3], tc::pack2(e0, e1));
+                            const __nv_bfloat162 pk = __floats2bfloat162_rn(e0, e1);
+                            packed[i] = *reinterpret_cast<const uint32_t*>(&pk);
+                        }
+                    }
+                    {
+                        const uint64_t s01 = tc::add2(tc::add2(acc[0], acc[1]), tc::add2(acc[2], acc[3]));
+                        float sa, sb;
+                        tc::unpack2(s01, sa, sb);
+                        l += sa + sb;
+                    }
+                    tc::tmem_st32(tm_s[q] + lane_base, packed);
+                    tc::tmem_st32(tm_s[q] + lane_base + 32, packed + 32);
+                    tc::wait_st();
+                    tc::fence_before_sync();
+                    tc::mbar_arrive(bp);
+                }
+                if (ok) ok = tc::mbar_wait(bo, (sp0 + nt - 1) & 1, abort_flag, kWaitLimit);
+                if (ok) tc::fence_after_sync();
+            }
+
+            // ---------------------------------------------------------------- epilogue
+            const long long unit_end = it.unit_begin + p.tiles_total;
+            const int c_first = static_cast<int>(((it.unit_begin + 1) * C + T - 1) / T) - 1;   // CTA of the unit's first step
+            const int c_last = static_cast<int>((unit_end * C + T - 1) / T) - 1;                // CTA of its last step
+            const int n_pieces = c_last - c_first + 1;
+            const float inv = l > 0.0f ? 1.0f / l : 0.0f;
+            if (n_pieces == 1) {
+                if (active && ok) {
+                    __nv_bfloat16* op = p.out + ((static_cast<size_t>(f) * p.d + qi) * p.n_q_heads + h * p.G + qg) * D;
+#pragma unroll
+                    for (int cc = 0; cc < D / 32; ++cc) {
+                        uint32_t o[32];
+                        tc::tmem_ld32(tm_o[q] + lane_base + cc * 32, o);
+                        tc::wait_ld();
+                        if (row_ok) {
+#pragma unroll
+                            for (int v4 = 0; v4 < 4; ++v4) {
+                                uint32_t w[4];
+#pragma unroll
+                                for (int x = 0; x < 4; ++x) {
+                                    const __nv_bfloat162 pk = __floats2bfloat162_rn(__uint_as_float(o[v4 * 8 + 2 * x]) * inv,
+                                                                                      __uint_as_float(o[v4 * 8 + 2 * x + 1]) * inv);
+                                    w[x] = *reinterpret_cast<const uint32_t*>(&pk);
+                                }
+                                *reinterpret_cast<uint4*>(op + cc * 32 + v4 * 8) = make_uint4(w[0], w[1], w[2], w[3]);
+                            }
+                        }
+                    }
+                }
+            } else {
+                // A piece that starts at the CTA's range start uses the CTA's slot 0, a later one
+                // (necessarily the CTA's last item) slot 1.
+                const int own_slot = blockIdx.x * 2 + (pos == range_begin ? 0 : 1);
+                if (active && ok) {
+                    float* po = a.part_o + (static_cast<size_t>(own_slot) * 256 + q * 128 + row_local) * D;
+#pragma unroll
+                    for (int cc = 0; cc < D / 32; ++cc) {
+                        uint32_t o[32];
+                        tc::tmem_ld32(tm_o[q] + lane_base + cc * 32, o);
+                        tc::wait_ld();
+#pragma unroll
+                        for (int v4 = 0; v4 < 8; ++v4)
+                            __stcg(reinterpret_cast<float4*>(po + cc * 32 + v4 * 4),
+                                   make_float4(__uint_as_float(o[v4 * 4]) * inv, __uint_as_float(o[v4 * 4 + 1]) * inv,
+                                               __uint_as_float(o[v4 * 4 + 2]) * inv, __uint_as_float(o[v4 * 4 + 3]) * inv));
+                    }
+                    __stcg(a.part_lse + static_cast<size_t>(own_slot) * 256 + q * 128 + row_local, m_used + log2f(l));
+                }
+                __threadfence();
+                tc::named_barrier(1, 256);
+                if (tid == 0) {
+                    const int gu = p.unit_base + it.unit;
+                    const int old = atomicAdd(a.unit_count + gu, 1);
+                    const int last = old == n_pieces - 1;
+                    if (last) a.unit_count[gu] = 0;          // every piece has arrived: ready for the next launch
+                    last_s = last;
+                }
+                tc::named_barrier(1, 256);
+                if (last_s) {
+                    // This CTA finished the unit's last outstanding piece: merge all of them.
+                    //   out = sum_s w_s O_s / sum_s w_s,  w_s = 2^(lse_s - max lse)
+                    __threadfence();
+                    constexpr int kLanes = D / 4;       // lanes that carry a float4 of the row
+                    for (int row = warp; row < rows_here; row += 8) {
+                        const int rr = rp * 256 + row;
+                        float M = -CUDART_INF_F;
+                        for (int pc = c_first; pc <= c_last; ++pc) {
+                            const int slot = pc * 2 + (it.unit_begin <= T * pc / C ? 0 : 1);
+                            M = fmaxf(M, __ldcg(a.part_lse + static_cast<size_t>(slot) * 256 + row));
+                        }
+                        float4 accv = make_float4(0.f, 0.f, 0.f, 0.f);
+                        float wsum = 0.0f;
+                        for (int pc = c_first; pc <= c_last; ++pc) {
+                            const int slot = pc * 2 + (it.unit_begin <= T * pc / C ? 0 : 1);
+                            const float w = exp2f(__ldcg(a.part_lse + static_cast<size_t>(slot) * 256 + row) - M);
+                            wsum += w;
+                            if (lane < kLanes) {
+                                const float4 o = __ldcg(reinterpret_cast<const float4*>(
+                                    a.part_o + (static_cast<size_t>(slot) * 256 + row) * D + lane * 4));
+                                accv.x = fmaf(w, o.x, accv.x); accv.y = fmaf(w, o.y, accv.y);
+                                accv.z = fmaf(w, o.z, accv.z); accv.w = fmaf(w, o.w, accv.w);
+                            }
+                        }
+                        if (lane < kLanes) {
+                            const float iw = 1.0f / wsum;
+                            const int i2 = rr / p.G, g2 = rr - i2 * p.G;
+                            __nv_bfloat16* op = p.out + ((static_cast<size_t>(f) * p.d + i2) * p.n_q_heads + h * p.G + g2) * D + lane * 4;
+                            const __nv_bfloat162 lo = __floats2bfloat162_rn(accv.x * iw, accv.y * iw);
+                            const __nv_bfloat162 hi = __floats2bfloat162_rn(accv.z * iw, accv.w * iw);
+                            *reinterpret_cast<uint2*>(op) = make_uint2(*reinterpret_cast<const uint32_t*>(&lo),
+                                                                       *reinterpret_cast<const uint32_t*>(&hi));
+                        }
+                    }
+                }
+            }
+            if (!ok) {
+                if (*abort_flag == 0) atomicCAS(a.status, 0, FDD_ERR_DEVICE_TIMEOUT);
+                *abort_flag = 1;
+            }
+            if (active) sp0 += nt;
+            pos += nt;
+            if (!end_of_item()) break;
+        }
+    }
+
+    tc::fence_before_sync();
+    __syncthreads();
+    if (warp == 9) tc::tmem_dealloc(tmem, 512);
+}
+
+bool make_call_maps(const AttnProblem& a, int D, TcSetMaps* m) {
+    const uint64_t eb = 2;
+    const int G = a.n_q_heads / a.n_kv_heads;
+    {
+        uint64_t dims[4] = {(uint64_t)D, (uint64_t)a.n_q_heads, (uint64_t)a.d, (uint64_t)a.n_forks};
+        uint64_t str[3] = {D * eb, a.n_q_heads * D * eb, (uint64_t)a.d * a.n_q_heads * D * eb};
+        uint32_t box[4] = {64, (uint32_t)G, (uint32_t)(128 / G), 1};
+        if (!tmap::encode_bf16(&m->q, a.q, 4, dims, str, box)) return false;
+    }
+    {
+        uint64_t dims[4] = {(uint64_t)D, (uint64_t)a.n_kv_heads, (uint64_t)a.d, (uint64_t)a.n_forks};
+        uint64_t str[3] = {D * eb, a.n_kv_heads * D * eb, (uint64_t)a.d * a.n_kv_heads * D * eb};
+        uint32_t box[4] = {64, 1, 64, 1};
+        if (!tmap::encode_bf16(&m->bk, a.k_blk, 4, dims, str, box)) return false;
+        if (!tmap::encode_bf16(&m->bv, a.v_blk, 4, dims, str, box)) return false;
+    }
+    return true;
+}
+
+bool make_cache_maps(const AttnProblem& a, int D, TcSetMaps* m) {
+    const uint64_t eb = 2;
+    if (a.suffix_len > 0) {
+        uint64_t dims[4] = {(uint64_t)D, (uint64_t)a.suffix_len, (uint64_t)a.n_kv_heads, (uint64_t)a.n_forks};
+        uint64_t str[3] = {D * eb, (uint64_t)a.suffix_capacity * D * eb, (uint64_t)a.n_kv_heads * a.suffix_capacity * D * eb};
+        uint32_t box[4] = {64, 64, 1, 1};
+        if (!tmap::encode_bf16(&m->sk, a.suffix_k, 4, dims, str, box)) return false;
+        if (!tmap::encode_bf16(&m->sv, a.suffix_v, 4, dims, str, box)) return false;
+    } else {
+        m->sk = m->bk; m->sv = m->bv;    // never used (no suffix tiles)
+    }
+    m->pk_tail = m->bk; m->pv_tail = m->bv;
+    if (a.prefix_len > 0) {
+        if (a.page_tokens == 0) {
+            uint64_t dims[3] = {(uint64_t)D, (uint64_t)a.prefix_len, (uint64_t)a.n_kv_heads};
+            uint64_t str[2] = {D * eb, (uint64_t)a.prefix_capacity * D * eb};
+            uint32_t box[3] = {64, 64, 1};
+            if (!tmap::encode_bf16(&m->pk, a.prefix_k, 3, dims, str, box)) return false;
+            if (!tmap::encode_bf16(&m->pv, a.prefix_v, 3, dims, str, box)) return false;
+        } else {
+            uint64_t dims[4] = {(uint64_t)D, (uint64_t)a.page_tokens, (uint64_t)a.n_kv_heads, (uint64_t)a.prefix_capacity};
+            uint64_t str[3] = {D * eb, (uint64_t)a.page_tokens * D * eb, (uint64_t)a.n_kv_heads * a.page_tokens * D * eb};
+            uint32_t box[4] = {64, 64, 1, 1};
+            if (!tmap::encode_bf16(&m->pk, a.prefix_k, 4, dims, str, box)) return false;
+            if (!tmap::encode_bf16(&m->pv, a.prefix_v, 4, dims, str, box)) return false;
+            const int tail = a.prefix_len % a.page_tokens;
+            if (tail) {
+                dims[1] = tail;
+                if (!tmap::encode_bf16(&m->pk_tail, a.prefix_k, 4, dims, str, box)) return false;
+                if (!tmap::encode_bf16(&m->pv_tail, a.prefix_v, 4, dims, str, box)) return false;
+            }
+        }
+    } else {
+        m->pk = m->bk; m->pv = m->bv;    // never used (no prefix tiles)
+    }
+    return true;
+}
+
+// Tensor maps of one scene, reusing the cached ones while the pointers and lengths they were
+// built from have not changed (the usual case: one set of buffers, many denoising steps).
+const TcSetMaps* maps_for(const AttnProblem& a, int D, TcMapCache* cache) {
+    const bool call_same = cache->valid && cache->q == a.q && cache->k_blk == a.k_blk && cache->v_blk == a.v_blk &&
+                           cache->d == a.d;
+    const bool cache_same = cache->valid && cache->suffix_len == a.suffix_len;
+    if (call_same && cache_same) return &cache->maps;
+    if (!call_same) {
+        if (!make_call_maps(a, D, &cache->maps)) { cache->valid = false; return nullptr; }
+    }
+    // the never-used entries of the cache part alias the call part, so it is rebuilt either way
+    if (!make_cache_maps(a, D, &cache->maps)) { cache->valid = false; return nullptr; }
+    cache->q = a.q; cache->k_blk = a.k_blk; cache->v_blk = a.v_blk; cache->d = a.d;
+    cache->suffix_len = a.suffix_len;
+    cache->valid = true;
+    return &cache->maps;
+}
+
+int emulated_exponentials() {
+    // How many of the 128 exponentials of a key tile go through the polynomial.  FDD_ATTN_EMU
+    // (0, 32, 48 or 64) overrides the default; every choice computes the same thing.
+    static int value = -1;
+    if (value < 0) {
+        value = 48;
+        if (const char* e = std::getenv("FDD_ATTN_EMU")) {
+            const int v = std::atoi(e);
+            if (v == 0 || v == 32 || v == 48 || v == 64) value = v;
+        }
+    }
+    return value;
+}
+
+template <int D, int MAXSETS, int EMU>
+cudaError_t launch_one(const TcArgs<MAXSETS>& args, unsigned ctas, cudaStream_t st) {
+    const int smem = TcShape<D>::kSmemBytes;
+    static bool configured = false;
+    if (!configured) {
+        cudaError_t e = cudaFuncSetAttribute(attn_ptc_kernel<D, MAXSETS, EMU>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        if (e != cudaSuccess) return e;
+        configured = true;
+    }
+    attn_ptc_kernel<D, MAXSETS, EMU><<<ctas, kTcThreads, smem, st>>>(args);
+    return cudaGetLastError();
+}
+
+template <int MAXSETS>
+cudaError_t launch_emu(const TcArgs<MAXSETS>& args, int head_dim, unsigned ctas, cudaStream_t st) {
+    if (head_dim == 64) return launch_one<64, MAXSETS, 0>(args, ctas, st);
+    switch (emulated_exponentials()) {
+        case 0: return launch_one<128, MAXSETS, 0>(args, ctas, st);
+        case 32: return launch_one<128, MAXSETS, 32>(args, ctas, st);
+        case 64: return launch_one<128, MAXSETS, 64>(args, ctas, st);
+        default: return launch_one<128, MAXSETS, 48>(args, ctas, st);
+    }
+}
+
+template <int MAXSETS>
+cudaError_t launch_group(fdd_ctx* ctx, const AttnProblem* probs, TcMapCache* const* caches, int n, int head_dim,
+                         cudaStream_t st) {
+    static TcArgs<MAXSETS> args;     // 1-20 KB, kept off the stack (a context is used by one host thread at a time)
+    long long steps = 0;
+    int units = 0;
+    for (int s = 0; s < n; ++s) {
+        const AttnProblem& a = probs[s];
+        const TcSetMaps* m = maps_for(a, head_dim, caches[s]);
+        if (!m) return cudaErrorInvalidValue;
+        args.maps[s] = *m;
+        SetParams& p = args.sets[s];
+        p.out = a.out;
+        p.page_table = a.page_table;
+        p.n_forks = a.n_forks; p.d = a.d; p.n_q_heads = a.n_q_heads;
+        p.G = a.n_q_heads / a.n_kv_heads;
+        p.R = a.d * p.G;
+        p.prefix_len = a.prefix_len; p.page_tokens = a.page_tokens; p.n_phys_pages = a.prefix_capacity;
+        p.suffix_len = a.suffix_len;
+        p.tiles_prefix = (a.prefix_len + kKeysPerTile - 1) / kKeysPerTile;
+        p.tiles_suffix = (a.suffix_len + kKeysPerTile - 1) / kKeysPerTile;
+        p.tiles_total = p.tiles_prefix + p.tiles_suffix + (a.d + kKeysPerTile - 1) / kKeysPerTile;
+        p.row_pairs = (p.R + 255) / 256;
+        p.units = a.n_kv_heads * p.row_pairs * a.n_forks;
+        p.causal = a.causal_in_block;
+        p.step_base = steps;
+        p.unit_base = units;
+        steps += static_cast<long long>(p.units) * p.tiles_total;
+        units += p.units;
+    }
+    if (units > ctx->attn_max_units) return cudaErrorInvalidValue;
+    long long ctas = steps / kMinTilesPerCta;
+    if (ctas > ctx->attn_max_ctas) ctas = ctx->attn_max_ctas;
+    if (ctas < 1) ctas = 1;
+    args.part_o = static_cast<float*>(ctx->ws_attn);
+    args.part_lse = args.part_o + static_cast<size_t>(2) * ctx->attn_max_ctas * 256 * head_dim;
+    args.unit_count = ctx->attn_unit_count;
+    args.status = ctx->d_status;
+    args.total_steps = steps;
+    args.n_sets = n;
+    args.scale_log2 = probs[0].scale * 1.4426950408889634f;
+    return launch_emu<MAXSETS>(args, head_dim, static_cast<unsigned>(ctas), st);
+}
+
+}  // namespace
+
+// Scratch of the split-unit merge: two partial slots (256 rows of D values + log-sum-exp) per CTA.
+size_t attention_ptc_workspace_bytes(int head_dim, int max_ctas) {
+    return static_cast<size_t>(2) * max_ctas * 256 * (head_dim + 1) * sizeof(float);
+}
+
+// One launch for up to kTcMaxSets scenes (all with the same soft-max scale).
+cudaError_t launch_attention_ptc(fdd_ctx* ctx, const AttnProblem* probs, TcMapCache* const* caches, int n,
+                                 int head_dim, cudaStream_t st, int* n_launches) {
+    if (n < 1 || n > kTcMaxSets) return cudaErrorInvalidValue;
+    *n_launches += 1;
+    if (n == 1) return launch_group<1>(ctx, probs, caches, n, head_dim, st);
+    return launch_group<kTcMaxSets>(ctx, probs, caches, n, head_dim, st);
+}

@@ -4,10 +4,10 @@
 #include <algorithm>
 #include <cstdarg>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <new>
 
-cudaError_t launch_attention_simple(const AttnProblem& p, int head_dim, cudaStream_t st);
 cudaError_t launch_attention_tc(fdd_ctx* ctx, const AttnProblem& a, int head_dim, cudaStream_t st, int* n_launches);
 bool attention_tc_supported(const AttnProblem& a, int head_dim);
 size_t attention_tc_workspace_bytes(int head_dim, int sm_count);
@@ -32,6 +32,17 @@ fdd_status cuda_fail(fdd_ctx* ctx, cudaError_t e, const char* what) {
 
 bool set_alive(const fdd_ctx* ctx, const fdd_forkset* s) {
     return s && std::find(ctx->live_sets.begin(), ctx->live_sets.end(), s) != ctx->live_sets.end();
+}
+
+// Bring-up switch: FDD_ATTN_IMPL=persistent selects the persistent multi-scene kernel,
+// anything else the one-CTA-per-unit kernel.
+bool use_persistent_attention() {
+    static int v = -1;
+    if (v < 0) {
+        const char* e = std::getenv("FDD_ATTN_IMPL");
+        v = (e && std::strcmp(e, "persistent") == 0) ? 1 : 0;
+    }
+    return v == 1;
 }
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
@@ -83,8 +94,18 @@ fdd_status fdd_create(const fdd_config* cfg, fdd_ctx** out) {
         e = cudaMalloc(&ctx->ws_unmask, ctx->ws_unmask_bytes);
     }
     if (e == cudaSuccess) {
-        ctx->ws_attn_bytes = attention_tc_workspace_bytes(cfg->head_dim, ctx->sm_count);
+        ctx->attn_max_ctas = ctx->sm_count > 0 ? ctx->sm_count : 148;
+        ctx->ws_attn_bytes = std::max(attention_tc_workspace_bytes(cfg->head_dim, ctx->sm_count),
+                                      attention_ptc_workspace_bytes(cfg->head_dim, ctx->attn_max_ctas));
         e = cudaMalloc(&ctx->ws_attn, ctx->ws_attn_bytes);
+    }
+    if (e == cudaSuccess) {
+        // one counter per attention unit: (KV head, pair of 128-row tiles, rollout)
+        const int G = cfg->n_q_heads / cfg->n_kv_heads;
+        const int row_pairs = (cfg->max_block * G + 255) / 256;
+        ctx->attn_max_units = cfg->n_kv_heads * row_pairs * cfg->max_forks;
+        e = cudaMalloc(&ctx->attn_unit_count, sizeof(int) * ctx->attn_max_units);
+        if (e == cudaSuccess) e = cudaMemset(ctx->attn_unit_count, 0, sizeof(int) * ctx->attn_max_units);
     }
     if (e != cudaSuccess) {
         fdd_destroy(ctx);
@@ -104,6 +125,7 @@ void fdd_destroy(fdd_ctx* ctx) {
     if (ctx->h_status) cudaFreeHost(ctx->h_status);
     if (ctx->ws_unmask) cudaFree(ctx->ws_unmask);
     if (ctx->ws_attn) cudaFree(ctx->ws_attn);
+    if (ctx->attn_unit_count) cudaFree(ctx->attn_unit_count);
     delete ctx;
 }
 
@@ -154,6 +176,7 @@ fdd_status fdd_fork(fdd_ctx* ctx, const void* const* prefix_k, const void* const
     s->suffix_v.assign(suffix_v, suffix_v + ctx->cfg.n_layers);
     s->suffix_capacity = suffix_capacity;
     s->suffix_len = 0;
+    s->map_cache.resize(ctx->cfg.n_layers);
     cudaError_t e = cudaMalloc(&s->d_seeds, sizeof(uint64_t) * n_forks);
     if (e == cudaSuccess) e = cudaMemcpy(s->d_seeds, seeds, sizeof(uint64_t) * n_forks, cudaMemcpyHostToDevice);
     if (e != cudaSuccess) {
@@ -198,9 +221,13 @@ fdd_status fdd_block_attn(fdd_ctx* ctx, fdd_forkset* const* sets, int n_sets, in
     if (layer < 0 || layer >= ctx->cfg.n_layers) return fail(ctx, FDD_ERR_SHAPE, "layer %d outside [0, %d)", layer, ctx->cfg.n_layers);
     if (!(scale > 0.0f)) return fail(ctx, FDD_ERR_INVALID_ARG, "scale must be positive");
     const fdd_config& c = ctx->cfg;
+    cudaStream_t st_ = static_cast<cudaStream_t>(stream);
+    const bool persistent = use_persistent_attention();
     size_t q_off = 0, kv_off = 0;
+    std::vector<AttnProblem> tc_probs;
+    std::vector<TcMapCache*> tc_caches;
     for (int s = 0; s < n_sets; ++s) {
-        const fdd_forkset* fs = sets[s];
+        fdd_forkset* fs = sets[s];
         AttnProblem p;
         p.q = static_cast<const __nv_bfloat16*>(q) + q_off;
         p.k_blk = static_cast<const __nv_bfloat16*>(k_blk) + kv_off;
@@ -222,12 +249,26 @@ fdd_status fdd_block_attn(fdd_ctx* ctx, fdd_forkset* const* sets, int n_sets, in
         p.suffix_capacity = fs->suffix_capacity;
         p.causal_in_block = causal_in_block ? 1 : 0;
         p.scale = scale;
-        int n_launches = 0;
-        cudaError_t e = launch_attention(ctx, p, c.head_dim, static_cast<cudaStream_t>(stream), &n_launches);
-        ctx->launches += n_launches;
-        if (e != cudaSuccess) return cuda_fail(ctx, e, "fdd_block_attn launch");
+        if (persistent && attention_tc_supported(p, c.head_dim)) {
+            // the persistent tensor-core kernel takes many scenes per launch
+            tc_probs.push_back(p);
+            tc_caches.push_back(&fs->map_cache[layer]);
+        } else {
+            int n_launches = 0;
+            cudaError_t e = launch_attention(ctx, p, c.head_dim, st_, &n_launches);
+            ctx->launches += n_launches;
+            if (e != cudaSuccess) return cuda_fail(ctx, e, "fdd_block_attn launch");
+        }
         q_off += static_cast<size_t>(fs->n_forks) * p.d * c.n_q_heads * c.head_dim;
         kv_off += static_cast<size_t>(fs->n_forks) * p.d * c.n_kv_heads * c.head_dim;
+    }
+    for (size_t first = 0; first < tc_probs.size(); first += kTcMaxSets) {
+        const int n = static_cast<int>(std::min<size_t>(kTcMaxSets, tc_probs.size() - first));
+        int n_launches = 0;
+        cudaError_t e = launch_attention_ptc(ctx, tc_probs.data() + first, tc_caches.data() + first, n, c.head_dim, st_,
+                                             &n_launches);
+        ctx->launches += n_launches;
+        if (e != cudaSuccess) return cuda_fail(ctx, e, "fdd_block_attn launch");
     }
     return FDD_OK;
 }
@@ -327,7 +368,12 @@ fdd_status fdd_poll_status(fdd_ctx* ctx, void* stream) {
     if (e == cudaSuccess) e = cudaStreamSynchronize(st);
     if (e != cudaSuccess) return cuda_fail(ctx, e, "fdd_poll_status");
     const int code = *ctx->h_status;
-    if (code != FDD_OK) return fail(ctx, code, "a kernel recorded device status %d", code);
+    if (code != FDD_OK) {
+        // a kernel that gave up may have left piece counters of the attention merge half counted
+        cudaMemsetAsync(ctx->attn_unit_count, 0, sizeof(int) * ctx->attn_max_units, st);
+        cudaStreamSynchronize(st);
+        return fail(ctx, code, "a kernel recorded device status %d", code);
+    }
     return FDD_OK;
 }
 

@@ -1,5 +1,6 @@
 // Internal declarations shared by the host API and the kernel files.
 #pragma once
+#include <cuda.h>
 #include <cuda_runtime.h>
 #include <cuda_bf16.h>
 #include <stdint.h>
@@ -7,6 +8,27 @@
 #include <vector>
 
 #include "fdd.h"
+
+// TMA tensor maps of one scene for the persistent tensor-core attention kernel.
+struct TcSetMaps {
+    CUtensorMap q;                  // (D, Hq, d, N)
+    CUtensorMap bk, bv;             // (D, Hkv, d, N)
+    CUtensorMap sk, sv;             // (D, S, Hkv, N)
+    CUtensorMap pk, pv;             // contiguous: (D, P, Hkv); paged: (D, 64, Hkv, pages)
+    CUtensorMap pk_tail, pv_tail;   // paged only: token dimension cut to the last page's fill
+};
+constexpr int kTcMaxSets = 16;      // scenes per attention launch
+
+// The maps last built for one (fork set, layer) and what they were built from.
+struct TcMapCache {
+    bool valid = false;
+    const void* q = nullptr;
+    const void* k_blk = nullptr;
+    const void* v_blk = nullptr;
+    int d = 0;
+    int suffix_len = -1;
+    TcSetMaps maps;
+};
 
 struct fdd_ctx {
     fdd_config cfg;
@@ -16,8 +38,11 @@ struct fdd_ctx {
     int* h_status = nullptr;          // pinned mirror
     void* ws_unmask = nullptr;        // per (row, chunk) partial reductions
     size_t ws_unmask_bytes = 0;
-    void* ws_attn = nullptr;          // split-KV partial outputs
+    void* ws_attn = nullptr;          // partial outputs of attention units cut between CTAs
     size_t ws_attn_bytes = 0;
+    int* attn_unit_count = nullptr;   // device [attn_max_units]: finished pieces per unit (self-resetting)
+    int attn_max_units = 0;
+    int attn_max_ctas = 0;
     uint64_t launches = 0;
     std::string last_error;
     std::vector<fdd_forkset*> live_sets;
@@ -34,6 +59,7 @@ struct fdd_forkset {
     int suffix_capacity = 0;
     int suffix_len = 0;
     uint64_t* d_seeds = nullptr;            // device [n_forks]
+    std::vector<TcMapCache> map_cache;      // per layer
 };
 
 // One scene's slice of a batched call, as the kernels see it.
@@ -81,6 +107,11 @@ static constexpr int kUnmaskChunk = 8192;   // vocabulary entries per CTA
 static inline int unmask_chunks(int vocab) { return (vocab + kUnmaskChunk - 1) / kUnmaskChunk; }
 
 cudaError_t launch_attention(fdd_ctx* ctx, const AttnProblem& p, int head_dim, cudaStream_t st, int* n_launches);
+cudaError_t launch_attention_simple(const AttnProblem& p, int head_dim, cudaStream_t st);
+bool attention_tc_supported(const AttnProblem& a, int head_dim);
+size_t attention_ptc_workspace_bytes(int head_dim, int max_ctas);
+cudaError_t launch_attention_ptc(fdd_ctx* ctx, const AttnProblem* probs, TcMapCache* const* caches, int n,
+                                 int head_dim, cudaStream_t st, int* n_launches);
 cudaError_t launch_unmask(fdd_ctx* ctx, const UnmaskProblem& p, cudaStream_t st, int* n_launches);
 cudaError_t launch_kv_commit(const __nv_bfloat16* k_blk, const __nv_bfloat16* v_blk,
                              __nv_bfloat16* suffix_k, __nv_bfloat16* suffix_v,

@@ -95,6 +95,62 @@ def test_attention_paged_prefix():
     _attention_case(w, n_blocks_before=1)
 
 
+def test_attention_many_scenes_one_call():
+    # a ragged serving batch in ONE call: scenes differ in prefix length, rollouts and block length;
+    # paged prefix with shuffled physical pages; every scene has an earlier block in its suffix
+    base = synth.workload("serving_mix")
+    scenes = (synth.Scene(64 * 5 + 9, 4, 16, 5, 2), synth.Scene(64 * 21, 1, 32, 10, 2),
+              synth.Scene(700, 3, 64, 19, 2), synth.Scene(130, 2, 32, 10, 2), synth.Scene(1, 1, 16, 5, 2))
+    w = synth.Workload("mix_small", base.n_q_heads, base.n_kv_heads, base.head_dim, 1024, "bf16", "peaked", 0.9, 1.0,
+                       scenes, page_tokens=64, seed=17)
+    ctx = harness.create_context(w)
+    try:
+        gs, refs, qs, ks, vs = [], [], [], [], []
+        for i, sc in enumerate(scenes):
+            g = harness.GpuScene(ctx, w, i, suffix_capacity=2 * sc.block_len)
+            pk, pv = synth.make_prefix(w, i)
+            ofs = ForkSet([pk], [pv], sc.n_forks, g.seeds)
+            _, kb, vb = synth.make_qkv(w, i, 0, 0, 0)
+            fdd.fdd_kv_commit(ctx, [g.forkset], 0, harness.bf16_tensor(kb), harness.bf16_tensor(vb), [sc.block_len], 1)
+            ofs.kv_commit(0, kb, vb)
+            q, k, v = synth.make_qkv(w, i, 0, 1, 0)
+            refs.append(pu.attention_oracle(w, (pk, pv), _suffix_from_oracle(ofs), q, k, v))
+            gs.append(g); qs.append(q); ks.append(k); vs.append(v)
+        pack = lambda xs: harness.bf16_tensor(np.concatenate([x.reshape(-1) for x in xs]))
+        qd, kd, vd = pack(qs), pack(ks), pack(vs)
+        out = torch.full_like(qd, float("nan"))
+        fdd.fdd_block_attn(ctx, [g.forkset for g in gs], 0, qd, kd, vd, out, [sc.block_len for sc in scenes],
+                           1.0 / np.sqrt(w.head_dim), 0)
+        fdd.fdd_poll_status(ctx)
+        got = out.float().cpu().numpy().astype(np.float64)
+        off = 0
+        for sc, ref in zip(scenes, refs):
+            n = ref.size
+            pu.assert_attention_close(got[off:off + n].reshape(ref.shape), ref)
+            off += n
+        assert off == got.size
+    finally:
+        fdd.fdd_destroy(ctx)
+
+
+def test_attention_repeated_calls_reuse_scratch():
+    # the scratch of the split-unit merge is reusable at once: the same call three times in a row
+    # (different inputs) stays correct
+    w = synth.workload("tts")
+    ctx = harness.create_context(w)
+    try:
+        scene = harness.GpuScene(ctx, w, 0)
+        pk, pv = synth.make_prefix(w, 0)
+        empty = ([np.zeros((0, w.n_kv_heads, w.head_dim), dtype=np.uint16)] * 8,) * 2
+        for step in range(3):
+            q, k, v = synth.make_qkv(w, 0, 0, 0, step)
+            got = pu.attention_gpu(ctx, scene, q, k, v)
+            ref = pu.attention_oracle(w, (pk, pv), empty, q, k, v, forks=[step, 7 - step])
+            pu.assert_attention_close(got[[step, 7 - step]], ref)
+    finally:
+        fdd.fdd_destroy(ctx)
+
+
 def test_prefix_is_never_written_and_forks_with_equal_inputs_agree():
     w = synth.small_variant(synth.workload("tts"), prefix_len=512, vocab=512, n_forks=4, n_blocks=1)
     ctx = harness.create_context(w)
