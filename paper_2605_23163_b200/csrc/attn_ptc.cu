@@ -701,13 +701,13 @@ const TcSetMaps* maps_for(const AttnProblem& a, int D, TcMapCache* cache) {
 
 int emulated_exponentials() {
     // How many of the 128 exponentials of a key tile go through the polynomial.  FDD_ATTN_EMU
-    // (0, 32, 48 or 64) overrides the default; every choice computes the same thing.
+    // (0, 16 or 32) overrides the default; every choice computes the same thing.
     static int value = -1;
     if (value < 0) {
-        value = 48;
+        value = 0;
         if (const char* e = std::getenv("FDD_ATTN_EMU")) {
             const int v = std::atoi(e);
-            if (v == 0 || v == 32 || v == 48 || v == 64) value = v;
+            if (v == 0 || v == 16 || v == 32) value = v;
         }
     }
     return value;
@@ -730,10 +730,9 @@ template <int MAXSETS>
 cudaError_t launch_emu(const TcArgs<MAXSETS>& args, int head_dim, unsigned ctas, cudaStream_t st) {
     if (head_dim == 64) return launch_one<64, MAXSETS, 0>(args, ctas, st);
     switch (emulated_exponentials()) {
-        case 0: return launch_one<128, MAXSETS, 0>(args, ctas, st);
+        case 16: return launch_one<128, MAXSETS, 16>(args, ctas, st);
         case 32: return launch_one<128, MAXSETS, 32>(args, ctas, st);
-        case 64: return launch_one<128, MAXSETS, 64>(args, ctas, st);
-        default: return launch_one<128, MAXSETS, 48>(args, ctas, st);
+        default: return launch_one<128, MAXSETS, 0>(args, ctas, st);
     }
 }
 
@@ -782,6 +781,15 @@ cudaError_t launch_group(fdd_ctx* ctx, const AttnProblem* probs, TcMapCache* con
 }
 
 }  // namespace
+
+// Whether the tensor-core kernel covers this problem.
+bool attention_tc_supported(const AttnProblem& a, int head_dim) {
+    const int G = a.n_q_heads / a.n_kv_heads;
+    if (head_dim != 64 && head_dim != 128) return false;
+    if (G < 1 || G > 16 || (G & (G - 1)) != 0) return false;
+    if (a.page_tokens != 0 && a.page_tokens != 64) return false;
+    return tmap::encode_fn() != nullptr;
+}
 
 // Scratch of the split-unit merge: two partial slots (256 rows of D values + log-sum-exp) per CTA.
 size_t attention_ptc_workspace_bytes(int head_dim, int max_ctas) {

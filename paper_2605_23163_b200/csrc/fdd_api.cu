@@ -8,9 +8,6 @@
 #include <cstring>
 #include <new>
 
-cudaError_t launch_attention_tc(fdd_ctx* ctx, const AttnProblem& a, int head_dim, cudaStream_t st, int* n_launches);
-bool attention_tc_supported(const AttnProblem& a, int head_dim);
-size_t attention_tc_workspace_bytes(int head_dim, int sm_count);
 
 namespace {
 
@@ -32,17 +29,6 @@ fdd_status cuda_fail(fdd_ctx* ctx, cudaError_t e, const char* what) {
 
 bool set_alive(const fdd_ctx* ctx, const fdd_forkset* s) {
     return s && std::find(ctx->live_sets.begin(), ctx->live_sets.end(), s) != ctx->live_sets.end();
-}
-
-// Bring-up switch: FDD_ATTN_IMPL=persistent selects the persistent multi-scene kernel,
-// anything else the one-CTA-per-unit kernel.
-bool use_persistent_attention() {
-    static int v = -1;
-    if (v < 0) {
-        const char* e = std::getenv("FDD_ATTN_IMPL");
-        v = (e && std::strcmp(e, "persistent") == 0) ? 1 : 0;
-    }
-    return v == 1;
 }
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
@@ -95,8 +81,7 @@ fdd_status fdd_create(const fdd_config* cfg, fdd_ctx** out) {
     }
     if (e == cudaSuccess) {
         ctx->attn_max_ctas = ctx->sm_count > 0 ? ctx->sm_count : 148;
-        ctx->ws_attn_bytes = std::max(attention_tc_workspace_bytes(cfg->head_dim, ctx->sm_count),
-                                      attention_ptc_workspace_bytes(cfg->head_dim, ctx->attn_max_ctas));
+        ctx->ws_attn_bytes = attention_ptc_workspace_bytes(cfg->head_dim, ctx->attn_max_ctas);
         e = cudaMalloc(&ctx->ws_attn, ctx->ws_attn_bytes);
     }
     if (e == cudaSuccess) {
@@ -222,7 +207,6 @@ fdd_status fdd_block_attn(fdd_ctx* ctx, fdd_forkset* const* sets, int n_sets, in
     if (!(scale > 0.0f)) return fail(ctx, FDD_ERR_INVALID_ARG, "scale must be positive");
     const fdd_config& c = ctx->cfg;
     cudaStream_t st_ = static_cast<cudaStream_t>(stream);
-    const bool persistent = use_persistent_attention();
     size_t q_off = 0, kv_off = 0;
     std::vector<AttnProblem> tc_probs;
     std::vector<TcMapCache*> tc_caches;
@@ -249,14 +233,14 @@ fdd_status fdd_block_attn(fdd_ctx* ctx, fdd_forkset* const* sets, int n_sets, in
         p.suffix_capacity = fs->suffix_capacity;
         p.causal_in_block = causal_in_block ? 1 : 0;
         p.scale = scale;
-        if (persistent && attention_tc_supported(p, c.head_dim)) {
-            // the persistent tensor-core kernel takes many scenes per launch
+        if (attention_tc_supported(p, c.head_dim)) {
+            // the tensor-core kernel takes many scenes per launch
             tc_probs.push_back(p);
             tc_caches.push_back(&fs->map_cache[layer]);
         } else {
-            int n_launches = 0;
-            cudaError_t e = launch_attention(ctx, p, c.head_dim, st_, &n_launches);
-            ctx->launches += n_launches;
+            // the CUDA-core kernel covers the remaining shapes (GQA groups that are not a power of two)
+            cudaError_t e = launch_attention_simple(p, c.head_dim, st_);
+            ctx->launches += 1;
             if (e != cudaSuccess) return cuda_fail(ctx, e, "fdd_block_attn launch");
         }
         q_off += static_cast<size_t>(fs->n_forks) * p.d * c.n_q_heads * c.head_dim;
@@ -378,10 +362,3 @@ fdd_status fdd_poll_status(fdd_ctx* ctx, void* stream) {
 }
 
 }  // extern "C"
-
-cudaError_t launch_attention(fdd_ctx* ctx, const AttnProblem& p, int head_dim, cudaStream_t st, int* n_launches) {
-    // The tensor-core kernel covers power-of-two GQA groups; the CUDA-core kernel the rest.
-    if (attention_tc_supported(p, head_dim)) return launch_attention_tc(ctx, p, head_dim, st, n_launches);
-    *n_launches += 1;
-    return launch_attention_simple(p, head_dim, st);
-}

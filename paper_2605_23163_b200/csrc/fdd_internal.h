@@ -106,7 +106,6 @@ struct UnmaskPartial {
 static constexpr int kUnmaskChunk = 8192;   // vocabulary entries per CTA
 static inline int unmask_chunks(int vocab) { return (vocab + kUnmaskChunk - 1) / kUnmaskChunk; }
 
-cudaError_t launch_attention(fdd_ctx* ctx, const AttnProblem& p, int head_dim, cudaStream_t st, int* n_launches);
 cudaError_t launch_attention_simple(const AttnProblem& p, int head_dim, cudaStream_t st);
 bool attention_tc_supported(const AttnProblem& a, int head_dim);
 size_t attention_ptc_workspace_bytes(int head_dim, int max_ctas);

@@ -160,8 +160,11 @@ def test_prefix_is_never_written_and_forks_with_equal_inputs_agree():
         q, k, v = synth.make_qkv(w, 0, 0, 0, 0)
         q, k, v = (np.repeat(x[:1], 4, axis=0) for x in (q, k, v))
         got = pu.attention_gpu(ctx, scene, q, k, v)
+        # Rollouts with equal inputs agree up to the rounding of the bf16 output: a unit may be cut
+        # between CTAs at a different key tile per rollout, which changes the summation order only.
         for f in range(1, 4):
-            assert np.array_equal(got[f], got[0])
+            assert np.max(np.abs(got[f] - got[0])) <= 2e-3
+            assert np.linalg.norm(got[f] - got[0]) <= 4e-3 * np.linalg.norm(got[0])
         fdd.fdd_kv_commit(ctx, [scene.forkset], 0, harness.bf16_tensor(k), harness.bf16_tensor(v), [k.shape[1]], 1)
         fdd.fdd_poll_status(ctx)
         for a, b in zip(before, scene.prefix_k + scene.prefix_v):
