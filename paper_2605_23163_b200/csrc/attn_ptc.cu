@@ -15,13 +15,17 @@
 // Warp roles (384 threads): warps 0-3 and 4-7 are the two soft-max groups (thread = one query
 // row = one TMEM lane), warp 8 lane 0 drives TMA, warp 9 lane 0 issues every tcgen05.mma, warps
 // 10-11 only donate their registers.
-// TMEM (512 columns): S0 | S1 | O0 | O1; the bf16 probabilities P overwrite the first half of
-// their S tile and feed the PV product straight from TMEM.  Per key tile and query tile:
-//   S = Q K^T (smem x smem)  ->  soft-max warps: running max (rescaling O only when the max moved
-//   by more than 2^8), P = exp2(S * c - m) -> TMEM  ->  O += P V (TMEM x smem, V keys-major).
-// The two query tiles ping-pong, so one tile's soft-max overlaps the other tile's MMAs.  The
-// exponentials of a tile are split between the special-function unit (ex2.approx) and a cubic
-// polynomial on the FMA pipe, because one ex2 per score needs as many cycles as the MMAs.
+// A staged 128-key tile is consumed in two halves of 64 keys, and every query tile owns TWO score
+// buffers, so the scores of the next half are already in TMEM while the soft-max warps work on
+// the current one: four independent S -> P -> PV chains keep the tensor pipe and the soft-max
+// warps busy at the same time.
+// TMEM (512 columns): S[q][b] at (2 q + b) * 64 (64 fp32 columns each) | O0 | O1 at 256; the bf16
+// probabilities P overwrite the first half of their S buffer and feed the PV product straight
+// from TMEM.  Per half tile and query tile:
+//   S = Q K^T (smem x smem, N = 64)  ->  soft-max warps: running max (rescaling O only when the
+//   max moved by more than 2^8), P = exp2(S * c - m) -> TMEM  ->  O += P V (TMEM x smem).
+// The exponentials can be split between the special-function unit (ex2.approx) and a cubic
+// polynomial on the FMA pipe (one ex2 per score needs as many cycles as the MMAs).
 // Every mbarrier wait is bounded; on a timeout the CTA records FDD_ERR_DEVICE_TIMEOUT, drains
 // and returns (TMEM is always freed).
 #include "fdd_internal.h"
@@ -181,7 +185,7 @@ attn_ptc_kernel(const __grid_constant__ TcArgs<MAXSETS> a) {
     const uint32_t v_s = k_s + kStages * Shape::kTileBytes;
 
     __shared__ __align__(8) unsigned long long bar_q_full, bar_k_full[kStages], bar_k_empty[kStages],
-        bar_v_full[kStages], bar_v_empty[kStages], bar_s_full[2], bar_p_full[2], bar_o_done[2];
+        bar_v_full[kStages], bar_v_empty[kStages], bar_s_full[2][2], bar_p_full[2][2], bar_o_done[2], bar_item_done;
     __shared__ uint32_t tmem_base_s;
     __shared__ int abort_s, last_s;
     volatile int* abort_flag = &abort_s;
@@ -197,6 +201,7 @@ attn_ptc_kernel(const __grid_constant__ TcArgs<MAXSETS> a) {
         abort_s = 0;
         last_s = 0;
         tc::mbar_init(tc::smem_u32(&bar_q_full), 1);
+        tc::mbar_init(tc::smem_u32(&bar_item_done), 1);
         for (int s = 0; s < kStages; ++s) {
             tc::mbar_init(tc::smem_u32(&bar_k_full[s]), 1);
             tc::mbar_init(tc::smem_u32(&bar_k_empty[s]), 1);
@@ -204,8 +209,10 @@ attn_ptc_kernel(const __grid_constant__ TcArgs<MAXSETS> a) {
             tc::mbar_init(tc::smem_u32(&bar_v_empty[s]), 1);
         }
         for (int q = 0; q < 2; ++q) {
-            tc::mbar_init(tc::smem_u32(&bar_s_full[q]), 1);
-            tc::mbar_init(tc::smem_u32(&bar_p_full[q]), 128);
+            for (int b = 0; b < 2; ++b) {
+                tc::mbar_init(tc::smem_u32(&bar_s_full[q][b]), 1);
+                tc::mbar_init(tc::smem_u32(&bar_p_full[q][b]), 128);
+            }
             tc::mbar_init(tc::smem_u32(&bar_o_done[q]), 1);
         }
         tc::fence_barrier_init();
@@ -218,7 +225,7 @@ attn_ptc_kernel(const __grid_constant__ TcArgs<MAXSETS> a) {
     __syncthreads();
     tc::fence_after_sync();
     const uint32_t tmem = tmem_base_s;
-    const uint32_t tm_s[2] = {tmem, tmem + 128};
+    const uint32_t tm_s[2][2] = {{tmem, tmem + 64}, {tmem + 128, tmem + 192}};
     const uint32_t tm_o[2] = {tmem + 256, tmem + 256 + D};
 
     // Each role runs its own copy of the item loop; all of them meet at the end of every item.
@@ -304,21 +311,23 @@ attn_ptc_kernel(const __grid_constant__ TcArgs<MAXSETS> a) {
                 const ItemView v = view_item(pos);
                 const int nt = v.nt, NQ = v.NQ;
                 if (lane == 0) {
-                    constexpr uint32_t kIdescQK = tc::idesc_bf16(128, 128, 0);
+                    constexpr uint32_t kIdescQK = tc::idesc_bf16(128, 64, 0);
                     constexpr uint32_t kIdescPV = tc::idesc_bf16(128, D, 1);
-                    auto issue_qk = [&](int q, int s) {
+                    // S[q][b] = Q[q] . K[keys 64 b .. 64 b + 63]^T
+                    auto issue_qk = [&](int q, int s, int b) {
 #pragma unroll
                         for (int k = 0; k < D / 16; ++k) {
                             const uint32_t off = (k >> 2) * Shape::kChunkBytes + (k & 3) * 32;
-                            tc::mma_ss(tm_s[q], tc::smem_desc_sw128(q_s + q * Shape::kTileBytes + off, 0, 1024),
-                                       tc::smem_desc_sw128(k_s + s * Shape::kTileBytes + off, 0, 1024), kIdescQK, k > 0);
+                            tc::mma_ss(tm_s[q][b], tc::smem_desc_sw128(q_s + q * Shape::kTileBytes + off, 0, 1024),
+                                       tc::smem_desc_sw128(k_s + s * Shape::kTileBytes + b * 8192 + off, 0, 1024), kIdescQK, k > 0);
                         }
                     };
-                    auto issue_pv = [&](int q, int s, int accumulate) {
+                    // O[q] (+)= P[q][b] . V[keys 64 b .. 64 b + 63]
+                    auto issue_pv = [&](int q, int s, int b, int accumulate) {
 #pragma unroll
-                        for (int j = 0; j < kKeysPerTile / 16; ++j)
-                            tc::mma_ts(tm_o[q], tm_s[q] + j * 8,
-                                       tc::smem_desc_sw128(v_s + s * Shape::kTileBytes + j * 2048, Shape::kChunkBytes, 1024),
+                        for (int j = 0; j < 4; ++j)
+                            tc::mma_ts(tm_o[q], tm_s[q][b] + j * 8,
+                                       tc::smem_desc_sw128(v_s + s * Shape::kTileBytes + (b * 4 + j) * 2048, Shape::kChunkBytes, 1024),
                                        kIdescPV, (accumulate || j > 0) ? 1u : 0u);
                     };
                     const int s0 = kv_cnt % kStages;
@@ -326,40 +335,47 @@ attn_ptc_kernel(const __grid_constant__ TcArgs<MAXSETS> a) {
                     ok = ok && tc::mbar_wait(tc::smem_u32(&bar_k_full[s0]), (kv_cnt / kStages) & 1, abort_flag, kWaitLimit);
                     if (ok) {
                         tc::fence_after_sync();
-                        for (int q = 0; q < NQ; ++q) {
-                            issue_qk(q, s0);
-                            tc::mma_commit(tc::smem_u32(&bar_s_full[q]));
-                        }
+                        for (int b = 0; b < 2; ++b)
+                            for (int q = 0; q < NQ; ++q) {
+                                issue_qk(q, s0, b);
+                                tc::mma_commit(tc::smem_u32(&bar_s_full[q][b]));
+                            }
                         tc::mma_commit(tc::smem_u32(&bar_k_empty[s0]));
                     }
+                    // The scores run one key tile ahead of the PV products.
                     for (int jl = 0; jl < nt && ok; ++jl) {
                         const uint32_t n = kv_cnt + jl;
                         const int s = n % kStages;
                         const uint32_t ph = (n / kStages) & 1;
-                        const int jn = jl + 1;
+                        const bool has_next = jl + 1 < nt;
                         const int sn = (n + 1) % kStages;
                         const uint32_t phn = ((n + 1) / kStages) & 1;
                         ok = tc::mbar_wait(tc::smem_u32(&bar_v_full[s]), ph, abort_flag, kWaitLimit);
-                        for (int q = 0; q < NQ && ok; ++q) {
-                            ok = tc::mbar_wait(tc::smem_u32(&bar_p_full[q]), (sp_cnt[q] + jl) & 1, abort_flag, kWaitLimit);
-                            if (!ok) break;
-                            tc::fence_after_sync();
-                            issue_pv(q, s, jl > 0);
-                            tc::mma_commit(tc::smem_u32(&bar_o_done[q]));
-                            if (jn < nt) {
-                                if (q == 0) {
-                                    ok = tc::mbar_wait(tc::smem_u32(&bar_k_full[sn]), phn, abort_flag, kWaitLimit);
-                                    if (!ok) break;
-                                    tc::fence_after_sync();
+                        for (int b = 0; b < 2 && ok; ++b) {
+                            for (int q = 0; q < NQ && ok; ++q) {
+                                ok = tc::mbar_wait(tc::smem_u32(&bar_p_full[q][b]), (sp_cnt[q] + jl) & 1, abort_flag, kWaitLimit);
+                                if (!ok) break;
+                                tc::fence_after_sync();
+                                issue_pv(q, s, b, jl > 0 || b > 0);
+                                tc::mma_commit(tc::smem_u32(&bar_o_done[q]));
+                                if (has_next) {
+                                    if (q == 0 && b == 0) {
+                                        ok = tc::mbar_wait(tc::smem_u32(&bar_k_full[sn]), phn, abort_flag, kWaitLimit);
+                                        if (!ok) break;
+                                        tc::fence_after_sync();
+                                    }
+                                    issue_qk(q, sn, b);
+                                    tc::mma_commit(tc::smem_u32(&bar_s_full[q][b]));
                                 }
-                                issue_qk(q, sn);
-                                tc::mma_commit(tc::smem_u32(&bar_s_full[q]));
                             }
                         }
                         if (!ok) break;
                         tc::mma_commit(tc::smem_u32(&bar_v_empty[s]));
-                        if (jn < nt) tc::mma_commit(tc::smem_u32(&bar_k_empty[sn]));
+                        if (has_next) tc::mma_commit(tc::smem_u32(&bar_k_empty[sn]));
                     }
+                    // One arrival per item once every MMA of the item has completed.  (bar_o_done cannot
+                    // serve here: the scores run ahead, so a waiter could be two of its phases behind.)
+                    if (ok) tc::mma_commit(tc::smem_u32(&bar_item_done));
                     if (!ok) {
                         if (*abort_flag == 0) atomicCAS(a.status, 0, FDD_ERR_DEVICE_TIMEOUT);
                         *abort_flag = 1;
@@ -386,8 +402,9 @@ attn_ptc_kernel(const __grid_constant__ TcArgs<MAXSETS> a) {
         const int q = warp >> 2;
         const int row_local = tid & 127;
         const uint32_t lane_base = (static_cast<uint32_t>(warp & 3) * 32u) << 16;
-        const uint32_t bs = tc::smem_u32(&bar_s_full[q]), bp = tc::smem_u32(&bar_p_full[q]), bo = tc::smem_u32(&bar_o_done[q]);
-        uint32_t sp0 = 0;                   // key tiles this group has handled so far
+        const uint32_t bo = tc::smem_u32(&bar_o_done[q]);
+        uint32_t sp0 = 0;                   // key tiles this group has handled so far (two PV commits each)
+        uint32_t item_cnt = 0;
         for (long long pos = range_begin; pos < range_end;) {
             const ItemView v = view_item(pos);
             const Item& it = v.it;
@@ -401,28 +418,33 @@ attn_ptc_kernel(const __grid_constant__ TcArgs<MAXSETS> a) {
             float m_used = -CUDART_INF_F, l = 0.0f;
             bool ok = true;
             if (active) {
+                constexpr int kHalf = 64;                   // keys per half tile
+                constexpr int kEmu = EMU / 2;               // emulated exponentials per half tile
                 const float c = a.scale_log2;
                 const uint64_t c2 = tc::pack2(c, c);
                 const float c_emu = c * (1.0f / 128.0f);
-                for (int jl = 0; jl < nt; ++jl) {
+                for (int hs = 0; hs < 2 * nt; ++hs) {
+                    const int jl = hs >> 1, b = hs & 1;
                     const TileInfo t = tile_info(p, it.t0 + jl);
-                    ok = tc::mbar_wait(bs, (sp0 + jl) & 1, abort_flag, kWaitLimit);
+                    ok = tc::mbar_wait(tc::smem_u32(&bar_s_full[q][b]), (sp0 + jl) & 1, abort_flag, kWaitLimit);
                     if (!ok) break;
                     tc::fence_after_sync();
-                    uint32_t sr[128];
-#pragma unroll
-                    for (int cc = 0; cc < 4; ++cc) tc::tmem_ld32(tm_s[q] + lane_base + cc * 32, sr + cc * 32);
+                    const uint32_t ts = tm_s[q][b] + lane_base;
+                    uint32_t sr[kHalf];
+                    tc::tmem_ld32(ts, sr);
+                    tc::tmem_ld32(ts + 32, sr + 32);
                     tc::wait_ld();
-                    int limit = t.nvalid;                               // keys [0, limit) are visible
+                    int limit = t.nvalid;                               // keys [0, limit) of the tile are visible
                     if (p.causal && t.segment == 2) limit = min(limit, qi - t.index * kKeysPerTile + 1);
-                    if (limit < kKeysPerTile) {
+                    limit -= b * kHalf;                                 // ... of this half
+                    if (limit < kHalf) {
 #pragma unroll
-                        for (int i = 0; i < 128; ++i)
+                        for (int i = 0; i < kHalf; ++i)
                             if (i >= limit) sr[i] = 0xFF800000u;        // -inf
                     }
                     float mx[4] = {-CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F};
 #pragma unroll
-                    for (int i = 0; i < 128; i += 8) {
+                    for (int i = 0; i < kHalf; i += 8) {
 #pragma unroll
                         for (int u = 0; u < 4; ++u)
                             mx[u] = tc::max3(mx[u], __uint_as_float(sr[i + 2 * u]), __uint_as_float(sr[i + 2 * u + 1]));
@@ -430,12 +452,13 @@ attn_ptc_kernel(const __grid_constant__ TcArgs<MAXSETS> a) {
                     const float tmax = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
                     float m_tile = tmax * c;
                     if (!(m_tile > -CUDART_INF_F)) m_tile = m_used > -CUDART_INF_F ? m_used : 0.0f;
-                    if (jl == 0) {
+                    if (hs == 0) {
                         m_used = m_tile;
                     } else {
                         const bool need = m_tile > m_used + 8.0f;
                         if (__any_sync(0xFFFFFFFFu, need)) {
-                            ok = tc::mbar_wait(bo, (sp0 + jl - 1) & 1, abort_flag, kWaitLimit);
+                            // O holds every PV product up to the previous half: wait for that one, rescale
+                            ok = tc::mbar_wait(bo, (2 * sp0 + hs - 1) & 1, abort_flag, kWaitLimit);
                             if (!ok) break;
                             tc::fence_after_sync();
                             const float alpha = need ? exp2f(m_used - m_tile) : 1.0f;
@@ -453,13 +476,13 @@ attn_ptc_kernel(const __grid_constant__ TcArgs<MAXSETS> a) {
                             if (need) m_used = m_tile;
                         }
                     }
-                    // P = 2^(S * c - m): the first 128 - EMU scores through ex2.approx, the rest
+                    // P = 2^(S * c - m): the first kHalf - kEmu scores through ex2.approx, the rest
                     // through the polynomial; row sums in four packed accumulators.
                     uint64_t acc[4] = {0ull, 0ull, 0ull, 0ull};
-                    uint32_t packed[64];
+                    uint32_t packed[kHalf / 2];
                     const uint64_t nm2 = tc::pack2(-m_used, -m_used);
 #pragma unroll
-                    for (int i = 0; i < (128 - EMU) / 2; ++i) {
+                    for (int i = 0; i < (kHalf - kEmu) / 2; ++i) {
                         const uint64_t x2 = tc::fma2(tc::pack2(__uint_as_float(sr[2 * i]), __uint_as_float(sr[2 * i + 1])), c2, nm2);
                         float x0, x1;
                         tc::unpack2(x2, x0, x1);
@@ -468,7 +491,7 @@ attn_ptc_kernel(const __grid_constant__ TcArgs<MAXSETS> a) {
                         const __nv_bfloat162 pk = __floats2bfloat162_rn(e0, e1);
                         packed[i] = *reinterpret_cast<const uint32_t*>(&pk);
                     }
-                    if (EMU > 0) {
+                    if (kEmu > 0) {
                         // y = (S * c - m + 112) / 128 clamped to [0, 1]; 2^(128 y - 112) = 2^n * 2^f with
                         // n = round(128 y), f = 128 y - n; 2^n enters through the exponent bits.
                         const float k_emu = (kExpShift - m_used) * (1.0f / 128.0f);
@@ -478,7 +501,7 @@ attn_ptc_kernel(const __grid_constant__ TcArgs<MAXSETS> a) {
                         const uint64_t p0_2 = tc::pack2(kPoly0, kPoly0), p1_2 = tc::pack2(kPoly1, kPoly1);
                         const uint64_t p2_2 = tc::pack2(kPoly2, kPoly2), p3_2 = tc::pack2(kPoly3, kPoly3);
 #pragma unroll
-                        for (int i = (128 - EMU) / 2; i < 64; ++i) {
+                        for (int i = (kHalf - kEmu) / 2; i < kHalf / 2; ++i) {
                             const float y0 = tc::fma_sat(__uint_as_float(sr[2 * i]), c_emu, k_emu);
                             const float y1 = tc::fma_sat(__uint_as_float(sr[2 * i + 1]), c_emu, k_emu);
                             const uint64_t y2 = tc::pack2(y0, y1);
@@ -504,13 +527,12 @@ attn_ptc_kernel(const __grid_constant__ TcArgs<MAXSETS> a) {
                         tc::unpack2(s01, sa, sb);
                         l += sa + sb;
                     }
-                    tc::tmem_st32(tm_s[q] + lane_base, packed);
-                    tc::tmem_st32(tm_s[q] + lane_base + 32, packed + 32);
+                    tc::tmem_st32(ts, packed);
                     tc::wait_st();
                     tc::fence_before_sync();
-                    tc::mbar_arrive(bp);
+                    tc::mbar_arrive(tc::smem_u32(&bar_p_full[q][b]));
                 }
-                if (ok) ok = tc::mbar_wait(bo, (sp0 + nt - 1) & 1, abort_flag, kWaitLimit);
+                if (ok) ok = tc::mbar_wait(tc::smem_u32(&bar_item_done), item_cnt & 1, abort_flag, kWaitLimit);
                 if (ok) tc::fence_after_sync();
             }
 
@@ -614,6 +636,7 @@ attn_ptc_kernel(const __grid_constant__ TcArgs<MAXSETS> a) {
                 *abort_flag = 1;
             }
             if (active) sp0 += nt;
+            ++item_cnt;
             pos += nt;
             if (!end_of_item()) break;
         }
