@@ -15,15 +15,15 @@
 // Warp roles (384 threads): warps 0-3 and 4-7 are the two soft-max groups (thread = one query
 // row = one TMEM lane), warp 8 lane 0 drives TMA, warp 9 lane 0 issues every tcgen05.mma, warps
 // 10-11 only donate their registers.
-// A staged 128-key tile is consumed in two halves of 64 keys, and every query tile owns TWO score
-// buffers, so the scores of the next half are already in TMEM while the soft-max warps work on
-// the current one: four independent S -> P -> PV chains keep the tensor pipe and the soft-max
-// warps busy at the same time.
-// TMEM (512 columns): S[q][b] at (2 q + b) * 64 (64 fp32 columns each) | O0 | O1 at 256; the bf16
-// probabilities P overwrite the first half of their S buffer and feed the PV product straight
-// from TMEM.  Per half tile and query tile:
-//   S = Q K^T (smem x smem, N = 64)  ->  soft-max warps: running max (rescaling O only when the
-//   max moved by more than 2^8), P = exp2(S * c - m) -> TMEM  ->  O += P V (TMEM x smem).
+// TMEM (512 columns): S | P0 | P1 | O0 | O1.  There is ONE fp32 score buffer S (128 columns) that the
+// two query tiles use in turn: a soft-max group copies its scores into registers and hands the
+// buffer back at once, so the next QK^T never waits for the exponentials.  The bf16 probabilities
+// go to a buffer of their own (P0 / P1, 64 columns) and feed the PV product straight from TMEM.
+// Per key tile and query tile:
+//   S = Q K^T (smem x smem)  ->  soft-max warps: running max (rescaling O only when the max moved
+//   by more than 2^8), P = exp2(S * c - m) -> TMEM  ->  O += P V (TMEM x smem, V keys-major).
+// The MMA warp issues QK(1, j), PV(1, j - 1), QK(0, j + 1), PV(0, j) in that order, which keeps the
+// tensor pipe fed while each soft-max group spends a whole period on one tile.
 // The exponentials can be split between the special-function unit (ex2.approx) and a cubic
 // polynomial on the FMA pipe (one ex2 per score needs as many cycles as the MMAs).
 // Every mbarrier wait is bounded; on a timeout the CTA records FDD_ERR_DEVICE_TIMEOUT, drains
@@ -185,7 +185,7 @@ attn_ptc_kernel(const __grid_constant__ TcArgs<MAXSETS> a) {
     const uint32_t v_s = k_s + kStages * Shape::kTileBytes;
 
     __shared__ __align__(8) unsigned long long bar_q_full, bar_k_full[kStages], bar_k_empty[kStages],
-        bar_v_full[kStages], bar_v_empty[kStages], bar_s_full[2][2], bar_p_full[2][2], bar_o_done[2], bar_item_done;
+        bar_v_full[kStages], bar_v_empty[kStages], bar_s_full[2], bar_s_free[2], bar_p_full[2], bar_o_done[2], bar_item_done;
     __shared__ uint32_t tmem_base_s;
     __shared__ int abort_s, last_s;
     volatile int* abort_flag = &abort_s;
@@ -209,11 +209,10 @@ attn_ptc_kernel(const __grid_constant__ TcArgs<MAXSETS> a) {
             tc::mbar_init(tc::smem_u32(&bar_v_empty[s]), 1);
         }
         for (int q = 0; q < 2; ++q) {
-            for (int b = 0; b < 2; ++b) {
-                tc::mbar_init(tc::smem_u32(&bar_s_full[q][b]), 1);
-                tc::mbar_init(tc::smem_u32(&bar_p_full[q][b]), 128);
-            }
-            tc::mbar_init(tc::smem_u32(&bar_o_done[q]), 1);
+            tc::mbar_init(tc::smem_u32(&bar_s_full[q]), 1);     // scores of query tile q are in S
+            tc::mbar_init(tc::smem_u32(&bar_s_free[q]), 128);   // group q has copied them out of S
+            tc::mbar_init(tc::smem_u32(&bar_p_full[q]), 128);   // group q has written P[q]
+            tc::mbar_init(tc::smem_u32(&bar_o_done[q]), 1);     // a PV product of query tile q has completed
         }
         tc::fence_barrier_init();
     }
@@ -225,7 +224,8 @@ attn_ptc_kernel(const __grid_constant__ TcArgs<MAXSETS> a) {
     __syncthreads();
     tc::fence_after_sync();
     const uint32_t tmem = tmem_base_s;
-    const uint32_t tm_s[2][2] = {{tmem, tmem + 64}, {tmem + 128, tmem + 192}};
+    const uint32_t tm_s = tmem;
+    const uint32_t tm_p[2] = {tmem + 128, tmem + 192};
     const uint32_t tm_o[2] = {tmem + 256, tmem + 256 + D};
 
     // Each role runs its own copy of the item loop; all of them meet at the end of every item.
@@ -310,73 +310,99 @@ attn_ptc_kernel(const __grid_constant__ TcArgs<MAXSETS> a) {
             for (long long pos = range_begin; pos < range_end;) {
                 const ItemView v = view_item(pos);
                 const int nt = v.nt, NQ = v.NQ;
-                if (lane == 0) {
-                    constexpr uint32_t kIdescQK = tc::idesc_bf16(128, 64, 0);
+                {
+                    // The whole warp runs this loop with warp-uniform values (so that descriptors and
+                    // addresses can live in uniform registers); one elected lane issues the MMAs.
+                    constexpr uint32_t kIdescQK = tc::idesc_bf16(128, 128, 0);
                     constexpr uint32_t kIdescPV = tc::idesc_bf16(128, D, 1);
-                    // S[q][b] = Q[q] . K[keys 64 b .. 64 b + 63]^T
-                    auto issue_qk = [&](int q, int s, int b) {
+                    // Descriptors are built once; inside the loops an operand address is one addition
+                    // (the address field counts 16-byte units and never carries out of its 14 bits).
+                    const uint64_t dq0 = tc::smem_desc_sw128(q_s, 0, 1024);
+                    const uint64_t dk0 = tc::smem_desc_sw128(k_s, 0, 1024);
+                    const uint64_t dv0 = tc::smem_desc_sw128(v_s, Shape::kChunkBytes, 1024);
+                    // S = Q[q] . K^T
+                    auto issue_qk = [&](int q, int s) {
+                        const uint64_t dq = dq0 + static_cast<uint32_t>((q * Shape::kTileBytes) >> 4);
+                        const uint64_t dk = dk0 + static_cast<uint32_t>((s * Shape::kTileBytes) >> 4);
 #pragma unroll
                         for (int k = 0; k < D / 16; ++k) {
-                            const uint32_t off = (k >> 2) * Shape::kChunkBytes + (k & 3) * 32;
-                            tc::mma_ss(tm_s[q][b], tc::smem_desc_sw128(q_s + q * Shape::kTileBytes + off, 0, 1024),
-                                       tc::smem_desc_sw128(k_s + s * Shape::kTileBytes + b * 8192 + off, 0, 1024), kIdescQK, k > 0);
+                            const uint32_t off = ((k >> 2) * Shape::kChunkBytes + (k & 3) * 32) >> 4;
+                            if (k == 0) tc::mma_ss_first(tm_s, dq + off, dk + off, kIdescQK);
+                            else tc::mma_ss_acc(tm_s, dq + off, dk + off, kIdescQK);
                         }
                     };
-                    // O[q] (+)= P[q][b] . V[keys 64 b .. 64 b + 63]
-                    auto issue_pv = [&](int q, int s, int b, int accumulate) {
+                    // O[q] (+)= P[q] . V
+                    auto issue_pv = [&](int q, int s, bool accumulate) {
+                        const uint64_t dv = dv0 + static_cast<uint32_t>((s * Shape::kTileBytes) >> 4);
+                        if (accumulate) tc::mma_ts_acc(tm_o[q], tm_p[q], dv, kIdescPV);
+                        else tc::mma_ts_first(tm_o[q], tm_p[q], dv, kIdescPV);
 #pragma unroll
-                        for (int j = 0; j < 4; ++j)
-                            tc::mma_ts(tm_o[q], tm_s[q][b] + j * 8,
-                                       tc::smem_desc_sw128(v_s + s * Shape::kTileBytes + (b * 4 + j) * 2048, Shape::kChunkBytes, 1024),
-                                       kIdescPV, (accumulate || j > 0) ? 1u : 0u);
+                        for (int j = 1; j < kKeysPerTile / 16; ++j)
+                            tc::mma_ts_acc(tm_o[q], tm_p[q] + j * 8, dv + static_cast<uint32_t>((j * 2048) >> 4), kIdescPV);
                     };
-                    const int s0 = kv_cnt % kStages;
-                    bool ok = tc::mbar_wait(tc::smem_u32(&bar_q_full), item_cnt & 1, abort_flag, kWaitLimit);
-                    ok = ok && tc::mbar_wait(tc::smem_u32(&bar_k_full[s0]), (kv_cnt / kStages) & 1, abort_flag, kWaitLimit);
-                    if (ok) {
+                    auto stage_of = [&](int jl) { return static_cast<int>((kv_cnt + jl) % kStages); };
+                    auto phase_of = [&](int jl) { return ((kv_cnt + jl) / kStages) & 1u; };
+                    auto wait = [&](unsigned long long* bar, uint32_t parity) {
+                        return tc::mbar_wait(tc::smem_u32(bar), parity & 1u, abort_flag, kWaitLimit);
+                    };
+                    // PV(q, jl): needs V tile jl and P[q] of that tile
+                    auto do_pv = [&](int q, int jl, bool first_user_of_v, bool last_user_of_v) {
+                        const int s = stage_of(jl);
+                        bool good = true;
+                        if (first_user_of_v) good = wait(&bar_v_full[s], phase_of(jl));
+                        good = good && wait(&bar_p_full[q], sp_cnt[q] + jl);
+                        good = __shfl_sync(0xFFFFFFFFu, good ? 1 : 0, 0) != 0;
+                        if (!good) return false;
                         tc::fence_after_sync();
-                        for (int b = 0; b < 2; ++b)
-                            for (int q = 0; q < NQ; ++q) {
-                                issue_qk(q, s0, b);
-                                tc::mma_commit(tc::smem_u32(&bar_s_full[q][b]));
-                            }
-                        tc::mma_commit(tc::smem_u32(&bar_k_empty[s0]));
-                    }
-                    // The scores run one key tile ahead of the PV products.
-                    for (int jl = 0; jl < nt && ok; ++jl) {
-                        const uint32_t n = kv_cnt + jl;
-                        const int s = n % kStages;
-                        const uint32_t ph = (n / kStages) & 1;
-                        const bool has_next = jl + 1 < nt;
-                        const int sn = (n + 1) % kStages;
-                        const uint32_t phn = ((n + 1) / kStages) & 1;
-                        ok = tc::mbar_wait(tc::smem_u32(&bar_v_full[s]), ph, abort_flag, kWaitLimit);
-                        for (int b = 0; b < 2 && ok; ++b) {
-                            for (int q = 0; q < NQ && ok; ++q) {
-                                ok = tc::mbar_wait(tc::smem_u32(&bar_p_full[q][b]), (sp_cnt[q] + jl) & 1, abort_flag, kWaitLimit);
-                                if (!ok) break;
-                                tc::fence_after_sync();
-                                issue_pv(q, s, b, jl > 0 || b > 0);
-                                tc::mma_commit(tc::smem_u32(&bar_o_done[q]));
-                                if (has_next) {
-                                    if (q == 0 && b == 0) {
-                                        ok = tc::mbar_wait(tc::smem_u32(&bar_k_full[sn]), phn, abort_flag, kWaitLimit);
-                                        if (!ok) break;
-                                        tc::fence_after_sync();
-                                    }
-                                    issue_qk(q, sn, b);
-                                    tc::mma_commit(tc::smem_u32(&bar_s_full[q][b]));
-                                }
-                            }
+                        if (tc::elect_one()) {
+                            issue_pv(q, s, jl > 0);
+                            tc::mma_commit(tc::smem_u32(&bar_o_done[q]));
+                            if (last_user_of_v) tc::mma_commit(tc::smem_u32(&bar_v_empty[s]));
                         }
-                        if (!ok) break;
-                        tc::mma_commit(tc::smem_u32(&bar_v_empty[s]));
-                        if (has_next) tc::mma_commit(tc::smem_u32(&bar_k_empty[sn]));
+                        __syncwarp();
+                        return true;
+                    };
+                    // QK(q, jl) into S: needs K tile jl and S handed back by its previous reader
+                    auto do_qk = [&](int q, int jl, bool first_user_of_k, bool last_user_of_k, int prev_q, uint32_t prev_idx,
+                                     bool has_prev) {
+                        const int s = stage_of(jl);
+                        bool good = true;
+                        if (first_user_of_k) good = wait(&bar_k_full[s], phase_of(jl));
+                        if (has_prev) good = good && wait(&bar_s_free[prev_q], prev_idx);
+                        good = __shfl_sync(0xFFFFFFFFu, good ? 1 : 0, 0) != 0;
+                        if (!good) return false;
+                        tc::fence_after_sync();
+                        if (tc::elect_one()) {
+                            issue_qk(q, s);
+                            tc::mma_commit(tc::smem_u32(&bar_s_full[q]));
+                            if (last_user_of_k) tc::mma_commit(tc::smem_u32(&bar_k_empty[s]));
+                        }
+                        __syncwarp();
+                        return true;
+                    };
+                    bool ok = __shfl_sync(0xFFFFFFFFu, wait(&bar_q_full, item_cnt) ? 1 : 0, 0) != 0;
+                    if (NQ == 2) {
+                        // order: QK(0,0) | QK(1,j) PV(1,j-1) QK(0,j+1) PV(0,j) | ... | PV(1,nt-1)
+                        ok = ok && do_qk(0, 0, true, false, 0, 0, false);
+                        for (int jl = 0; jl < nt && ok; ++jl) {
+                            ok = do_qk(1, jl, false, true, 0, sp_cnt[0] + jl, true);
+                            if (ok && jl > 0) ok = do_pv(1, jl - 1, false, true);
+                            if (ok && jl + 1 < nt) ok = do_qk(0, jl + 1, true, false, 1, sp_cnt[1] + jl, true);
+                            if (ok) ok = do_pv(0, jl, true, false);
+                        }
+                        if (ok) ok = do_pv(1, nt - 1, false, true);
+                    } else {
+                        // order: QK(0,0) | QK(0,j+1) PV(0,j) | ...
+                        ok = ok && do_qk(0, 0, true, true, 0, 0, false);
+                        for (int jl = 0; jl < nt && ok; ++jl) {
+                            if (jl + 1 < nt) ok = do_qk(0, jl + 1, true, true, 0, sp_cnt[0] + jl, true);
+                            if (ok) ok = do_pv(0, jl, true, true);
+                        }
                     }
                     // One arrival per item once every MMA of the item has completed.  (bar_o_done cannot
                     // serve here: the scores run ahead, so a waiter could be two of its phases behind.)
-                    if (ok) tc::mma_commit(tc::smem_u32(&bar_item_done));
-                    if (!ok) {
+                    if (ok && tc::elect_one()) tc::mma_commit(tc::smem_u32(&bar_item_done));
+                    if (!ok && lane == 0) {
                         if (*abort_flag == 0) atomicCAS(a.status, 0, FDD_ERR_DEVICE_TIMEOUT);
                         *abort_flag = 1;
                     }
@@ -403,7 +429,7 @@ attn_ptc_kernel(const __grid_constant__ TcArgs<MAXSETS> a) {
         const int row_local = tid & 127;
         const uint32_t lane_base = (static_cast<uint32_t>(warp & 3) * 32u) << 16;
         const uint32_t bo = tc::smem_u32(&bar_o_done[q]);
-        uint32_t sp0 = 0;                   // key tiles this group has handled so far (two PV commits each)
+        uint32_t sp0 = 0;                   // key tiles this group has handled so far
         uint32_t item_cnt = 0;
         for (long long pos = range_begin; pos < range_end;) {
             const ItemView v = view_item(pos);
@@ -418,33 +444,32 @@ attn_ptc_kernel(const __grid_constant__ TcArgs<MAXSETS> a) {
             float m_used = -CUDART_INF_F, l = 0.0f;
             bool ok = true;
             if (active) {
-                constexpr int kHalf = 64;                   // keys per half tile
-                constexpr int kEmu = EMU / 2;               // emulated exponentials per half tile
                 const float c = a.scale_log2;
                 const uint64_t c2 = tc::pack2(c, c);
                 const float c_emu = c * (1.0f / 128.0f);
-                for (int hs = 0; hs < 2 * nt; ++hs) {
-                    const int jl = hs >> 1, b = hs & 1;
+                const uint32_t bs = tc::smem_u32(&bar_s_full[q]), bf = tc::smem_u32(&bar_s_free[q]);
+                const uint32_t bp = tc::smem_u32(&bar_p_full[q]);
+                for (int jl = 0; jl < nt; ++jl) {
                     const TileInfo t = tile_info(p, it.t0 + jl);
-                    ok = tc::mbar_wait(tc::smem_u32(&bar_s_full[q][b]), (sp0 + jl) & 1, abort_flag, kWaitLimit);
+                    ok = tc::mbar_wait(bs, (sp0 + jl) & 1, abort_flag, kWaitLimit);
                     if (!ok) break;
                     tc::fence_after_sync();
-                    const uint32_t ts = tm_s[q][b] + lane_base;
-                    uint32_t sr[kHalf];
-                    tc::tmem_ld32(ts, sr);
-                    tc::tmem_ld32(ts + 32, sr + 32);
-                    tc::wait_ld();
-                    int limit = t.nvalid;                               // keys [0, limit) of the tile are visible
-                    if (p.causal && t.segment == 2) limit = min(limit, qi - t.index * kKeysPerTile + 1);
-                    limit -= b * kHalf;                                 // ... of this half
-                    if (limit < kHalf) {
+                    uint32_t sr[128];
 #pragma unroll
-                        for (int i = 0; i < kHalf; ++i)
+                    for (int cc = 0; cc < 4; ++cc) tc::tmem_ld32(tm_s + lane_base + cc * 32, sr + cc * 32);
+                    tc::wait_ld();
+                    tc::fence_before_sync();
+                    tc::mbar_arrive(bf);                                // S may be overwritten now
+                    int limit = t.nvalid;                               // keys [0, limit) are visible
+                    if (p.causal && t.segment == 2) limit = min(limit, qi - t.index * kKeysPerTile + 1);
+                    if (limit < kKeysPerTile) {
+#pragma unroll
+                        for (int i = 0; i < 128; ++i)
                             if (i >= limit) sr[i] = 0xFF800000u;        // -inf
                     }
                     float mx[4] = {-CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F};
 #pragma unroll
-                    for (int i = 0; i < kHalf; i += 8) {
+                    for (int i = 0; i < 128; i += 8) {
 #pragma unroll
                         for (int u = 0; u < 4; ++u)
                             mx[u] = tc::max3(mx[u], __uint_as_float(sr[i + 2 * u]), __uint_as_float(sr[i + 2 * u + 1]));
@@ -452,14 +477,15 @@ attn_ptc_kernel(const __grid_constant__ TcArgs<MAXSETS> a) {
                     const float tmax = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
                     float m_tile = tmax * c;
                     if (!(m_tile > -CUDART_INF_F)) m_tile = m_used > -CUDART_INF_F ? m_used : 0.0f;
-                    if (hs == 0) {
+                    if (jl == 0) {
                         m_used = m_tile;
                     } else {
+                        // The previous PV of this query tile must be complete before P is overwritten
+                        // (and before O is rescaled).  It is one phase behind at most.
+                        ok = tc::mbar_wait(bo, (sp0 + jl - 1) & 1, abort_flag, kWaitLimit);
+                        if (!ok) break;
                         const bool need = m_tile > m_used + 8.0f;
                         if (__any_sync(0xFFFFFFFFu, need)) {
-                            // O holds every PV product up to the previous half: wait for that one, rescale
-                            ok = tc::mbar_wait(bo, (2 * sp0 + hs - 1) & 1, abort_flag, kWaitLimit);
-                            if (!ok) break;
                             tc::fence_after_sync();
                             const float alpha = need ? exp2f(m_used - m_tile) : 1.0f;
 #pragma unroll
@@ -476,13 +502,13 @@ attn_ptc_kernel(const __grid_constant__ TcArgs<MAXSETS> a) {
                             if (need) m_used = m_tile;
                         }
                     }
-                    // P = 2^(S * c - m): the first kHalf - kEmu scores through ex2.approx, the rest
+                    // P = 2^(S * c - m): the first 128 - EMU scores through ex2.approx, the rest
                     // through the polynomial; row sums in four packed accumulators.
                     uint64_t acc[4] = {0ull, 0ull, 0ull, 0ull};
-                    uint32_t packed[kHalf / 2];
+                    uint32_t packed[64];
                     const uint64_t nm2 = tc::pack2(-m_used, -m_used);
 #pragma unroll
-                    for (int i = 0; i < (kHalf - kEmu) / 2; ++i) {
+                    for (int i = 0; i < (128 - EMU) / 2; ++i) {
                         const uint64_t x2 = tc::fma2(tc::pack2(__uint_as_float(sr[2 * i]), __uint_as_float(sr[2 * i + 1])), c2, nm2);
                         float x0, x1;
                         tc::unpack2(x2, x0, x1);
@@ -491,7 +517,7 @@ attn_ptc_kernel(const __grid_constant__ TcArgs<MAXSETS> a) {
                         const __nv_bfloat162 pk = __floats2bfloat162_rn(e0, e1);
                         packed[i] = *reinterpret_cast<const uint32_t*>(&pk);
                     }
-                    if (kEmu > 0) {
+                    if (EMU > 0) {
                         // y = (S * c - m + 112) / 128 clamped to [0, 1]; 2^(128 y - 112) = 2^n * 2^f with
                         // n = round(128 y), f = 128 y - n; 2^n enters through the exponent bits.
                         const float k_emu = (kExpShift - m_used) * (1.0f / 128.0f);
@@ -501,7 +527,7 @@ attn_ptc_kernel(const __grid_constant__ TcArgs<MAXSETS> a) {
                         const uint64_t p0_2 = tc::pack2(kPoly0, kPoly0), p1_2 = tc::pack2(kPoly1, kPoly1);
                         const uint64_t p2_2 = tc::pack2(kPoly2, kPoly2), p3_2 = tc::pack2(kPoly3, kPoly3);
 #pragma unroll
-                        for (int i = (kHalf - kEmu) / 2; i < kHalf / 2; ++i) {
+                        for (int i = (128 - EMU) / 2; i < 64; ++i) {
                             const float y0 = tc::fma_sat(__uint_as_float(sr[2 * i]), c_emu, k_emu);
                             const float y1 = tc::fma_sat(__uint_as_float(sr[2 * i + 1]), c_emu, k_emu);
                             const uint64_t y2 = tc::pack2(y0, y1);
@@ -527,10 +553,11 @@ attn_ptc_kernel(const __grid_constant__ TcArgs<MAXSETS> a) {
                         tc::unpack2(s01, sa, sb);
                         l += sa + sb;
                     }
-                    tc::tmem_st32(ts, packed);
+                    tc::tmem_st32(tm_p[q] + lane_base, packed);
+                    tc::tmem_st32(tm_p[q] + lane_base + 32, packed + 32);
                     tc::wait_st();
                     tc::fence_before_sync();
-                    tc::mbar_arrive(tc::smem_u32(&bar_p_full[q][b]));
+                    tc::mbar_arrive(bp);
                 }
                 if (ok) ok = tc::mbar_wait(tc::smem_u32(&bar_item_done), item_cnt & 1, abort_flag, kWaitLimit);
                 if (ok) tc::fence_after_sync();
