@@ -13,8 +13,9 @@
 // nobody waits) merges the pieces and writes the bf16 rows.
 //
 // Warp roles (384 threads): warps 0-3 and 4-7 are the two soft-max groups (thread = one query
-// row = one TMEM lane), warp 8 lane 0 drives TMA, warp 9 lane 0 issues every tcgen05.mma, warps
-// 10-11 only donate their registers.
+// row = one TMEM lane), warp 8 lane 0 drives TMA, warps 9 and 10 issue the tcgen05.mma (one lane each:
+// warp 9 the score products, warp 10 the output products), warp
+// 11 only donates its registers.
 // TMEM (512 columns): S | P0 | P1 | O0 | O1.  There is ONE fp32 score buffer S (128 columns) that the
 // two query tiles use in turn: a soft-max group copies its scores into registers and hands the
 // buffer back at once, so the next QK^T never waits for the exponentials.  The bf16 probabilities
@@ -264,16 +265,20 @@ attn_ptc_kernel(const __grid_constant__ TcArgs<MAXSETS> a) {
             uint32_t kv_cnt = 0;            // K/V tiles staged so far: ring stage and phase carry over between items
             for (long long pos = range_begin; pos < range_end;) {
                 const ItemView v = view_item(pos);
-                if (lane == 0) {
+                {
+                    // warp-uniform loop, one elected lane issues the copies
                     const SetParams& p = a.sets[v.it.s];
                     const TcSetMaps& maps = a.maps[v.it.s];
-                    tc::prefetch_tmap(&maps.q);
                     const uint32_t bq = tc::smem_u32(&bar_q_full);
-                    tc::mbar_arrive_expect_tx(bq, v.NQ * Shape::kTileBytes);
-                    for (int q = 0; q < v.NQ; ++q)
-                        for (int ch = 0; ch < Shape::kChunks; ++ch)
-                            tc::tma_load_4d(q_s + q * Shape::kTileBytes + ch * Shape::kChunkBytes, &maps.q, bq, ch * 64,
-                                            v.h * p.G, (v.rp * 2 + q) * (128 / p.G), v.f);
+                    if (tc::elect_one()) {
+                        tc::prefetch_tmap(&maps.q);
+                        tc::mbar_arrive_expect_tx(bq, v.NQ * Shape::kTileBytes);
+                        for (int q = 0; q < v.NQ; ++q)
+                            for (int ch = 0; ch < Shape::kChunks; ++ch)
+                                tc::tma_load_4d(q_s + q * Shape::kTileBytes + ch * Shape::kChunkBytes, &maps.q, bq, ch * 64,
+                                                v.h * p.G, (v.rp * 2 + q) * (128 / p.G), v.f);
+                    }
+                    __syncwarp();
                     bool ok = true;
                     for (int jl = 0; jl < v.nt && ok; ++jl) {
                         const TileInfo t = tile_info(p, v.it.t0 + jl);
@@ -283,15 +288,23 @@ attn_ptc_kernel(const __grid_constant__ TcArgs<MAXSETS> a) {
                         const CUtensorMap* mk = t.segment == 0 ? &maps.pk : (t.segment == 1 ? &maps.sk : &maps.bk);
                         const CUtensorMap* mv = t.segment == 0 ? &maps.pv : (t.segment == 1 ? &maps.sv : &maps.bv);
                         ok = tc::mbar_wait(tc::smem_u32(&bar_k_empty[s]), ph ^ 1, abort_flag, kWaitLimit);
+                        ok = __shfl_sync(0xFFFFFFFFu, ok ? 1 : 0, 0) != 0;
                         if (!ok) break;
-                        tc::mbar_arrive_expect_tx(tc::smem_u32(&bar_k_full[s]), Shape::kTileBytes);
-                        load_kv_tile<D>(p, mk, &maps.pk_tail, t, k_s + s * Shape::kTileBytes, tc::smem_u32(&bar_k_full[s]), v.h, v.f);
+                        if (tc::elect_one()) {
+                            tc::mbar_arrive_expect_tx(tc::smem_u32(&bar_k_full[s]), Shape::kTileBytes);
+                            load_kv_tile<D>(p, mk, &maps.pk_tail, t, k_s + s * Shape::kTileBytes, tc::smem_u32(&bar_k_full[s]), v.h, v.f);
+                        }
+                        __syncwarp();
                         ok = tc::mbar_wait(tc::smem_u32(&bar_v_empty[s]), ph ^ 1, abort_flag, kWaitLimit);
+                        ok = __shfl_sync(0xFFFFFFFFu, ok ? 1 : 0, 0) != 0;
                         if (!ok) break;
-                        tc::mbar_arrive_expect_tx(tc::smem_u32(&bar_v_full[s]), Shape::kTileBytes);
-                        load_kv_tile<D>(p, mv, &maps.pv_tail, t, v_s + s * Shape::kTileBytes, tc::smem_u32(&bar_v_full[s]), v.h, v.f);
+                        if (tc::elect_one()) {
+                            tc::mbar_arrive_expect_tx(tc::smem_u32(&bar_v_full[s]), Shape::kTileBytes);
+                            load_kv_tile<D>(p, mv, &maps.pv_tail, t, v_s + s * Shape::kTileBytes, tc::smem_u32(&bar_v_full[s]), v.h, v.f);
+                        }
+                        __syncwarp();
                     }
-                    if (!ok) {
+                    if (!ok && lane == 0) {
                         if (*abort_flag == 0) atomicCAS(a.status, 0, FDD_ERR_DEVICE_TIMEOUT);
                         *abort_flag = 1;
                         const long long t0 = clock64();          // let copies already in flight land
@@ -303,8 +316,12 @@ attn_ptc_kernel(const __grid_constant__ TcArgs<MAXSETS> a) {
                 pos += v.nt;
                 if (!end_of_item()) break;
             }
-        } else if (warp == 9) {
-            // ------------------------------------------------------------------ MMA issuer
+        } else if (warp == 9 || warp == 10) {
+            // ------------------------------------------------------------------ MMA issuers
+            // Warp 9 issues every QK^T, warp 10 every PV: while one of them checks the barriers of its
+            // next product, the other one's MMAs keep the tensor pipe busy.  Nothing orders the two
+            // streams against each other but the barriers (S handed back, P written).
+            const bool qk_role = warp == 9;
             uint32_t kv_cnt = 0, item_cnt = 0;
             uint32_t sp_cnt[2] = {0, 0};    // key tiles handled so far per query tile
             for (long long pos = range_begin; pos < range_end;) {
@@ -380,28 +397,27 @@ attn_ptc_kernel(const __grid_constant__ TcArgs<MAXSETS> a) {
                         __syncwarp();
                         return true;
                     };
-                    bool ok = __shfl_sync(0xFFFFFFFFu, wait(&bar_q_full, item_cnt) ? 1 : 0, 0) != 0;
-                    if (NQ == 2) {
-                        // order: QK(0,0) | QK(1,j) PV(1,j-1) QK(0,j+1) PV(0,j) | ... | PV(1,nt-1)
-                        ok = ok && do_qk(0, 0, true, false, 0, 0, false);
+                    bool ok = true;
+                    if (qk_role) {
+                        // scores: QK(0,0) | QK(1,j) QK(0,j+1) | ...   (S is one buffer: each product waits
+                        // until the group that owned the previous scores has copied them out)
+                        ok = __shfl_sync(0xFFFFFFFFu, wait(&bar_q_full, item_cnt) ? 1 : 0, 0) != 0;
+                        ok = ok && do_qk(0, 0, true, NQ == 1, 0, 0, false);
                         for (int jl = 0; jl < nt && ok; ++jl) {
-                            ok = do_qk(1, jl, false, true, 0, sp_cnt[0] + jl, true);
-                            if (ok && jl > 0) ok = do_pv(1, jl - 1, false, true);
-                            if (ok && jl + 1 < nt) ok = do_qk(0, jl + 1, true, false, 1, sp_cnt[1] + jl, true);
-                            if (ok) ok = do_pv(0, jl, true, false);
+                            if (NQ == 2) ok = do_qk(1, jl, false, true, 0, sp_cnt[0] + jl, true);
+                            if (ok && jl + 1 < nt) ok = do_qk(0, jl + 1, true, NQ == 1, NQ - 1, sp_cnt[NQ - 1] + jl, true);
                         }
-                        if (ok) ok = do_pv(1, nt - 1, false, true);
                     } else {
-                        // order: QK(0,0) | QK(0,j+1) PV(0,j) | ...
-                        ok = ok && do_qk(0, 0, true, true, 0, 0, false);
+                        // outputs: PV(1,j-1) PV(0,j) | ... | PV(1,nt-1), in the order the P tiles appear
                         for (int jl = 0; jl < nt && ok; ++jl) {
-                            if (jl + 1 < nt) ok = do_qk(0, jl + 1, true, true, 0, sp_cnt[0] + jl, true);
-                            if (ok) ok = do_pv(0, jl, true, true);
+                            if (NQ == 2 && jl > 0) ok = do_pv(1, jl - 1, false, true);
+                            if (ok) ok = do_pv(0, jl, true, NQ == 1);
                         }
+                        if (ok && NQ == 2) ok = do_pv(1, nt - 1, false, true);
+                        // One arrival per item once every PV (hence every MMA) of the item has completed.
+                        // (bar_o_done cannot serve here: a waiter could be two of its phases behind.)
+                        if (ok && tc::elect_one()) tc::mma_commit(tc::smem_u32(&bar_item_done));
                     }
-                    // One arrival per item once every MMA of the item has completed.  (bar_o_done cannot
-                    // serve here: the scores run ahead, so a waiter could be two of its phases behind.)
-                    if (ok && tc::elect_one()) tc::mma_commit(tc::smem_u32(&bar_item_done));
                     if (!ok && lane == 0) {
                         if (*abort_flag == 0) atomicCAS(a.status, 0, FDD_ERR_DEVICE_TIMEOUT);
                         *abort_flag = 1;
@@ -477,15 +493,18 @@ attn_ptc_kernel(const __grid_constant__ TcArgs<MAXSETS> a) {
                     const float tmax = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
                     float m_tile = tmax * c;
                     if (!(m_tile > -CUDART_INF_F)) m_tile = m_used > -CUDART_INF_F ? m_used : 0.0f;
+                    // The previous PV of this query tile must be complete before P is overwritten and
+                    // before O is rescaled (it is one phase behind at most).  Usually only the first
+                    // matters, so the wait sits after the exponentials.
+                    bool pv_done = jl == 0;
                     if (jl == 0) {
                         m_used = m_tile;
                     } else {
-                        // The previous PV of this query tile must be complete before P is overwritten
-                        // (and before O is rescaled).  It is one phase behind at most.
-                        ok = tc::mbar_wait(bo, (sp0 + jl - 1) & 1, abort_flag, kWaitLimit);
-                        if (!ok) break;
                         const bool need = m_tile > m_used + 8.0f;
                         if (__any_sync(0xFFFFFFFFu, need)) {
+                            ok = tc::mbar_wait(bo, (sp0 + jl - 1) & 1, abort_flag, kWaitLimit);
+                            if (!ok) break;
+                            pv_done = true;
                             tc::fence_after_sync();
                             const float alpha = need ? exp2f(m_used - m_tile) : 1.0f;
 #pragma unroll
@@ -552,6 +571,11 @@ attn_ptc_kernel(const __grid_constant__ TcArgs<MAXSETS> a) {
                         float sa, sb;
                         tc::unpack2(s01, sa, sb);
                         l += sa + sb;
+                    }
+                    if (!pv_done) {
+                        ok = tc::mbar_wait(bo, (sp0 + jl - 1) & 1, abort_flag, kWaitLimit);
+                        if (!ok) break;
+                        tc::fence_after_sync();
                     }
                     tc::tmem_st32(tm_p[q] + lane_base, packed);
                     tc::tmem_st32(tm_p[q] + lane_base + 32, packed + 32);
