@@ -8,7 +8,8 @@ generator.  The reading used by this repository: Philox4x32 with 10 rounds
 SC'11), keyed by the rollout's 64-bit seed, with the counter made of the
 vocabulary index, the position inside the block, the denoising step and the
 block index, so that a draw depends on nothing but (seed, block, step,
-position, vocabulary id).
+position, vocabulary id).  Each uniform is assembled from two streams: an 8-bit
+coarse value (16 ids per Philox block) and 23 fine bits (4 ids per block).
 
 Two implementations live here on purpose: a scalar one on Python integers that
 follows the published round function literally, and a numpy one used for whole
@@ -69,28 +70,59 @@ def philox4x32_vec(c0, c1, c2, c3, k0, k1, rounds=10):
     return c0, c1, c2, c3
 
 
-def uniform_from_word(x):
-    """Map a 32-bit word to the open interval (0, 1).
+FINE_STREAM = 1 << 31   # added to the position word of the counter for the second stream
 
-    u = ((x >> 9) + 0.5) * 2**-23: the top 23 bits, centred in their bin.  Every
-    value is exactly representable in fp32 as well as fp64 (24 significant
-    bits), lies in [2**-24, 1 - 2**-24], and so -ln(-ln(u)) is always finite.
+
+def uniform_from_parts(coarse, fine):
+    """Map an 8-bit coarse value and a 23-bit fine value to the open interval (0, 1).
+
+    u = (coarse + (fine + 0.5) * 2**-23) / 256: the coarse byte picks one of 256
+    equal bins, the fine bits a point inside it, centred in its sub-bin.  u is a
+    multiple of 2**-32 in [2**-32, 1 - 2**-32], so -ln(-ln(u)) is always finite
+    (between -3.1 and 22.2).
     """
-    x = np.asarray(x, dtype=np.uint64)
-    return ((x >> np.uint64(9)).astype(np.float64) + 0.5) * (2.0 ** -23)
+    coarse = np.asarray(coarse, dtype=np.float64)
+    fine = np.asarray(fine, dtype=np.float64)
+    return (coarse + (fine + 0.5) * (2.0 ** -23)) / 256.0
 
 
-def gumbel_row(seed, block_idx, step, position, vocab):
-    """Standard Gumbel noise g[v] = -ln(-ln(u[v])) for one row of a block.
-
-    Counter = (v // 4, position, step, block_idx), key = (seed low word, seed
-    high word); vocabulary id v takes output word v % 4 of its counter.
-    """
+def coarse_bytes(seed, block_idx, step, position, vocab):
+    """The coarse byte of every vocabulary id of one row: id v takes byte v % 16
+    (little-endian inside the four output words) of the Philox block with
+    counter (v // 16, position, step, block_idx)."""
     seed = int(seed) & 0xFFFFFFFFFFFFFFFF
-    nctr = (vocab + 3) // 4
+    nctr = (vocab + 15) // 16
     ctr = np.arange(nctr, dtype=np.uint64)
     w = philox4x32_vec(ctr, np.uint64(position), np.uint64(step), np.uint64(block_idx),
                        seed & MASK32, seed >> 32)
+    words = np.stack(w, axis=1).reshape(-1)                       # word k of block c at 4 c + k
+    shifts = np.array([0, 8, 16, 24], dtype=np.uint64)
+    return ((words[:, None] >> shifts[None, :]) & np.uint64(0xFF)).reshape(-1)[:vocab]
+
+
+def fine_bits(seed, block_idx, step, position, vocab):
+    """The 23 fine bits of every vocabulary id of one row: id v takes the top 23
+    bits of word v % 4 of the Philox block with counter
+    (v // 4, position + 2**31, step, block_idx) (a second stream: the position
+    word never reaches 2**31 otherwise)."""
+    seed = int(seed) & 0xFFFFFFFFFFFFFFFF
+    nctr = (vocab + 3) // 4
+    ctr = np.arange(nctr, dtype=np.uint64)
+    w = philox4x32_vec(ctr, np.uint64(position + FINE_STREAM), np.uint64(step), np.uint64(block_idx),
+                       seed & MASK32, seed >> 32)
     words = np.stack(w, axis=1).reshape(-1)[:vocab]
-    u = uniform_from_word(words)
+    return words >> np.uint64(9)
+
+
+def gumbel_row(seed, block_idx, step, position, vocab):
+    """Standard Gumbel noise g[v] = -ln(-ln(u[v])) for one row of a block, with
+    u[v] = uniform_from_parts(coarse byte of v, fine bits of v).  A draw depends
+    on nothing but (seed, block, step, position, vocabulary id).
+
+    The uniform is split in two so that an implementation can bound a draw from
+    its coarse byte alone (one Philox block per 16 ids) and spend the second
+    Philox block only on the few ids whose bound can still win the arg-max.
+    """
+    u = uniform_from_parts(coarse_bytes(seed, block_idx, step, position, vocab),
+                           fine_bits(seed, block_idx, step, position, vocab))
     return -np.log(-np.log(u))

@@ -269,6 +269,10 @@ fdd_status fdd_unmask(fdd_ctx* ctx, fdd_forkset* const* sets, int n_sets, const 
         return fail(ctx, FDD_ERR_INVALID_ARG, "logits/tokens/state/n_committed/n_left is NULL");
     if (!(temperature >= 0.0f)) return fail(ctx, FDD_ERR_INVALID_ARG, "temperature must be >= 0");
     if (threshold != threshold) return fail(ctx, FDD_ERR_INVALID_ARG, "threshold is NaN");
+    for (int s = 0; s < n_sets; ++s)
+        if (sets[s]->n_forks * block_len[s] > kUnmaskMaxRows)
+            return fail(ctx, FDD_ERR_CAPACITY, "set %d: %d rollouts x %d positions exceed %d rows per set", s,
+                        sets[s]->n_forks, block_len[s], kUnmaskMaxRows);
     const fdd_config& c = ctx->cfg;
     const size_t esz = c.logits_dtype == FDD_LOGITS_BF16 ? 2 : 4;
     size_t row_off = 0;

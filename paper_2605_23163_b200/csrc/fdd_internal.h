@@ -103,7 +103,8 @@ struct UnmaskPartial {
     int pad[3];
 };
 
-static constexpr int kUnmaskChunk = 8192;   // vocabulary entries per CTA
+static constexpr int kUnmaskChunk = 8192;   // vocabulary entries per work item
+static constexpr int kUnmaskMaxRows = 4096; // rollouts x positions of one set (the kernel compacts them in shared memory)
 static inline int unmask_chunks(int vocab) { return (vocab + kUnmaskChunk - 1) / kUnmaskChunk; }
 
 cudaError_t launch_attention_simple(const AttnProblem& p, int head_dim, cudaStream_t st);

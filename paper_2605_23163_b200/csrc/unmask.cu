@@ -1,10 +1,22 @@
 // Confidence-threshold parallel unmasking: vocabulary-wide soft-max statistics and
 // (Gumbel-perturbed) arg-max per MASKED row, then the per-rollout commit rule.
 //
-// Kernel 1 (unmask_partial_kernel): one CTA per (row, chunk).  A CTA streams one chunk of one
-// row of logits from HBM exactly once with 16-byte loads, keeps it in registers, and
-// reduces it to (max, sum exp, best perturbed score, its vocabulary id and logit).  Rows
-// whose position is not MASKED exit at once, so only the rows the method needs are read.
+// Kernel 1 (unmask_partial_kernel): a persistent grid walks the (MASKED row, 8192-logit chunk)
+// pairs of the call.  A CTA streams its chunk from HBM exactly once with 32-byte loads (16
+// consecutive logits per thread and load), keeps it in registers and reduces it to (max, sum exp,
+// best perturbed score, its vocabulary id and logit).  Rows that are not MASKED are never read.
+//
+// Noise (temperature > 0).  The uniform behind every Gumbel draw has two parts: a coarse byte c
+// (one Philox block serves 16 vocabulary ids) and 23 fine bits (one block per 4 ids).  The byte
+// alone bounds the draw, g < -ln(-ln((c + 1) / 256)) for c < 255, which is what makes the
+// kernel cheap: every id gets its coarse byte, but the second Philox block and the two
+// logarithms are spent only on
+//   (1) the ids with c = 255 (one in 256), whose best exact score L is a lower bound of the
+//       chunk's best score, and
+//   (2) the ids of threads whose largest logit could still beat L with the largest draw a
+//       byte below 255 allows (g < 5.5433), filtered once more by their own byte's bound.
+// Any id left out cannot reach L, so the arg-max (lowest id on ties) is exact.
+//
 // Kernel 2 (unmask_finalize_kernel): one CTA per rollout merges the chunk records of its
 // rows, forms the confidences and applies the threshold / at-least-one rule.
 #include "fdd_internal.h"
@@ -15,9 +27,15 @@ namespace {
 
 constexpr int kThreads = 256;
 constexpr int kPerThread = kUnmaskChunk / kThreads;   // 32 vocabulary entries per thread
+constexpr int kGroup = 16;                            // consecutive entries per load and per coarse Philox block
+constexpr int kGroups = kPerThread / kGroup;          // 2
+constexpr int kMaxCand = 1024;                        // c = 255 ids kept per chunk (32 expected)
+constexpr int kMaxRows = kUnmaskMaxRows;               // rows whose state fits the CTA's compaction buffer
+constexpr float kGumbelBelow255 = 5.5440f;            // > -ln(-ln(255/256)) = 5.54322, with rounding slack
 
 constexpr uint32_t kPhiloxM0 = 0xD2511F53u, kPhiloxM1 = 0xCD9E8D57u;
 constexpr uint32_t kPhiloxW0 = 0x9E3779B9u, kPhiloxW1 = 0xBB67AE85u;
+constexpr uint32_t kFineStream = 0x80000000u;         // added to the position word for the fine bits
 
 // Philox4x32 with 10 rounds (Salmon et al., SC'11), written from the published round function.
 __device__ __forceinline__ uint4 philox4x32_10(uint4 c, uint2 k) {
@@ -31,31 +49,55 @@ __device__ __forceinline__ uint4 philox4x32_10(uint4 c, uint2 k) {
     return c;
 }
 
-// g = -ln(-ln(u)), u = (k + 0.5) * 2^-23 with k the top 23 bits of the word; u is exact in fp32.
-__device__ __forceinline__ float gumbel_from_bits(uint32_t k23) {
-    const float u = (static_cast<float>(k23) + 0.5f) * 1.1920928955078125e-07f;
-    return -logf(-logf(u));
+// g = -ln(-ln(u)), u = (c + (f + 0.5) 2^-23) / 256.  Near u = 1 the inner logarithm goes through
+// 1 - u, which fp32 holds almost exactly there.
+__device__ __forceinline__ float gumbel_exact(uint32_t c, uint32_t f23) {
+    float inner;                                        // -ln(u) > 0
+    if (c >= 128u) {
+        const float y = (static_cast<float>(255u - c) + (8388608.0f - static_cast<float>(f23) - 0.5f) * 1.1920928955078125e-07f)
+                        * 0.00390625f;                  // 1 - u
+        inner = -log1pf(-y);
+    } else {
+        const float a = static_cast<float>(c) + (static_cast<float>(f23) + 0.5f) * 1.1920928955078125e-07f;   // 256 u
+        inner = 5.545177444479562f - logf(a);
+    }
+    return -logf(inner);
 }
 
-template <typename T> struct LogitVec;
-template <> struct LogitVec<__nv_bfloat16> {
-    static constexpr int kVec = 8;
-    __device__ static void load(const __nv_bfloat16* p, float* out) {
-        const uint4 raw = __ldcs(reinterpret_cast<const uint4*>(p));
-        const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
+// Upper bound of the draws with coarse byte c < 255 (c = 255 has no useful bound).
+__device__ __forceinline__ float gumbel_bound(uint32_t c) {
+    return -logf(-logf(static_cast<float>(c + 1u) * 0.00390625f)) + 1e-3f;
+}
+
+__device__ __forceinline__ void load32(const void* p, uint32_t (&r)[8]) {
+    asm volatile("ld.global.L1::no_allocate.v8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
+                 : "l"(p));
+}
+
+template <typename T> struct Logit;
+template <> struct Logit<__nv_bfloat16> {
+    // 16 consecutive logits from one 32-byte load
+    __device__ static void load16(const __nv_bfloat16* p, float* out) {
+        uint32_t w[8];
+        load32(p, w);
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
+        for (int i = 0; i < 8; ++i) {
             out[2 * i] = __uint_as_float(w[i] << 16);
             out[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u);
         }
     }
     __device__ static float load1(const __nv_bfloat16* p) { return __bfloat162float(*p); }
 };
-template <> struct LogitVec<float> {
-    static constexpr int kVec = 4;
-    __device__ static void load(const float* p, float* out) {
-        const float4 raw = __ldcs(reinterpret_cast<const float4*>(p));
-        out[0] = raw.x; out[1] = raw.y; out[2] = raw.z; out[3] = raw.w;
+template <> struct Logit<float> {
+    __device__ static void load16(const float* p, float* out) {
+        uint32_t w[8];
+        load32(p, w);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) out[i] = __uint_as_float(w[i]);
+        load32(p + 8, w);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) out[8 + i] = __uint_as_float(w[i]);
     }
     __device__ static float load1(const float* p) { return *p; }
 };
@@ -69,124 +111,211 @@ __device__ __forceinline__ Best better(const Best& a, const Best& b) {
     if (b.score > a.score || (b.score == a.score && b.index < a.index)) return b;
     return a;
 }
+__device__ __forceinline__ Best warp_best(Best b) {
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) {
+        Best o;
+        o.score = __shfl_xor_sync(0xFFFFFFFFu, b.score, off);
+        o.logit = __shfl_xor_sync(0xFFFFFFFFu, b.logit, off);
+        o.index = __shfl_xor_sync(0xFFFFFFFFu, b.index, off);
+        b = better(b, o);
+    }
+    return b;
+}
 
 template <typename T>
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kThreads, 3)
 unmask_partial_kernel(const T* __restrict__ logits, const uint8_t* __restrict__ state,
                       const uint64_t* __restrict__ seeds, UnmaskPartial* __restrict__ partial,
-                      int d, int vocab, int n_chunks, float temperature,
+                      int rows, int d, int vocab, int n_chunks, float temperature,
                       uint32_t block_idx, uint32_t step, int vec_ok) {
-    const int row = blockIdx.x / n_chunks;
-    if (state[row] != FDD_MASKED) return;
-    const int chunk = blockIdx.x - row * n_chunks;
-    const int tid = threadIdx.x;
-    constexpr int kVec = LogitVec<T>::kVec;
-    constexpr int kIter = kPerThread / kVec;
-
-    __shared__ float g_upper[256];     // upper bound of the Gumbel value per top-8-bit bin
-    __shared__ float red_max[kThreads / 32], red_sum[kThreads / 32];
+    __shared__ uint16_t s_rows[kMaxRows];               // MASKED rows, ascending
+    __shared__ int s_n_rows;
+    __shared__ int s_warp_count[kThreads / 32];
+    __shared__ uint16_t s_cand[kMaxCand];               // chunk-local ids with coarse byte 255
+    __shared__ int s_n_cand;
+    __shared__ float red_max[kThreads / 32], red_sum[kThreads / 32], red_score[kThreads / 32];
     __shared__ Best red_best[kThreads / 32];
 
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const bool noisy = temperature != 0.0f;
-    if (noisy) {
-        const uint32_t k_hi = ((static_cast<uint32_t>(tid) + 1u) << 15) - 1u;
-        g_upper[tid] = gumbel_from_bits(k_hi) + 1e-3f;
-    }
 
-    const T* row_ptr = logits + static_cast<size_t>(row) * vocab;
-    const int chunk_base = chunk * kUnmaskChunk;
-
-    float val[kPerThread];
-#pragma unroll
-    for (int it = 0; it < kIter; ++it) {
-        const int v0 = chunk_base + (it * kThreads + tid) * kVec;
-        if (vec_ok && v0 + kVec <= vocab) {
-            LogitVec<T>::load(row_ptr + v0, &val[it * kVec]);
-        } else {
-#pragma unroll
-            for (int j = 0; j < kVec; ++j)
-                val[it * kVec + j] = (v0 + j < vocab) ? LogitVec<T>::load1(row_ptr + v0 + j) : -CUDART_INF_F;
+    // Every CTA compacts the list of MASKED rows for itself (the state array is a few KB).
+    {
+        int base = 0;
+        for (int r0 = 0; r0 < rows; r0 += kThreads) {
+            const int r = r0 + tid;
+            const bool m = r < rows && state[r] == FDD_MASKED;
+            const unsigned bal = __ballot_sync(0xFFFFFFFFu, m);
+            if (lane == 0) s_warp_count[warp] = __popc(bal);
+            __syncthreads();
+            int before = base;
+            for (int w2 = 0; w2 < warp; ++w2) before += s_warp_count[w2];
+            if (m) s_rows[before + __popc(bal & ((1u << lane) - 1u))] = static_cast<uint16_t>(r);
+            for (int w2 = 0; w2 < kThreads / 32; ++w2) base += s_warp_count[w2];
+            __syncthreads();
         }
+        if (tid == 0) s_n_rows = base;
+        __syncthreads();
     }
+    const int n_items = s_n_rows * n_chunks;
 
-    float m = -CUDART_INF_F;
-#pragma unroll
-    for (int i = 0; i < kPerThread; ++i) m = fmaxf(m, val[i]);
-    float s = 0.0f;
-    if (m > -CUDART_INF_F) {
-#pragma unroll
-        for (int i = 0; i < kPerThread; ++i) s += __expf(val[i] - m);
-    }
+    for (int item = blockIdx.x; item < n_items; item += gridDim.x) {
+        const int row = s_rows[item / n_chunks];
+        const int chunk = item - (item / n_chunks) * n_chunks;
+        const T* row_ptr = logits + static_cast<size_t>(row) * vocab;
+        const int chunk_base = chunk * kUnmaskChunk;
+        if (tid == 0) s_n_cand = 0;
 
-    Best best{-CUDART_INF_F, -CUDART_INF_F, 0x7FFFFFFF};
-    if (!noisy) {
+        // ---- stream the chunk: 2 x 16 consecutive logits per thread
+        float val[kPerThread];
 #pragma unroll
-        for (int it = 0; it < kIter; ++it) {
+        for (int g = 0; g < kGroups; ++g) {
+            const int v0 = chunk_base + (g * kThreads + tid) * kGroup;
+            if (vec_ok && v0 + kGroup <= vocab) {
+                Logit<T>::load16(row_ptr + v0, &val[g * kGroup]);
+            } else {
 #pragma unroll
-            for (int j = 0; j < kVec; ++j) {
-                const float l = val[it * kVec + j];
-                if (l > best.score) best = Best{l, l, chunk_base + (it * kThreads + tid) * kVec + j};
+                for (int j = 0; j < kGroup; ++j)
+                    val[g * kGroup + j] = (v0 + j < vocab) ? Logit<T>::load1(row_ptr + v0 + j) : -CUDART_INF_F;
             }
         }
-    } else {
-        __syncthreads();                       // g_upper ready
-        const int fork = row / d, pos = row - fork * d;
-        const uint64_t seed = seeds[fork];
-        const uint2 key = make_uint2(static_cast<uint32_t>(seed), static_cast<uint32_t>(seed >> 32));
+
+        // ---- soft-max statistics of the thread's 32 logits
+        float m = -CUDART_INF_F;
 #pragma unroll
-        for (int it = 0; it < kIter; ++it) {
-            const int v0 = chunk_base + (it * kThreads + tid) * kVec;
+        for (int i = 0; i < kPerThread; ++i) m = fmaxf(m, val[i]);
+        float s = 0.0f;
+        if (m > -CUDART_INF_F) {
+            const float ml = m * 1.4426950408889634f;
+            float s4[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-            for (int q4 = 0; q4 < kVec / 4; ++q4) {
-                const int vq = v0 + q4 * 4;
-                if (vq >= vocab) continue;
-                const uint4 r = philox4x32_10(make_uint4(static_cast<uint32_t>(vq >> 2), pos, step, block_idx), key);
-                const uint32_t w[4] = {r.x, r.y, r.z, r.w};
+            for (int i = 0; i < kPerThread; ++i) s4[i & 3] += exp2f(fmaf(val[i], 1.4426950408889634f, -ml));
+            s = (s4[0] + s4[1]) + (s4[2] + s4[3]);
+        }
+
+        Best best{-CUDART_INF_F, -CUDART_INF_F, 0x7FFFFFFF};
+        if (!noisy) {
+            // arg-max of the logits themselves; the thread maximum is known, find its first place
+            if (m > -CUDART_INF_F) {
+                int at = kPerThread;
 #pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    const float l = val[it * kVec + q4 * 4 + j];
-                    const uint32_t k23 = w[j] >> 9;
-                    // cheap test first: even the largest Gumbel value of this bin cannot reach the best
-                    const float bound = fmaf(temperature, g_upper[k23 >> 15], l);
-                    if (bound >= best.score && l > -CUDART_INF_F) {
-                        const float sc = fmaf(temperature, gumbel_from_bits(k23), l);
-                        if (sc > best.score) best = Best{sc, l, vq + j};
+                for (int i = kPerThread - 1; i >= 0; --i)
+                    if (val[i] == m) at = i;
+                const int g = at / kGroup;
+                best = Best{m, m, chunk_base + (g * kThreads + tid) * kGroup + (at - g * kGroup)};
+            }
+        } else {
+            const int fork = row / d, pos = row - fork * d;
+            const uint64_t seed = seeds[fork];
+            const uint2 key = make_uint2(static_cast<uint32_t>(seed), static_cast<uint32_t>(seed >> 32));
+            // ---- coarse bytes: one Philox block per 16 ids; ids with byte 255 go to the candidate list
+            uint32_t cw[kGroups][4];
+            __syncthreads();                            // s_n_cand is zero
+#pragma unroll
+            for (int g = 0; g < kGroups; ++g) {
+                const int v0 = chunk_base + (g * kThreads + tid) * kGroup;
+                const uint4 r = philox4x32_10(make_uint4(static_cast<uint32_t>(v0 >> 4), pos, step, block_idx), key);
+                cw[g][0] = r.x; cw[g][1] = r.y; cw[g][2] = r.z; cw[g][3] = r.w;
+            }
+            uint32_t any = 0;
+            uint32_t hit[kGroups][4];
+#pragma unroll
+            for (int g = 0; g < kGroups; ++g)
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    // 0x80 in every byte of the word that equals 255
+                    const uint32_t z = ~cw[g][k];
+                    hit[g][k] = ~(((z & 0x7F7F7F7Fu) + 0x7F7F7F7Fu) | z | 0x7F7F7F7Fu);
+                    any |= hit[g][k];
+                }
+            if (any) {
+#pragma unroll
+                for (int g = 0; g < kGroups; ++g)
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) {
+                        uint32_t h = hit[g][k];
+                        while (h) {
+                            const int j = (__ffs(h) - 1) >> 3;
+                            h &= h - 1;
+                            const int local = (g * kThreads + tid) * kGroup + k * 4 + j;
+                            if (chunk_base + local < vocab) {
+                                const int slot = atomicAdd(&s_n_cand, 1);
+                                if (slot < kMaxCand) s_cand[slot] = static_cast<uint16_t>(local);
+                            }
+                        }
                     }
+            }
+            __syncthreads();
+            // ---- exact scores of the candidates: their best is a lower bound L of the chunk's best
+            const int n_cand = s_n_cand;
+            const bool overflow = n_cand > kMaxCand;    // (never for random bytes) then nothing is pruned
+            if (!overflow) {
+                for (int c = tid; c < n_cand; c += kThreads) {
+                    const int v = chunk_base + s_cand[c];
+                    const float l = Logit<T>::load1(row_ptr + v);
+                    const uint4 r = philox4x32_10(make_uint4(static_cast<uint32_t>(v >> 2), pos | kFineStream, step, block_idx), key);
+                    const uint32_t w4[4] = {r.x, r.y, r.z, r.w};
+                    const float sc = fmaf(temperature, gumbel_exact(255u, w4[v & 3] >> 9), l);
+                    best = better(best, Best{sc, l, v});
+                }
+            }
+            float lb = best.score;
+#pragma unroll
+            for (int off = 16; off > 0; off >>= 1) lb = fmaxf(lb, __shfl_xor_sync(0xFFFFFFFFu, lb, off));
+            if (lane == 0) red_score[warp] = lb;
+            __syncthreads();
+            lb = red_score[0];
+#pragma unroll
+            for (int w2 = 1; w2 < kThreads / 32; ++w2) lb = fmaxf(lb, red_score[w2]);
+            if (overflow) lb = -CUDART_INF_F;
+            // ---- ids whose byte is below 255 (or every id after an overflow) that can still reach L
+            const float reach = lb - temperature * kGumbelBelow255 - 1e-3f;
+            if (m >= reach) {
+#pragma unroll
+                for (int i = 0; i < kPerThread; ++i) {          // unrolled: val[] must stay in registers
+                    const float l = val[i];
+                    if (!(l >= reach) || l == -CUDART_INF_F) continue;
+                    const int g = i / kGroup, e = i - g * kGroup;
+                    const uint32_t c = (cw[g][e >> 2] >> ((e & 3) * 8)) & 0xFFu;
+                    if (c == 255u && !overflow) continue;                  // handled as a candidate
+                    if (c < 255u && fmaf(temperature, gumbel_bound(c), l) < lb) continue;
+                    const int v = chunk_base + (g * kThreads + tid) * kGroup + e;
+                    const uint4 r = philox4x32_10(make_uint4(static_cast<uint32_t>(v >> 2), pos | kFineStream, step, block_idx), key);
+                    const uint32_t w4[4] = {r.x, r.y, r.z, r.w};
+                    const float sc = fmaf(temperature, gumbel_exact(c, w4[v & 3] >> 9), l);
+                    best = better(best, Best{sc, l, v});
                 }
             }
         }
-    }
 
-    // block reduction
+        // ---- block reduction
 #pragma unroll
-    for (int off = 16; off > 0; off >>= 1) {
-        const float m2 = __shfl_xor_sync(0xFFFFFFFFu, m, off);
-        const float s2 = __shfl_xor_sync(0xFFFFFFFFu, s, off);
-        const float mn = fmaxf(m, m2);
-        if (mn > -CUDART_INF_F) s = s * __expf(m - mn) + s2 * __expf(m2 - mn);
-        m = mn;
-        Best o;
-        o.score = __shfl_xor_sync(0xFFFFFFFFu, best.score, off);
-        o.logit = __shfl_xor_sync(0xFFFFFFFFu, best.logit, off);
-        o.index = __shfl_xor_sync(0xFFFFFFFFu, best.index, off);
-        best = better(best, o);
-    }
-    const int warp = tid >> 5, lane = tid & 31;
-    if (lane == 0) { red_max[warp] = m; red_sum[warp] = s; red_best[warp] = best; }
-    __syncthreads();
-    if (tid == 0) {
-        float M = red_max[0], S = red_sum[0];
-        Best B = red_best[0];
-        for (int w2 = 1; w2 < kThreads / 32; ++w2) {
-            const float mn = fmaxf(M, red_max[w2]);
-            if (mn > -CUDART_INF_F) S = S * __expf(M - mn) + red_sum[w2] * __expf(red_max[w2] - mn);
-            M = mn;
-            B = better(B, red_best[w2]);
+        for (int off = 16; off > 0; off >>= 1) {
+            const float m2 = __shfl_xor_sync(0xFFFFFFFFu, m, off);
+            const float s2 = __shfl_xor_sync(0xFFFFFFFFu, s, off);
+            const float mn = fmaxf(m, m2);
+            if (mn > -CUDART_INF_F) s = s * __expf(m - mn) + s2 * __expf(m2 - mn);
+            m = mn;
         }
-        UnmaskPartial out;
-        out.row_max = M; out.sum_exp = S; out.best_score = B.score; out.best_logit = B.logit;
-        out.best_index = B.index; out.pad[0] = out.pad[1] = out.pad[2] = 0;
-        partial[static_cast<size_t>(row) * n_chunks + chunk] = out;
+        best = warp_best(best);
+        if (lane == 0) { red_max[warp] = m; red_sum[warp] = s; red_best[warp] = best; }
+        __syncthreads();
+        if (tid == 0) {
+            float M = red_max[0], S = red_sum[0];
+            Best B = red_best[0];
+            for (int w2 = 1; w2 < kThreads / 32; ++w2) {
+                const float mn = fmaxf(M, red_max[w2]);
+                if (mn > -CUDART_INF_F) S = S * __expf(M - mn) + red_sum[w2] * __expf(red_max[w2] - mn);
+                M = mn;
+                B = better(B, red_best[w2]);
+            }
+            UnmaskPartial out;
+            out.row_max = M; out.sum_exp = S; out.best_score = B.score; out.best_logit = B.logit;
+            out.best_index = B.index; out.pad[0] = out.pad[1] = out.pad[2] = 0;
+            partial[static_cast<size_t>(row) * n_chunks + chunk] = out;
+        }
+        __syncthreads();                                // red_* and the candidate list are reused by the next item
     }
 }
 
@@ -251,30 +380,51 @@ unmask_finalize_kernel(const UnmaskPartial* __restrict__ partial, int32_t* __res
     }
 }
 
+
 }  // namespace
 
-cudaError_t launch_unmask(fdd_ctx* ctx, const UnmaskProblem& p, cudaStream_t st, int* n_launches) {
+namespace {
+
+// Both entry points launch the same two kernels; only the home of the records differs.
+cudaError_t launch_unmask_kernels(const UnmaskProblem& p, UnmaskPartial* partial, cudaStream_t st) {
     const int rows = p.n_forks * p.d;
+    if (rows > kMaxRows) return cudaErrorInvalidValue;
     const int n_chunks = unmask_chunks(p.vocab);
-    UnmaskPartial* partial = static_cast<UnmaskPartial*>(ctx->ws_unmask);
-    const dim3 grid(static_cast<unsigned>(n_chunks) * static_cast<unsigned>(rows));
+    static int sm_count = 0;
+    if (sm_count == 0) {
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess ||
+            cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sm_count <= 0)
+            sm_count = 148;
+    }
+    long long items = static_cast<long long>(rows) * n_chunks;
+    long long ctas = static_cast<long long>(sm_count) * 3;      // persistent: as many CTAs as fit on the SMs
+    if (ctas > items) ctas = items;
+    if (ctas < 1) ctas = 1;
+    const dim3 grid(static_cast<unsigned>(ctas));
     if (p.logits_dtype == FDD_LOGITS_BF16) {
-        const int vec_ok = (p.vocab % 8 == 0) && (reinterpret_cast<uintptr_t>(p.logits) % 16 == 0);
+        const int vec_ok = (p.vocab % 16 == 0) && (reinterpret_cast<uintptr_t>(p.logits) % 32 == 0);
         unmask_partial_kernel<__nv_bfloat16><<<grid, kThreads, 0, st>>>(
-            static_cast<const __nv_bfloat16*>(p.logits), p.state, p.seeds, partial, p.d, p.vocab,
+            static_cast<const __nv_bfloat16*>(p.logits), p.state, p.seeds, partial, rows, p.d, p.vocab,
             n_chunks, p.temperature, p.block_idx, p.step, vec_ok);
     } else {
-        const int vec_ok = (p.vocab % 4 == 0) && (reinterpret_cast<uintptr_t>(p.logits) % 16 == 0);
+        const int vec_ok = (p.vocab % 8 == 0) && (reinterpret_cast<uintptr_t>(p.logits) % 32 == 0);
         unmask_partial_kernel<float><<<grid, kThreads, 0, st>>>(
-            static_cast<const float*>(p.logits), p.state, p.seeds, partial, p.d, p.vocab,
+            static_cast<const float*>(p.logits), p.state, p.seeds, partial, rows, p.d, p.vocab,
             n_chunks, p.temperature, p.block_idx, p.step, vec_ok);
     }
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     unmask_finalize_kernel<<<p.n_forks, 128, 0, st>>>(partial, p.tokens, p.state, p.n_committed,
                                                      p.n_left, p.conf, p.d, n_chunks, p.threshold);
-    *n_launches += 2;
     return cudaGetLastError();
+}
+
+}  // namespace
+
+cudaError_t launch_unmask(fdd_ctx* ctx, const UnmaskProblem& p, cudaStream_t st, int* n_launches) {
+    *n_launches += 2;
+    return launch_unmask_kernels(p, static_cast<UnmaskPartial*>(ctx->ws_unmask), st);
 }
 
 // -------------------------------------------------------------------------------------------------
@@ -348,28 +498,12 @@ extern "C" fdd_status fdd_unmask_static(const void* logits, int logits_dtype, in
         g_static_ptr[dev] = static_cast<UnmaskPartial*>(p);
         g_static_ready[dev] = true;
     }
-    UnmaskPartial* partial = g_static_ptr[dev];
-    cudaStream_t st = static_cast<cudaStream_t>(stream);
-    const int rows = n_forks * block_len;
-    const int n_chunks = unmask_chunks(vocab);
-    const dim3 grid(static_cast<unsigned>(n_chunks) * static_cast<unsigned>(rows));
-    if (logits_dtype == FDD_LOGITS_BF16) {
-        const int vec_ok = (vocab % 8 == 0) && (reinterpret_cast<uintptr_t>(logits) % 16 == 0);
-        unmask_partial_kernel<__nv_bfloat16><<<grid, kThreads, 0, st>>>(
-            static_cast<const __nv_bfloat16*>(logits), state, seeds, partial, block_len, vocab, n_chunks,
-            temperature, block_idx, step, vec_ok);
-    } else {
-        const int vec_ok = (vocab % 4 == 0) && (reinterpret_cast<uintptr_t>(logits) % 16 == 0);
-        unmask_partial_kernel<float><<<grid, kThreads, 0, st>>>(
-            static_cast<const float*>(logits), state, seeds, partial, block_len, vocab, n_chunks,
-            temperature, block_idx, step, vec_ok);
-    }
-    e = cudaGetLastError();
-    if (e == cudaSuccess) {
-        unmask_finalize_kernel<<<n_forks, 128, 0, st>>>(partial, tokens, state, n_committed, n_left, conf,
-                                                       block_len, n_chunks, threshold);
-        e = cudaGetLastError();
-    }
+    UnmaskProblem p;
+    p.logits = logits; p.tokens = tokens; p.state = state; p.seeds = seeds;
+    p.n_committed = n_committed; p.n_left = n_left; p.conf = conf;
+    p.n_forks = n_forks; p.d = block_len; p.vocab = vocab; p.logits_dtype = logits_dtype;
+    p.threshold = threshold; p.temperature = temperature; p.block_idx = block_idx; p.step = step;
+    e = launch_unmask_kernels(p, g_static_ptr[dev], static_cast<cudaStream_t>(stream));
     if (e != cudaSuccess) {
         if (err && err_len) snprintf(err, err_len, "fdd_unmask_static: launch failed: %s", cudaGetErrorString(e));
         return FDD_ERR_CUDA;

@@ -7,7 +7,8 @@ import numpy as np
 import pytest
 
 from oracle import MASKED, COMMITTED, SCAFFOLD
-from oracle.philox import (gumbel_row, philox4x32_scalar, philox4x32_vec, uniform_from_word)
+from oracle.philox import (coarse_bytes, fine_bits, gumbel_row, philox4x32_scalar, philox4x32_vec,
+                           uniform_from_parts)
 from oracle.unmask import unmask_step
 
 GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
@@ -44,14 +45,16 @@ def test_philox_vectorised_equals_scalar():
         assert [int(o[0]) for o in out] == expect
 
 
-def test_uniform_map_is_open_interval_and_fp32_exact():
-    x = np.array([0, 1, 511, 512, 2 ** 31, 2 ** 32 - 1], dtype=np.uint64)
-    u = uniform_from_word(x)
-    assert u[0] == 2.0 ** -24 and u[-1] == 1.0 - 2.0 ** -24
-    assert u[1] == u[2] == u[0] and u[3] == 3 * 2.0 ** -24
-    np.testing.assert_array_equal(u.astype(np.float32).astype(np.float64), u)
+def test_uniform_map_is_open_interval_and_monotone():
+    c = np.array([0, 0, 0, 1, 127, 128, 255, 255])
+    f = np.array([0, 1, 2 ** 23 - 1, 0, 2 ** 23 - 1, 0, 0, 2 ** 23 - 1])
+    u = uniform_from_parts(c, f)
+    assert u[0] == 2.0 ** -32 and u[-1] == 1.0 - 2.0 ** -32
+    assert np.all(np.diff(u) > 0)                      # ordered by (coarse, fine)
+    assert u[3] - u[2] == 2.0 ** -31                   # bins tile (0, 1) without gap or overlap
+    assert np.all(u * 2.0 ** 32 == np.round(u * 2.0 ** 32))
     g = -np.log(-np.log(u))
-    assert np.all(np.isfinite(g))
+    assert np.all(np.isfinite(g)) and -3.1 < g[0] and g[-1] < 22.2
 
 
 def test_gumbel_row_layout_and_independence_from_vocab_size():
@@ -59,16 +62,37 @@ def test_gumbel_row_layout_and_independence_from_vocab_size():
     a = gumbel_row(seed, 3, 2, 5, 37)
     b = gumbel_row(seed, 3, 2, 5, 64)
     np.testing.assert_array_equal(a, b[:37])
-    # entry v is word v % 4 of counter (v // 4, pos, step, block) under key (lo, hi)
+    key = (seed & 0xFFFFFFFF, seed >> 32)
+    # coarse: byte v % 16 of counter (v // 16, pos, step, block); fine: top 23 bits of word v % 4 of
+    # counter (v // 4, pos + 2^31, step, block); both under key (lo, hi)
     for v in (0, 5, 18, 36):
-        w = philox4x32_scalar((v // 4, 5, 2, 3), (seed & 0xFFFFFFFF, seed >> 32))[v % 4]
-        u = ((w >> 9) + 0.5) * 2.0 ** -23
+        cw = philox4x32_scalar((v // 16, 5, 2, 3), key)[(v % 16) // 4]
+        c = (cw >> (8 * (v % 4))) & 0xFF
+        f = philox4x32_scalar((v // 4, 5 + 2 ** 31, 2, 3), key)[v % 4] >> 9
+        u = (c + (f + 0.5) * 2.0 ** -23) / 256.0
         assert a[v] == -math.log(-math.log(u))
+        assert coarse_bytes(seed, 3, 2, 5, 37)[v] == c and fine_bits(seed, 3, 2, 5, 37)[v] == f
     # every counter field and the seed matter
     for other in (gumbel_row(seed + 1, 3, 2, 5, 37), gumbel_row(seed, 4, 2, 5, 37),
                   gumbel_row(seed, 3, 1, 5, 37), gumbel_row(seed, 3, 2, 6, 37),
                   gumbel_row(seed ^ (1 << 40), 3, 2, 5, 37)):
         assert not np.array_equal(a, other)
+
+
+def test_coarse_byte_bounds_the_draw():
+    # what lets an implementation skip the second stream: g < -ln(-ln((c + 1) / 256)) for c < 255
+    g = gumbel_row(777, 1, 4, 9, 50000)
+    c = coarse_bytes(777, 1, 4, 9, 50000).astype(np.float64)
+    low = c < 255
+    with np.errstate(divide="ignore"):
+        upper = -np.log(-np.log((c + 1.0) / 256.0))
+        lower = -np.log(-np.log(c / 256.0))
+    assert np.all(g[low] < upper[low]) and np.all(g[c > 0] > lower[c > 0])
+    # the two streams are not the same numbers: coarse bytes are uncorrelated with the fine bits
+    f = fine_bits(777, 1, 4, 9, 50000).astype(np.float64)
+    assert abs(np.corrcoef(c, f)[0, 1]) < 0.02
+    counts = np.bincount(c.astype(int), minlength=256)
+    assert counts.min() > 120 and counts.max() < 280    # 50000 / 256 = 195 expected per bin
 
 
 def test_gumbel_uniformity_ks():
