@@ -1,10 +1,11 @@
 // Confidence-threshold parallel unmasking: vocabulary-wide soft-max statistics and
 // (Gumbel-perturbed) arg-max per MASKED row, then the per-rollout commit rule.
 //
-// Kernel 1 (unmask_partial_kernel): a persistent grid walks the (MASKED row, 8192-logit chunk)
-// pairs of the call.  A CTA streams its chunk from HBM exactly once with 32-byte loads (16
-// consecutive logits per thread and load), keeps it in registers and reduces it to (max, sum exp,
-// best perturbed score, its vocabulary id and logit).  Rows that are not MASKED are never read.
+// Kernel 1 (unmask_partial_kernel): a persistent grid walks the (MASKED row, segment) pairs of the
+// call; with many MASKED rows a segment is a whole row, with few the rows are cut so that every
+// SM has work.  A CTA streams its segment from HBM once with 32-byte loads (16 consecutive logits
+// per thread and load) and keeps running soft-max statistics; nothing but the few logits that can
+// win the arg-max is looked at twice.  Rows that are not MASKED are never read.
 //
 // Noise (temperature > 0).  The uniform behind every Gumbel draw has two parts: a coarse byte c
 // (one Philox block serves 16 vocabulary ids) and 23 fine bits (one block per 4 ids).  The byte
@@ -12,12 +13,12 @@
 // kernel cheap: every id gets its coarse byte, but the second Philox block and the two
 // logarithms are spent only on
 //   (1) the ids with c = 255 (one in 256), whose best exact score L is a lower bound of the
-//       chunk's best score, and
+//       segment's best score, and
 //   (2) the ids of threads whose largest logit could still beat L with the largest draw a
 //       byte below 255 allows (g < 5.5433), filtered once more by their own byte's bound.
 // Any id left out cannot reach L, so the arg-max (lowest id on ties) is exact.
 //
-// Kernel 2 (unmask_finalize_kernel): one CTA per rollout merges the chunk records of its
+// Kernel 2 (unmask_finalize_kernel): one CTA per rollout merges the segment records of its
 // rows, forms the confidences and applies the threshold / at-least-one rule.
 #include "fdd_internal.h"
 
@@ -26,25 +27,40 @@
 namespace {
 
 constexpr int kThreads = 256;
-constexpr int kPerThread = kUnmaskChunk / kThreads;   // 32 vocabulary entries per thread
 constexpr int kGroup = 16;                            // consecutive entries per load and per coarse Philox block
-constexpr int kGroups = kPerThread / kGroup;          // 2
-constexpr int kMaxCand = 1024;                        // c = 255 ids kept per chunk (32 expected)
-constexpr int kMaxRows = kUnmaskMaxRows;               // rows whose state fits the CTA's compaction buffer
+constexpr int kSegQuantum = kThreads * kGroup;        // segment lengths are multiples of this (4096)
+constexpr int kMaxCand = 1536;                        // c = 255 ids kept per segment (594 expected for a 152k row)
+constexpr int kMaxRows = kUnmaskMaxRows;              // rows whose state fits the CTA's compaction buffer
 constexpr float kGumbelBelow255 = 5.5440f;            // > -ln(-ln(255/256)) = 5.54322, with rounding slack
+constexpr float kLog2e = 1.4426950408889634f;
 
 constexpr uint32_t kPhiloxM0 = 0xD2511F53u, kPhiloxM1 = 0xCD9E8D57u;
 constexpr uint32_t kPhiloxW0 = 0x9E3779B9u, kPhiloxW1 = 0xBB67AE85u;
 constexpr uint32_t kFineStream = 0x80000000u;         // added to the position word for the fine bits
 
-// Philox4x32 with 10 rounds (Salmon et al., SC'11), written from the published round function.
-__device__ __forceinline__ uint4 philox4x32_10(uint4 c, uint2 k) {
+// Round keys of Philox4x32-10 for one 64-bit key (the key schedule does not depend on the counter).
+struct PhiloxKeys {
+    uint32_t k0[10], k1[10];
+};
+__device__ __forceinline__ PhiloxKeys philox_keys(uint64_t seed) {
+    PhiloxKeys k;
+    uint32_t a = static_cast<uint32_t>(seed), b = static_cast<uint32_t>(seed >> 32);
 #pragma unroll
     for (int r = 0; r < 10; ++r) {
-        if (r > 0) { k.x += kPhiloxW0; k.y += kPhiloxW1; }
-        const uint32_t hi0 = __umulhi(kPhiloxM0, c.x), lo0 = kPhiloxM0 * c.x;
-        const uint32_t hi1 = __umulhi(kPhiloxM1, c.z), lo1 = kPhiloxM1 * c.z;
-        c = make_uint4(hi1 ^ c.y ^ k.x, lo1, hi0 ^ c.w ^ k.y, lo0);
+        k.k0[r] = a; k.k1[r] = b;
+        a += kPhiloxW0; b += kPhiloxW1;
+    }
+    return k;
+}
+// Philox4x32 with 10 rounds (Salmon et al., SC'11), written from the published round function:
+// (c0, c1, c2, c3) -> (hi(M1 c2) ^ c1 ^ k0, lo(M1 c2), hi(M0 c0) ^ c3 ^ k1, lo(M0 c0)).
+__device__ __forceinline__ uint4 philox4x32_10(uint4 c, const PhiloxKeys& k) {
+#pragma unroll
+    for (int r = 0; r < 10; ++r) {
+        const uint64_t p0 = static_cast<uint64_t>(kPhiloxM0) * c.x;
+        const uint64_t p1 = static_cast<uint64_t>(kPhiloxM1) * c.z;
+        c = make_uint4(static_cast<uint32_t>(p1 >> 32) ^ c.y ^ k.k0[r], static_cast<uint32_t>(p1),
+                       static_cast<uint32_t>(p0 >> 32) ^ c.w ^ k.k1[r], static_cast<uint32_t>(p0));
     }
     return c;
 }
@@ -67,6 +83,17 @@ __device__ __forceinline__ float gumbel_exact(uint32_t c, uint32_t f23) {
 // Upper bound of the draws with coarse byte c < 255 (c = 255 has no useful bound).
 __device__ __forceinline__ float gumbel_bound(uint32_t c) {
     return -logf(-logf(static_cast<float>(c + 1u) * 0.00390625f)) + 1e-3f;
+}
+
+__device__ __forceinline__ float ex2_fast(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+__device__ __forceinline__ float max3f(float a, float b, float c) {
+    float d;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
 }
 
 __device__ __forceinline__ void load32(const void* p, uint32_t (&r)[8]) {
@@ -102,6 +129,17 @@ template <> struct Logit<float> {
     __device__ static float load1(const float* p) { return *p; }
 };
 
+// 16 logits starting at vocabulary id v0 (a multiple of 16); ids >= vocab read as -inf.
+template <typename T>
+__device__ __forceinline__ void load_group(const T* row_ptr, int v0, int vocab, int vec_ok, float* val) {
+    if (vec_ok && v0 + kGroup <= vocab) {
+        Logit<T>::load16(row_ptr + v0, val);
+    } else {
+#pragma unroll
+        for (int j = 0; j < kGroup; ++j) val[j] = (v0 + j < vocab) ? Logit<T>::load1(row_ptr + v0 + j) : -CUDART_INF_F;
+    }
+}
+
 struct Best {
     float score, logit;
     int index;
@@ -132,7 +170,7 @@ unmask_partial_kernel(const T* __restrict__ logits, const uint8_t* __restrict__ 
     __shared__ uint16_t s_rows[kMaxRows];               // MASKED rows, ascending
     __shared__ int s_n_rows;
     __shared__ int s_warp_count[kThreads / 32];
-    __shared__ uint16_t s_cand[kMaxCand];               // chunk-local ids with coarse byte 255
+    __shared__ int s_cand[kMaxCand];                    // vocabulary ids with coarse byte 255
     __shared__ int s_n_cand;
     __shared__ float red_max[kThreads / 32], red_sum[kThreads / 32], red_score[kThreads / 32];
     __shared__ Best red_best[kThreads / 32];
@@ -155,106 +193,97 @@ unmask_partial_kernel(const T* __restrict__ logits, const uint8_t* __restrict__ 
             for (int w2 = 0; w2 < kThreads / 32; ++w2) base += s_warp_count[w2];
             __syncthreads();
         }
-        if (tid == 0) s_n_rows = base;
+        if (tid == 0) { s_n_rows = base; s_n_cand = 0; }
         __syncthreads();
     }
-    const int n_items = s_n_rows * n_chunks;
+    const int n_rows = s_n_rows;
+    if (n_rows == 0) return;
+    // Segments per row: one when there are plenty of rows, more (up to n_chunks) when the rows
+    // alone would leave SMs idle.  Every CTA derives the same numbers.
+    int segs = (2 * static_cast<int>(gridDim.x) + n_rows - 1) / n_rows;
+    segs = max(1, min(segs, n_chunks));
+    const int seg_len = ((vocab + segs - 1) / segs + kSegQuantum - 1) / kSegQuantum * kSegQuantum;
+    segs = (vocab + seg_len - 1) / seg_len;
+    const int n_items = n_rows * segs;
 
     for (int item = blockIdx.x; item < n_items; item += gridDim.x) {
-        const int row = s_rows[item / n_chunks];
-        const int chunk = item - (item / n_chunks) * n_chunks;
+        const int row = s_rows[item / segs];
+        const int seg = item - (item / segs) * segs;
         const T* row_ptr = logits + static_cast<size_t>(row) * vocab;
-        const int chunk_base = chunk * kUnmaskChunk;
-        if (tid == 0) s_n_cand = 0;
+        const int seg_begin = seg * seg_len;
+        const int seg_end = min(vocab, seg_begin + seg_len);
+        const int fork = row / d, pos = row - fork * d;
+        PhiloxKeys keys;
+        if (noisy) keys = philox_keys(seeds[fork]);
 
-        // ---- stream the chunk: 2 x 16 consecutive logits per thread
-        float val[kPerThread];
-#pragma unroll
-        for (int g = 0; g < kGroups; ++g) {
-            const int v0 = chunk_base + (g * kThreads + tid) * kGroup;
-            if (vec_ok && v0 + kGroup <= vocab) {
-                Logit<T>::load16(row_ptr + v0, &val[g * kGroup]);
-            } else {
-#pragma unroll
-                for (int j = 0; j < kGroup; ++j)
-                    val[g * kGroup + j] = (v0 + j < vocab) ? Logit<T>::load1(row_ptr + v0 + j) : -CUDART_INF_F;
-            }
-        }
-
-        // ---- soft-max statistics of the thread's 32 logits
-        float m = -CUDART_INF_F;
-#pragma unroll
-        for (int i = 0; i < kPerThread; ++i) m = fmaxf(m, val[i]);
-        float s = 0.0f;
-        if (m > -CUDART_INF_F) {
-            const float ml = m * 1.4426950408889634f;
-            float s4[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-            for (int i = 0; i < kPerThread; ++i) s4[i & 3] += exp2f(fmaf(val[i], 1.4426950408889634f, -ml));
-            s = (s4[0] + s4[1]) + (s4[2] + s4[3]);
-        }
-
+        // ---- pass 1: stream the segment; running soft-max statistics, coarse bytes, candidates
+        float m = -CUDART_INF_F, s = 0.0f;             // thread's running max and sum exp(l - m)
         Best best{-CUDART_INF_F, -CUDART_INF_F, 0x7FFFFFFF};
-        if (!noisy) {
-            // arg-max of the logits themselves; the thread maximum is known, find its first place
-            if (m > -CUDART_INF_F) {
-                int at = kPerThread;
+        for (int v0 = seg_begin + tid * kGroup; v0 < seg_end; v0 += kSegQuantum) {
+            float val[kGroup];
+            load_group(row_ptr, v0, vocab, vec_ok, val);
+            float g4[4];
 #pragma unroll
-                for (int i = kPerThread - 1; i >= 0; --i)
-                    if (val[i] == m) at = i;
-                const int g = at / kGroup;
-                best = Best{m, m, chunk_base + (g * kThreads + tid) * kGroup + (at - g * kGroup)};
+            for (int u = 0; u < 4; ++u) g4[u] = max3f(val[4 * u], val[4 * u + 1], fmaxf(val[4 * u + 2], val[4 * u + 3]));
+            const float gm = fmaxf(fmaxf(g4[0], g4[1]), fmaxf(g4[2], g4[3]));
+            if (gm > -CUDART_INF_F) {
+                if (!noisy && gm > m) {
+                    // greedy: the arg-max so far moves into this group; find its first place
+                    int at = kGroup;
+#pragma unroll
+                    for (int i = kGroup - 1; i >= 0; --i)
+                        if (val[i] == gm) at = i;
+                    best = Best{gm, gm, v0 + at};
+                }
+                const float mn = fmaxf(m, gm);
+                const float mnl = mn * kLog2e;
+                float s4[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+                for (int i = 0; i < kGroup; ++i) s4[i & 3] += ex2_fast(fmaf(val[i], kLog2e, -mnl));
+                // rescale by 2^((m - mn) log2e): exactly 1 while the maximum stands (the rounded mnl must
+                // not enter here, or a factor 1 + 1e-7 would compound over the groups)
+                s = s * ex2_fast((m - mn) * kLog2e) + ((s4[0] + s4[1]) + (s4[2] + s4[3]));
+                m = mn;
             }
-        } else {
-            const int fork = row / d, pos = row - fork * d;
-            const uint64_t seed = seeds[fork];
-            const uint2 key = make_uint2(static_cast<uint32_t>(seed), static_cast<uint32_t>(seed >> 32));
-            // ---- coarse bytes: one Philox block per 16 ids; ids with byte 255 go to the candidate list
-            uint32_t cw[kGroups][4];
-            __syncthreads();                            // s_n_cand is zero
-#pragma unroll
-            for (int g = 0; g < kGroups; ++g) {
-                const int v0 = chunk_base + (g * kThreads + tid) * kGroup;
-                const uint4 r = philox4x32_10(make_uint4(static_cast<uint32_t>(v0 >> 4), pos, step, block_idx), key);
-                cw[g][0] = r.x; cw[g][1] = r.y; cw[g][2] = r.z; cw[g][3] = r.w;
-            }
-            uint32_t any = 0;
-            uint32_t hit[kGroups][4];
-#pragma unroll
-            for (int g = 0; g < kGroups; ++g)
+            if (noisy) {
+                const uint4 r = philox4x32_10(make_uint4(static_cast<uint32_t>(v0 >> 4), pos, step, block_idx), keys);
+                const uint32_t cw[4] = {r.x, r.y, r.z, r.w};
+                uint32_t hit[4], any = 0;
 #pragma unroll
                 for (int k = 0; k < 4; ++k) {
                     // 0x80 in every byte of the word that equals 255
-                    const uint32_t z = ~cw[g][k];
-                    hit[g][k] = ~(((z & 0x7F7F7F7Fu) + 0x7F7F7F7Fu) | z | 0x7F7F7F7Fu);
-                    any |= hit[g][k];
+                    const uint32_t z = ~cw[k];
+                    hit[k] = ~(((z & 0x7F7F7F7Fu) + 0x7F7F7F7Fu) | z | 0x7F7F7F7Fu);
+                    any |= hit[k];
                 }
-            if (any) {
-#pragma unroll
-                for (int g = 0; g < kGroups; ++g)
+                if (any) {
 #pragma unroll
                     for (int k = 0; k < 4; ++k) {
-                        uint32_t h = hit[g][k];
+                        uint32_t h = hit[k];
                         while (h) {
                             const int j = (__ffs(h) - 1) >> 3;
                             h &= h - 1;
-                            const int local = (g * kThreads + tid) * kGroup + k * 4 + j;
-                            if (chunk_base + local < vocab) {
+                            const int v = v0 + k * 4 + j;
+                            if (v < vocab) {
                                 const int slot = atomicAdd(&s_n_cand, 1);
-                                if (slot < kMaxCand) s_cand[slot] = static_cast<uint16_t>(local);
+                                if (slot < kMaxCand) s_cand[slot] = v;
                             }
                         }
                     }
+                }
             }
+        }
+
+        if (noisy) {
             __syncthreads();
-            // ---- exact scores of the candidates: their best is a lower bound L of the chunk's best
+            // ---- exact scores of the candidates: their best is a lower bound L of the segment's best
             const int n_cand = s_n_cand;
             const bool overflow = n_cand > kMaxCand;    // (never for random bytes) then nothing is pruned
             if (!overflow) {
                 for (int c = tid; c < n_cand; c += kThreads) {
-                    const int v = chunk_base + s_cand[c];
+                    const int v = s_cand[c];
                     const float l = Logit<T>::load1(row_ptr + v);
-                    const uint4 r = philox4x32_10(make_uint4(static_cast<uint32_t>(v >> 2), pos | kFineStream, step, block_idx), key);
+                    const uint4 r = philox4x32_10(make_uint4(static_cast<uint32_t>(v >> 2), pos | kFineStream, step, block_idx), keys);
                     const uint32_t w4[4] = {r.x, r.y, r.z, r.w};
                     const float sc = fmaf(temperature, gumbel_exact(255u, w4[v & 3] >> 9), l);
                     best = better(best, Best{sc, l, v});
@@ -269,22 +298,33 @@ unmask_partial_kernel(const T* __restrict__ logits, const uint8_t* __restrict__ 
 #pragma unroll
             for (int w2 = 1; w2 < kThreads / 32; ++w2) lb = fmaxf(lb, red_score[w2]);
             if (overflow) lb = -CUDART_INF_F;
-            // ---- ids whose byte is below 255 (or every id after an overflow) that can still reach L
+            // ---- pass 2: a thread whose largest logit can still reach L goes over its groups again
             const float reach = lb - temperature * kGumbelBelow255 - 1e-3f;
             if (m >= reach) {
+                for (int v0 = seg_begin + tid * kGroup; v0 < seg_end; v0 += kSegQuantum) {
+                    float val[kGroup];
+                    load_group(row_ptr, v0, vocab, vec_ok, val);
+                    bool some = false;
 #pragma unroll
-                for (int i = 0; i < kPerThread; ++i) {          // unrolled: val[] must stay in registers
-                    const float l = val[i];
-                    if (!(l >= reach) || l == -CUDART_INF_F) continue;
-                    const int g = i / kGroup, e = i - g * kGroup;
-                    const uint32_t c = (cw[g][e >> 2] >> ((e & 3) * 8)) & 0xFFu;
-                    if (c == 255u && !overflow) continue;                  // handled as a candidate
-                    if (c < 255u && fmaf(temperature, gumbel_bound(c), l) < lb) continue;
-                    const int v = chunk_base + (g * kThreads + tid) * kGroup + e;
-                    const uint4 r = philox4x32_10(make_uint4(static_cast<uint32_t>(v >> 2), pos | kFineStream, step, block_idx), key);
-                    const uint32_t w4[4] = {r.x, r.y, r.z, r.w};
-                    const float sc = fmaf(temperature, gumbel_exact(c, w4[v & 3] >> 9), l);
-                    best = better(best, Best{sc, l, v});
+                    for (int i = 0; i < kGroup; ++i) some = some || (val[i] >= reach && val[i] > -CUDART_INF_F);
+                    if (!some) continue;
+                    const uint4 rc = philox4x32_10(make_uint4(static_cast<uint32_t>(v0 >> 4), pos, step, block_idx), keys);
+                    const uint32_t cw[4] = {rc.x, rc.y, rc.z, rc.w};
+                    for (int i = 0; i < kGroup; ++i) {
+                        float l = -CUDART_INF_F;
+                        uint32_t word = 0;
+#pragma unroll
+                        for (int x = 0; x < kGroup; ++x) if (x == i) { l = val[x]; word = cw[x >> 2]; }
+                        if (!(l >= reach) || l == -CUDART_INF_F) continue;
+                        const uint32_t c = (word >> ((i & 3) * 8)) & 0xFFu;
+                        if (c == 255u && !overflow) continue;                  // handled as a candidate
+                        if (c < 255u && fmaf(temperature, gumbel_bound(c), l) < lb) continue;
+                        const int v = v0 + i;
+                        const uint4 r = philox4x32_10(make_uint4(static_cast<uint32_t>(v >> 2), pos | kFineStream, step, block_idx), keys);
+                        const uint32_t w4[4] = {r.x, r.y, r.z, r.w};
+                        const float sc = fmaf(temperature, gumbel_exact(c, w4[v & 3] >> 9), l);
+                        best = better(best, Best{sc, l, v});
+                    }
                 }
             }
         }
@@ -312,8 +352,11 @@ unmask_partial_kernel(const T* __restrict__ logits, const uint8_t* __restrict__ 
             }
             UnmaskPartial out;
             out.row_max = M; out.sum_exp = S; out.best_score = B.score; out.best_logit = B.logit;
-            out.best_index = B.index; out.pad[0] = out.pad[1] = out.pad[2] = 0;
-            partial[static_cast<size_t>(row) * n_chunks + chunk] = out;
+            out.best_index = B.index;
+            out.pad[0] = segs;                          // how many records this row has (read from record 0)
+            out.pad[1] = out.pad[2] = 0;
+            partial[static_cast<size_t>(row) * n_chunks + seg] = out;
+            s_n_cand = 0;
         }
         __syncthreads();                                // red_* and the candidate list are reused by the next item
     }
@@ -339,11 +382,12 @@ unmask_finalize_kernel(const UnmaskPartial* __restrict__ partial, int32_t* __res
         masked = state[row] == FDD_MASKED;
         if (masked) {
             const UnmaskPartial* p = partial + static_cast<size_t>(row) * n_chunks;
+            const int n_rec = p[0].pad[0];              // records the first kernel wrote for this row
             float M = -CUDART_INF_F;
-            for (int c = 0; c < n_chunks; ++c) M = fmaxf(M, p[c].row_max);
+            for (int c = 0; c < n_rec; ++c) M = fmaxf(M, p[c].row_max);
             float S = 0.0f;
             Best B{-CUDART_INF_F, -CUDART_INF_F, 0x7FFFFFFF};
-            for (int c = 0; c < n_chunks; ++c) {
+            for (int c = 0; c < n_rec; ++c) {
                 S += p[c].sum_exp * expf(p[c].row_max - M);
                 B = better(B, Best{p[c].best_score, p[c].best_logit, p[c].best_index});
             }
@@ -397,10 +441,7 @@ cudaError_t launch_unmask_kernels(const UnmaskProblem& p, UnmaskPartial* partial
             cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sm_count <= 0)
             sm_count = 148;
     }
-    long long items = static_cast<long long>(rows) * n_chunks;
-    long long ctas = static_cast<long long>(sm_count) * 3;      // persistent: as many CTAs as fit on the SMs
-    if (ctas > items) ctas = items;
-    if (ctas < 1) ctas = 1;
+    const long long ctas = static_cast<long long>(sm_count) * 3;      // persistent: as many CTAs as fit on the SMs
     const dim3 grid(static_cast<unsigned>(ctas));
     if (p.logits_dtype == FDD_LOGITS_BF16) {
         const int vec_ok = (p.vocab % 16 == 0) && (reinterpret_cast<uintptr_t>(p.logits) % 32 == 0);
