@@ -38,29 +38,17 @@ constexpr uint32_t kPhiloxM0 = 0xD2511F53u, kPhiloxM1 = 0xCD9E8D57u;
 constexpr uint32_t kPhiloxW0 = 0x9E3779B9u, kPhiloxW1 = 0xBB67AE85u;
 constexpr uint32_t kFineStream = 0x80000000u;         // added to the position word for the fine bits
 
-// Round keys of Philox4x32-10 for one 64-bit key (the key schedule does not depend on the counter).
-struct PhiloxKeys {
-    uint32_t k0[10], k1[10];
-};
-__device__ __forceinline__ PhiloxKeys philox_keys(uint64_t seed) {
-    PhiloxKeys k;
-    uint32_t a = static_cast<uint32_t>(seed), b = static_cast<uint32_t>(seed >> 32);
-#pragma unroll
-    for (int r = 0; r < 10; ++r) {
-        k.k0[r] = a; k.k1[r] = b;
-        a += kPhiloxW0; b += kPhiloxW1;
-    }
-    return k;
-}
 // Philox4x32 with 10 rounds (Salmon et al., SC'11), written from the published round function:
-// (c0, c1, c2, c3) -> (hi(M1 c2) ^ c1 ^ k0, lo(M1 c2), hi(M0 c0) ^ c3 ^ k1, lo(M0 c0)).
-__device__ __forceinline__ uint4 philox4x32_10(uint4 c, const PhiloxKeys& k) {
+// (c0, c1, c2, c3) -> (hi(M1 c2) ^ c1 ^ k0, lo(M1 c2), hi(M0 c0) ^ c3 ^ k1, lo(M0 c0)), the key
+// bumped by the Weyl constants between rounds.
+__device__ __forceinline__ uint4 philox4x32_10(uint4 c, uint2 k) {
 #pragma unroll
     for (int r = 0; r < 10; ++r) {
+        if (r > 0) { k.x += kPhiloxW0; k.y += kPhiloxW1; }
         const uint64_t p0 = static_cast<uint64_t>(kPhiloxM0) * c.x;
         const uint64_t p1 = static_cast<uint64_t>(kPhiloxM1) * c.z;
-        c = make_uint4(static_cast<uint32_t>(p1 >> 32) ^ c.y ^ k.k0[r], static_cast<uint32_t>(p1),
-                       static_cast<uint32_t>(p0 >> 32) ^ c.w ^ k.k1[r], static_cast<uint32_t>(p0));
+        c = make_uint4(static_cast<uint32_t>(p1 >> 32) ^ c.y ^ k.x, static_cast<uint32_t>(p1),
+                       static_cast<uint32_t>(p0 >> 32) ^ c.w ^ k.y, static_cast<uint32_t>(p0));
     }
     return c;
 }
@@ -102,12 +90,13 @@ __device__ __forceinline__ void load32(const void* p, uint32_t (&r)[8]) {
                  : "l"(p));
 }
 
+// A group = 16 consecutive logits.  fetch() starts the 32-byte loads of a group into raw words,
+// widen() turns the words into fp32 once they are needed (so several groups can be in flight).
 template <typename T> struct Logit;
 template <> struct Logit<__nv_bfloat16> {
-    // 16 consecutive logits from one 32-byte load
-    __device__ static void load16(const __nv_bfloat16* p, float* out) {
-        uint32_t w[8];
-        load32(p, w);
+    static constexpr int kWords = 8;
+    __device__ static void fetch(const __nv_bfloat16* p, uint32_t (&w)[kWords]) { load32(p, w); }
+    __device__ static void widen(const uint32_t (&w)[kWords], float* out) {
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
             out[2 * i] = __uint_as_float(w[i] << 16);
@@ -117,14 +106,17 @@ template <> struct Logit<__nv_bfloat16> {
     __device__ static float load1(const __nv_bfloat16* p) { return __bfloat162float(*p); }
 };
 template <> struct Logit<float> {
-    __device__ static void load16(const float* p, float* out) {
-        uint32_t w[8];
-        load32(p, w);
+    static constexpr int kWords = 16;
+    __device__ static void fetch(const float* p, uint32_t (&w)[kWords]) {
+        uint32_t a[8], b[8];
+        load32(p, a);
+        load32(p + 8, b);
 #pragma unroll
-        for (int i = 0; i < 8; ++i) out[i] = __uint_as_float(w[i]);
-        load32(p + 8, w);
+        for (int i = 0; i < 8; ++i) { w[i] = a[i]; w[8 + i] = b[i]; }
+    }
+    __device__ static void widen(const uint32_t (&w)[kWords], float* out) {
 #pragma unroll
-        for (int i = 0; i < 8; ++i) out[8 + i] = __uint_as_float(w[i]);
+        for (int i = 0; i < 16; ++i) out[i] = __uint_as_float(w[i]);
     }
     __device__ static float load1(const float* p) { return *p; }
 };
@@ -133,7 +125,9 @@ template <> struct Logit<float> {
 template <typename T>
 __device__ __forceinline__ void load_group(const T* row_ptr, int v0, int vocab, int vec_ok, float* val) {
     if (vec_ok && v0 + kGroup <= vocab) {
-        Logit<T>::load16(row_ptr + v0, val);
+        uint32_t w[Logit<T>::kWords];
+        Logit<T>::fetch(row_ptr + v0, w);
+        Logit<T>::widen(w, val);
     } else {
 #pragma unroll
         for (int j = 0; j < kGroup; ++j) val[j] = (v0 + j < vocab) ? Logit<T>::load1(row_ptr + v0 + j) : -CUDART_INF_F;
@@ -172,6 +166,8 @@ unmask_partial_kernel(const T* __restrict__ logits, const uint8_t* __restrict__ 
     __shared__ int s_warp_count[kThreads / 32];
     __shared__ int s_cand[kMaxCand];                    // vocabulary ids with coarse byte 255
     __shared__ int s_n_cand;
+    __shared__ uint16_t s_redo[kThreads];               // threads whose groups pass 2 goes over again
+    __shared__ int s_n_redo;
     __shared__ float red_max[kThreads / 32], red_sum[kThreads / 32], red_score[kThreads / 32];
     __shared__ Best red_best[kThreads / 32];
 
@@ -193,7 +189,7 @@ unmask_partial_kernel(const T* __restrict__ logits, const uint8_t* __restrict__ 
             for (int w2 = 0; w2 < kThreads / 32; ++w2) base += s_warp_count[w2];
             __syncthreads();
         }
-        if (tid == 0) { s_n_rows = base; s_n_cand = 0; }
+        if (tid == 0) { s_n_rows = base; s_n_cand = 0; s_n_redo = 0; }
         __syncthreads();
     }
     const int n_rows = s_n_rows;
@@ -213,15 +209,24 @@ unmask_partial_kernel(const T* __restrict__ logits, const uint8_t* __restrict__ 
         const int seg_begin = seg * seg_len;
         const int seg_end = min(vocab, seg_begin + seg_len);
         const int fork = row / d, pos = row - fork * d;
-        PhiloxKeys keys;
-        if (noisy) keys = philox_keys(seeds[fork]);
+        uint2 keys = make_uint2(0u, 0u);
+        if (noisy) {
+            const uint64_t seed = seeds[fork];
+            keys = make_uint2(static_cast<uint32_t>(seed), static_cast<uint32_t>(seed >> 32));
+        }
 
         // ---- pass 1: stream the segment; running soft-max statistics, coarse bytes, candidates
         float m = -CUDART_INF_F, s = 0.0f;             // thread's running max and sum exp(l - m)
         Best best{-CUDART_INF_F, -CUDART_INF_F, 0x7FFFFFFF};
-        for (int v0 = seg_begin + tid * kGroup; v0 < seg_end; v0 += kSegQuantum) {
+        // One group: `w` holds its raw words if it could be fetched with the wide loads.
+        auto process = [&](int v0, const uint32_t (&w)[Logit<T>::kWords]) {
             float val[kGroup];
-            load_group(row_ptr, v0, vocab, vec_ok, val);
+            if (vec_ok && v0 + kGroup <= vocab) {
+                Logit<T>::widen(w, val);
+            } else {
+#pragma unroll
+                for (int j = 0; j < kGroup; ++j) val[j] = (v0 + j < vocab) ? Logit<T>::load1(row_ptr + v0 + j) : -CUDART_INF_F;
+            }
             float g4[4];
 #pragma unroll
             for (int u = 0; u < 4; ++u) g4[u] = max3f(val[4 * u], val[4 * u + 1], fmaxf(val[4 * u + 2], val[4 * u + 3]));
@@ -272,6 +277,24 @@ unmask_partial_kernel(const T* __restrict__ logits, const uint8_t* __restrict__ 
                     }
                 }
             }
+        };
+        auto fetch = [&](int v0, uint32_t (&w)[Logit<T>::kWords]) {
+            if (vec_ok && v0 < seg_end && v0 + kGroup <= vocab) Logit<T>::fetch(row_ptr + v0, w);
+        };
+        {
+            // two register buffers take turns: the next group's load is in flight while this one is reduced
+            uint32_t wa[Logit<T>::kWords], wb[Logit<T>::kWords];
+            int v0 = seg_begin + tid * kGroup;
+            fetch(v0, wa);
+            while (v0 < seg_end) {
+                fetch(v0 + kSegQuantum, wb);
+                process(v0, wa);
+                if (v0 + kSegQuantum < seg_end) {
+                    fetch(v0 + 2 * kSegQuantum, wa);
+                    process(v0 + kSegQuantum, wb);
+                }
+                v0 += 2 * kSegQuantum;
+            }
         }
 
         if (noisy) {
@@ -298,33 +321,42 @@ unmask_partial_kernel(const T* __restrict__ logits, const uint8_t* __restrict__ 
 #pragma unroll
             for (int w2 = 1; w2 < kThreads / 32; ++w2) lb = fmaxf(lb, red_score[w2]);
             if (overflow) lb = -CUDART_INF_F;
-            // ---- pass 2: a thread whose largest logit can still reach L goes over its groups again
+            // ---- pass 2: the groups of every thread whose largest logit can still reach L are gone over
+            // again, by the whole CTA (one group per thread), not by that thread alone
             const float reach = lb - temperature * kGumbelBelow255 - 1e-3f;
             if (m >= reach) {
-                for (int v0 = seg_begin + tid * kGroup; v0 < seg_end; v0 += kSegQuantum) {
-                    float val[kGroup];
-                    load_group(row_ptr, v0, vocab, vec_ok, val);
-                    bool some = false;
+                const int slot = atomicAdd(&s_n_redo, 1);
+                if (slot < kThreads) s_redo[slot] = static_cast<uint16_t>(tid);
+            }
+            __syncthreads();
+            const int n_redo = min(s_n_redo, kThreads);
+            const int groups_per_thread = (seg_end - seg_begin + kSegQuantum - 1) / kSegQuantum;
+            for (int w = tid; w < n_redo * groups_per_thread; w += kThreads) {
+                const int owner = s_redo[w / groups_per_thread];
+                const int v0 = seg_begin + owner * kGroup + (w % groups_per_thread) * kSegQuantum;
+                if (v0 >= seg_end) continue;
+                float val[kGroup];
+                load_group(row_ptr, v0, vocab, vec_ok, val);
+                bool some = false;
 #pragma unroll
-                    for (int i = 0; i < kGroup; ++i) some = some || (val[i] >= reach && val[i] > -CUDART_INF_F);
-                    if (!some) continue;
-                    const uint4 rc = philox4x32_10(make_uint4(static_cast<uint32_t>(v0 >> 4), pos, step, block_idx), keys);
-                    const uint32_t cw[4] = {rc.x, rc.y, rc.z, rc.w};
-                    for (int i = 0; i < kGroup; ++i) {
-                        float l = -CUDART_INF_F;
-                        uint32_t word = 0;
+                for (int i = 0; i < kGroup; ++i) some = some || (val[i] >= reach && val[i] > -CUDART_INF_F);
+                if (!some) continue;
+                const uint4 rc = philox4x32_10(make_uint4(static_cast<uint32_t>(v0 >> 4), pos, step, block_idx), keys);
+                const uint32_t cw[4] = {rc.x, rc.y, rc.z, rc.w};
+                for (int i = 0; i < kGroup; ++i) {
+                    float l = -CUDART_INF_F;
+                    uint32_t word = 0;
 #pragma unroll
-                        for (int x = 0; x < kGroup; ++x) if (x == i) { l = val[x]; word = cw[x >> 2]; }
-                        if (!(l >= reach) || l == -CUDART_INF_F) continue;
-                        const uint32_t c = (word >> ((i & 3) * 8)) & 0xFFu;
-                        if (c == 255u && !overflow) continue;                  // handled as a candidate
-                        if (c < 255u && fmaf(temperature, gumbel_bound(c), l) < lb) continue;
-                        const int v = v0 + i;
-                        const uint4 r = philox4x32_10(make_uint4(static_cast<uint32_t>(v >> 2), pos | kFineStream, step, block_idx), keys);
-                        const uint32_t w4[4] = {r.x, r.y, r.z, r.w};
-                        const float sc = fmaf(temperature, gumbel_exact(c, w4[v & 3] >> 9), l);
-                        best = better(best, Best{sc, l, v});
-                    }
+                    for (int x = 0; x < kGroup; ++x) if (x == i) { l = val[x]; word = cw[x >> 2]; }
+                    if (!(l >= reach) || l == -CUDART_INF_F) continue;
+                    const uint32_t c = (word >> ((i & 3) * 8)) & 0xFFu;
+                    if (c == 255u && !overflow) continue;                  // handled as a candidate
+                    if (c < 255u && fmaf(temperature, gumbel_bound(c), l) < lb) continue;
+                    const int v = v0 + i;
+                    const uint4 r = philox4x32_10(make_uint4(static_cast<uint32_t>(v >> 2), pos | kFineStream, step, block_idx), keys);
+                    const uint32_t w4[4] = {r.x, r.y, r.z, r.w};
+                    const float sc = fmaf(temperature, gumbel_exact(c, w4[v & 3] >> 9), l);
+                    best = better(best, Best{sc, l, v});
                 }
             }
         }
@@ -357,6 +389,7 @@ unmask_partial_kernel(const T* __restrict__ logits, const uint8_t* __restrict__ 
             out.pad[1] = out.pad[2] = 0;
             partial[static_cast<size_t>(row) * n_chunks + seg] = out;
             s_n_cand = 0;
+            s_n_redo = 0;
         }
         __syncthreads();                                // red_* and the candidate list are reused by the next item
     }
