@@ -26,6 +26,9 @@ if ROOT not in sys.path:
 
 METRIC = "committed tokens/s per denoise step (N forks, shared prefix)"
 UNIT = "tokens/s"
+# DRAM bytes (read + write) of one attention launch at the long_prefix workload, from the ncu capture
+# summarised in profiles/attn_ptc_long_prefix.md; None for other workloads or once the kernel changed.
+ATTN_DRAM_BYTES_PER_LAUNCH = {"long_prefix": 157.0e6}
 PRE_STEPS = 6      # distinct per-step input sets kept resident; later steps cycle through them (--pre-steps)
 
 
@@ -102,7 +105,7 @@ def _attn_flops(w, sc, suffix_len):
 def run_ours(args):
     import torch
     from concurrent.futures import ThreadPoolExecutor
-    from paper_2605_23163_b200 import fdd, harness, synth
+    from paper_2605_23163_b200 import fdd, harness, replicas, synth
 
     rank = int(os.environ.get("RANK", 0))
     world = int(os.environ.get("WORLD_SIZE", 1))
@@ -114,8 +117,7 @@ def run_ours(args):
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     fdd.lib()
     w = synth.workload(args.workload)
-    if world > 1:     # every rank decodes its own scene replica (different seed)
-        w = synth.Workload(**{**w.__dict__, "seed": w.seed + 100 * rank})
+    w = replicas.replica_workload(w, rank)     # every rank decodes its own scene (different seed)
     sc = w.scenes[0]
     L = args.layers
     ctx = harness.create_context(w, n_layers=L)
@@ -146,6 +148,7 @@ def run_ours(args):
     all_tokens = int(state0.size)
 
     attn_events = []
+    unmask_events = []          # (start, end, MASKED rows on entry) of every timed unmask call
 
     def decode_block(inputs, timed_attn):
         """One step of the benchmark: the whole block loop for all rollouts.  `inputs(t)` returns
@@ -156,6 +159,7 @@ def run_ours(args):
         tokens.copy_(tokens0_d, non_blocking=True)
         state.copy_(state0_d, non_blocking=True)
         t = 0
+        masked_rows = value_tokens
         while True:
             q, k, v, lg = inputs(t)
             for layer in range(L):
@@ -166,11 +170,18 @@ def run_ours(args):
                 if timed_attn:
                     e1.record(stream)
                     attn_events.append((e0, e1))
+            if timed_attn:
+                u0, u1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                u0.record(stream)
             fdd.fdd_unmask(ctx, [fs], lg, tokens, state, [d], w.threshold, w.temperature, 0, t, n_comm, n_left)
+            if timed_attn:
+                u1.record(stream)
+                unmask_events.append((u0, u1, masked_rows))
             n_left_host.copy_(n_left, non_blocking=True)
             stream.synchronize()
             t += 1
-            if int(n_left_host.sum()) == 0 or t >= d:
+            masked_rows = int(n_left_host.sum())
+            if masked_rows == 0 or t >= d:
                 break
         for layer in range(L):
             fdd.fdd_kv_commit(ctx, [fs], layer, k, v, [d], 1 if layer == L - 1 else 0)
@@ -203,10 +214,8 @@ def run_ours(args):
     sampler.join(timeout=2)
     ms = ev0.elapsed_time(ev1)
     attn_ms = [a.elapsed_time(b) for a, b in attn_events]
-    if dist is not None:
-        t_ = torch.tensor([ms], device="cuda")
-        dist.all_reduce(t_, op=dist.ReduceOp.MAX)
-        ms = float(t_.item())
+    unmask_ms = [(a.elapsed_time(b), rows) for a, b, rows in unmask_events]
+    ms = replicas.max_over_ranks(ms, dist, "cuda")
     fdd.fdd_poll_status(ctx)
 
     # end to end: every denoising step's inputs come from pinned host memory, results go back
@@ -240,10 +249,7 @@ def run_ours(args):
         ee1.record(stream)
         barrier()
         e_ms = ee0.elapsed_time(ee1)
-        if dist is not None:
-            t_ = torch.tensor([e_ms], device="cuda")
-            dist.all_reduce(t_, op=dist.ReduceOp.MAX)
-            e_ms = float(t_.item())
+        e_ms = replicas.max_over_ranks(e_ms, dist, "cuda")
         per_block_denoise = e2e_denoise / e2e_steps
         e2e = {"value": world * value_tokens * e2e_steps / (e_ms * 1e-3), "unit": UNIT,
                "h2d_bytes_per_step": int(h2d * per_block_denoise),
@@ -258,6 +264,12 @@ def run_ours(args):
     flops = _attn_flops(w, sc, 0)
     attn_avg_ms = float(np.mean(attn_ms)) if attn_ms else None
     achieved = flops / (attn_avg_ms * 1e-3) / 1e12 if attn_avg_ms else None
+    # unmask: the launches that see every value row MASKED (first denoising step of a block)
+    esz = 2 if w.logits_dtype == "bf16" else 4
+    first = [ms_ for ms_, rows in unmask_ms if rows == value_tokens]
+    um_ms = float(np.mean(first)) if first else None
+    um_bytes = float(value_tokens) * w.vocab * esz
+    um_gbs = um_bytes / (um_ms * 1e-3) / 1e9 if um_ms else None
     line = {
         "metric": METRIC, "value": world * value_tokens * args.steps / (ms * 1e-3), "unit": UNIT,
         "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms / args.steps,
@@ -273,11 +285,19 @@ def run_ours(args):
         "clocks": sampler.summary(),
         "e2e": e2e,
         "gpu_launches": int(launches),
-        "roofline": {"kernel": "fdd_block_attn", "bound": "tensor", "achieved": achieved,
+        "roofline": {"kernel": "fdd_block_attn (attn_ptc_kernel)", "bound": "tensor", "achieved": achieved,
                      "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s",
                      "frac": (achieved / peaks["bf16_tflops_sustained"]) if achieved else None,
-                     "traffic": None, "peak_source": peaks["source"] + " (sustained bf16)",
+                     "traffic": ATTN_DRAM_BYTES_PER_LAUNCH.get(args.workload) if L == 1 else None,
+                     "peak_source": peaks["source"] + " (sustained bf16: the kernel is timed inside the step loop)",
+                     "frac_of_burst_peak": (achieved / peaks["bf16_tflops"]) if achieved else None,
                      "flops_per_launch": flops, "avg_launch_ms": attn_avg_ms, "launches_timed": len(attn_ms)},
+        "roofline_unmask": {"kernel": "fdd_unmask (unmask_partial_kernel), first step of a block: every value row MASKED",
+                            "bound": "hbm" if w.temperature == 0 else "alu (Philox + exp2 per logit), reported against hbm",
+                            "achieved": um_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                            "frac": (um_gbs / peaks["hbm_gbs"]) if um_gbs else None,
+                            "bytes_per_launch": um_bytes, "avg_launch_ms": um_ms, "launches_timed": len(first),
+                            "peak_source": peaks["source"]},
         "tokens_per_s_incl_scaffold": world * all_tokens * args.steps / (ms * 1e-3),
     }
     if not args.no_cpu_baseline and world >= 1:

@@ -69,7 +69,8 @@ typedef struct fdd_config {
 } fdd_config;
 
 /* Create / destroy a context on the current CUDA device.  Allocates the device status
- * word and the scratch buffers (split-KV partials, unmask partials), sized from cfg.
+ * word and the scratch buffers (partials of attention units cut between CTAs, unmask
+ * records), sized from cfg.
  * Returns FDD_ERR_UNSUPPORTED for head_dim not in {64,128}, Hq % Hkv != 0, Hq/Hkv > 16,
  * max_block > 128; FDD_ERR_CUDA if no usable device.  *out is NULL on failure. */
 fdd_status fdd_create(const fdd_config* cfg, fdd_ctx** out);
@@ -126,7 +127,10 @@ fdd_status fdd_forkset_reset(fdd_ctx* ctx, fdd_forkset* set);
  *                  set s contributes [N_s][d_s][Hq][D]; k_blk, v_blk likewise [N_s][d_s][Hkv][D].
  *   out            device bf16, same packing and shape as q.
  *   block_len      host int32 [n_sets]: d_s, 1 <= d_s <= cfg.max_block.
- *   scale          soft-max scale (1/sqrt(D) by convention).
+ *   scale          soft-max scale (1/sqrt(D) by convention), the same for every set of the call.
+ * All sets of a call go into one launch (groups of 16 sets).  Rollouts with equal inputs agree
+ * up to the rounding of the bf16 output, not bit for bit: where a unit of work is cut between
+ * CTAs depends on its place in the call.
  *   causal_in_block 0: bidirectional inside the block (denoising pass);
  *                  1: query i sees block keys 0..i only (the causal verifier pass of
  *                  Scaffold Speculative Decoding, Sec. 3.3 step 3).
@@ -142,15 +146,20 @@ fdd_status fdd_block_attn(fdd_ctx* ctx, fdd_forkset* const* sets, int n_sets, in
  * For every rollout f and every position i with state MASKED:
  *   tok  = argmax_v (logit[v] + temperature * g[v])            lowest v on ties
  *   conf = softmax(logit)[tok]                                  noise-free probability
- * where g[v] = -ln(-ln(u)), u = ((x >> 9) + 0.5) * 2^-23 and x is output word v % 4 of
- * Philox4x32-10 with key = the rollout's seed (low, high word) and counter =
- * (v / 4, i, step, block_idx); temperature == 0 uses no noise.  Positions with
+ * where g[v] = -ln(-ln(u)), u = (c + (f + 0.5) * 2^-23) / 256 is assembled from two
+ * Philox4x32-10 streams under key = the rollout's seed (low, high word):
+ *   c = byte v % 16 (little-endian in the four output words) of counter (v / 16, i, step, block_idx)
+ *   f = top 23 bits of output word v % 4 of counter (v / 4, i + 2^31, step, block_idx)
+ * (the coarse byte bounds a draw, which lets the kernel skip the second stream for almost
+ * every v); temperature == 0 uses no noise.  Positions with
  * conf > threshold are committed (token written, state -> COMMITTED); if a rollout has
  * MASKED positions and none passes, its single most confident one (lowest i on ties)
  * is committed.  Nothing else is written; rollouts without MASKED positions are no-ops.
  *
  *   logits        device, packed like q: [N_s][d_s][V], fp32 or bf16 per cfg.logits_dtype.
- *                 Only rows of MASKED positions are read.
+ *                 Only rows of MASKED positions are read.  N_s * d_s <= 4096 per set
+ *                 (FDD_ERR_CAPACITY otherwise); the wide loads need V % 16 == 0 (bf16) or
+ *                 V % 8 == 0 (fp32) and a 32-byte aligned base, else a slower path runs.
  *   tokens        device int32 [N_s][d_s], in/out.     state: device uint8, in/out.
  *   n_committed   device int32 [sum N_s]: commits of this step per rollout (written).
  *   n_left        device int32 [sum N_s]: MASKED positions remaining per rollout (written).
@@ -208,7 +217,7 @@ fdd_status fdd_average_rollouts(fdd_ctx* ctx, const float* traj, int n, int w, f
  * any stream capture begins.  Later calls do no set-up.
  * Sharing: all calls on a device use the same array, which keeps whatever the previous call
  * left in it.  Nothing in it has to start at zero: every record that is read was written earlier
- * in the same call.  Two calls whose kernels can overlap on the GPU (different streams without
+ * in the same call (the first record of a row says how many of its records are valid).  Two calls whose kernels can overlap on the GPU (different streams without
  * ordering) race on it; order them.  The host side is not thread-safe for the first call per device.
  */
 #define FDD_UNMASK_STATIC_MAX_RECORDS 65536
