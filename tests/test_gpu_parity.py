@@ -151,6 +151,115 @@ def test_attention_repeated_calls_reuse_scratch():
         fdd.fdd_destroy(ctx)
 
 
+def test_serving_mix_full_size_one_call():
+    # the ragged serving batch at full size: 16 scenes (prefix 2048..12288 tokens in shuffled pages,
+    # 1/4/16 rollouts, blocks of 16/32/64) in ONE attention call and ONE unmask call; the oracle
+    # checks one rollout of every third scene (attention) and of three scenes (unmask)
+    w = synth.workload("serving_mix")
+    ctx = harness.create_context(w)
+    try:
+        scenes = w.scenes
+        gs = [harness.GpuScene(ctx, w, i) for i in range(len(scenes))]
+        qs, ks, vs = zip(*[synth.make_qkv(w, i, 0, 0, 0) for i in range(len(scenes))])
+        pack = lambda xs: harness.bf16_tensor(np.concatenate([x.reshape(-1) for x in xs]))
+        qd, kd, vd = pack(qs), pack(ks), pack(vs)
+        out = torch.full_like(qd, float("nan"))
+        n0 = fdd.fdd_launch_count(ctx)
+        fdd.fdd_block_attn(ctx, [g.forkset for g in gs], 0, qd, kd, vd, out, [sc.block_len for sc in scenes],
+                           1.0 / np.sqrt(w.head_dim), 0)
+        fdd.fdd_poll_status(ctx)
+        assert fdd.fdd_launch_count(ctx) - n0 == 1
+        got = out.float().cpu().numpy().astype(np.float64)
+        assert np.all(np.isfinite(got))
+        off = 0
+        for i, sc in enumerate(scenes):
+            n = qs[i].size
+            if i % 3 == 0:
+                f = (i * 5) % sc.n_forks
+                pk, pv = synth.make_prefix(w, i)
+                empty = ([np.zeros((0, w.n_kv_heads, w.head_dim), dtype=np.uint16)] * sc.n_forks,) * 2
+                ref = pu.attention_oracle(w, (pk, pv), empty, qs[i], ks[i], vs[i], forks=[f])
+                pu.assert_attention_close(got[off:off + n].reshape(qs[i].shape)[[f]], ref)
+            off += n
+        # unmask: all 16 scenes in one call; logits rows are generated for the checked rollouts only
+        # (the other rollouts of a checked scene reuse them, unchecked scenes get one shared row)
+        checked = {2: 0, 7: None, 11: None}
+        for i in (7, 11):
+            checked[i] = scenes[i].n_forks - 1
+        toks, sts, lgs = [], [], []
+        shared_row = synth.make_logits_row(w, 0, 0, 0, 0, 0)
+        for i, sc in enumerate(scenes):
+            t_, s_ = synth.make_block_template(w, i, 0)
+            lg = np.empty((sc.n_forks, sc.block_len, w.vocab), dtype=np.uint16)
+            lg[:] = shared_row
+            if i in checked:
+                frozen = set(synth.scaffold_positions(w, i, 0).tolist())
+                for pos in range(sc.block_len):
+                    if pos not in frozen:
+                        lg[:, pos] = synth.make_logits_row(w, i, 0, 0, checked[i], pos)
+            toks.append(t_); sts.append(s_); lgs.append(lg)
+        lg_d = harness.bf16_tensor(np.concatenate([x.reshape(-1) for x in lgs]))
+        tok_d = torch.from_numpy(np.concatenate([x.reshape(-1) for x in toks])).cuda()
+        st_d = torch.from_numpy(np.concatenate([x.reshape(-1) for x in sts])).cuda()
+        total_forks = sum(sc.n_forks for sc in scenes)
+        n_comm = torch.full((total_forks,), -7, dtype=torch.int32, device="cuda")
+        n_left = torch.full((total_forks,), -7, dtype=torch.int32, device="cuda")
+        conf = torch.zeros(tok_d.shape, dtype=torch.float32, device="cuda")
+        fdd.fdd_unmask(ctx, [g.forkset for g in gs], lg_d, tok_d, st_d, [sc.block_len for sc in scenes],
+                       w.threshold, w.temperature, 0, 0, n_comm, n_left, conf)
+        fdd.fdd_poll_status(ctx)
+        tok_h, st_h, conf_h = tok_d.cpu().numpy(), st_d.cpu().numpy(), conf.cpu().numpy()
+        nc_h, nl_h = n_comm.cpu().numpy(), n_left.cpu().numpy()
+        assert np.all(nc_h >= 1) and np.all(nl_h >= 0)
+        row_off = fork_off = 0
+        ambiguous = 0
+        for i, sc in enumerate(scenes):
+            rows = sc.n_forks * sc.block_len
+            if i in checked:
+                f = checked[i]
+                sl = slice(row_off + f * sc.block_len, row_off + (f + 1) * sc.block_len)
+                ref = unmask_step(pu.widen_logits(w, lgs[i][[f]]), toks[i][[f]], sts[i][[f]], gs[i].seeds[[f]],
+                                  w.threshold, w.temperature, 0, 0)
+                sub = dict(tokens=tok_h[sl][None], state=st_h[sl][None], conf=conf_h[sl][None],
+                           n_committed=nc_h[fork_off + f:fork_off + f + 1], n_left=nl_h[fork_off + f:fork_off + f + 1])
+                info = pu.compare_unmask(sub, ref, toks[i][[f]], sts[i][[f]], w.threshold)
+                ambiguous += len(info["ambiguous_forks"])
+            row_off += rows
+            fork_off += sc.n_forks
+        assert ambiguous <= 1
+    finally:
+        fdd.fdd_destroy(ctx)
+
+
+def test_attention_largest_block_and_group():
+    # the limits of the interface: block of 128 positions, 16 query heads per KV head (2048 stacked
+    # rows per rollout and KV head = 8 row pairs), head_dim 64, with an earlier block in the suffix
+    sc = synth.Scene(prefix_len=389, n_forks=2, block_len=128, n_scaffold=30, n_blocks=2)
+    w = synth.Workload("wide", 16, 1, 64, 512, "bf16", "peaked", 0.9, 1.0, (sc,), qkv_sigma=0.5, seed=31)
+    ctx = harness.create_context(w)
+    try:
+        scene = harness.GpuScene(ctx, w, 0, suffix_capacity=256)
+        pk, pv = synth.make_prefix(w, 0)
+        ofs = ForkSet([pk], [pv], 2, scene.seeds)
+        _, kb, vb = synth.make_qkv(w, 0, 0, 0, 0)
+        fdd.fdd_kv_commit(ctx, [scene.forkset], 0, harness.bf16_tensor(kb), harness.bf16_tensor(vb), [128], 1)
+        ofs.kv_commit(0, kb, vb)
+        q, k, v = synth.make_qkv(w, 0, 0, 1, 0)
+        for causal in (False, True):
+            got = pu.attention_gpu(ctx, scene, q, k, v, causal=causal)
+            ref = pu.attention_oracle(w, (pk, pv), _suffix_from_oracle(ofs), q, k, v, causal=causal)
+            pu.assert_attention_close(got, ref)
+    finally:
+        fdd.fdd_destroy(ctx)
+
+
+def test_attention_group_of_three_uses_the_cuda_core_kernel():
+    # a GQA group that is not a power of two is outside the tensor-core kernel's row stacking
+    sc = synth.Scene(prefix_len=150, n_forks=2, block_len=20, n_scaffold=5, n_blocks=1)
+    w = synth.Workload("g3", 6, 2, 64, 512, "bf16", "peaked", 0.9, 1.0, (sc,), qkv_sigma=0.5, seed=32)
+    _attention_case(w)
+
+
 def test_prefix_is_never_written_and_forks_with_equal_inputs_agree():
     w = synth.small_variant(synth.workload("tts"), prefix_len=512, vocab=512, n_forks=4, n_blocks=1)
     ctx = harness.create_context(w)
