@@ -157,7 +157,7 @@ fdd_status fdd_block_attn(fdd_ctx* ctx, fdd_forkset* const* sets, int n_sets, in
  * is committed.  Nothing else is written; rollouts without MASKED positions are no-ops.
  *
  *   logits        device, packed like q: [N_s][d_s][V], fp32 or bf16 per cfg.logits_dtype.
- *                 Only rows of MASKED positions are read.  N_s * d_s <= 4096 per set
+ *                 Only rows of MASKED positions are read.  N_s * d_s <= 8192 per set
  *                 (FDD_ERR_CAPACITY otherwise); the wide loads need V % 16 == 0 (bf16) or
  *                 V % 8 == 0 (fp32) and a 32-byte aligned base, else a slower path runs.
  *   tokens        device int32 [N_s][d_s], in/out.     state: device uint8, in/out.

@@ -269,26 +269,38 @@ fdd_status fdd_unmask(fdd_ctx* ctx, fdd_forkset* const* sets, int n_sets, const 
         return fail(ctx, FDD_ERR_INVALID_ARG, "logits/tokens/state/n_committed/n_left is NULL");
     if (!(temperature >= 0.0f)) return fail(ctx, FDD_ERR_INVALID_ARG, "temperature must be >= 0");
     if (threshold != threshold) return fail(ctx, FDD_ERR_INVALID_ARG, "threshold is NaN");
-    for (int s = 0; s < n_sets; ++s)
-        if (sets[s]->n_forks * block_len[s] > kUnmaskMaxRows)
-            return fail(ctx, FDD_ERR_CAPACITY, "set %d: %d rollouts x %d positions exceed %d rows per set", s,
-                        sets[s]->n_forks, block_len[s], kUnmaskMaxRows);
     const fdd_config& c = ctx->cfg;
     const size_t esz = c.logits_dtype == FDD_LOGITS_BF16 ? 2 : 4;
+    // Sets go to the kernels in groups of at most kUnmaskMaxSets sets and kUnmaskMaxRows rows.
     size_t row_off = 0;
     int fork_off = 0;
-    for (int s = 0; s < n_sets; ++s) {
-        const fdd_forkset* fs = sets[s];
+    int s = 0;
+    while (s < n_sets) {
         UnmaskProblem p;
+        p.sets.n_sets = 0;
+        p.sets.row_off[0] = 0;
+        p.sets.fork_off[0] = 0;
+        while (s < n_sets && p.sets.n_sets < kUnmaskMaxSets) {
+            const fdd_forkset* fs = sets[s];
+            const int rows = fs->n_forks * block_len[s];
+            if (rows > kUnmaskMaxRows)
+                return fail(ctx, FDD_ERR_CAPACITY, "set %d: %d rollouts x %d positions exceed %d rows per set", s,
+                            fs->n_forks, block_len[s], kUnmaskMaxRows);
+            const int k = p.sets.n_sets;
+            if (p.sets.row_off[k] + rows > kUnmaskMaxRows) break;
+            p.sets.d[k] = block_len[s];
+            p.sets.seeds[k] = fs->d_seeds;
+            p.sets.row_off[k + 1] = p.sets.row_off[k] + rows;
+            p.sets.fork_off[k + 1] = p.sets.fork_off[k] + fs->n_forks;
+            ++p.sets.n_sets;
+            ++s;
+        }
         p.logits = static_cast<const char*>(logits) + row_off * c.vocab * esz;
         p.tokens = tokens + row_off;
         p.state = state + row_off;
-        p.seeds = fs->d_seeds;
         p.n_committed = n_committed + fork_off;
         p.n_left = n_left + fork_off;
         p.conf = conf ? conf + row_off : nullptr;
-        p.n_forks = fs->n_forks;
-        p.d = block_len[s];
         p.vocab = c.vocab;
         p.logits_dtype = c.logits_dtype;
         p.threshold = threshold;
@@ -299,8 +311,8 @@ fdd_status fdd_unmask(fdd_ctx* ctx, fdd_forkset* const* sets, int n_sets, const 
         cudaError_t e = launch_unmask(ctx, p, static_cast<cudaStream_t>(stream), &n_launches);
         ctx->launches += n_launches;
         if (e != cudaSuccess) return cuda_fail(ctx, e, "fdd_unmask launch");
-        row_off += static_cast<size_t>(fs->n_forks) * p.d;
-        fork_off += fs->n_forks;
+        row_off += static_cast<size_t>(p.sets.row_off[p.sets.n_sets]);
+        fork_off += p.sets.fork_off[p.sets.n_sets];
     }
     return FDD_OK;
 }

@@ -80,15 +80,26 @@ struct AttnProblem {
     float scale;
 };
 
+constexpr int kUnmaskMaxSets = 16;          // scenes per unmask launch
+
+// Several scenes of one unmask call, packed in set order (rows = rollouts x positions).
+struct UnmaskSets {
+    int n_sets;
+    int row_off[kUnmaskMaxSets + 1];        // first row of each set (and the total)
+    int fork_off[kUnmaskMaxSets + 1];       // first rollout of each set (and the total)
+    int d[kUnmaskMaxSets];                  // block length of each set
+    const uint64_t* seeds[kUnmaskMaxSets];  // device [n_forks of the set]
+};
+
 struct UnmaskProblem {
     const void* logits;     // [rows][V]
     int32_t* tokens;        // [rows]
     uint8_t* state;         // [rows]
-    const uint64_t* seeds;  // device [n_forks]
-    int32_t* n_committed;   // [n_forks]
-    int32_t* n_left;        // [n_forks]
+    int32_t* n_committed;   // [forks]
+    int32_t* n_left;        // [forks]
     float* conf;            // [rows] or nullptr
-    int n_forks, d, vocab, logits_dtype;
+    UnmaskSets sets;
+    int vocab, logits_dtype;
     float threshold, temperature;
     uint32_t block_idx, step;
 };
@@ -104,7 +115,7 @@ struct UnmaskPartial {
 };
 
 static constexpr int kUnmaskChunk = 8192;   // vocabulary entries per work item
-static constexpr int kUnmaskMaxRows = 4096; // rollouts x positions of one set (the kernel compacts them in shared memory)
+static constexpr int kUnmaskMaxRows = 8192; // rollouts x positions of one launch (the kernel compacts them in shared memory)
 static inline int unmask_chunks(int vocab) { return (vocab + kUnmaskChunk - 1) / kUnmaskChunk; }
 
 cudaError_t launch_attention_simple(const AttnProblem& p, int head_dim, cudaStream_t st);

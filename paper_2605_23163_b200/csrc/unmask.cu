@@ -158,9 +158,10 @@ __device__ __forceinline__ Best warp_best(Best b) {
 template <typename T>
 __global__ void __launch_bounds__(kThreads, 3)
 unmask_partial_kernel(const T* __restrict__ logits, const uint8_t* __restrict__ state,
-                      const uint64_t* __restrict__ seeds, UnmaskPartial* __restrict__ partial,
-                      int rows, int d, int vocab, int n_chunks, float temperature,
+                      const __grid_constant__ UnmaskSets sets, UnmaskPartial* __restrict__ partial,
+                      int vocab, int n_chunks, float temperature,
                       uint32_t block_idx, uint32_t step, int vec_ok) {
+    const int rows = sets.row_off[sets.n_sets];
     __shared__ uint16_t s_rows[kMaxRows];               // MASKED rows, ascending
     __shared__ int s_n_rows;
     __shared__ int s_warp_count[kThreads / 32];
@@ -208,10 +209,13 @@ unmask_partial_kernel(const T* __restrict__ logits, const uint8_t* __restrict__ 
         const T* row_ptr = logits + static_cast<size_t>(row) * vocab;
         const int seg_begin = seg * seg_len;
         const int seg_end = min(vocab, seg_begin + seg_len);
-        const int fork = row / d, pos = row - fork * d;
+        int set = 0;
+        while (set + 1 < sets.n_sets && row >= sets.row_off[set + 1]) ++set;
+        const int local = row - sets.row_off[set];
+        const int fork = local / sets.d[set], pos = local - fork * sets.d[set];   // rollout inside its set
         uint2 keys = make_uint2(0u, 0u);
         if (noisy) {
-            const uint64_t seed = seeds[fork];
+            const uint64_t seed = sets.seeds[set][fork];
             keys = make_uint2(static_cast<uint32_t>(seed), static_cast<uint32_t>(seed >> 32));
         }
 
@@ -399,15 +403,19 @@ __global__ void __launch_bounds__(128)
 unmask_finalize_kernel(const UnmaskPartial* __restrict__ partial, int32_t* __restrict__ tokens,
                        uint8_t* __restrict__ state, int32_t* __restrict__ n_committed,
                        int32_t* __restrict__ n_left, float* __restrict__ conf_out,
-                       int d, int n_chunks, float threshold) {
-    const int fork = blockIdx.x;
+                       const __grid_constant__ UnmaskSets sets, int n_chunks, float threshold) {
+    const int fork = blockIdx.x;                        // rollout index over all sets of the call
     const int i = threadIdx.x;
+    int set = 0;
+    while (set + 1 < sets.n_sets && fork >= sets.fork_off[set + 1]) ++set;
+    const int d = sets.d[set];
+    const int row0 = sets.row_off[set] + (fork - sets.fork_off[set]) * d;
     __shared__ float s_conf[128];
     __shared__ int s_masked, s_pass;
     if (i == 0) { s_masked = 0; s_pass = 0; }
     __syncthreads();
 
-    const int row = fork * d + i;
+    const int row = row0 + i;
     bool masked = false;
     float conf = -1.0f;
     int tok = 0;
@@ -464,7 +472,8 @@ namespace {
 
 // Both entry points launch the same two kernels; only the home of the records differs.
 cudaError_t launch_unmask_kernels(const UnmaskProblem& p, UnmaskPartial* partial, cudaStream_t st) {
-    const int rows = p.n_forks * p.d;
+    const int rows = p.sets.row_off[p.sets.n_sets];
+    const int forks = p.sets.fork_off[p.sets.n_sets];
     if (rows > kMaxRows) return cudaErrorInvalidValue;
     const int n_chunks = unmask_chunks(p.vocab);
     static int sm_count = 0;
@@ -479,18 +488,18 @@ cudaError_t launch_unmask_kernels(const UnmaskProblem& p, UnmaskPartial* partial
     if (p.logits_dtype == FDD_LOGITS_BF16) {
         const int vec_ok = (p.vocab % 16 == 0) && (reinterpret_cast<uintptr_t>(p.logits) % 32 == 0);
         unmask_partial_kernel<__nv_bfloat16><<<grid, kThreads, 0, st>>>(
-            static_cast<const __nv_bfloat16*>(p.logits), p.state, p.seeds, partial, rows, p.d, p.vocab,
+            static_cast<const __nv_bfloat16*>(p.logits), p.state, p.sets, partial, p.vocab,
             n_chunks, p.temperature, p.block_idx, p.step, vec_ok);
     } else {
         const int vec_ok = (p.vocab % 8 == 0) && (reinterpret_cast<uintptr_t>(p.logits) % 32 == 0);
         unmask_partial_kernel<float><<<grid, kThreads, 0, st>>>(
-            static_cast<const float*>(p.logits), p.state, p.seeds, partial, rows, p.d, p.vocab,
+            static_cast<const float*>(p.logits), p.state, p.sets, partial, p.vocab,
             n_chunks, p.temperature, p.block_idx, p.step, vec_ok);
     }
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
-    unmask_finalize_kernel<<<p.n_forks, 128, 0, st>>>(partial, p.tokens, p.state, p.n_committed,
-                                                     p.n_left, p.conf, p.d, n_chunks, p.threshold);
+    unmask_finalize_kernel<<<forks, 128, 0, st>>>(partial, p.tokens, p.state, p.n_committed,
+                                                 p.n_left, p.conf, p.sets, n_chunks, p.threshold);
     return cudaGetLastError();
 }
 
@@ -573,9 +582,13 @@ extern "C" fdd_status fdd_unmask_static(const void* logits, int logits_dtype, in
         g_static_ready[dev] = true;
     }
     UnmaskProblem p;
-    p.logits = logits; p.tokens = tokens; p.state = state; p.seeds = seeds;
+    p.logits = logits; p.tokens = tokens; p.state = state;
     p.n_committed = n_committed; p.n_left = n_left; p.conf = conf;
-    p.n_forks = n_forks; p.d = block_len; p.vocab = vocab; p.logits_dtype = logits_dtype;
+    p.sets.n_sets = 1;
+    p.sets.row_off[0] = 0; p.sets.row_off[1] = n_forks * block_len;
+    p.sets.fork_off[0] = 0; p.sets.fork_off[1] = n_forks;
+    p.sets.d[0] = block_len; p.sets.seeds[0] = seeds;
+    p.vocab = vocab; p.logits_dtype = logits_dtype;
     p.threshold = threshold; p.temperature = temperature; p.block_idx = block_idx; p.step = step;
     e = launch_unmask_kernels(p, g_static_ptr[dev], static_cast<cudaStream_t>(stream));
     if (e != cudaSuccess) {

@@ -205,9 +205,11 @@ def test_serving_mix_full_size_one_call():
         n_comm = torch.full((total_forks,), -7, dtype=torch.int32, device="cuda")
         n_left = torch.full((total_forks,), -7, dtype=torch.int32, device="cuda")
         conf = torch.zeros(tok_d.shape, dtype=torch.float32, device="cuda")
+        n0 = fdd.fdd_launch_count(ctx)
         fdd.fdd_unmask(ctx, [g.forkset for g in gs], lg_d, tok_d, st_d, [sc.block_len for sc in scenes],
                        w.threshold, w.temperature, 0, 0, n_comm, n_left, conf)
         fdd.fdd_poll_status(ctx)
+        assert fdd.fdd_launch_count(ctx) - n0 == 2        # all scenes in one pair of launches
         tok_h, st_h, conf_h = tok_d.cpu().numpy(), st_d.cpu().numpy(), conf.cpu().numpy()
         nc_h, nl_h = n_comm.cpu().numpy(), n_left.cpu().numpy()
         assert np.all(nc_h >= 1) and np.all(nl_h >= 0)
