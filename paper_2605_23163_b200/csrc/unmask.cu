@@ -78,6 +78,25 @@ __device__ __forceinline__ float ex2_fast(float x) {
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
 }
+// two fp32 values in one 64-bit register for the packed fp32x2 instructions of sm_100
+__device__ __forceinline__ uint64_t pack2(float lo, float hi) {
+    uint64_t d;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(d) : "f"(lo), "f"(hi));
+    return d;
+}
+__device__ __forceinline__ void unpack2(uint64_t v, float& lo, float& hi) {
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
+    uint64_t d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
+    uint64_t d;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
 __device__ __forceinline__ float max3f(float a, float b, float c) {
     float d;
     asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
@@ -155,7 +174,7 @@ __device__ __forceinline__ Best warp_best(Best b) {
     return b;
 }
 
-template <typename T>
+template <typename T, bool NOISY>
 __global__ void __launch_bounds__(kThreads, 3)
 unmask_partial_kernel(const T* __restrict__ logits, const uint8_t* __restrict__ state,
                       const __grid_constant__ UnmaskSets sets, UnmaskPartial* __restrict__ partial,
@@ -173,7 +192,7 @@ unmask_partial_kernel(const T* __restrict__ logits, const uint8_t* __restrict__ 
     __shared__ Best red_best[kThreads / 32];
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const bool noisy = temperature != 0.0f;
+    constexpr bool noisy = NOISY;                       // temperature > 0
 
     // Every CTA compacts the list of MASKED rows for itself (the state array is a few KB).
     {
@@ -246,29 +265,35 @@ unmask_partial_kernel(const T* __restrict__ logits, const uint8_t* __restrict__ 
                 }
                 const float mn = fmaxf(m, gm);
                 const float mnl = mn * kLog2e;
-                float s4[4] = {0.f, 0.f, 0.f, 0.f};
+                const uint64_t l2e2 = pack2(kLog2e, kLog2e), nm2 = pack2(-mnl, -mnl);
+                uint64_t s2[2] = {0ull, 0ull};
 #pragma unroll
-                for (int i = 0; i < kGroup; ++i) s4[i & 3] += ex2_fast(fmaf(val[i], kLog2e, -mnl));
+                for (int i = 0; i < kGroup; i += 2) {
+                    float x0, x1;
+                    unpack2(fma2(pack2(val[i], val[i + 1]), l2e2, nm2), x0, x1);
+                    s2[(i >> 1) & 1] = add2(s2[(i >> 1) & 1], pack2(ex2_fast(x0), ex2_fast(x1)));
+                }
+                float sa, sb;
+                unpack2(add2(s2[0], s2[1]), sa, sb);
                 // rescale by 2^((m - mn) log2e): exactly 1 while the maximum stands (the rounded mnl must
                 // not enter here, or a factor 1 + 1e-7 would compound over the groups)
-                s = s * ex2_fast((m - mn) * kLog2e) + ((s4[0] + s4[1]) + (s4[2] + s4[3]));
+                s = s * ex2_fast((m - mn) * kLog2e) + (sa + sb);
                 m = mn;
             }
             if (noisy) {
                 const uint4 r = philox4x32_10(make_uint4(static_cast<uint32_t>(v0 >> 4), pos, step, block_idx), keys);
                 const uint32_t cw[4] = {r.x, r.y, r.z, r.w};
-                uint32_t hit[4], any = 0;
+                // Does any of the 16 bytes equal 255?  (~w - 0x01010101) & w & 0x80808080 is non-zero
+                // exactly when the word has such a byte (a borrow can mark a byte above a real one
+                // too, so the places are found again, exactly, on the rare path).
+                uint32_t any = 0;
 #pragma unroll
-                for (int k = 0; k < 4; ++k) {
-                    // 0x80 in every byte of the word that equals 255
-                    const uint32_t z = ~cw[k];
-                    hit[k] = ~(((z & 0x7F7F7F7Fu) + 0x7F7F7F7Fu) | z | 0x7F7F7F7Fu);
-                    any |= hit[k];
-                }
+                for (int k = 0; k < 4; ++k) any |= (0xFEFEFEFEu - cw[k]) & cw[k] & 0x80808080u;
                 if (any) {
 #pragma unroll
                     for (int k = 0; k < 4; ++k) {
-                        uint32_t h = hit[k];
+                        const uint32_t z = ~cw[k];
+                        uint32_t h = ~(((z & 0x7F7F7F7Fu) + 0x7F7F7F7Fu) | z | 0x7F7F7F7Fu);   // 0x80 where the byte is 255
                         while (h) {
                             const int j = (__ffs(h) - 1) >> 3;
                             h &= h - 1;
@@ -285,7 +310,7 @@ unmask_partial_kernel(const T* __restrict__ logits, const uint8_t* __restrict__ 
         auto fetch = [&](int v0, uint32_t (&w)[Logit<T>::kWords]) {
             if (vec_ok && v0 < seg_end && v0 + kGroup <= vocab) Logit<T>::fetch(row_ptr + v0, w);
         };
-        {
+        if (noisy || sizeof(T) == 4) {
             // two register buffers take turns: the next group's load is in flight while this one is reduced
             uint32_t wa[Logit<T>::kWords], wb[Logit<T>::kWords];
             int v0 = seg_begin + tid * kGroup;
@@ -298,6 +323,22 @@ unmask_partial_kernel(const T* __restrict__ logits, const uint8_t* __restrict__ 
                     process(v0 + kSegQuantum, wb);
                 }
                 v0 += 2 * kSegQuantum;
+            }
+        } else {
+            // the greedy step has little arithmetic per logit to hide the memory latency behind: four
+            // buffers, three loads in flight
+            uint32_t wa[Logit<T>::kWords], wb[Logit<T>::kWords], wc[Logit<T>::kWords], wd[Logit<T>::kWords];
+            int v0 = seg_begin + tid * kGroup;
+            fetch(v0, wa);
+            fetch(v0 + kSegQuantum, wb);
+            fetch(v0 + 2 * kSegQuantum, wc);
+            while (v0 < seg_end) {
+                fetch(v0 + 3 * kSegQuantum, wd);
+                process(v0, wa);
+                if (v0 + kSegQuantum < seg_end) { fetch(v0 + 4 * kSegQuantum, wa); process(v0 + kSegQuantum, wb); }
+                if (v0 + 2 * kSegQuantum < seg_end) { fetch(v0 + 5 * kSegQuantum, wb); process(v0 + 2 * kSegQuantum, wc); }
+                if (v0 + 3 * kSegQuantum < seg_end) { fetch(v0 + 6 * kSegQuantum, wc); process(v0 + 3 * kSegQuantum, wd); }
+                v0 += 4 * kSegQuantum;
             }
         }
 
@@ -487,14 +528,24 @@ cudaError_t launch_unmask_kernels(const UnmaskProblem& p, UnmaskPartial* partial
     const dim3 grid(static_cast<unsigned>(ctas));
     if (p.logits_dtype == FDD_LOGITS_BF16) {
         const int vec_ok = (p.vocab % 16 == 0) && (reinterpret_cast<uintptr_t>(p.logits) % 32 == 0);
-        unmask_partial_kernel<__nv_bfloat16><<<grid, kThreads, 0, st>>>(
-            static_cast<const __nv_bfloat16*>(p.logits), p.state, p.sets, partial, p.vocab,
-            n_chunks, p.temperature, p.block_idx, p.step, vec_ok);
+        if (p.temperature != 0.0f)
+            unmask_partial_kernel<__nv_bfloat16, true><<<grid, kThreads, 0, st>>>(
+                static_cast<const __nv_bfloat16*>(p.logits), p.state, p.sets, partial, p.vocab,
+                n_chunks, p.temperature, p.block_idx, p.step, vec_ok);
+        else
+            unmask_partial_kernel<__nv_bfloat16, false><<<grid, kThreads, 0, st>>>(
+                static_cast<const __nv_bfloat16*>(p.logits), p.state, p.sets, partial, p.vocab,
+                n_chunks, p.temperature, p.block_idx, p.step, vec_ok);
     } else {
         const int vec_ok = (p.vocab % 8 == 0) && (reinterpret_cast<uintptr_t>(p.logits) % 32 == 0);
-        unmask_partial_kernel<float><<<grid, kThreads, 0, st>>>(
-            static_cast<const float*>(p.logits), p.state, p.sets, partial, p.vocab,
-            n_chunks, p.temperature, p.block_idx, p.step, vec_ok);
+        if (p.temperature != 0.0f)
+            unmask_partial_kernel<float, true><<<grid, kThreads, 0, st>>>(
+                static_cast<const float*>(p.logits), p.state, p.sets, partial, p.vocab,
+                n_chunks, p.temperature, p.block_idx, p.step, vec_ok);
+        else
+            unmask_partial_kernel<float, false><<<grid, kThreads, 0, st>>>(
+                static_cast<const float*>(p.logits), p.state, p.sets, partial, p.vocab,
+                n_chunks, p.temperature, p.block_idx, p.step, vec_ok);
     }
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
