@@ -7,6 +7,7 @@
  *   fdd_block_attn       block-causal attention of the current block    (Sec. 3.1, "Block-Causal Diffusion")
  *   fdd_unmask           confidence-threshold parallel unmasking        (Sec. 3.3, "Section Diffusion";
  *                                                                        Sec. 3.2 scaffold; Sec. 3.1 "visible tokens fixed")
+ *   fdd_ss_draft/_accept draft and accept scan of Scaffold Speculative Decoding (Sec. 3.3, Algorithm)
  *   fdd_kv_commit        append the finished block to each private cache (Sec. 3.3 cache reuse; Sec. 3.4 fork)
  *   fdd_average_rollouts equal-weight mean of N trajectories            (Sec. 3.4, trajectory averaging)
  *
@@ -24,7 +25,7 @@
  *   - A context and its fork sets must be used from one host thread at a time.
  *
  * Position state codes (uint8): 0 = MASKED (to be decoded), 1 = COMMITTED, 2 = SCAFFOLD
- * (frozen structural token, Sec. 3.2).
+ * (frozen structural token, Sec. 3.2), 3 = DRAFT (between fdd_ss_draft and fdd_ss_accept).
  */
 #ifndef FDD_H_
 #define FDD_H_
@@ -49,6 +50,7 @@ typedef int fdd_status;
 #define FDD_MASKED    0
 #define FDD_COMMITTED 1
 #define FDD_SCAFFOLD  2
+#define FDD_DRAFT     3   /* drafted, not yet verified (Scaffold Speculative Decoding only) */
 
 #define FDD_LOGITS_F32  0
 #define FDD_LOGITS_BF16 1
@@ -170,6 +172,33 @@ fdd_status fdd_unmask(fdd_ctx* ctx, fdd_forkset* const* sets, int n_sets, const 
                       int32_t* tokens, uint8_t* state, const int32_t* block_len,
                       float threshold, float temperature, uint32_t block_idx, uint32_t step,
                       int32_t* n_committed, int32_t* n_left, float* conf, void* stream);
+
+/*
+ * fdd_ss_draft, fdd_ss_accept -- Scaffold Speculative Decoding (Sec. 3.3, Algorithm steps 1-3).
+ * Scaffold positions are accepted as they are (step 1: they are never read or written).
+ *
+ * fdd_ss_draft (step 2): `logits` are the diffusion head's, from one bidirectional pass
+ * (fdd_block_attn with causal_in_block = 0).  Every MASKED position gets
+ * argmax_v (logit[v] + temperature * g[v]) (noise and packing as in fdd_unmask) and the state
+ * FDD_DRAFT.  n_drafted / n_left: device int32 [sum N_s], drafts written / MASKED left (0).
+ *
+ * fdd_ss_accept (step 3): `ar_logits[f][i]` are the AR head's logits FOR position i from one causal
+ * pass over the block (fdd_block_attn with causal_in_block = 1).  Per rollout, over the FDD_DRAFT
+ * positions from left to right: the draft is accepted (state -> COMMITTED) while it equals the
+ * verifier's token argmax_v (ar_logit[v] + temperature * g[v]) (temperature > 0: the sampled
+ * verifier of Sec. 3.4); at the first mismatch the verifier's token replaces the draft and is
+ * accepted, and every later FDD_DRAFT position goes back to MASKED for the next draft / verify
+ * cycle.  n_accepted: positions that became COMMITTED in this call; n_left: MASKED afterwards.
+ * Only rows in state FDD_DRAFT are read.  Limits as for fdd_unmask.
+ */
+fdd_status fdd_ss_draft(fdd_ctx* ctx, fdd_forkset* const* sets, int n_sets, const void* logits,
+                        int32_t* tokens, uint8_t* state, const int32_t* block_len,
+                        float temperature, uint32_t block_idx, uint32_t step,
+                        int32_t* n_drafted, int32_t* n_left, void* stream);
+fdd_status fdd_ss_accept(fdd_ctx* ctx, fdd_forkset* const* sets, int n_sets, const void* ar_logits,
+                         int32_t* tokens, uint8_t* state, const int32_t* block_len,
+                         float temperature, uint32_t block_idx, uint32_t step,
+                         int32_t* n_accepted, int32_t* n_left, void* stream);
 
 /*
  * fdd_kv_commit -- Sec. 3.3 / 3.4: a finished block's K/V join the cache of the rollout

@@ -257,10 +257,10 @@ fdd_status fdd_block_attn(fdd_ctx* ctx, fdd_forkset* const* sets, int n_sets, in
     return FDD_OK;
 }
 
-fdd_status fdd_unmask(fdd_ctx* ctx, fdd_forkset* const* sets, int n_sets, const void* logits,
-                      int32_t* tokens, uint8_t* state, const int32_t* block_len,
-                      float threshold, float temperature, uint32_t block_idx, uint32_t step,
-                      int32_t* n_committed, int32_t* n_left, float* conf, void* stream) {
+static fdd_status unmask_like(fdd_ctx* ctx, fdd_forkset* const* sets, int n_sets, const void* logits,
+                              int32_t* tokens, uint8_t* state, const int32_t* block_len,
+                              float threshold, float temperature, uint32_t block_idx, uint32_t step,
+                              int32_t* n_committed, int32_t* n_left, float* conf, void* stream, int mode) {
     if (!ctx) return FDD_ERR_INVALID_ARG;
     int total = 0;
     fdd_status st = check_sets(ctx, sets, n_sets, block_len, &total);
@@ -308,13 +308,38 @@ fdd_status fdd_unmask(fdd_ctx* ctx, fdd_forkset* const* sets, int n_sets, const 
         p.block_idx = block_idx;
         p.step = step;
         int n_launches = 0;
-        cudaError_t e = launch_unmask(ctx, p, static_cast<cudaStream_t>(stream), &n_launches);
+        cudaError_t e = launch_unmask(ctx, p, static_cast<cudaStream_t>(stream), &n_launches, mode);
         ctx->launches += n_launches;
         if (e != cudaSuccess) return cuda_fail(ctx, e, "fdd_unmask launch");
         row_off += static_cast<size_t>(p.sets.row_off[p.sets.n_sets]);
         fork_off += p.sets.fork_off[p.sets.n_sets];
     }
     return FDD_OK;
+}
+
+fdd_status fdd_unmask(fdd_ctx* ctx, fdd_forkset* const* sets, int n_sets, const void* logits,
+                      int32_t* tokens, uint8_t* state, const int32_t* block_len,
+                      float threshold, float temperature, uint32_t block_idx, uint32_t step,
+                      int32_t* n_committed, int32_t* n_left, float* conf, void* stream) {
+    return unmask_like(ctx, sets, n_sets, logits, tokens, state, block_len, threshold, temperature, block_idx, step,
+                       n_committed, n_left, conf, stream, 0);
+}
+
+fdd_status fdd_ss_draft(fdd_ctx* ctx, fdd_forkset* const* sets, int n_sets, const void* logits,
+                        int32_t* tokens, uint8_t* state, const int32_t* block_len,
+                        float temperature, uint32_t block_idx, uint32_t step,
+                        int32_t* n_drafted, int32_t* n_left, void* stream) {
+    // every MASKED position passes a threshold below any probability
+    return unmask_like(ctx, sets, n_sets, logits, tokens, state, block_len, -1.0f, temperature, block_idx, step,
+                       n_drafted, n_left, nullptr, stream, 1);
+}
+
+fdd_status fdd_ss_accept(fdd_ctx* ctx, fdd_forkset* const* sets, int n_sets, const void* ar_logits,
+                         int32_t* tokens, uint8_t* state, const int32_t* block_len,
+                         float temperature, uint32_t block_idx, uint32_t step,
+                         int32_t* n_accepted, int32_t* n_left, void* stream) {
+    return unmask_like(ctx, sets, n_sets, ar_logits, tokens, state, block_len, 0.0f, temperature, block_idx, step,
+                       n_accepted, n_left, nullptr, stream, 2);
 }
 
 fdd_status fdd_kv_commit(fdd_ctx* ctx, fdd_forkset* const* sets, int n_sets, int layer,

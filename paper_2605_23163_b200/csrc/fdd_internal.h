@@ -123,7 +123,7 @@ bool attention_tc_supported(const AttnProblem& a, int head_dim);
 size_t attention_ptc_workspace_bytes(int head_dim, int max_ctas);
 cudaError_t launch_attention_ptc(fdd_ctx* ctx, const AttnProblem* probs, TcMapCache* const* caches, int n,
                                  int head_dim, cudaStream_t st, int* n_launches);
-cudaError_t launch_unmask(fdd_ctx* ctx, const UnmaskProblem& p, cudaStream_t st, int* n_launches);
+cudaError_t launch_unmask(fdd_ctx* ctx, const UnmaskProblem& p, cudaStream_t st, int* n_launches, int mode = 0);
 cudaError_t launch_kv_commit(const __nv_bfloat16* k_blk, const __nv_bfloat16* v_blk,
                              __nv_bfloat16* suffix_k, __nv_bfloat16* suffix_v,
                              int n_forks, int d, int n_kv_heads, int head_dim,

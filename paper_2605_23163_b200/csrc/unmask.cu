@@ -179,9 +179,9 @@ __global__ void __launch_bounds__(kThreads, 3)
 unmask_partial_kernel(const T* __restrict__ logits, const uint8_t* __restrict__ state,
                       const __grid_constant__ UnmaskSets sets, UnmaskPartial* __restrict__ partial,
                       int vocab, int n_chunks, float temperature,
-                      uint32_t block_idx, uint32_t step, int vec_ok) {
+                      uint32_t block_idx, uint32_t step, int vec_ok, int select_state) {
     const int rows = sets.row_off[sets.n_sets];
-    __shared__ uint16_t s_rows[kMaxRows];               // MASKED rows, ascending
+    __shared__ uint16_t s_rows[kMaxRows];               // the selected rows (MASKED, or DRAFT for the verifier), ascending
     __shared__ int s_n_rows;
     __shared__ int s_warp_count[kThreads / 32];
     __shared__ int s_cand[kMaxCand];                    // vocabulary ids with coarse byte 255
@@ -199,7 +199,7 @@ unmask_partial_kernel(const T* __restrict__ logits, const uint8_t* __restrict__ 
         int base = 0;
         for (int r0 = 0; r0 < rows; r0 += kThreads) {
             const int r = r0 + tid;
-            const bool m = r < rows && state[r] == FDD_MASKED;
+            const bool m = r < rows && state[r] == select_state;
             const unsigned bal = __ballot_sync(0xFFFFFFFFu, m);
             if (lane == 0) s_warp_count[warp] = __popc(bal);
             __syncthreads();
@@ -444,7 +444,7 @@ __global__ void __launch_bounds__(128)
 unmask_finalize_kernel(const UnmaskPartial* __restrict__ partial, int32_t* __restrict__ tokens,
                        uint8_t* __restrict__ state, int32_t* __restrict__ n_committed,
                        int32_t* __restrict__ n_left, float* __restrict__ conf_out,
-                       const __grid_constant__ UnmaskSets sets, int n_chunks, float threshold) {
+                       const __grid_constant__ UnmaskSets sets, int n_chunks, float threshold, int commit_state) {
     const int fork = blockIdx.x;                        // rollout index over all sets of the call
     const int i = threadIdx.x;
     int set = 0;
@@ -497,7 +497,7 @@ unmask_finalize_kernel(const UnmaskPartial* __restrict__ partial, int32_t* __res
     }
     if (commit && i < d) {
         tokens[row] = tok;
-        state[row] = FDD_COMMITTED;
+        state[row] = static_cast<uint8_t>(commit_state);
     }
     if (i == 0) {
         const int nc = (n_masked == 0) ? 0 : (n_pass > 0 ? n_pass : 1);
@@ -507,12 +507,68 @@ unmask_finalize_kernel(const UnmaskPartial* __restrict__ partial, int32_t* __res
 }
 
 
+// Accept scan of Scaffold Speculative Decoding: one CTA per rollout.  The first kernel has left, for
+// every DRAFT row, the verifier's token (arg-max of its perturbed logits).  Going left to right, a
+// draft is accepted while it equals the verifier's token; at the first mismatch the verifier's token
+// replaces it and every later draft goes back to MASKED.
+__global__ void __launch_bounds__(128)
+ss_accept_kernel(const UnmaskPartial* __restrict__ partial, int32_t* __restrict__ tokens,
+                 uint8_t* __restrict__ state, int32_t* __restrict__ n_accepted, int32_t* __restrict__ n_left,
+                 const __grid_constant__ UnmaskSets sets, int n_chunks) {
+    const int fork = blockIdx.x;
+    const int i = threadIdx.x;
+    int set = 0;
+    while (set + 1 < sets.n_sets && fork >= sets.fork_off[set + 1]) ++set;
+    const int d = sets.d[set];
+    const int row = sets.row_off[set] + (fork - sets.fork_off[set]) * d + i;
+    __shared__ int s_first_mismatch, s_accepted, s_masked;
+    if (i == 0) { s_first_mismatch = 0x7FFFFFFF; s_accepted = 0; s_masked = 0; }
+    __syncthreads();
+    int st = FDD_SCAFFOLD, tok = 0;
+    bool draft = false, mismatch = false;
+    if (i < d) {
+        st = state[row];
+        draft = st == FDD_DRAFT;
+        if (draft) {
+            const UnmaskPartial* p = partial + static_cast<size_t>(row) * n_chunks;
+            const int n_rec = p[0].pad[0];
+            Best B{-CUDART_INF_F, -CUDART_INF_F, 0x7FFFFFFF};
+            for (int c = 0; c < n_rec; ++c) B = better(B, Best{p[c].best_score, p[c].best_logit, p[c].best_index});
+            tok = B.index;
+            mismatch = tok != tokens[row];
+            if (mismatch) atomicMin(&s_first_mismatch, i);
+        }
+    }
+    __syncthreads();
+    const int stop = s_first_mismatch;                  // position of the replacement token, if any
+    if (draft) {
+        if (i <= stop) {
+            if (i == stop) tokens[row] = tok;           // the verifier's token, always accepted
+            state[row] = FDD_COMMITTED;
+            atomicAdd(&s_accepted, 1);
+        } else {
+            state[row] = FDD_MASKED;                    // discarded draft
+            atomicAdd(&s_masked, 1);
+        }
+    } else if (i < d && st == FDD_MASKED) {
+        atomicAdd(&s_masked, 1);
+    }
+    __syncthreads();
+    if (i == 0) {
+        n_accepted[fork] = s_accepted;
+        n_left[fork] = s_masked;
+    }
+}
+
 }  // namespace
 
 namespace {
 
 // Both entry points launch the same two kernels; only the home of the records differs.
-cudaError_t launch_unmask_kernels(const UnmaskProblem& p, UnmaskPartial* partial, cudaStream_t st) {
+// mode 0: unmasking step; 1: draft of Scaffold Speculative Decoding (every MASKED row becomes DRAFT);
+// 2: its accept scan (rows in state DRAFT are read, then the scan runs).
+cudaError_t launch_unmask_kernels(const UnmaskProblem& p, UnmaskPartial* partial, cudaStream_t st, int mode = 0) {
+    const int select_state = mode == 2 ? FDD_DRAFT : FDD_MASKED;
     const int rows = p.sets.row_off[p.sets.n_sets];
     const int forks = p.sets.fork_off[p.sets.n_sets];
     if (rows > kMaxRows) return cudaErrorInvalidValue;
@@ -531,34 +587,37 @@ cudaError_t launch_unmask_kernels(const UnmaskProblem& p, UnmaskPartial* partial
         if (p.temperature != 0.0f)
             unmask_partial_kernel<__nv_bfloat16, true><<<grid, kThreads, 0, st>>>(
                 static_cast<const __nv_bfloat16*>(p.logits), p.state, p.sets, partial, p.vocab,
-                n_chunks, p.temperature, p.block_idx, p.step, vec_ok);
+                n_chunks, p.temperature, p.block_idx, p.step, vec_ok, select_state);
         else
             unmask_partial_kernel<__nv_bfloat16, false><<<grid, kThreads, 0, st>>>(
                 static_cast<const __nv_bfloat16*>(p.logits), p.state, p.sets, partial, p.vocab,
-                n_chunks, p.temperature, p.block_idx, p.step, vec_ok);
+                n_chunks, p.temperature, p.block_idx, p.step, vec_ok, select_state);
     } else {
         const int vec_ok = (p.vocab % 8 == 0) && (reinterpret_cast<uintptr_t>(p.logits) % 32 == 0);
         if (p.temperature != 0.0f)
             unmask_partial_kernel<float, true><<<grid, kThreads, 0, st>>>(
                 static_cast<const float*>(p.logits), p.state, p.sets, partial, p.vocab,
-                n_chunks, p.temperature, p.block_idx, p.step, vec_ok);
+                n_chunks, p.temperature, p.block_idx, p.step, vec_ok, select_state);
         else
             unmask_partial_kernel<float, false><<<grid, kThreads, 0, st>>>(
                 static_cast<const float*>(p.logits), p.state, p.sets, partial, p.vocab,
-                n_chunks, p.temperature, p.block_idx, p.step, vec_ok);
+                n_chunks, p.temperature, p.block_idx, p.step, vec_ok, select_state);
     }
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
-    unmask_finalize_kernel<<<forks, 128, 0, st>>>(partial, p.tokens, p.state, p.n_committed,
-                                                 p.n_left, p.conf, p.sets, n_chunks, p.threshold);
+    if (mode == 2)
+        ss_accept_kernel<<<forks, 128, 0, st>>>(partial, p.tokens, p.state, p.n_committed, p.n_left, p.sets, n_chunks);
+    else
+        unmask_finalize_kernel<<<forks, 128, 0, st>>>(partial, p.tokens, p.state, p.n_committed, p.n_left, p.conf,
+                                                     p.sets, n_chunks, p.threshold, mode == 1 ? FDD_DRAFT : FDD_COMMITTED);
     return cudaGetLastError();
 }
 
 }  // namespace
 
-cudaError_t launch_unmask(fdd_ctx* ctx, const UnmaskProblem& p, cudaStream_t st, int* n_launches) {
+cudaError_t launch_unmask(fdd_ctx* ctx, const UnmaskProblem& p, cudaStream_t st, int* n_launches, int mode) {
     *n_launches += 2;
-    return launch_unmask_kernels(p, static_cast<UnmaskPartial*>(ctx->ws_unmask), st);
+    return launch_unmask_kernels(p, static_cast<UnmaskPartial*>(ctx->ws_unmask), st, mode);
 }
 
 // -------------------------------------------------------------------------------------------------

@@ -15,13 +15,13 @@ LIB_PATH = os.path.join(_PKG, "libfdd.so")
 FDD_OK = 0
 FDD_ERR_INVALID_ARG, FDD_ERR_SHAPE, FDD_ERR_CAPACITY, FDD_ERR_STATE = -1, -2, -3, -4
 FDD_ERR_CUDA, FDD_ERR_DEVICE_TIMEOUT, FDD_ERR_UNSUPPORTED = -5, -6, -7
-FDD_MASKED, FDD_COMMITTED, FDD_SCAFFOLD = 0, 1, 2
+FDD_MASKED, FDD_COMMITTED, FDD_SCAFFOLD, FDD_DRAFT = 0, 1, 2, 3
 FDD_LOGITS_F32, FDD_LOGITS_BF16 = 0, 1
 
 EXPORTS = (
     "fdd_create", "fdd_destroy", "fdd_last_error", "fdd_launch_count", "fdd_fork",
     "fdd_forkset_free", "fdd_forkset_suffix_len", "fdd_forkset_reset", "fdd_block_attn",
-    "fdd_unmask", "fdd_kv_commit", "fdd_average_rollouts", "fdd_poll_status", "fdd_unmask_static",
+    "fdd_unmask", "fdd_ss_draft", "fdd_ss_accept", "fdd_kv_commit", "fdd_average_rollouts", "fdd_poll_status", "fdd_unmask_static",
 )
 FDD_UNMASK_STATIC_MAX_RECORDS = 65536
 
@@ -74,6 +74,9 @@ def lib():
     L.fdd_block_attn.restype = i32
     L.fdd_unmask.argtypes = [vp, vpp, i32, vp, vp, vp, ip, f32, f32, u32, u32, vp, vp, vp, vp]
     L.fdd_unmask.restype = i32
+    for fn in (L.fdd_ss_draft, L.fdd_ss_accept):
+        fn.argtypes = [vp, vpp, i32, vp, vp, vp, ip, f32, u32, u32, vp, vp, vp]
+        fn.restype = i32
     L.fdd_kv_commit.argtypes = [vp, vpp, i32, i32, vp, vp, ip, i32, vp]
     L.fdd_kv_commit.restype = i32
     L.fdd_average_rollouts.argtypes = [vp, vp, i32, i32, vp, vp]
@@ -189,6 +192,20 @@ def fdd_unmask(ctx, sets, logits, tokens, state, block_len, threshold, temperatu
         ctx, _ptr_array(sets), len(sets), _ptr(logits), _ptr(tokens), _ptr(state),
         _i32_array(block_len), float(threshold), float(temperature), int(block_idx), int(step),
         _ptr(n_committed), _ptr(n_left), _ptr(conf), _stream(stream)))
+
+
+def fdd_ss_draft(ctx, sets, logits, tokens, state, block_len, temperature, block_idx, step, n_drafted, n_left,
+                 stream=None):
+    return _check(ctx, lib().fdd_ss_draft(
+        ctx, _ptr_array(sets), len(sets), _ptr(logits), _ptr(tokens), _ptr(state), _i32_array(block_len),
+        float(temperature), int(block_idx), int(step), _ptr(n_drafted), _ptr(n_left), _stream(stream)))
+
+
+def fdd_ss_accept(ctx, sets, ar_logits, tokens, state, block_len, temperature, block_idx, step, n_accepted, n_left,
+                  stream=None):
+    return _check(ctx, lib().fdd_ss_accept(
+        ctx, _ptr_array(sets), len(sets), _ptr(ar_logits), _ptr(tokens), _ptr(state), _i32_array(block_len),
+        float(temperature), int(block_idx), int(step), _ptr(n_accepted), _ptr(n_left), _stream(stream)))
 
 
 def fdd_kv_commit(ctx, sets, layer, k_blk, v_blk, block_len, advance, stream=None):

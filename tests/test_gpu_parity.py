@@ -442,6 +442,67 @@ def test_unmask_long_prefix_full_size_step0():
 
 
 # ---------------------------------------------------------------------------------------------
+# Scaffold Speculative Decoding: draft and accept scan
+# ---------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("temperature", [0.0, 0.9])
+def test_ss_draft_and_accept_cycles_match_oracle(temperature):
+    from oracle.ss import DRAFT, ss_accept, ss_draft
+    w = synth.small_variant(synth.workload("tts"), prefix_len=64, vocab=8192 + 4096, n_forks=5, n_blocks=1)
+    sc = w.scenes[0]
+    ctx = harness.create_context(w)
+    try:
+        scene = harness.GpuScene(ctx, w, 0)
+        tokens, state = synth.make_block_template(w, 0, 0)
+        n_a = torch.full((sc.n_forks,), -7, dtype=torch.int32, device="cuda")
+        n_l = torch.full((sc.n_forks,), -7, dtype=torch.int32, device="cuda")
+        g = np.random.default_rng(77)
+        cycle = 0
+        while np.any(state == MASKED):
+            # draft
+            logits = synth.make_logits(w, 0, 0, cycle, rows="all")
+            tok_d, st_d = torch.from_numpy(tokens).cuda(), torch.from_numpy(state).cuda()
+            fdd.fdd_ss_draft(ctx, [scene.forkset], harness.logits_tensor(w, logits), tok_d, st_d, [sc.block_len],
+                             temperature, 0, 2 * cycle, n_a, n_l)
+            fdd.fdd_poll_status(ctx)
+            ref_t, ref_s = ss_draft(pu.widen_logits(w, logits), tokens, state, scene.seeds, temperature, 0, 2 * cycle)
+            margins = unmask_step(pu.widen_logits(w, logits), tokens, state, scene.seeds, -1.0, temperature, 0,
+                                  2 * cycle)["score_margin"]
+            got_t, got_s = tok_d.cpu().numpy(), st_d.cpu().numpy()
+            assert np.array_equal(got_s, ref_s) and not np.any(got_s == MASKED)
+            clear = margins > pu.SCORE_MARGIN
+            assert np.array_equal(got_t[clear], ref_t[clear]) and clear.mean() > 0.99
+            assert np.array_equal(n_a.cpu().numpy(), (state == MASKED).sum(axis=1)) and not n_l.cpu().numpy().any()
+            tokens, state = ref_t, ref_s                    # continue from the oracle's drafts
+            # verifier logits: agrees with the first k_f drafts of rollout f, then with nothing in particular
+            ar = (g.standard_normal((sc.n_forks, sc.block_len, w.vocab)) * 0.5).astype(np.float32)
+            for f in range(sc.n_forks):
+                drafts = np.nonzero(state[f] == DRAFT)[0]
+                k = int(g.integers(0, len(drafts) + 1)) if f else len(drafts)      # rollout 0: all accepted
+                for i in drafts[:k]:
+                    ar[f, i, tokens[f, i]] = 12.0
+            ar_bits = synth.f32_to_bf16_bits(ar)
+            tok_d, st_d = torch.from_numpy(tokens).cuda(), torch.from_numpy(state).cuda()
+            fdd.fdd_ss_accept(ctx, [scene.forkset], harness.bf16_tensor(ar_bits), tok_d, st_d, [sc.block_len],
+                              temperature, 0, 2 * cycle + 1, n_a, n_l)
+            fdd.fdd_poll_status(ctx)
+            ref = ss_accept(pu.widen_logits(w, ar_bits), tokens, state, scene.seeds, temperature, 0, 2 * cycle + 1)
+            got_t, got_s = tok_d.cpu().numpy(), st_d.cpu().numpy()
+            for f in range(sc.n_forks):
+                if np.all(ref["score_margin"][f] > pu.SCORE_MARGIN):
+                    assert np.array_equal(got_t[f], ref["tokens"][f]) and np.array_equal(got_s[f], ref["state"][f])
+                    assert n_a.cpu().numpy()[f] == ref["n_accepted"][f] and n_l.cpu().numpy()[f] == ref["n_left"][f]
+            keep = state == SCAFFOLD
+            assert np.array_equal(got_t[keep], tokens[keep]) and np.all(got_s[keep] == SCAFFOLD)
+            assert not np.any(got_s == DRAFT)
+            tokens, state = ref["tokens"], ref["state"]
+            cycle += 1
+            assert cycle <= sc.block_len
+        assert cycle >= 2
+    finally:
+        fdd.fdd_destroy(ctx)
+
+
+# ---------------------------------------------------------------------------------------------
 # whole block loop, averaging
 # ---------------------------------------------------------------------------------------------
 def test_block_loop_matches_oracle_and_averages():
