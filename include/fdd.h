@@ -8,6 +8,7 @@
  *   fdd_unmask           confidence-threshold parallel unmasking        (Sec. 3.3, "Section Diffusion";
  *                                                                        Sec. 3.2 scaffold; Sec. 3.1 "visible tokens fixed")
  *   fdd_ss_draft/_accept draft and accept scan of Scaffold Speculative Decoding (Sec. 3.3, Algorithm)
+ *   fdd_plan_blocks      section-aligned blocks of the output template         (Sec. 3.2)
  *   fdd_kv_commit        append the finished block to each private cache (Sec. 3.3 cache reuse; Sec. 3.4 fork)
  *   fdd_average_rollouts equal-weight mean of N trajectories            (Sec. 3.4, trajectory averaging)
  *
@@ -255,6 +256,23 @@ fdd_status fdd_unmask_static(const void* logits, int logits_dtype, int n_forks, 
                              float threshold, float temperature, uint32_t block_idx, uint32_t step,
                              int32_t* n_committed, int32_t* n_left, float* conf, void* stream,
                              char* err, size_t err_len);
+
+/*
+ * fdd_plan_blocks -- Sec. 3.2 "Section-Aligned Blocks": block borders follow section borders, and
+ * section s with E_s editable (value) positions is cut into ceil(E_s / d) blocks.  Host code only.
+ * Inside a section the blocks are filled from the left with d editable positions each (the last
+ * takes the rest); a block ends right after its last editable position, the section's last block
+ * at the section's end, so scaffold tokens travel with the value tokens that follow them; a
+ * section without editable positions is one block that needs no decoding.
+ *   editable       host uint8 [length]: 1 = value position, 0 = scaffold
+ *   section_end    host int32 [n_sections]: exclusive end of each section, non-decreasing, last == length
+ *   block_begin, block_end, block_section   host int32 [capacity], written: block b covers positions
+ *                  [block_begin[b], block_end[b]) of section block_section[b]; *n_blocks = their number
+ * FDD_ERR_CAPACITY if more than `capacity` blocks are needed, FDD_ERR_INVALID_ARG for bad arguments.
+ */
+fdd_status fdd_plan_blocks(const uint8_t* editable, const int32_t* section_end, int n_sections,
+                           int length, int d, int32_t* block_begin, int32_t* block_end,
+                           int32_t* block_section, int capacity, int* n_blocks);
 
 /* Synchronise `stream` and return the device status word: FDD_OK, or the first error a
  * kernel recorded (FDD_ERR_DEVICE_TIMEOUT).  Reading clears it. */

@@ -21,7 +21,7 @@ FDD_LOGITS_F32, FDD_LOGITS_BF16 = 0, 1
 EXPORTS = (
     "fdd_create", "fdd_destroy", "fdd_last_error", "fdd_launch_count", "fdd_fork",
     "fdd_forkset_free", "fdd_forkset_suffix_len", "fdd_forkset_reset", "fdd_block_attn",
-    "fdd_unmask", "fdd_ss_draft", "fdd_ss_accept", "fdd_kv_commit", "fdd_average_rollouts", "fdd_poll_status", "fdd_unmask_static",
+    "fdd_unmask", "fdd_ss_draft", "fdd_ss_accept", "fdd_kv_commit", "fdd_average_rollouts", "fdd_poll_status", "fdd_unmask_static", "fdd_plan_blocks",
 )
 FDD_UNMASK_STATIC_MAX_RECORDS = 65536
 
@@ -217,6 +217,25 @@ def fdd_kv_commit(ctx, sets, layer, k_blk, v_blk, block_len, advance, stream=Non
 def fdd_average_rollouts(ctx, traj, n, w, out, stream=None):
     return _check(ctx, lib().fdd_average_rollouts(ctx, _ptr(traj), int(n), int(w), _ptr(out),
                                                   _stream(stream)))
+
+
+def fdd_plan_blocks(editable, section_end, d, capacity=4096):
+    """Host-side block planner; returns a list of (begin, end, section)."""
+    import numpy as np
+    ed = np.ascontiguousarray(editable, dtype=np.uint8)
+    en = np.ascontiguousarray(section_end, dtype=np.int32)
+    bb, be, bs = (np.zeros(capacity, dtype=np.int32) for _ in range(3))
+    n = ctypes.c_int(0)
+    L = lib()
+    L.fdd_plan_blocks.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.c_int, ctypes.c_int,
+                                  ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int,
+                                  ctypes.POINTER(ctypes.c_int)]
+    L.fdd_plan_blocks.restype = ctypes.c_int
+    st = L.fdd_plan_blocks(ed.ctypes.data, en.ctypes.data, len(en), len(ed), int(d), bb.ctypes.data, be.ctypes.data,
+                           bs.ctypes.data, capacity, ctypes.byref(n))
+    if st < 0:
+        raise FddError(st, "fdd_plan_blocks failed")
+    return [(int(bb[i]), int(be[i]), int(bs[i])) for i in range(n.value)]
 
 
 def fdd_poll_status(ctx, stream=None):
