@@ -118,22 +118,34 @@ def run_ours(args):
     fdd.lib()
     w = synth.workload(args.workload)
     w = replicas.replica_workload(w, rank)     # every rank decodes its own scene (different seed)
+    # A workload is one scene or a batch of independent scenes (the serving mix): every call below
+    # takes all of them at once, packed in scene order.
+    n_scenes = len(w.scenes)
     sc = w.scenes[0]
     L = args.layers
     ctx = harness.create_context(w, n_layers=L)
-    scene = harness.GpuScene(ctx, w, 0, n_layers=L, suffix_capacity=sc.block_len)
+    gscenes = [harness.GpuScene(ctx, w, i, n_layers=L, suffix_capacity=w.scenes[i].block_len) for i in range(n_scenes)]
+    for g in gscenes:                      # the benchmark forks anew for every block
+        g.free()
     stream = torch.cuda.current_stream()
     scale = 1.0 / np.sqrt(w.head_dim)
-    d, N = sc.block_len, sc.n_forks
+    ds = [s_.block_len for s_ in w.scenes]
+    Ns = [s_.n_forks for s_ in w.scenes]
+    d, N = max(ds), sum(Ns)
 
     pool = ThreadPoolExecutor(max_workers=max(1, len(os.sched_getaffinity(0))))
-    host_steps = [_gen_step_inputs(w, 0, 0, t, pool) for t in range(PRE_STEPS)]
+    host_steps = []
+    for t in range(PRE_STEPS):
+        per_scene = [_gen_step_inputs(w, i, 0, t, pool) for i in range(n_scenes)]
+        host_steps.append(tuple(np.concatenate([x[j].reshape(-1) for x in per_scene]) for j in range(4)))
     pool.shutdown()
     dev_steps = []
     for q, k, v, lg in host_steps:
         dev_steps.append(tuple([harness.bf16_tensor(q), harness.bf16_tensor(k), harness.bf16_tensor(v),
                                 harness.logits_tensor(w, lg)]))
-    tokens0, state0 = synth.make_block_template(w, 0, 0)
+    templates = [synth.make_block_template(w, i, 0) for i in range(n_scenes)]
+    tokens0 = np.concatenate([t_.reshape(-1) for t_, _ in templates])
+    state0 = np.concatenate([s_.reshape(-1) for _, s_ in templates])
     tokens0_d = torch.from_numpy(tokens0).cuda()
     state0_d = torch.from_numpy(state0).cuda()
     tokens = torch.empty_like(tokens0_d)
@@ -142,8 +154,8 @@ def run_ours(args):
     n_comm = torch.zeros(N, dtype=torch.int32, device="cuda")
     n_left = torch.zeros(N, dtype=torch.int32, device="cuda")
     n_left_host = torch.zeros(N, dtype=torch.int32).pin_memory()
-    traj = torch.from_numpy(synth.tokens_to_trajectory(w, tokens0, state0)).cuda()
-    traj_out = torch.zeros((w.waypoints, 2), dtype=torch.float32, device="cuda")
+    trajs = [torch.from_numpy(synth.tokens_to_trajectory(w, t_, s_)).cuda() for t_, s_ in templates]
+    traj_out = torch.zeros((n_scenes, w.waypoints, 2), dtype=torch.float32, device="cuda")
     value_tokens = int((state0 == synth.MASKED).sum())
     all_tokens = int(state0.size)
 
@@ -153,9 +165,8 @@ def run_ours(args):
     def decode_block(inputs, timed_attn):
         """One step of the benchmark: the whole block loop for all rollouts.  `inputs(t)` returns
         device tensors (q, k, v, logits) of denoising step t."""
-        fs = fdd.fdd_fork(ctx, scene.prefix_k, scene.prefix_v, scene.page_table, sc.prefix_len,
-                          scene.prefix_capacity, N, scene.seeds, scene.suffix_k, scene.suffix_v,
-                          scene.suffix_capacity)
+        fs = [fdd.fdd_fork(ctx, g.prefix_k, g.prefix_v, g.page_table, g.sc.prefix_len, g.prefix_capacity,
+                           g.sc.n_forks, g.seeds, g.suffix_k, g.suffix_v, g.suffix_capacity) for g in gscenes]
         tokens.copy_(tokens0_d, non_blocking=True)
         state.copy_(state0_d, non_blocking=True)
         t = 0
@@ -166,14 +177,14 @@ def run_ours(args):
                 if timed_attn:
                     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
                     e0.record(stream)
-                fdd.fdd_block_attn(ctx, [fs], layer, q, k, v, out, [d], scale, 0)
+                fdd.fdd_block_attn(ctx, fs, layer, q, k, v, out, ds, scale, 0)
                 if timed_attn:
                     e1.record(stream)
                     attn_events.append((e0, e1))
             if timed_attn:
                 u0, u1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
                 u0.record(stream)
-            fdd.fdd_unmask(ctx, [fs], lg, tokens, state, [d], w.threshold, w.temperature, 0, t, n_comm, n_left)
+            fdd.fdd_unmask(ctx, fs, lg, tokens, state, ds, w.threshold, w.temperature, 0, t, n_comm, n_left)
             if timed_attn:
                 u1.record(stream)
                 unmask_events.append((u0, u1, masked_rows))
@@ -184,9 +195,11 @@ def run_ours(args):
             if masked_rows == 0 or t >= d:
                 break
         for layer in range(L):
-            fdd.fdd_kv_commit(ctx, [fs], layer, k, v, [d], 1 if layer == L - 1 else 0)
-        fdd.fdd_average_rollouts(ctx, traj, N, w.waypoints, traj_out)
-        fdd.fdd_forkset_free(ctx, fs)
+            fdd.fdd_kv_commit(ctx, fs, layer, k, v, ds, 1 if layer == L - 1 else 0)
+        for i in range(n_scenes):
+            fdd.fdd_average_rollouts(ctx, trajs[i], Ns[i], w.waypoints, traj_out[i])
+        for f_ in fs:
+            fdd.fdd_forkset_free(ctx, f_)
         return t
 
     resident = lambda t: dev_steps[t % PRE_STEPS]
@@ -225,7 +238,7 @@ def run_ours(args):
                         for a in hs) for hs in host_steps]
         stage = [torch.empty_like(x) for x in dev_steps[0]]
         tok_host = torch.zeros_like(tokens0_d, device="cpu").pin_memory()
-        traj_host = torch.zeros((w.waypoints, 2), dtype=torch.float32).pin_memory()
+        traj_host = torch.zeros((n_scenes, w.waypoints, 2), dtype=torch.float32).pin_memory()
         h2d = sum(x.numel() * x.element_size() for x in pinned[0])
         d2h_step = n_left_host.numel() * 4
 
@@ -261,7 +274,7 @@ def run_ours(args):
             dist.destroy_process_group()
         return
     peaks = _peaks()
-    flops = _attn_flops(w, sc, 0)
+    flops = sum(_attn_flops(w, s_, 0) for s_ in w.scenes)
     attn_avg_ms = float(np.mean(attn_ms)) if attn_ms else None
     achieved = flops / (attn_avg_ms * 1e-3) / 1e12 if attn_avg_ms else None
     # unmask: the launches that see every value row MASKED (first denoising step of a block)
@@ -275,7 +288,8 @@ def run_ours(args):
         "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms / args.steps,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
         "data": "synthetic",
-        "config": {"workload": args.workload, "n_forks": N, "block_len": d, "prefix_len": sc.prefix_len,
+        "config": {"workload": args.workload, "scenes": n_scenes, "n_forks": N, "block_len": d,
+                   "prefix_len": sc.prefix_len if n_scenes == 1 else [s_.prefix_len for s_ in w.scenes],
                    "heads": f"{w.n_q_heads}q/{w.n_kv_heads}kv", "head_dim": w.head_dim, "vocab": w.vocab,
                    "layers": L, "threshold": w.threshold, "temperature": w.temperature,
                    "denoise_steps_per_block": denoise_steps / args.steps,

@@ -42,7 +42,7 @@ namespace {
 constexpr int kTcThreads = 384;
 constexpr int kKeysPerTile = 128;
 constexpr long long kWaitLimit = 4000000000LL;   // about two seconds of SM clocks
-constexpr int kMinTilesPerCta = 4;               // do not cut the work finer than this
+constexpr int kMinTilesPerCta = 8;               // do not cut the work finer than this (every cut costs a merge)
 // Registers per thread after the hand-over.  The CTA starts with 384 x 168; 8 soft-max warps x
 // kRegsSoftmax + 4 other warps x kRegsOther must not exceed that (2 * 208 + 88 = 3 * 168).
 constexpr int kRegsSoftmax = 208;
@@ -649,35 +649,59 @@ attn_ptc_kernel(const __grid_constant__ TcArgs<MAXSETS> a) {
                     // This CTA finished the unit's last outstanding piece: merge all of them.
                     //   out = sum_s w_s O_s / sum_s w_s,  w_s = 2^(lse_s - max lse)
                     __threadfence();
+                    // A warp takes eight rows at a time (lane = four columns), so that the loads of a
+                    // piece are eight independent 512-byte rows in flight, not one after the other.
                     constexpr int kLanes = D / 4;       // lanes that carry a float4 of the row
-                    for (int row = warp; row < rows_here; row += 8) {
-                        const int rr = rp * 256 + row;
-                        float M = -CUDART_INF_F;
-                        for (int pc = c_first; pc <= c_last; ++pc) {
-                            const int slot = pc * 2 + (it.unit_begin <= T * pc / C ? 0 : 1);
-                            M = fmaxf(M, __ldcg(a.part_lse + static_cast<size_t>(slot) * 256 + row));
+                    constexpr int kBatch = 8;
+                    auto slot_of = [&](int pc) { return pc * 2 + (it.unit_begin <= T * pc / C ? 0 : 1); };
+                    for (int row0 = warp * kBatch; row0 < rows_here; row0 += 8 * kBatch) {
+                        float M[kBatch], wsum[kBatch];
+                        float4 accv[kBatch];
+#pragma unroll
+                        for (int j = 0; j < kBatch; ++j) {
+                            M[j] = -CUDART_INF_F; wsum[j] = 0.0f;
+                            accv[j] = make_float4(0.f, 0.f, 0.f, 0.f);
                         }
-                        float4 accv = make_float4(0.f, 0.f, 0.f, 0.f);
-                        float wsum = 0.0f;
                         for (int pc = c_first; pc <= c_last; ++pc) {
-                            const int slot = pc * 2 + (it.unit_begin <= T * pc / C ? 0 : 1);
-                            const float w = exp2f(__ldcg(a.part_lse + static_cast<size_t>(slot) * 256 + row) - M);
-                            wsum += w;
-                            if (lane < kLanes) {
-                                const float4 o = __ldcg(reinterpret_cast<const float4*>(
-                                    a.part_o + (static_cast<size_t>(slot) * 256 + row) * D + lane * 4));
-                                accv.x = fmaf(w, o.x, accv.x); accv.y = fmaf(w, o.y, accv.y);
-                                accv.z = fmaf(w, o.z, accv.z); accv.w = fmaf(w, o.w, accv.w);
+                            const float* lse = a.part_lse + static_cast<size_t>(slot_of(pc)) * 256 + row0;
+#pragma unroll
+                            for (int j = 0; j < kBatch; ++j)
+                                if (row0 + j < rows_here) M[j] = fmaxf(M[j], __ldcg(lse + j));
+                        }
+                        for (int pc = c_first; pc <= c_last; ++pc) {
+                            const int slot = slot_of(pc);
+                            const float* lse = a.part_lse + static_cast<size_t>(slot) * 256 + row0;
+                            const float* po = a.part_o + (static_cast<size_t>(slot) * 256 + row0) * D + lane * 4;
+                            float wj[kBatch];
+                            float4 oj[kBatch];
+#pragma unroll
+                            for (int j = 0; j < kBatch; ++j) {
+                                const bool live = row0 + j < rows_here;
+                                wj[j] = live ? __ldcg(lse + j) : -CUDART_INF_F;
+                                oj[j] = (live && lane < kLanes) ? __ldcg(reinterpret_cast<const float4*>(po + static_cast<size_t>(j) * D))
+                                                                : make_float4(0.f, 0.f, 0.f, 0.f);
+                            }
+#pragma unroll
+                            for (int j = 0; j < kBatch; ++j) {
+                                const float wgt = (row0 + j < rows_here) ? exp2f(wj[j] - M[j]) : 0.0f;
+                                wsum[j] += wgt;
+                                accv[j].x = fmaf(wgt, oj[j].x, accv[j].x); accv[j].y = fmaf(wgt, oj[j].y, accv[j].y);
+                                accv[j].z = fmaf(wgt, oj[j].z, accv[j].z); accv[j].w = fmaf(wgt, oj[j].w, accv[j].w);
                             }
                         }
                         if (lane < kLanes) {
-                            const float iw = 1.0f / wsum;
-                            const int i2 = rr / p.G, g2 = rr - i2 * p.G;
-                            __nv_bfloat16* op = p.out + ((static_cast<size_t>(f) * p.d + i2) * p.n_q_heads + h * p.G + g2) * D + lane * 4;
-                            const __nv_bfloat162 lo = __floats2bfloat162_rn(accv.x * iw, accv.y * iw);
-                            const __nv_bfloat162 hi = __floats2bfloat162_rn(accv.z * iw, accv.w * iw);
-                            *reinterpret_cast<uint2*>(op) = make_uint2(*reinterpret_cast<const uint32_t*>(&lo),
-                                                                       *reinterpret_cast<const uint32_t*>(&hi));
+#pragma unroll
+                            for (int j = 0; j < kBatch; ++j) {
+                                if (row0 + j >= rows_here) continue;
+                                const int rr = rp * 256 + row0 + j;
+                                const float iw = 1.0f / wsum[j];
+                                const int i2 = rr / p.G, g2 = rr - i2 * p.G;
+                                __nv_bfloat16* op = p.out + ((static_cast<size_t>(f) * p.d + i2) * p.n_q_heads + h * p.G + g2) * D + lane * 4;
+                                const __nv_bfloat162 lo = __floats2bfloat162_rn(accv[j].x * iw, accv[j].y * iw);
+                                const __nv_bfloat162 hi = __floats2bfloat162_rn(accv[j].z * iw, accv[j].w * iw);
+                                *reinterpret_cast<uint2*>(op) = make_uint2(*reinterpret_cast<const uint32_t*>(&lo),
+                                                                           *reinterpret_cast<const uint32_t*>(&hi));
+                            }
                         }
                     }
                 }
