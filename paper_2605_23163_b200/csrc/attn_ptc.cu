@@ -189,6 +189,8 @@ attn_ptc_kernel(const __grid_constant__ TcArgs<MAXSETS> a) {
         bar_v_full[kStages], bar_v_empty[kStages], bar_s_full[2], bar_s_free[2], bar_p_full[2], bar_o_done[2], bar_item_done;
     __shared__ uint32_t tmem_base_s;
     __shared__ int abort_s, last_s;
+    constexpr int kMaxPieces = 160;                     // a unit is cut by CTA borders: at most one piece per CTA
+    __shared__ int slot_s[kMaxPieces];                  // scratch slot of every piece of the unit being merged
     volatile int* abort_flag = &abort_s;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -649,49 +651,65 @@ attn_ptc_kernel(const __grid_constant__ TcArgs<MAXSETS> a) {
                     // This CTA finished the unit's last outstanding piece: merge all of them.
                     //   out = sum_s w_s O_s / sum_s w_s,  w_s = 2^(lse_s - max lse)
                     __threadfence();
-                    // A warp takes eight rows at a time (lane = four columns), so that the loads of a
-                    // piece are eight independent 512-byte rows in flight, not one after the other.
+                    // A warp takes four rows at a time (lane = four columns) and up to eight pieces at
+                    // once: 32 independent 512-byte row reads (plus their log-sum-exps) are in flight
+                    // before the first one is used; more than eight pieces are folded in chunk by chunk
+                    // with a running maximum.
                     constexpr int kLanes = D / 4;       // lanes that carry a float4 of the row
-                    constexpr int kBatch = 8;
-                    auto slot_of = [&](int pc) { return pc * 2 + (it.unit_begin <= T * pc / C ? 0 : 1); };
-                    for (int row0 = warp * kBatch; row0 < rows_here; row0 += 8 * kBatch) {
-                        float M[kBatch], wsum[kBatch];
-                        float4 accv[kBatch];
+                    constexpr int kRowsB = 4, kPC = 8;
+                    if (tid < n_pieces && tid < kMaxPieces) {
+                        const int pc = c_first + tid;
+                        slot_s[tid] = pc * 2 + (it.unit_begin <= T * pc / C ? 0 : 1);
+                    }
+                    tc::named_barrier(1, 256);
+                    for (int row0 = warp * kRowsB; row0 < rows_here; row0 += 8 * kRowsB) {
+                        float M[kRowsB], wsum[kRowsB];
+                        float4 accv[kRowsB];
 #pragma unroll
-                        for (int j = 0; j < kBatch; ++j) {
+                        for (int j = 0; j < kRowsB; ++j) {
                             M[j] = -CUDART_INF_F; wsum[j] = 0.0f;
                             accv[j] = make_float4(0.f, 0.f, 0.f, 0.f);
                         }
-                        for (int pc = c_first; pc <= c_last; ++pc) {
-                            const float* lse = a.part_lse + static_cast<size_t>(slot_of(pc)) * 256 + row0;
+                        for (int k0 = 0; k0 < n_pieces; k0 += kPC) {
+                            float ls[kPC][kRowsB];
+                            float4 ov[kPC][kRowsB];
 #pragma unroll
-                            for (int j = 0; j < kBatch; ++j)
-                                if (row0 + j < rows_here) M[j] = fmaxf(M[j], __ldcg(lse + j));
-                        }
-                        for (int pc = c_first; pc <= c_last; ++pc) {
-                            const int slot = slot_of(pc);
-                            const float* lse = a.part_lse + static_cast<size_t>(slot) * 256 + row0;
-                            const float* po = a.part_o + (static_cast<size_t>(slot) * 256 + row0) * D + lane * 4;
-                            float wj[kBatch];
-                            float4 oj[kBatch];
+                            for (int k = 0; k < kPC; ++k) {
+                                const bool live_p = k0 + k < n_pieces;
+                                const int slot = slot_s[min(k0 + k, n_pieces - 1)];
+                                const float* lse = a.part_lse + static_cast<size_t>(slot) * 256 + row0;
+                                const float* po = a.part_o + (static_cast<size_t>(slot) * 256 + row0) * D + lane * 4;
 #pragma unroll
-                            for (int j = 0; j < kBatch; ++j) {
-                                const bool live = row0 + j < rows_here;
-                                wj[j] = live ? __ldcg(lse + j) : -CUDART_INF_F;
-                                oj[j] = (live && lane < kLanes) ? __ldcg(reinterpret_cast<const float4*>(po + static_cast<size_t>(j) * D))
-                                                                : make_float4(0.f, 0.f, 0.f, 0.f);
+                                for (int j = 0; j < kRowsB; ++j) {
+                                    const bool live = live_p && row0 + j < rows_here;
+                                    ls[k][j] = live ? __ldcg(lse + j) : -CUDART_INF_F;
+                                    ov[k][j] = (live && lane < kLanes) ? __ldcg(reinterpret_cast<const float4*>(po + static_cast<size_t>(j) * D))
+                                                                       : make_float4(0.f, 0.f, 0.f, 0.f);
+                                }
                             }
 #pragma unroll
-                            for (int j = 0; j < kBatch; ++j) {
-                                const float wgt = (row0 + j < rows_here) ? exp2f(wj[j] - M[j]) : 0.0f;
-                                wsum[j] += wgt;
-                                accv[j].x = fmaf(wgt, oj[j].x, accv[j].x); accv[j].y = fmaf(wgt, oj[j].y, accv[j].y);
-                                accv[j].z = fmaf(wgt, oj[j].z, accv[j].z); accv[j].w = fmaf(wgt, oj[j].w, accv[j].w);
+                            for (int j = 0; j < kRowsB; ++j) {
+                                float mc = ls[0][j];
+#pragma unroll
+                                for (int k = 1; k < kPC; ++k) mc = fmaxf(mc, ls[k][j]);
+                                const float mn = fmaxf(M[j], mc);
+                                if (mn == -CUDART_INF_F) continue;              // nothing live in this row yet
+                                const float keep = exp2f(M[j] - mn);           // 0 on the first chunk (M = -inf)
+                                wsum[j] *= keep;
+                                accv[j].x *= keep; accv[j].y *= keep; accv[j].z *= keep; accv[j].w *= keep;
+                                M[j] = mn;
+#pragma unroll
+                                for (int k = 0; k < kPC; ++k) {
+                                    const float wgt = exp2f(ls[k][j] - mn);    // 0 for a piece that is not there
+                                    wsum[j] += wgt;
+                                    accv[j].x = fmaf(wgt, ov[k][j].x, accv[j].x); accv[j].y = fmaf(wgt, ov[k][j].y, accv[j].y);
+                                    accv[j].z = fmaf(wgt, ov[k][j].z, accv[j].z); accv[j].w = fmaf(wgt, ov[k][j].w, accv[j].w);
+                                }
                             }
                         }
                         if (lane < kLanes) {
 #pragma unroll
-                            for (int j = 0; j < kBatch; ++j) {
+                            for (int j = 0; j < kRowsB; ++j) {
                                 if (row0 + j >= rows_here) continue;
                                 const int rr = rp * 256 + row0 + j;
                                 const float iw = 1.0f / wsum[j];
@@ -865,7 +883,12 @@ cudaError_t launch_group(fdd_ctx* ctx, const AttnProblem* probs, TcMapCache* con
         units += p.units;
     }
     if (units > ctx->attn_max_units) return cudaErrorInvalidValue;
-    long long ctas = steps / kMinTilesPerCta;
+    static int min_tiles = 0;
+    if (min_tiles == 0) {
+        min_tiles = kMinTilesPerCta;
+        if (const char* e = std::getenv("FDD_ATTN_MIN_TILES")) { const int v = std::atoi(e); if (v >= 1 && v <= 64) min_tiles = v; }
+    }
+    long long ctas = steps / min_tiles;
     if (ctas > ctx->attn_max_ctas) ctas = ctx->attn_max_ctas;
     if (ctas < 1) ctas = 1;
     args.part_o = static_cast<float*>(ctx->ws_attn);
