@@ -274,6 +274,19 @@ fdd_status fdd_plan_blocks(const uint8_t* editable, const int32_t* section_end, 
                            int length, int d, int32_t* block_begin, int32_t* block_end,
                            int32_t* block_section, int capacity, int* n_blocks);
 
+/*
+ * fdd_upload_masked_rows -- host-to-device copy of exactly the logits rows the next fdd_unmask
+ * will read (Sec. 3.3: only MASKED value positions are decoded; everything else is never read).
+ * For callers whose logits live in host memory.
+ *   host_logits   host (pinned for an asynchronous copy) [rows][V], dtype per cfg.logits_dtype
+ *   dev_logits    device buffer of the same shape; rows that are not copied keep their old bytes
+ *   host_state    host uint8 [rows]: the state array as the caller last read it from the device
+ *   bytes_copied  optional: bytes enqueued
+ * One cudaMemcpyAsync per run of consecutive MASKED rows, on `stream`; returns without waiting.
+ */
+fdd_status fdd_upload_masked_rows(fdd_ctx* ctx, const void* host_logits, void* dev_logits,
+                                  const uint8_t* host_state, int rows, size_t* bytes_copied, void* stream);
+
 /* Synchronise `stream` and return the device status word: FDD_OK, or the first error a
  * kernel recorded (FDD_ERR_DEVICE_TIMEOUT).  Reading clears it. */
 fdd_status fdd_poll_status(fdd_ctx* ctx, void* stream);

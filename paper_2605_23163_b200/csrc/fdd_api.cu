@@ -385,6 +385,31 @@ fdd_status fdd_average_rollouts(fdd_ctx* ctx, const float* traj, int n, int w, f
     return FDD_OK;
 }
 
+fdd_status fdd_upload_masked_rows(fdd_ctx* ctx, const void* host_logits, void* dev_logits,
+                                  const uint8_t* host_state, int rows, size_t* bytes_copied, void* stream) {
+    if (!ctx) return FDD_ERR_INVALID_ARG;
+    if (bytes_copied) *bytes_copied = 0;
+    if (!host_logits || !dev_logits || !host_state || rows < 0)
+        return fail(ctx, FDD_ERR_INVALID_ARG, "host_logits/dev_logits/host_state is NULL or rows < 0");
+    const size_t row_bytes = static_cast<size_t>(ctx->cfg.vocab) * (ctx->cfg.logits_dtype == FDD_LOGITS_BF16 ? 2 : 4);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    size_t total = 0;
+    int r = 0;
+    while (r < rows) {
+        if (host_state[r] != FDD_MASKED) { ++r; continue; }
+        int e = r + 1;
+        while (e < rows && host_state[e] == FDD_MASKED) ++e;            // one copy per run of MASKED rows
+        const size_t off = static_cast<size_t>(r) * row_bytes, len = static_cast<size_t>(e - r) * row_bytes;
+        cudaError_t err = cudaMemcpyAsync(static_cast<char*>(dev_logits) + off, static_cast<const char*>(host_logits) + off,
+                                          len, cudaMemcpyHostToDevice, st);
+        if (err != cudaSuccess) return cuda_fail(ctx, err, "fdd_upload_masked_rows copy");
+        total += len;
+        r = e;
+    }
+    if (bytes_copied) *bytes_copied = total;
+    return FDD_OK;
+}
+
 fdd_status fdd_poll_status(fdd_ctx* ctx, void* stream) {
     if (!ctx) return FDD_ERR_INVALID_ARG;
     cudaStream_t st = static_cast<cudaStream_t>(stream);

@@ -21,7 +21,7 @@ FDD_LOGITS_F32, FDD_LOGITS_BF16 = 0, 1
 EXPORTS = (
     "fdd_create", "fdd_destroy", "fdd_last_error", "fdd_launch_count", "fdd_fork",
     "fdd_forkset_free", "fdd_forkset_suffix_len", "fdd_forkset_reset", "fdd_block_attn",
-    "fdd_unmask", "fdd_ss_draft", "fdd_ss_accept", "fdd_kv_commit", "fdd_average_rollouts", "fdd_poll_status", "fdd_unmask_static", "fdd_plan_blocks",
+    "fdd_unmask", "fdd_ss_draft", "fdd_ss_accept", "fdd_kv_commit", "fdd_average_rollouts", "fdd_poll_status", "fdd_unmask_static", "fdd_plan_blocks", "fdd_upload_masked_rows",
 )
 FDD_UNMASK_STATIC_MAX_RECORDS = 65536
 
@@ -236,6 +236,19 @@ def fdd_plan_blocks(editable, section_end, d, capacity=4096):
     if st < 0:
         raise FddError(st, "fdd_plan_blocks failed")
     return [(int(bb[i]), int(be[i]), int(bs[i])) for i in range(n.value)]
+
+
+def fdd_upload_masked_rows(ctx, host_logits, dev_logits, host_state, stream=None):
+    """host_logits: pinned CPU tensor [rows, V]; dev_logits: CUDA tensor of the same shape;
+    host_state: CPU uint8 tensor [rows].  Returns the bytes enqueued."""
+    L = lib()
+    L.fdd_upload_masked_rows.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int,
+                                         ctypes.POINTER(ctypes.c_size_t), ctypes.c_void_p]
+    L.fdd_upload_masked_rows.restype = ctypes.c_int
+    n = ctypes.c_size_t(0)
+    _check(ctx, L.fdd_upload_masked_rows(ctx, _ptr(host_logits), _ptr(dev_logits), _ptr(host_state),
+                                          int(host_state.numel()), ctypes.byref(n), _stream(stream)))
+    return int(n.value)
 
 
 def fdd_poll_status(ctx, stream=None):

@@ -568,6 +568,31 @@ def test_average_cancellation_and_single_rollout():
         fdd.fdd_destroy(ctx)
 
 
+def test_upload_masked_rows_copies_exactly_the_rows_that_are_read():
+    w = synth.small_variant(synth.workload("tts"), prefix_len=64, vocab=4096, n_forks=3, n_blocks=1)
+    sc = w.scenes[0]
+    ctx = harness.create_context(w)
+    try:
+        rows = sc.n_forks * sc.block_len
+        g = np.random.default_rng(3)
+        host = torch.from_numpy(g.integers(-30000, 30000, size=(rows, w.vocab), dtype=np.int16)).pin_memory()
+        dev = torch.full((rows, w.vocab), 77, dtype=torch.int16, device="cuda")
+        _, state = synth.make_block_template(w, 0, 0)
+        state = state.reshape(-1).copy()
+        state[5] = COMMITTED                                   # break a run of MASKED rows
+        st = torch.from_numpy(state)
+        n = fdd.fdd_upload_masked_rows(ctx, host, dev, st)
+        torch.cuda.synchronize()
+        masked = state == MASKED
+        assert n == int(masked.sum()) * w.vocab * 2
+        got = dev.cpu().numpy()
+        assert np.array_equal(got[masked], host.numpy()[masked])
+        assert np.all(got[~masked] == 77)
+        assert fdd.fdd_upload_masked_rows(ctx, host, dev, torch.full((rows,), COMMITTED, dtype=torch.uint8)) == 0
+    finally:
+        fdd.fdd_destroy(ctx)
+
+
 # ---------------------------------------------------------------------------------------------
 # host-side error paths (nothing is launched)
 # ---------------------------------------------------------------------------------------------
