@@ -551,6 +551,48 @@ def test_block_loop_matches_oracle_and_averages():
         fdd.fdd_destroy(ctx)
 
 
+def test_tts_full_size_block_loop_sampled_rollouts():
+    # the test-time-scaling configuration at full size (8 rollouts, 4096-token prefix, vocabulary
+    # 151936, Gumbel noise): the whole loop of one block runs on the GPU; every step the oracle
+    # re-does two rollouts from the same state, and attention is checked at the first and last step
+    w = synth.workload("tts")
+    sc = w.scenes[0]
+    ctx = harness.create_context(w)
+    try:
+        scene = harness.GpuScene(ctx, w, 0)
+        pk, pv = synth.make_prefix(w, 0)
+        empty = ([np.zeros((0, w.n_kv_heads, w.head_dim), dtype=np.uint16)] * sc.n_forks,) * 2
+        tokens, state = synth.make_block_template(w, 0, 0)
+        sample = [1, 6]
+        step, ambiguous = 0, 0
+        while np.any(state == MASKED):
+            q, k, v = synth.make_qkv(w, 0, 0, 0, step)
+            got_attn = pu.attention_gpu(ctx, scene, q, k, v)
+            if step == 0 or int((state == MASKED).sum()) <= 3 * sc.n_forks:
+                ref_attn = pu.attention_oracle(w, (pk, pv), empty, q, k, v, forks=sample)
+                pu.assert_attention_close(got_attn[sample], ref_attn)
+            logits = synth.make_logits(w, 0, 0, step, rows="value")
+            got = pu.unmask_gpu(ctx, scene, logits, tokens, state, w.threshold, w.temperature, 0, step)
+            ref = unmask_step(pu.widen_logits(w, logits[sample]), tokens[sample], state[sample], scene.seeds[sample],
+                              w.threshold, w.temperature, 0, step)
+            sub = {k_: v_[sample] for k_, v_ in got.items()}
+            ambiguous += len(pu.compare_unmask(sub, ref, tokens[sample], state[sample], w.threshold)["ambiguous_forks"])
+            assert np.all(got["n_committed"][(state == MASKED).any(axis=1)] >= 1)
+            tokens, state = got["tokens"], got["state"]
+            step += 1
+            assert step <= sc.block_len
+        assert ambiguous <= 1 and 2 <= step <= 22
+        fdd.fdd_kv_commit(ctx, [scene.forkset], 0, harness.bf16_tensor(k), harness.bf16_tensor(v), [sc.block_len], 1)
+        traj = synth.tokens_to_trajectory(w, tokens, state)
+        out = torch.zeros((w.waypoints, 2), dtype=torch.float32, device="cuda")
+        fdd.fdd_average_rollouts(ctx, torch.from_numpy(traj).cuda(), sc.n_forks, w.waypoints, out)
+        fdd.fdd_poll_status(ctx)
+        ref_t = average_rollouts(traj)
+        assert np.all(np.abs(out.cpu().numpy() - ref_t) <= 1e-5 * np.maximum(np.abs(ref_t), 1e-30) + 1e-30)
+    finally:
+        fdd.fdd_destroy(ctx)
+
+
 def test_average_cancellation_and_single_rollout():
     ctx = fdd.fdd_create(4, 1, 64, 64)
     try:
