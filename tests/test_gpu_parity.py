@@ -262,6 +262,83 @@ def test_attention_group_of_three_uses_the_cuda_core_kernel():
     _attention_case(w)
 
 
+def test_more_scenes_and_rows_than_one_launch_takes():
+    # 18 scenes (more than the 16 of one attention / unmask launch) and, separately, three sets of
+    # 4096 rows each (more than the 8192 rows of one unmask launch): the calls split the work
+    scenes = tuple(synth.Scene(prefix_len=70 + 13 * i, n_forks=1 + i % 3, block_len=16, n_scaffold=4, n_blocks=1)
+                   for i in range(18))
+    w = synth.Workload("many", 8, 2, 64, 640, "bf16", "peaked", 0.9, 0.7, scenes, qkv_sigma=0.5, seed=41)
+    ctx = harness.create_context(w)
+    try:
+        gs = [harness.GpuScene(ctx, w, i) for i in range(len(scenes))]
+        qs, ks, vs = zip(*[synth.make_qkv(w, i, 0, 0, 0) for i in range(len(scenes))])
+        pack = lambda xs: harness.bf16_tensor(np.concatenate([x.reshape(-1) for x in xs]))
+        qd, kd, vd = pack(qs), pack(ks), pack(vs)
+        out = torch.full_like(qd, float("nan"))
+        n0 = fdd.fdd_launch_count(ctx)
+        fdd.fdd_block_attn(ctx, [g.forkset for g in gs], 0, qd, kd, vd, out, [16] * 18, 0.125, 0)
+        fdd.fdd_poll_status(ctx)
+        assert fdd.fdd_launch_count(ctx) - n0 == 2
+        got = out.float().cpu().numpy().astype(np.float64)
+        off = 0
+        for i, sc in enumerate(scenes):
+            pk, pv = synth.make_prefix(w, i)
+            empty = ([np.zeros((0, w.n_kv_heads, w.head_dim), dtype=np.uint16)] * sc.n_forks,) * 2
+            ref = pu.attention_oracle(w, (pk, pv), empty, qs[i], ks[i], vs[i], scale=0.125)
+            pu.assert_attention_close(got[off:off + ref.size].reshape(ref.shape), ref)
+            off += ref.size
+        toks, sts, lgs = zip(*[synth.make_block_template(w, i, 0) + (synth.make_logits(w, i, 0, 0, rows="all"),)
+                               for i in range(len(scenes))])
+        flat = lambda xs: np.concatenate([x.reshape(-1) for x in xs])
+        tok_d, st_d = torch.from_numpy(flat(toks)).cuda(), torch.from_numpy(flat(sts)).cuda()
+        nf = sum(sc.n_forks for sc in scenes)
+        n_c = torch.zeros(nf, dtype=torch.int32, device="cuda"); n_l = torch.zeros(nf, dtype=torch.int32, device="cuda")
+        n0 = fdd.fdd_launch_count(ctx)
+        fdd.fdd_unmask(ctx, [g.forkset for g in gs], harness.bf16_tensor(flat(lgs)), tok_d, st_d, [16] * 18,
+                       w.threshold, w.temperature, 0, 0, n_c, n_l)
+        fdd.fdd_poll_status(ctx)
+        assert fdd.fdd_launch_count(ctx) - n0 == 4
+        tok_h, st_h = tok_d.cpu().numpy(), st_d.cpu().numpy()
+        off = foff = 0
+        for i, sc in enumerate(scenes):
+            rows = sc.n_forks * 16
+            ref = unmask_step(pu.widen_logits(w, lgs[i]), toks[i], sts[i], gs[i].seeds, w.threshold, w.temperature, 0, 0)
+            sub = dict(tokens=tok_h[off:off + rows].reshape(sc.n_forks, 16), state=st_h[off:off + rows].reshape(sc.n_forks, 16),
+                       conf=None, n_committed=n_c.cpu().numpy()[foff:foff + sc.n_forks], n_left=n_l.cpu().numpy()[foff:foff + sc.n_forks])
+            assert len(pu.compare_unmask(sub, ref, toks[i], sts[i], w.threshold)["ambiguous_forks"]) <= 1
+            off += rows; foff += sc.n_forks
+    finally:
+        fdd.fdd_destroy(ctx)
+    # rows: 3 sets x (32 rollouts x 128 positions) = 12288 rows > 8192 per launch
+    big = tuple(synth.Scene(prefix_len=16, n_forks=32, block_len=128, n_scaffold=40, n_blocks=1) for _ in range(3))
+    w = synth.Workload("rows", 4, 1, 64, 512, "f32", "peaked", 0.6, 1.1, big, seed=42)
+    ctx = harness.create_context(w)
+    try:
+        gs = [harness.GpuScene(ctx, w, i) for i in range(3)]
+        toks, sts, lgs = zip(*[synth.make_block_template(w, i, 0) + (synth.make_logits(w, i, 0, 0, rows="all"),)
+                               for i in range(3)])
+        flat = lambda xs: np.concatenate([x.reshape(-1) for x in xs])
+        tok_d, st_d = torch.from_numpy(flat(toks)).cuda(), torch.from_numpy(flat(sts)).cuda()
+        n_c = torch.zeros(96, dtype=torch.int32, device="cuda"); n_l = torch.zeros(96, dtype=torch.int32, device="cuda")
+        n0 = fdd.fdd_launch_count(ctx)
+        fdd.fdd_unmask(ctx, [g.forkset for g in gs], torch.from_numpy(flat(lgs)).cuda(), tok_d, st_d, [128] * 3,
+                       w.threshold, w.temperature, 0, 0, n_c, n_l)
+        fdd.fdd_poll_status(ctx)
+        assert fdd.fdd_launch_count(ctx) - n0 == 4                 # two sets, then one
+        tok_h, st_h = tok_d.cpu().numpy().reshape(3, 32, 128), st_d.cpu().numpy().reshape(3, 32, 128)
+        amb = 0
+        for i in (0, 2):
+            f = [3, 30]
+            ref = unmask_step(lgs[i][f].astype(np.float64), toks[i][f], sts[i][f], gs[i].seeds[f], w.threshold,
+                              w.temperature, 0, 0)
+            sub = dict(tokens=tok_h[i][f], state=st_h[i][f], conf=None,
+                       n_committed=n_c.cpu().numpy().reshape(3, 32)[i][f], n_left=n_l.cpu().numpy().reshape(3, 32)[i][f])
+            amb += len(pu.compare_unmask(sub, ref, toks[i][f], sts[i][f], w.threshold)["ambiguous_forks"])
+        assert amb <= 1
+    finally:
+        fdd.fdd_destroy(ctx)
+
+
 def test_prefix_is_never_written_and_forks_with_equal_inputs_agree():
     w = synth.small_variant(synth.workload("tts"), prefix_len=512, vocab=512, n_forks=4, n_blocks=1)
     ctx = harness.create_context(w)
