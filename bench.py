@@ -29,6 +29,7 @@ UNIT = "tokens/s"
 # DRAM bytes (read + write) of one attention launch at the long_prefix workload, from the ncu capture
 # summarised in profiles/attn_ptc_long_prefix.md; None for other workloads or once the kernel changed.
 ATTN_DRAM_BYTES_PER_LAUNCH = {"long_prefix": 170.5e6}
+LOOKAHEAD = True   # enqueue step t + 1 before the host has read the counts of step t (--no-lookahead)
 PRE_STEPS = 6      # distinct per-step input sets kept resident; later steps cycle through them (--pre-steps)
 
 
@@ -159,41 +160,79 @@ def run_ours(args):
     value_tokens = int((state0 == synth.MASKED).sum())
     all_tokens = int(state0.size)
 
-    attn_events = []
-    unmask_events = []          # (start, end, MASKED rows on entry) of every timed unmask call
+    # MASKED positions per rollout at the start of a block: the gate of the first attention call
+    n_left0_d = torch.from_numpy(np.concatenate(
+        [(s_ == synth.MASKED).sum(axis=1).astype(np.int32) for _, s_ in templates])).cuda()
+    n_left_hosts = [torch.zeros(N, dtype=torch.int32).pin_memory() for _ in range(2)]
+    step_done = [torch.cuda.Event(), torch.cuda.Event()]
 
-    def decode_block(inputs, timed_attn):
+    attn_events = []            # [start, end, rollouts still decoding] of every timed attention call
+    unmask_events = []          # [start, end, MASKED rows on entry] of every timed unmask call
+
+    def decode_block(inputs, timed_attn, lookahead):
         """One step of the benchmark: the whole block loop for all rollouts.  `inputs(t)` returns
-        device tensors (q, k, v, logits) of denoising step t."""
+        device tensors (q, k, v, logits) of denoising step t.  Attention is gated by the n_left
+        array of the step before, so rollouts that have finished their block cost nothing; with
+        `lookahead` step t + 1 is enqueued before the host has seen the result of step t (once
+        every rollout is done its kernels return at once), which keeps the GPU busy while the host
+        reads the counts."""
         fs = [fdd.fdd_fork(ctx, g.prefix_k, g.prefix_v, g.page_table, g.sc.prefix_len, g.prefix_capacity,
                            g.sc.n_forks, g.seeds, g.suffix_k, g.suffix_v, g.suffix_capacity) for g in gscenes]
         tokens.copy_(tokens0_d, non_blocking=True)
         state.copy_(state0_d, non_blocking=True)
-        t = 0
-        masked_rows = value_tokens
-        while True:
+        n_left.copy_(n_left0_d, non_blocking=True)
+        kv_of = [None, None]
+        pending = [None, None]      # the event records of a step, completed once its entry counts are known
+
+        def enqueue(t):
             q, k, v, lg = inputs(t)
+            kv_of[t % 2] = (k, v)
+            recs = []
             for layer in range(L):
                 if timed_attn:
                     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
                     e0.record(stream)
-                fdd.fdd_block_attn(ctx, fs, layer, q, k, v, out, ds, scale, 0)
+                fdd.fdd_block_attn_gated(ctx, fs, layer, q, k, v, out, ds, scale, 0, n_left)
                 if timed_attn:
                     e1.record(stream)
-                    attn_events.append((e0, e1))
+                    recs.append([e0, e1, None])
+                    attn_events.append(recs[-1])
             if timed_attn:
                 u0, u1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
                 u0.record(stream)
             fdd.fdd_unmask(ctx, fs, lg, tokens, state, ds, w.threshold, w.temperature, 0, t, n_comm, n_left)
             if timed_attn:
                 u1.record(stream)
-                unmask_events.append((u0, u1, masked_rows))
-            n_left_host.copy_(n_left, non_blocking=True)
-            stream.synchronize()
+                recs.append([u0, u1, None])
+                unmask_events.append(recs[-1])
+            n_left_hosts[t % 2].copy_(n_left, non_blocking=True)
+            step_done[t % 2].record(stream)
+            pending[t % 2] = recs
+
+        def entry_counts(t, rollouts, rows):
+            for r in pending[t % 2][:-1]:
+                r[2] = rollouts
+            if pending[t % 2]:
+                pending[t % 2][-1][2] = rows
+
+        enqueue(0)
+        entry_counts(0, N, value_tokens)
+        t = 0
+        while True:
+            if lookahead and t + 1 < d:
+                enqueue(t + 1)
+            step_done[t % 2].synchronize()
+            left = n_left_hosts[t % 2]
+            masked_rows = int(left.sum())
             t += 1
-            masked_rows = int(n_left_host.sum())
+            if lookahead and t < d:
+                entry_counts(t, int((left != 0).sum()), masked_rows)
             if masked_rows == 0 or t >= d:
                 break
+            if not lookahead:
+                enqueue(t)
+                entry_counts(t, int((left != 0).sum()), masked_rows)
+        k, v = kv_of[(t - 1) % 2]
         for layer in range(L):
             fdd.fdd_kv_commit(ctx, fs, layer, k, v, ds, 1 if layer == L - 1 else 0)
         for i in range(n_scenes):
@@ -210,7 +249,7 @@ def run_ours(args):
         torch.cuda.synchronize()
 
     for _ in range(args.warmup):
-        n_denoise = decode_block(resident, False)
+        n_denoise = decode_block(resident, False, LOOKAHEAD)
     barrier()
     sampler = ClockSampler(local)
     sampler.start()
@@ -219,14 +258,15 @@ def run_ours(args):
     ev0.record(stream)
     denoise_steps = 0
     for _ in range(args.steps):
-        denoise_steps += decode_block(resident, True)
+        denoise_steps += decode_block(resident, True, LOOKAHEAD)
     ev1.record(stream)
     barrier()
     launches = fdd.fdd_launch_count(ctx) - launches0
     sampler.stop_flag = True
     sampler.join(timeout=2)
     ms = ev0.elapsed_time(ev1)
-    attn_ms = [a.elapsed_time(b) for a, b in attn_events]
+    attn_all = [(a.elapsed_time(b), n) for a, b, n in attn_events]
+    attn_ms = [ms_ for ms_, n in attn_all if n == N]          # launches in which every rollout decodes
     unmask_ms = [(a.elapsed_time(b), rows) for a, b, rows in unmask_events]
     ms = replicas.max_over_ranks(ms, dist, "cuda")
     fdd.fdd_poll_status(ctx)
@@ -256,14 +296,14 @@ def run_ours(args):
             return tuple(stage)
 
         e2e_steps = max(1, min(args.steps, args.e2e_steps))
-        decode_block(from_host, False)
+        decode_block(from_host, False, False)
         barrier()
         ee0, ee1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         ee0.record(stream)
         e2e_denoise = 0
         h2d_total[0] = 0
         for _ in range(e2e_steps):
-            e2e_denoise += decode_block(from_host, False)
+            e2e_denoise += decode_block(from_host, False, False)
             tok_host.copy_(tokens, non_blocking=True)
             traj_host.copy_(traj_out, non_blocking=True)
             stream.synchronize()
@@ -303,6 +343,9 @@ def run_ours(args):
                    "denoise_steps_per_block": denoise_steps / args.steps,
                    "value_tokens_per_block": value_tokens, "tokens_incl_scaffold_per_block": all_tokens,
                    "l2": "per-step inputs (logits) larger than L2",
+                   "step_pipeline": ("attention gated by n_left; step t+1 enqueued before the host reads step t"
+                                     if LOOKAHEAD else "attention gated by n_left; one step in flight"),
+                   "rollouts_decoding_per_attention_call": float(np.mean([n for _, n in attn_all])) if attn_all else None,
                    "replicas": "independent scene per GPU, no collective"},
         "clocks": sampler.summary(),
         "e2e": e2e,
@@ -313,7 +356,9 @@ def run_ours(args):
                      "traffic": ATTN_DRAM_BYTES_PER_LAUNCH.get(args.workload) if L == 1 else None,
                      "peak_source": peaks["source"] + " (sustained bf16: the kernel is timed inside the step loop)",
                      "frac_of_burst_peak": (achieved / peaks["bf16_tflops"]) if achieved else None,
-                     "flops_per_launch": flops, "avg_launch_ms": attn_avg_ms, "launches_timed": len(attn_ms)},
+                     "flops_per_launch": flops, "avg_launch_ms": attn_avg_ms, "launches_timed": len(attn_ms),
+                     "launches": "those in which every rollout still decodes (first step of a block)",
+                     "avg_ms_all_launches": float(np.mean([ms_ for ms_, _ in attn_all])) if attn_all else None},
         "roofline_unmask": {"kernel": "fdd_unmask (unmask_partial_kernel), first step of a block: every value row MASKED",
                             "bound": "hbm" if w.temperature == 0 else "alu (Philox + exp2 per logit), reported against hbm",
                             "achieved": um_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
@@ -418,7 +463,7 @@ def run_reference(args):
 
 
 def main():
-    global PRE_STEPS
+    global PRE_STEPS, LOOKAHEAD
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=40)
@@ -430,10 +475,13 @@ def main():
     ap.add_argument("--pre-steps", type=int, default=PRE_STEPS,
                     help="distinct per-step input sets kept resident on the device")
     ap.add_argument("--cpu-budget", type=float, default=20.0)
+    ap.add_argument("--no-lookahead", action="store_true",
+                    help="enqueue a denoising step only after the host has read the counts of the one before")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     PRE_STEPS = max(1, args.pre_steps)
+    LOOKAHEAD = not args.no_lookahead
     if args.impl == "reference":
         run_reference(args)
     else:

@@ -144,6 +144,24 @@ fdd_status fdd_block_attn(fdd_ctx* ctx, fdd_forkset* const* sets, int n_sets, in
                           void* stream);
 
 /*
+ * fdd_block_attn_gated -- fdd_block_attn for the rollouts that still decode.  Under the
+ * confidence threshold of Sec. 3.3 the rollouts of a batch finish their block after different
+ * numbers of denoising steps; a rollout whose block is complete needs no further attention.
+ *
+ *   gate   device int32 [sum N_s], rollouts in set order, read by the kernel when it runs (the
+ *          n_left array that fdd_unmask wrote in the step before fits as it is): rollout r takes
+ *          part if gate[r] != 0; otherwise its rows of out are left untouched and none of its
+ *          keys are read.  NULL: every rollout takes part (fdd_block_attn).
+ * The work of the launch is laid out on the device from the gate values, so a caller may enqueue
+ * the next step before it has seen the result of this one: once every entry is 0 the launch
+ * returns at once.  With a gate a call takes at most 2048 rollouts (FDD_ERR_CAPACITY beyond).  Everything else as fdd_block_attn.
+ */
+fdd_status fdd_block_attn_gated(fdd_ctx* ctx, fdd_forkset* const* sets, int n_sets, int layer,
+                                const void* q, const void* k_blk, const void* v_blk, void* out,
+                                const int32_t* block_len, float scale, int causal_in_block,
+                                const int32_t* gate, void* stream);
+
+/*
  * fdd_unmask -- one parallel unmasking step (Sec. 3.3 "iteratively unmasks value
  * positions"; Sec. 3.1: visible tokens stay fixed; Sec. 3.2: scaffold never rewritten).
  * For every rollout f and every position i with state MASKED:

@@ -42,6 +42,7 @@ namespace {
 constexpr int kTcThreads = 384;
 constexpr int kKeysPerTile = 128;
 constexpr long long kWaitLimit = 4000000000LL;   // about two seconds of SM clocks
+constexpr int kMaxGatedForks = kAttnMaxGatedForks;   // rollouts of one launch when any scene has a gate
 constexpr int kMinTilesPerCta = 8;               // do not cut the work finer than this (every cut costs a merge)
 // Registers per thread after the hand-over.  The CTA starts with 384 x 168; 8 soft-max warps x
 // kRegsSoftmax + 4 other warps x kRegsOther must not exceed that (2 * 208 + 88 = 3 * 168).
@@ -52,9 +53,9 @@ static_assert(2 * kRegsSoftmax + kRegsOther <= 3 * 168, "register hand-over exce
 struct SetParams {
     __nv_bfloat16* out;
     const int32_t* page_table;
-    long long step_base;       // first global tile step of this scene
-    int unit_base;             // first global unit id of this scene
-    int units;                 // Hkv * row_pairs * n_forks
+    const int32_t* gate;       // per rollout, 0 = skip it; nullptr = every rollout takes part
+    int fork_base;             // rollouts of the scenes before this one (index into the kernel's list)
+    int units_per_fork;        // Hkv * row_pairs
     int n_forks, d, n_q_heads, G, R;
     int prefix_len, page_tokens, n_phys_pages, suffix_len;
     int tiles_prefix, tiles_suffix, tiles_total;
@@ -70,7 +71,7 @@ struct TcArgs {
     float* part_lse;           // [2 * ctas][256] log2-domain log-sum-exp of the partial
     int* unit_count;           // pieces finished per unit (self-resetting)
     int* status;
-    long long total_steps;
+    int min_tiles;             // do not cut the work into ranges shorter than this
     int n_sets;
     float scale_log2;
 };
@@ -147,13 +148,14 @@ struct Item {
     long long unit_begin;      // global tile step of the unit's tile 0
 };
 
+// step_base[s]: first global tile step of scene s (scenes laid end to end, skipped rollouts left out)
 template <int MAXSETS>
-__device__ __forceinline__ Item locate(const TcArgs<MAXSETS>& a, long long pos, long long end) {
+__device__ __forceinline__ Item locate(const TcArgs<MAXSETS>& a, const long long* step_base, long long pos, long long end) {
     Item it;
     int s = 0;
-    while (s + 1 < a.n_sets && pos >= a.sets[s + 1].step_base) ++s;
+    while (s + 1 < a.n_sets && pos >= step_base[s + 1]) ++s;
     const SetParams& p = a.sets[s];
-    const long long rel = pos - p.step_base;
+    const long long rel = pos - step_base[s];
     it.s = s;
     it.unit = static_cast<int>(rel / p.tiles_total);
     it.t0 = static_cast<int>(rel - static_cast<long long>(it.unit) * p.tiles_total);
@@ -193,10 +195,46 @@ attn_ptc_kernel(const __grid_constant__ TcArgs<MAXSETS> a) {
     __shared__ int slot_s[kMaxPieces];                  // scratch slot of every piece of the unit being merged
     volatile int* abort_flag = &abort_s;
 
+    // The rollouts that take part (gate != 0), scene after scene, and the layout of the work that
+    // follows from them.  Every CTA derives the same lists from the same gate values.
+    __shared__ unsigned short fork_s[kMaxGatedForks];
+    __shared__ int n_act_s[MAXSETS], unit_base_s[MAXSETS];
+    __shared__ long long step_base_s[MAXSETS + 1];
+
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
-    const long long T = a.total_steps;
-    const long long C = gridDim.x;
+    for (int s = warp; s < a.n_sets; s += kTcThreads / 32) {
+        const SetParams& p = a.sets[s];
+        int cnt = p.n_forks;
+        if (p.gate != nullptr) {
+            cnt = 0;
+            for (int j0 = 0; j0 < p.n_forks; j0 += 32) {
+                const int j = j0 + lane;
+                const bool on = j < p.n_forks && __ldcg(p.gate + j) != 0;
+                const unsigned m = __ballot_sync(0xffffffffu, on);
+                if (on) fork_s[p.fork_base + cnt + __popc(m & ((1u << lane) - 1u))] = static_cast<unsigned short>(j);
+                cnt += __popc(m);
+            }
+        }
+        if (lane == 0) n_act_s[s] = cnt;
+    }
+    __syncthreads();
+    if (tid == 0) {
+        long long steps = 0;
+        int units = 0;
+        for (int s = 0; s < a.n_sets; ++s) {
+            step_base_s[s] = steps;
+            unit_base_s[s] = units;
+            const int u = a.sets[s].units_per_fork * n_act_s[s];
+            steps += static_cast<long long>(u) * a.sets[s].tiles_total;
+            units += u;
+        }
+        step_base_s[a.n_sets] = steps;
+    }
+    __syncthreads();
+    const long long T = step_base_s[a.n_sets];
+    const long long C = max(1LL, min(static_cast<long long>(gridDim.x), T / a.min_tiles));
+    if (T == 0 || blockIdx.x >= C) return;          // nothing (left) to do: before any barrier or TMEM exists
     const long long range_begin = T * blockIdx.x / C;
     const long long range_end = T * (blockIdx.x + 1) / C;
 
@@ -238,10 +276,12 @@ attn_ptc_kernel(const __grid_constant__ TcArgs<MAXSETS> a) {
     };
     auto view_item = [&](long long pos) {
         ItemView v;
-        v.it = locate(a, pos, range_end);
+        v.it = locate(a, step_base_s, pos, range_end);
         const SetParams& p = a.sets[v.it.s];
         int idx = v.it.unit;
-        v.f = idx % p.n_forks; idx /= p.n_forks;
+        const int n_act = n_act_s[v.it.s];
+        v.f = idx % n_act; idx /= n_act;
+        if (p.gate != nullptr) v.f = fork_s[p.fork_base + v.f];
         v.rp = idx % p.row_pairs; idx /= p.row_pairs;
         v.h = idx;
         v.nt = v.it.t1 - v.it.t0;
@@ -640,7 +680,7 @@ attn_ptc_kernel(const __grid_constant__ TcArgs<MAXSETS> a) {
                 __threadfence();
                 tc::named_barrier(1, 256);
                 if (tid == 0) {
-                    const int gu = p.unit_base + it.unit;
+                    const int gu = unit_base_s[it.s] + it.unit;
                     const int old = atomicAdd(a.unit_count + gu, 1);
                     const int last = old == n_pieces - 1;
                     if (last) a.unit_count[gu] = 0;          // every piece has arrived: ready for the next launch
@@ -857,7 +897,8 @@ cudaError_t launch_group(fdd_ctx* ctx, const AttnProblem* probs, TcMapCache* con
                          cudaStream_t st) {
     static TcArgs<MAXSETS> args;     // 1-20 KB, kept off the stack (a context is used by one host thread at a time)
     long long steps = 0;
-    int units = 0;
+    int units = 0, forks = 0;
+    bool gated = false;
     for (int s = 0; s < n; ++s) {
         const AttnProblem& a = probs[s];
         const TcSetMaps* m = maps_for(a, head_dim, caches[s]);
@@ -875,14 +916,17 @@ cudaError_t launch_group(fdd_ctx* ctx, const AttnProblem* probs, TcMapCache* con
         p.tiles_suffix = (a.suffix_len + kKeysPerTile - 1) / kKeysPerTile;
         p.tiles_total = p.tiles_prefix + p.tiles_suffix + (a.d + kKeysPerTile - 1) / kKeysPerTile;
         p.row_pairs = (p.R + 255) / 256;
-        p.units = a.n_kv_heads * p.row_pairs * a.n_forks;
+        p.units_per_fork = a.n_kv_heads * p.row_pairs;
         p.causal = a.causal_in_block;
-        p.step_base = steps;
-        p.unit_base = units;
-        steps += static_cast<long long>(p.units) * p.tiles_total;
-        units += p.units;
+        p.gate = a.gate;
+        p.fork_base = forks;
+        gated = gated || a.gate != nullptr;
+        forks += a.n_forks;
+        steps += static_cast<long long>(p.units_per_fork) * a.n_forks * p.tiles_total;
+        units += p.units_per_fork * a.n_forks;
     }
     if (units > ctx->attn_max_units) return cudaErrorInvalidValue;
+    if (gated && forks > kMaxGatedForks) return cudaErrorInvalidValue;
     static int min_tiles = 0;
     if (min_tiles == 0) {
         min_tiles = kMinTilesPerCta;
@@ -895,7 +939,7 @@ cudaError_t launch_group(fdd_ctx* ctx, const AttnProblem* probs, TcMapCache* con
     args.part_lse = args.part_o + static_cast<size_t>(2) * ctx->attn_max_ctas * 256 * head_dim;
     args.unit_count = ctx->attn_unit_count;
     args.status = ctx->d_status;
-    args.total_steps = steps;
+    args.min_tiles = min_tiles;
     args.n_sets = n;
     args.scale_log2 = probs[0].scale * 1.4426950408889634f;
     return launch_emu<MAXSETS>(args, head_dim, static_cast<unsigned>(ctas), st);

@@ -50,6 +50,7 @@ attn_simple_kernel(const AttnProblem a) {
     const int r0 = blockIdx.x * kRows;
     const int h = blockIdx.y;      // KV head
     const int f = blockIdx.z;      // rollout
+    if (a.gate != nullptr && a.gate[f] == 0) return;   // the whole CTA: this rollout sits the call out
     const int tid = threadIdx.x;
     const int rr = tid >> 3;       // local row
     const int t8 = tid & 7;

@@ -196,6 +196,14 @@ fdd_status fdd_forkset_reset(fdd_ctx* ctx, fdd_forkset* set) {
 fdd_status fdd_block_attn(fdd_ctx* ctx, fdd_forkset* const* sets, int n_sets, int layer,
                           const void* q, const void* k_blk, const void* v_blk, void* out,
                           const int32_t* block_len, float scale, int causal_in_block, void* stream) {
+    return fdd_block_attn_gated(ctx, sets, n_sets, layer, q, k_blk, v_blk, out, block_len, scale, causal_in_block,
+                                nullptr, stream);
+}
+
+fdd_status fdd_block_attn_gated(fdd_ctx* ctx, fdd_forkset* const* sets, int n_sets, int layer,
+                                const void* q, const void* k_blk, const void* v_blk, void* out,
+                                const int32_t* block_len, float scale, int causal_in_block,
+                                const int32_t* gate, void* stream) {
     if (!ctx) return FDD_ERR_INVALID_ARG;
     int total = 0;
     fdd_status st = check_sets(ctx, sets, n_sets, block_len, &total);
@@ -205,9 +213,12 @@ fdd_status fdd_block_attn(fdd_ctx* ctx, fdd_forkset* const* sets, int n_sets, in
         return fail(ctx, FDD_ERR_INVALID_ARG, "q/k_blk/v_blk/out must be 16-byte aligned");
     if (layer < 0 || layer >= ctx->cfg.n_layers) return fail(ctx, FDD_ERR_SHAPE, "layer %d outside [0, %d)", layer, ctx->cfg.n_layers);
     if (!(scale > 0.0f)) return fail(ctx, FDD_ERR_INVALID_ARG, "scale must be positive");
+    if (gate && total > kAttnMaxGatedForks)
+        return fail(ctx, FDD_ERR_CAPACITY, "%d rollouts in one gated call exceed %d", total, kAttnMaxGatedForks);
     const fdd_config& c = ctx->cfg;
     cudaStream_t st_ = static_cast<cudaStream_t>(stream);
     size_t q_off = 0, kv_off = 0;
+    int fork_off = 0;
     std::vector<AttnProblem> tc_probs;
     std::vector<TcMapCache*> tc_caches;
     for (int s = 0; s < n_sets; ++s) {
@@ -233,6 +244,8 @@ fdd_status fdd_block_attn(fdd_ctx* ctx, fdd_forkset* const* sets, int n_sets, in
         p.suffix_capacity = fs->suffix_capacity;
         p.causal_in_block = causal_in_block ? 1 : 0;
         p.scale = scale;
+        p.gate = gate ? gate + fork_off : nullptr;
+        fork_off += fs->n_forks;
         if (attention_tc_supported(p, c.head_dim)) {
             // the tensor-core kernel takes many scenes per launch
             tc_probs.push_back(p);

@@ -78,8 +78,10 @@ struct AttnProblem {
     int suffix_len, suffix_capacity;
     int causal_in_block;
     float scale;
+    const int32_t* gate;           // device [N], 0 = leave the rollout out; nullptr = all take part
 };
 
+constexpr int kAttnMaxGatedForks = 2048;    // rollouts of one fdd_block_attn_gated call
 constexpr int kUnmaskMaxSets = 16;          // scenes per unmask launch
 
 // Several scenes of one unmask call, packed in set order (rows = rollouts x positions).

@@ -20,7 +20,7 @@ FDD_LOGITS_F32, FDD_LOGITS_BF16 = 0, 1
 
 EXPORTS = (
     "fdd_create", "fdd_destroy", "fdd_last_error", "fdd_launch_count", "fdd_fork",
-    "fdd_forkset_free", "fdd_forkset_suffix_len", "fdd_forkset_reset", "fdd_block_attn",
+    "fdd_forkset_free", "fdd_forkset_suffix_len", "fdd_forkset_reset", "fdd_block_attn", "fdd_block_attn_gated",
     "fdd_unmask", "fdd_ss_draft", "fdd_ss_accept", "fdd_kv_commit", "fdd_average_rollouts", "fdd_poll_status", "fdd_unmask_static", "fdd_plan_blocks", "fdd_upload_masked_rows",
 )
 FDD_UNMASK_STATIC_MAX_RECORDS = 65536
@@ -72,6 +72,8 @@ def lib():
     L.fdd_forkset_reset.restype = i32
     L.fdd_block_attn.argtypes = [vp, vpp, i32, i32, vp, vp, vp, vp, ip, f32, i32, vp]
     L.fdd_block_attn.restype = i32
+    L.fdd_block_attn_gated.argtypes = [vp, vpp, i32, i32, vp, vp, vp, vp, ip, f32, i32, vp, vp]
+    L.fdd_block_attn_gated.restype = i32
     L.fdd_unmask.argtypes = [vp, vpp, i32, vp, vp, vp, ip, f32, f32, u32, u32, vp, vp, vp, vp]
     L.fdd_unmask.restype = i32
     for fn in (L.fdd_ss_draft, L.fdd_ss_accept):
@@ -184,6 +186,13 @@ def fdd_block_attn(ctx, sets, layer, q, k_blk, v_blk, out, block_len, scale, cau
     return _check(ctx, lib().fdd_block_attn(
         ctx, _ptr_array(sets), len(sets), int(layer), _ptr(q), _ptr(k_blk), _ptr(v_blk), _ptr(out),
         _i32_array(block_len), float(scale), int(causal_in_block), _stream(stream)))
+
+
+def fdd_block_attn_gated(ctx, sets, layer, q, k_blk, v_blk, out, block_len, scale, causal_in_block, gate,
+                         stream=None):
+    return _check(ctx, lib().fdd_block_attn_gated(
+        ctx, _ptr_array(sets), len(sets), int(layer), _ptr(q), _ptr(k_blk), _ptr(v_blk), _ptr(out),
+        _i32_array(block_len), float(scale), int(causal_in_block), _ptr(gate), _stream(stream)))
 
 
 def fdd_unmask(ctx, sets, logits, tokens, state, block_len, threshold, temperature, block_idx, step,

@@ -133,6 +133,76 @@ def test_attention_many_scenes_one_call():
         fdd.fdd_destroy(ctx)
 
 
+def test_attention_gated_rollouts_are_skipped_and_the_rest_is_unchanged():
+    # fdd_block_attn_gated: rollouts whose gate entry is 0 sit the call out (their rows of out keep
+    # what was there), every other rollout gets what the ungated call gives, whatever the mix:
+    # some rollouts of a scene, a whole scene, everything, nothing.  The gate is the n_left array of
+    # an unmask step, so any non-zero value counts as "still decoding".
+    base = synth.workload("serving_mix")
+    scenes = (synth.Scene(64 * 9 + 5, 5, 32, 10, 1), synth.Scene(64 * 30, 2, 64, 19, 1),
+              synth.Scene(333, 37, 16, 5, 1), synth.Scene(64, 1, 16, 5, 1))
+    w = synth.Workload("gated", base.n_q_heads, base.n_kv_heads, base.head_dim, 1024, "bf16", "peaked", 0.9, 1.0,
+                       scenes, page_tokens=64, seed=23)
+    ctx = harness.create_context(w)
+    try:
+        gs, refs, qs, ks, vs = [], [], [], [], []
+        for i, sc in enumerate(scenes):
+            gs.append(harness.GpuScene(ctx, w, i))
+            pk, pv = synth.make_prefix(w, i)
+            q, k, v = synth.make_qkv(w, i, 0, 0, 0)
+            empty = ([np.zeros((0, w.n_kv_heads, w.head_dim), dtype=np.uint16)] * sc.n_forks,) * 2
+            refs.append(pu.attention_oracle(w, (pk, pv), empty, q, k, v))
+            qs.append(q); ks.append(k); vs.append(v)
+        pack = lambda xs: harness.bf16_tensor(np.concatenate([x.reshape(-1) for x in xs]))
+        qd, kd, vd = pack(qs), pack(ks), pack(vs)
+        n_total = sum(sc.n_forks for sc in scenes)
+        rng = np.random.default_rng(5)
+        some = rng.integers(0, 3, n_total).astype(np.int32) * 7          # about a third are 0
+        some[5:7] = 0                                                    # scene 1 sits out as a whole
+        gates = [some, np.ones(n_total, np.int32), np.zeros(n_total, np.int32),
+                 (np.arange(n_total) == 11).astype(np.int32)]
+        for gate in gates:
+            out = torch.full_like(qd, float("nan"))
+            n0 = fdd.fdd_launch_count(ctx)
+            fdd.fdd_block_attn_gated(ctx, [g.forkset for g in gs], 0, qd, kd, vd, out,
+                                     [sc.block_len for sc in scenes], 1.0 / np.sqrt(w.head_dim), 0,
+                                     torch.from_numpy(gate).cuda())
+            fdd.fdd_poll_status(ctx)
+            assert fdd.fdd_launch_count(ctx) - n0 == 1
+            got = out.float().cpu().numpy().astype(np.float64)
+            off = fork = 0
+            for sc, ref in zip(scenes, refs):
+                rows = got[off:off + ref.size].reshape(ref.shape)
+                for f in range(sc.n_forks):
+                    if gate[fork + f]:
+                        pu.assert_attention_close(rows[f], ref[f])
+                    else:
+                        assert np.all(np.isnan(rows[f])), "a skipped rollout was written"
+                off += ref.size; fork += sc.n_forks
+    finally:
+        fdd.fdd_destroy(ctx)
+    # the CUDA-core kernel (GQA group of three) honours the gate as well
+    w = synth.Workload("g3_gated", 6, 2, 64, 256, "f32", "peaked", 0.9, 0.0,
+                       (synth.Scene(prefix_len=100, n_forks=3, block_len=16, n_scaffold=5, n_blocks=1),), seed=13)
+    ctx = harness.create_context(w)
+    try:
+        g = harness.GpuScene(ctx, w, 0)
+        pk, pv = synth.make_prefix(w, 0)
+        q, k, v = synth.make_qkv(w, 0, 0, 0, 0)
+        empty = ([np.zeros((0, w.n_kv_heads, w.head_dim), dtype=np.uint16)] * 3,) * 2
+        ref = pu.attention_oracle(w, (pk, pv), empty, q, k, v)
+        out = torch.full((q.size,), float("nan"), dtype=torch.bfloat16, device="cuda")
+        fdd.fdd_block_attn_gated(ctx, [g.forkset], 0, harness.bf16_tensor(q), harness.bf16_tensor(k),
+                                 harness.bf16_tensor(v), out, [16], 1.0 / np.sqrt(w.head_dim), 0,
+                                 torch.tensor([4, 0, 1], dtype=torch.int32, device="cuda"))
+        fdd.fdd_poll_status(ctx)
+        got = out.float().cpu().numpy().astype(np.float64).reshape(ref.shape)
+        pu.assert_attention_close(got[[0, 2]], ref[[0, 2]])
+        assert np.all(np.isnan(got[1]))
+    finally:
+        fdd.fdd_destroy(ctx)
+
+
 def test_attention_repeated_calls_reuse_scratch():
     # the scratch of the split-unit merge is reusable at once: the same call three times in a row
     # (different inputs) stays correct
@@ -624,6 +694,78 @@ def test_block_loop_matches_oracle_and_averages():
         ref = average_rollouts(traj)
         got = out.cpu().numpy().astype(np.float64)
         assert np.all(np.abs(got - ref) <= 1e-5 * np.maximum(np.abs(ref), 1e-30) + 1e-30)
+    finally:
+        fdd.fdd_destroy(ctx)
+
+
+def test_pipelined_block_loop_gated_attention_one_step_ahead():
+    # The loop as a server runs it: everything stays on the device, attention is gated by the
+    # n_left array of the step before, and step t + 1 is enqueued before the host has read the
+    # counts of step t.  Every step is recorded on the device and re-done by the oracle afterwards:
+    # rollouts that still decode get the oracle's attention, finished ones are never written, the
+    # step enqueued after the block was complete does nothing at all.
+    w = synth.small_variant(synth.workload("tts"), prefix_len=300, vocab=2048, n_forks=6)
+    sc = w.scenes[0]
+    N, d = sc.n_forks, sc.block_len
+    ctx = harness.create_context(w)
+    try:
+        scene = harness.GpuScene(ctx, w, 0)
+        pk, pv = synth.make_prefix(w, 0)
+        empty = ([np.zeros((0, w.n_kv_heads, w.head_dim), dtype=np.uint16)] * N,) * 2
+        tokens0, state0 = synth.make_block_template(w, 0, 0)
+        tokens = torch.from_numpy(tokens0).cuda()
+        state = torch.from_numpy(state0).cuda()
+        n_left = torch.from_numpy((state0 == MASKED).sum(axis=1).astype(np.int32)).cuda()
+        n_comm = torch.zeros(N, dtype=torch.int32, device="cuda")
+        hosts = [torch.zeros(N, dtype=torch.int32).pin_memory() for _ in range(2)]
+        done = [torch.cuda.Event(), torch.cuda.Event()]
+        stream = torch.cuda.current_stream()
+        inputs, rec = [], []
+        scale = 1.0 / np.sqrt(w.head_dim)
+
+        def enqueue(t):
+            q, k, v = synth.make_qkv(w, 0, 0, 0, t)
+            lg = synth.make_logits(w, 0, 0, t, rows="all")
+            inputs.append((q, k, v, lg))
+            out = torch.full((q.size,), float("nan"), dtype=torch.bfloat16, device="cuda")
+            fdd.fdd_block_attn_gated(ctx, [scene.forkset], 0, harness.bf16_tensor(q), harness.bf16_tensor(k),
+                                     harness.bf16_tensor(v), out, [d], scale, 0, n_left)
+            fdd.fdd_unmask(ctx, [scene.forkset], harness.logits_tensor(w, lg), tokens, state, [d], w.threshold,
+                           w.temperature, 0, t, n_comm, n_left)
+            rec.append((out, tokens.clone(), state.clone(), n_comm.clone(), n_left.clone()))
+            hosts[t % 2].copy_(n_left, non_blocking=True)
+            done[t % 2].record(stream)
+
+        enqueue(0)
+        t = 0
+        while True:
+            if t + 1 < d:
+                enqueue(t + 1)
+            done[t % 2].synchronize()
+            left = int(hosts[t % 2].sum())
+            t += 1
+            if left == 0 or t >= d:
+                break
+        torch.cuda.synchronize()
+        fdd.fdd_poll_status(ctx)
+        assert 2 <= t < d and len(rec) == t + 1
+        tok_in, st_in, ambiguous = tokens0, state0, 0
+        for step, ((q, k, v, lg), (out, tok, st, nc, nl)) in enumerate(zip(inputs, rec)):
+            decoding = np.nonzero((st_in == MASKED).any(axis=1))[0]
+            got_attn = out.float().cpu().numpy().astype(np.float64).reshape(N, d, w.n_q_heads, w.head_dim)
+            if len(decoding):
+                ref_attn = pu.attention_oracle(w, (pk, pv), empty, q, k, v, forks=decoding)
+                pu.assert_attention_close(got_attn[decoding], ref_attn)
+            idle = np.setdiff1d(np.arange(N), decoding)
+            assert np.all(np.isnan(got_attn[idle])), "attention wrote rows of a rollout that had finished"
+            got = dict(tokens=tok.cpu().numpy(), state=st.cpu().numpy(), conf=None,
+                       n_committed=nc.cpu().numpy(), n_left=nl.cpu().numpy())
+            ref = unmask_step(pu.widen_logits(w, lg), tok_in, st_in, scene.seeds, w.threshold, w.temperature, 0, step)
+            ambiguous += len(pu.compare_unmask(got, ref, tok_in, st_in, w.threshold)["ambiguous_forks"])
+            tok_in, st_in = got["tokens"], got["state"]
+        assert ambiguous <= 1
+        assert not np.any(st_in == MASKED)
+        assert step == t and len(decoding) == 0          # the last recorded step ran after the block was complete
     finally:
         fdd.fdd_destroy(ctx)
 
