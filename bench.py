@@ -164,6 +164,12 @@ def run_ours(args):
     n_left0_d = torch.from_numpy(np.concatenate(
         [(s_ == synth.MASKED).sum(axis=1).astype(np.int32) for _, s_ in templates])).cuda()
     n_left_hosts = [torch.zeros(N, dtype=torch.int32).pin_memory() for _ in range(2)]
+    n_left_views = [t_.numpy() for t_ in n_left_hosts]          # the host reads the counts through these
+    # arguments that are the same in every call are marshalled once
+    ds_c = fdd.i32_array(ds)
+    fork_args = [(fdd.ptr_array(g.prefix_k), fdd.ptr_array(g.prefix_v), g.page_table, g.sc.prefix_len,
+                  g.prefix_capacity, g.sc.n_forks, fdd.u64_array(g.seeds), fdd.ptr_array(g.suffix_k),
+                  fdd.ptr_array(g.suffix_v), g.suffix_capacity) for g in gscenes]
     step_done = [torch.cuda.Event(), torch.cuda.Event()]
 
     attn_events = []            # [start, end, rollouts still decoding] of every timed attention call
@@ -176,8 +182,8 @@ def run_ours(args):
         `lookahead` step t + 1 is enqueued before the host has seen the result of step t (once
         every rollout is done its kernels return at once), which keeps the GPU busy while the host
         reads the counts."""
-        fs = [fdd.fdd_fork(ctx, g.prefix_k, g.prefix_v, g.page_table, g.sc.prefix_len, g.prefix_capacity,
-                           g.sc.n_forks, g.seeds, g.suffix_k, g.suffix_v, g.suffix_capacity) for g in gscenes]
+        fs_list = [fdd.fdd_fork(ctx, *fa) for fa in fork_args]
+        fs = fdd.ptr_array(fs_list)
         tokens.copy_(tokens0_d, non_blocking=True)
         state.copy_(state0_d, non_blocking=True)
         n_left.copy_(n_left0_d, non_blocking=True)
@@ -192,7 +198,7 @@ def run_ours(args):
                 if timed_attn:
                     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
                     e0.record(stream)
-                fdd.fdd_block_attn_gated(ctx, fs, layer, q, k, v, out, ds, scale, 0, n_left)
+                fdd.fdd_block_attn_gated(ctx, fs, layer, q, k, v, out, ds_c, scale, 0, n_left)
                 if timed_attn:
                     e1.record(stream)
                     recs.append([e0, e1, None])
@@ -200,7 +206,7 @@ def run_ours(args):
             if timed_attn:
                 u0, u1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
                 u0.record(stream)
-            fdd.fdd_unmask(ctx, fs, lg, tokens, state, ds, w.threshold, w.temperature, 0, t, n_comm, n_left)
+            fdd.fdd_unmask(ctx, fs, lg, tokens, state, ds_c, w.threshold, w.temperature, 0, t, n_comm, n_left)
             if timed_attn:
                 u1.record(stream)
                 recs.append([u0, u1, None])
@@ -222,7 +228,7 @@ def run_ours(args):
             if lookahead and t + 1 < d:
                 enqueue(t + 1)
             step_done[t % 2].synchronize()
-            left = n_left_hosts[t % 2]
+            left = n_left_views[t % 2]
             masked_rows = int(left.sum())
             t += 1
             if lookahead and t < d:
@@ -234,10 +240,10 @@ def run_ours(args):
                 entry_counts(t, int((left != 0).sum()), masked_rows)
         k, v = kv_of[(t - 1) % 2]
         for layer in range(L):
-            fdd.fdd_kv_commit(ctx, fs, layer, k, v, ds, 1 if layer == L - 1 else 0)
+            fdd.fdd_kv_commit(ctx, fs, layer, k, v, ds_c, 1 if layer == L - 1 else 0)
         for i in range(n_scenes):
             fdd.fdd_average_rollouts(ctx, trajs[i], Ns[i], w.waypoints, traj_out[i])
-        for f_ in fs:
+        for f_ in fs_list:
             fdd.fdd_forkset_free(ctx, f_)
         return t
 

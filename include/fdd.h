@@ -23,7 +23,9 @@
  *     detected on the host before anything is launched and returned synchronously.
  *   - No call aborts, throws or prints.  A negative fdd_status is an error; the text
  *     is available from fdd_last_error().
- *   - A context and its fork sets must be used from one host thread at a time.
+ *   - A context and its fork sets must be used from one host thread at a time.  The calls
+ *     on one context share its scratch buffers, so the work they enqueue has to execute in
+ *     call order: use one stream per context, or order the streams yourself.
  *
  * Position state codes (uint8): 0 = MASKED (to be decoded), 1 = COMMITTED, 2 = SCAFFOLD
  * (frozen structural token, Sec. 3.2), 3 = DRAFT (between fdd_ss_draft and fdd_ss_accept).
@@ -101,7 +103,8 @@ uint64_t fdd_launch_count(const fdd_ctx* ctx);
  *   prefix_len          valid prefix tokens (>= 0).
  *   prefix_capacity     tokens per head (contiguous) or number of physical pages (paged).
  *   n_forks             N >= 1, <= cfg.max_forks.
- *   seeds               host uint64 [N]: the noise key of each rollout (copied).
+ *   seeds               host uint64 [N]: the noise key of each rollout (copied; the first call
+ *                       that samples stores them on the device, in stream order).
  *   suffix_k, suffix_v  host arrays [L] of device pointers, bf16 [N][Hkv][suffix_capacity][D],
  *                       caller-owned, written by fdd_kv_commit only.
  *   suffix_capacity     tokens each rollout may append per layer.
@@ -111,6 +114,8 @@ fdd_status fdd_fork(fdd_ctx* ctx, const void* const* prefix_k, const void* const
                     int n_forks, const uint64_t* seeds,
                     void* const* suffix_k, void* const* suffix_v, int suffix_capacity,
                     fdd_forkset** out);
+/* Neither fdd_fork nor fdd_forkset_free waits for the device; a set may be freed while the
+ * work enqueued for it is still running (its caches are the caller's to keep alive). */
 fdd_status fdd_forkset_free(fdd_ctx* ctx, fdd_forkset* set);
 /* Committed private tokens per rollout (same for every rollout of a set); < 0 on error. */
 int fdd_forkset_suffix_len(const fdd_forkset* set);

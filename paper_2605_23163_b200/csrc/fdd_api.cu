@@ -27,6 +27,48 @@ fdd_status cuda_fail(fdd_ctx* ctx, cudaError_t e, const char* what) {
     return fail(ctx, FDD_ERR_CUDA, "%s: %s", what, cudaGetErrorString(e));
 }
 
+// Seeds travel to the device as kernel arguments: stream-ordered like everything else, no
+// staging buffer, no allocation, no synchronisation.
+constexpr size_t kMapPoolEntries = 64;
+constexpr int kSeedsPerLaunch = 240;
+struct SeedChunk {
+    uint64_t value[kSeedsPerLaunch];
+    uint64_t* dst[kSeedsPerLaunch];
+    int n;
+};
+
+__global__ void seed_store_kernel(const __grid_constant__ SeedChunk c) {
+    const int i = threadIdx.x;
+    if (i < c.n) *c.dst[i] = c.value[i];
+}
+
+// Store the seeds of every set of the call that has not been used for sampling yet.
+cudaError_t ensure_seeds(fdd_ctx* ctx, fdd_forkset* const* sets, int n_sets, cudaStream_t st) {
+    static SeedChunk chunk;        // 4 KB, kept off the stack (a context is used by one host thread at a time)
+    chunk.n = 0;
+    auto flush = [&]() -> cudaError_t {
+        if (chunk.n == 0) return cudaSuccess;
+        seed_store_kernel<<<1, 256, 0, st>>>(chunk);
+        ctx->launches += 1;
+        chunk.n = 0;
+        return cudaGetLastError();
+    };
+    for (int s = 0; s < n_sets; ++s) {
+        fdd_forkset* fs = sets[s];
+        if (fs->seeds_on_device) continue;
+        for (int f = 0; f < fs->n_forks; ++f) {
+            chunk.value[chunk.n] = fs->h_seeds[f];
+            chunk.dst[chunk.n] = fs->d_seeds + f;
+            if (++chunk.n == kSeedsPerLaunch) {
+                cudaError_t e = flush();
+                if (e != cudaSuccess) return e;
+            }
+        }
+        fs->seeds_on_device = true;
+    }
+    return flush();
+}
+
 bool set_alive(const fdd_ctx* ctx, const fdd_forkset* s) {
     return s && std::find(ctx->live_sets.begin(), ctx->live_sets.end(), s) != ctx->live_sets.end();
 }
@@ -106,6 +148,7 @@ void fdd_destroy(fdd_ctx* ctx) {
         if (s->d_seeds) cudaFree(s->d_seeds);
         delete s;
     }
+    for (const fdd_ctx::SeedBuf& b : ctx->seed_pool) cudaFree(b.ptr);
     if (ctx->d_status) cudaFree(ctx->d_status);
     if (ctx->h_status) cudaFreeHost(ctx->h_status);
     if (ctx->ws_unmask) cudaFree(ctx->ws_unmask);
@@ -161,13 +204,36 @@ fdd_status fdd_fork(fdd_ctx* ctx, const void* const* prefix_k, const void* const
     s->suffix_v.assign(suffix_v, suffix_v + ctx->cfg.n_layers);
     s->suffix_capacity = suffix_capacity;
     s->suffix_len = 0;
+    // the tensor maps of an earlier set over the same caches serve again
+    for (size_t i = 0; i < ctx->map_pool.size(); ++i) {
+        TcMapPoolEntry& m = ctx->map_pool[i];
+        if (m.n_forks == n_forks && m.prefix_len == prefix_len && m.prefix_capacity == prefix_capacity &&
+            m.suffix_capacity == suffix_capacity && m.prefix_k == s->prefix_k && m.prefix_v == s->prefix_v &&
+            m.suffix_k == s->suffix_k && m.suffix_v == s->suffix_v) {
+            s->map_cache = std::move(m.maps);
+            ctx->map_pool.erase(ctx->map_pool.begin() + i);
+            break;
+        }
+    }
     s->map_cache.resize(ctx->cfg.n_layers);
-    cudaError_t e = cudaMalloc(&s->d_seeds, sizeof(uint64_t) * n_forks);
-    if (e == cudaSuccess) e = cudaMemcpy(s->d_seeds, seeds, sizeof(uint64_t) * n_forks, cudaMemcpyHostToDevice);
-    if (e != cudaSuccess) {
-        if (s->d_seeds) cudaFree(s->d_seeds);
-        delete s;
-        return cuda_fail(ctx, e, "fdd_fork seeds");
+    s->h_seeds.assign(seeds, seeds + n_forks);
+    // A seed buffer left by a freed set serves again (the smallest that is large enough); only a
+    // context that has never held this many rollouts allocates.
+    int best = -1;
+    for (size_t i = 0; i < ctx->seed_pool.size(); ++i)
+        if (ctx->seed_pool[i].cap >= n_forks && (best < 0 || ctx->seed_pool[i].cap < ctx->seed_pool[best].cap))
+            best = static_cast<int>(i);
+    if (best >= 0) {
+        s->d_seeds = ctx->seed_pool[best].ptr;
+        s->seed_cap = ctx->seed_pool[best].cap;
+        ctx->seed_pool.erase(ctx->seed_pool.begin() + best);
+    } else {
+        s->seed_cap = std::max(n_forks, 64);
+        cudaError_t e = cudaMalloc(&s->d_seeds, sizeof(uint64_t) * s->seed_cap);
+        if (e != cudaSuccess) {
+            delete s;
+            return cuda_fail(ctx, e, "fdd_fork seeds");
+        }
     }
     ctx->live_sets.push_back(s);
     *out = s;
@@ -179,7 +245,13 @@ fdd_status fdd_forkset_free(fdd_ctx* ctx, fdd_forkset* set) {
     auto it = std::find(ctx->live_sets.begin(), ctx->live_sets.end(), set);
     if (!set || it == ctx->live_sets.end()) return fail(ctx, FDD_ERR_STATE, "fork set is not live (double free?)");
     ctx->live_sets.erase(it);
-    cudaFree(set->d_seeds);
+    // Work of the set may still be in flight: the buffer is not freed (that would wait for the
+    // device) but kept; whoever gets it next writes it in stream order, after that work.
+    ctx->seed_pool.push_back({set->d_seeds, set->seed_cap});
+    if (ctx->map_pool.size() >= kMapPoolEntries) ctx->map_pool.erase(ctx->map_pool.begin());
+    ctx->map_pool.push_back({std::move(set->prefix_k), std::move(set->prefix_v), std::move(set->suffix_k),
+                             std::move(set->suffix_v), set->n_forks, set->prefix_len, set->prefix_capacity,
+                             set->suffix_capacity, std::move(set->map_cache)});
     delete set;
     return FDD_OK;
 }
@@ -284,6 +356,10 @@ static fdd_status unmask_like(fdd_ctx* ctx, fdd_forkset* const* sets, int n_sets
     if (threshold != threshold) return fail(ctx, FDD_ERR_INVALID_ARG, "threshold is NaN");
     const fdd_config& c = ctx->cfg;
     const size_t esz = c.logits_dtype == FDD_LOGITS_BF16 ? 2 : 4;
+    if (temperature > 0.0f) {
+        cudaError_t e = ensure_seeds(ctx, sets, n_sets, static_cast<cudaStream_t>(stream));
+        if (e != cudaSuccess) return cuda_fail(ctx, e, "seed upload");
+    }
     // Sets go to the kernels in groups of at most kUnmaskMaxSets sets and kUnmaskMaxRows rows.
     size_t row_off = 0;
     int fork_off = 0;

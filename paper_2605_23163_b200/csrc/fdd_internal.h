@@ -30,6 +30,15 @@ struct TcMapCache {
     TcSetMaps maps;
 };
 
+// Tensor maps of a freed fork set, kept for a later set over the same caches (a server forks the
+// same prefix block after block).
+struct TcMapPoolEntry {
+    std::vector<const void*> prefix_k, prefix_v;
+    std::vector<void*> suffix_k, suffix_v;
+    int n_forks, prefix_len, prefix_capacity, suffix_capacity;
+    std::vector<TcMapCache> maps;
+};
+
 struct fdd_ctx {
     fdd_config cfg;
     int device = 0;
@@ -46,6 +55,9 @@ struct fdd_ctx {
     uint64_t launches = 0;
     std::string last_error;
     std::vector<fdd_forkset*> live_sets;
+    struct SeedBuf { uint64_t* ptr; int cap; };
+    std::vector<SeedBuf> seed_pool;   // device seed buffers of freed fork sets, kept for the next fork
+    std::vector<TcMapPoolEntry> map_pool;
 };
 
 struct fdd_forkset {
@@ -58,7 +70,10 @@ struct fdd_forkset {
     std::vector<void*> suffix_k, suffix_v;
     int suffix_capacity = 0;
     int suffix_len = 0;
-    uint64_t* d_seeds = nullptr;            // device [n_forks]
+    uint64_t* d_seeds = nullptr;            // device [seed_cap], from the context's pool
+    int seed_cap = 0;
+    std::vector<uint64_t> h_seeds;          // the caller's seeds, stored on the device by the first call that needs them
+    bool seeds_on_device = false;
     std::vector<TcMapCache> map_cache;      // per layer
 };
 

@@ -106,6 +106,8 @@ def _ptr(t):
 
 
 def _stream(stream):
+    if isinstance(stream, ctypes.c_void_p):
+        return stream
     if stream is None:
         import torch
         return ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
@@ -121,6 +123,8 @@ def _check(ctx, status):
 
 
 def _ptr_array(items):
+    if isinstance(items, ctypes.Array):      # marshalled earlier by ptr_array()
+        return items
     arr = (ctypes.c_void_p * len(items))()
     for i, t in enumerate(items):
         p = _ptr(t)
@@ -129,7 +133,26 @@ def _ptr_array(items):
 
 
 def _i32_array(vals):
+    if isinstance(vals, ctypes.Array):       # marshalled earlier by i32_array()
+        return vals
     return (ctypes.c_int32 * len(vals))(*[int(v) for v in vals])
+
+
+def ptr_array(items):
+    """Marshal a list of tensors / handles once; the result can be passed wherever the binding
+    takes such a list (saves the conversion in a loop that passes the same list every step)."""
+    return _ptr_array(items)
+
+
+def i32_array(vals):
+    """Marshal a list of ints once (see ptr_array)."""
+    return _i32_array(vals)
+
+
+def u64_array(vals):
+    """Marshal a list of 64-bit seeds once (see ptr_array)."""
+    vals = [int(s) & 0xFFFFFFFFFFFFFFFF for s in vals]
+    return (ctypes.c_uint64 * len(vals))(*vals)
 
 
 def fdd_create(n_q_heads, n_kv_heads, head_dim, vocab, n_layers=1, page_tokens=0, max_block=64,
@@ -158,8 +181,7 @@ def fdd_launch_count(ctx):
 def fdd_fork(ctx, prefix_k, prefix_v, page_table, prefix_len, prefix_capacity, n_forks, seeds,
              suffix_k, suffix_v, suffix_capacity):
     """prefix_k/v, suffix_k/v: per-layer lists of CUDA tensors; seeds: iterable of N ints."""
-    seeds = [int(s) & 0xFFFFFFFFFFFFFFFF for s in seeds]
-    seed_arr = (ctypes.c_uint64 * len(seeds))(*seeds)
+    seed_arr = seeds if isinstance(seeds, ctypes.Array) else u64_array(seeds)
     out = ctypes.c_void_p()
     st = lib().fdd_fork(ctx, _ptr_array(prefix_k), _ptr_array(prefix_v), _ptr(page_table),
                         int(prefix_len), int(prefix_capacity), int(n_forks), seed_arr,
