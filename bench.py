@@ -118,6 +118,8 @@ def run_ours(args):
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     fdd.lib()
     w = synth.workload(args.workload)
+    if args.n_forks:                           # rollout sweep: same shapes, another number of rollouts
+        w = synth.small_variant(w, n_forks=args.n_forks, name=w.name)
     w = replicas.replica_workload(w, rank)     # every rank decodes its own scene (different seed)
     # A workload is one scene or a batch of independent scenes (the serving mix): every call below
     # takes all of them at once, packed in scene order.
@@ -272,6 +274,7 @@ def run_ours(args):
     sampler.join(timeout=2)
     ms = ev0.elapsed_time(ev1)
     attn_all = [(a.elapsed_time(b), n) for a, b, n in attn_events]
+    rollout_steps = sum(n for _, n in attn_all) / L     # (rollout, step) pairs that decoded
     attn_ms = [ms_ for ms_, n in attn_all if n == N]          # launches in which every rollout decodes
     unmask_ms = [(a.elapsed_time(b), rows) for a, b, rows in unmask_events]
     ms = replicas.max_over_ranks(ms, dist, "cuda")
@@ -347,6 +350,8 @@ def run_ours(args):
                    "heads": f"{w.n_q_heads}q/{w.n_kv_heads}kv", "head_dim": w.head_dim, "vocab": w.vocab,
                    "layers": L, "threshold": w.threshold, "temperature": w.temperature,
                    "denoise_steps_per_block": denoise_steps / args.steps,
+                   # value tokens a rollout commits per denoising step it takes part in (the paper's Tok/Step)
+                   "tokens_per_step_per_rollout": (value_tokens * args.steps / rollout_steps) if rollout_steps else None,
                    "value_tokens_per_block": value_tokens, "tokens_incl_scaffold_per_block": all_tokens,
                    "l2": "per-step inputs (logits) larger than L2",
                    "step_pipeline": ("attention gated by n_left; step t+1 enqueued before the host reads step t"
@@ -359,7 +364,7 @@ def run_ours(args):
         "roofline": {"kernel": "fdd_block_attn (attn_ptc_kernel)", "bound": "tensor", "achieved": achieved,
                      "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s",
                      "frac": (achieved / peaks["bf16_tflops_sustained"]) if achieved else None,
-                     "traffic": ATTN_DRAM_BYTES_PER_LAUNCH.get(args.workload) if L == 1 else None,
+                     "traffic": ATTN_DRAM_BYTES_PER_LAUNCH.get(args.workload) if L == 1 and not args.n_forks else None,
                      "peak_source": peaks["source"] + " (sustained bf16: the kernel is timed inside the step loop)",
                      "frac_of_burst_peak": (achieved / peaks["bf16_tflops"]) if achieved else None,
                      "flops_per_launch": flops, "avg_launch_ms": attn_avg_ms, "launches_timed": len(attn_ms),
@@ -477,6 +482,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="long_prefix")
     ap.add_argument("--layers", type=int, default=1)
+    ap.add_argument("--n-forks", type=int, default=0, help="override the number of rollouts of every scene")
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--pre-steps", type=int, default=PRE_STEPS,
                     help="distinct per-step input sets kept resident on the device")
