@@ -67,7 +67,7 @@ template <int MAXSETS>
 struct TcArgs {
     TcSetMaps maps[MAXSETS];
     SetParams sets[MAXSETS];
-    float* part_o;             // [2 * ctas][256][D] normalised partial outputs
+    float* part_o;             // [2 * ctas][D / 4][256] float4: normalised partial outputs, column-major per slot
     float* part_lse;           // [2 * ctas][256] log2-domain log-sum-exp of the partial
     int* unit_count;           // pieces finished per unit (self-resetting)
     int* status;
@@ -174,6 +174,53 @@ constexpr float kPoly1 = 0.6932609677314758f * kPolyScale;
 constexpr float kPoly2 = 0.2426108568906784f * kPolyScale;
 constexpr float kPoly3 = 0.055171459913253784f * kPolyScale;
 constexpr float kRoundMagic = 12582912.0f;                    // 1.5 * 2^23: adding it rounds to an integer
+
+// Merge of a unit cut between CTAs, one output row:  out = sum_k w_k O_k,  w_k = 2^(lse_k - M) / sum.
+// Partials lie column-major in their slots ([D / 4][256 rows] float4).  CB columns x 32 / CB pieces
+// are read per round trip.
+template <int D, int CB>
+__device__ __forceinline__ void merge_row(const float* part_o, const float* part_lse, const int* slot_s, int n_pieces,
+                                          int row, float M, float inv_wsum, __nv_bfloat16* op) {
+    constexpr int NC4 = D / 4;
+    constexpr int CBE = CB < NC4 ? CB : NC4;        // columns per batch
+    constexpr int PC = 32 / CBE;                    // pieces per chunk
+    const float4* po4 = reinterpret_cast<const float4*>(part_o);
+    for (int c0 = 0; c0 < NC4; c0 += CBE) {
+        float4 acc[CBE];
+#pragma unroll
+        for (int c = 0; c < CBE; ++c) acc[c] = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int k0 = 0; k0 < n_pieces; k0 += PC) {
+            float ls[PC];
+            float4 ov[PC][CBE];
+#pragma unroll
+            for (int k = 0; k < PC; ++k) {
+                const bool live = k0 + k < n_pieces;
+                const size_t slot = slot_s[min(k0 + k, n_pieces - 1)];
+                ls[k] = live ? __ldcg(part_lse + slot * 256 + row) : -CUDART_INF_F;
+#pragma unroll
+                for (int c = 0; c < CBE; ++c)
+                    ov[k][c] = live ? __ldcg(po4 + (slot * NC4 + c0 + c) * 256 + row) : make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+#pragma unroll
+            for (int k = 0; k < PC; ++k) {
+                const float wgt = exp2f(ls[k] - M) * inv_wsum;      // 0 for a piece that is not there
+#pragma unroll
+                for (int c = 0; c < CBE; ++c) {
+                    acc[c].x = fmaf(wgt, ov[k][c].x, acc[c].x); acc[c].y = fmaf(wgt, ov[k][c].y, acc[c].y);
+                    acc[c].z = fmaf(wgt, ov[k][c].z, acc[c].z); acc[c].w = fmaf(wgt, ov[k][c].w, acc[c].w);
+                }
+            }
+        }
+#pragma unroll
+        for (int c = 0; c < CBE; c += 2) {
+            const __nv_bfloat162 b0 = __floats2bfloat162_rn(acc[c].x, acc[c].y), b1 = __floats2bfloat162_rn(acc[c].z, acc[c].w);
+            const __nv_bfloat162 b2 = __floats2bfloat162_rn(acc[c + 1].x, acc[c + 1].y), b3 = __floats2bfloat162_rn(acc[c + 1].z, acc[c + 1].w);
+            *reinterpret_cast<uint4*>(op + (c0 + c) * 4) =
+                make_uint4(*reinterpret_cast<const uint32_t*>(&b0), *reinterpret_cast<const uint32_t*>(&b1),
+                           *reinterpret_cast<const uint32_t*>(&b2), *reinterpret_cast<const uint32_t*>(&b3));
+        }
+    }
+}
 
 template <int D, int MAXSETS, int EMU>
 __global__ void __launch_bounds__(kTcThreads, 1)
@@ -493,7 +540,7 @@ attn_ptc_kernel(const __grid_constant__ TcArgs<MAXSETS> a) {
             const ItemView v = view_item(pos);
             const Item& it = v.it;
             const SetParams& p = a.sets[it.s];
-            const int f = v.f, rp = v.rp, h = v.h, nt = v.nt, rows_here = v.rows_here;
+            const int f = v.f, rp = v.rp, h = v.h, nt = v.nt;
             const bool active = q < v.NQ;
             const int r = rp * 256 + q * 128 + row_local;       // row inside the unit
             const bool row_ok = r < p.R;
@@ -663,7 +710,9 @@ attn_ptc_kernel(const __grid_constant__ TcArgs<MAXSETS> a) {
                 // (necessarily the CTA's last item) slot 1.
                 const int own_slot = blockIdx.x * 2 + (pos == range_begin ? 0 : 1);
                 if (active && ok) {
-                    float* po = a.part_o + (static_cast<size_t>(own_slot) * 256 + q * 128 + row_local) * D;
+                    // column-major inside the slot ([D / 4 float4 columns][256 rows]): the 32 rows of a
+                    // warp make one contiguous 512-byte store, and the merge reads them back the same way
+                    float4* po = reinterpret_cast<float4*>(a.part_o) + static_cast<size_t>(own_slot) * (D / 4) * 256 + q * 128 + row_local;
 #pragma unroll
                     for (int cc = 0; cc < D / 32; ++cc) {
                         uint32_t o[32];
@@ -671,7 +720,7 @@ attn_ptc_kernel(const __grid_constant__ TcArgs<MAXSETS> a) {
                         tc::wait_ld();
 #pragma unroll
                         for (int v4 = 0; v4 < 8; ++v4)
-                            __stcg(reinterpret_cast<float4*>(po + cc * 32 + v4 * 4),
+                            __stcg(po + (cc * 8 + v4) * 256,
                                    make_float4(__uint_as_float(o[v4 * 4]) * inv, __uint_as_float(o[v4 * 4 + 1]) * inv,
                                                __uint_as_float(o[v4 * 4 + 2]) * inv, __uint_as_float(o[v4 * 4 + 3]) * inv));
                     }
@@ -691,76 +740,40 @@ attn_ptc_kernel(const __grid_constant__ TcArgs<MAXSETS> a) {
                     // This CTA finished the unit's last outstanding piece: merge all of them.
                     //   out = sum_s w_s O_s / sum_s w_s,  w_s = 2^(lse_s - max lse)
                     __threadfence();
-                    // A warp takes four rows at a time (lane = four columns) and up to eight pieces at
-                    // once: 32 independent 512-byte row reads (plus their log-sum-exps) are in flight
-                    // before the first one is used; more than eight pieces are folded in chunk by chunk
-                    // with a running maximum.
-                    constexpr int kLanes = D / 4;       // lanes that carry a float4 of the row
-                    constexpr int kRowsB = 4, kPC = 8;
+                    // Thread = row, as in the writer (tid = q * 128 + row_local is the row inside the unit).
+                    // First the row's weights: M = max lse, 1 / sum 2^(lse - M), the log-sum-exps read eight
+                    // at a time.  Then the columns, in batches sized so that 32 independent 16-byte reads
+                    // are in flight per thread whatever the number of pieces.
                     if (tid < n_pieces && tid < kMaxPieces) {
                         const int pc = c_first + tid;
                         slot_s[tid] = pc * 2 + (it.unit_begin <= T * pc / C ? 0 : 1);
                     }
                     tc::named_barrier(1, 256);
-                    for (int row0 = warp * kRowsB; row0 < rows_here; row0 += 8 * kRowsB) {
-                        float M[kRowsB], wsum[kRowsB];
-                        float4 accv[kRowsB];
+                    if (row_ok) {
+                        float M = -CUDART_INF_F, wsum = 0.0f;
+                        for (int k0 = 0; k0 < n_pieces; k0 += 8) {
+                            float ls[8];
 #pragma unroll
-                        for (int j = 0; j < kRowsB; ++j) {
-                            M[j] = -CUDART_INF_F; wsum[j] = 0.0f;
-                            accv[j] = make_float4(0.f, 0.f, 0.f, 0.f);
-                        }
-                        for (int k0 = 0; k0 < n_pieces; k0 += kPC) {
-                            float ls[kPC][kRowsB];
-                            float4 ov[kPC][kRowsB];
+                            for (int k = 0; k < 8; ++k)
+                                ls[k] = k0 + k < n_pieces ? __ldcg(a.part_lse + static_cast<size_t>(slot_s[min(k0 + k, n_pieces - 1)]) * 256 + tid)
+                                                          : -CUDART_INF_F;
+                            float mc = ls[0];
 #pragma unroll
-                            for (int k = 0; k < kPC; ++k) {
-                                const bool live_p = k0 + k < n_pieces;
-                                const int slot = slot_s[min(k0 + k, n_pieces - 1)];
-                                const float* lse = a.part_lse + static_cast<size_t>(slot) * 256 + row0;
-                                const float* po = a.part_o + (static_cast<size_t>(slot) * 256 + row0) * D + lane * 4;
+                            for (int k = 1; k < 8; ++k) mc = fmaxf(mc, ls[k]);
+                            const float mn = fmaxf(M, mc);
+                            if (mn > -CUDART_INF_F) {
+                                wsum *= exp2f(M - mn);                  // 0 the first time (M = -inf)
 #pragma unroll
-                                for (int j = 0; j < kRowsB; ++j) {
-                                    const bool live = live_p && row0 + j < rows_here;
-                                    ls[k][j] = live ? __ldcg(lse + j) : -CUDART_INF_F;
-                                    ov[k][j] = (live && lane < kLanes) ? __ldcg(reinterpret_cast<const float4*>(po + static_cast<size_t>(j) * D))
-                                                                       : make_float4(0.f, 0.f, 0.f, 0.f);
-                                }
-                            }
-#pragma unroll
-                            for (int j = 0; j < kRowsB; ++j) {
-                                float mc = ls[0][j];
-#pragma unroll
-                                for (int k = 1; k < kPC; ++k) mc = fmaxf(mc, ls[k][j]);
-                                const float mn = fmaxf(M[j], mc);
-                                if (mn == -CUDART_INF_F) continue;              // nothing live in this row yet
-                                const float keep = exp2f(M[j] - mn);           // 0 on the first chunk (M = -inf)
-                                wsum[j] *= keep;
-                                accv[j].x *= keep; accv[j].y *= keep; accv[j].z *= keep; accv[j].w *= keep;
-                                M[j] = mn;
-#pragma unroll
-                                for (int k = 0; k < kPC; ++k) {
-                                    const float wgt = exp2f(ls[k][j] - mn);    // 0 for a piece that is not there
-                                    wsum[j] += wgt;
-                                    accv[j].x = fmaf(wgt, ov[k][j].x, accv[j].x); accv[j].y = fmaf(wgt, ov[k][j].y, accv[j].y);
-                                    accv[j].z = fmaf(wgt, ov[k][j].z, accv[j].z); accv[j].w = fmaf(wgt, ov[k][j].w, accv[j].w);
-                                }
+                                for (int k = 0; k < 8; ++k) wsum += exp2f(ls[k] - mn);
+                                M = mn;
                             }
                         }
-                        if (lane < kLanes) {
-#pragma unroll
-                            for (int j = 0; j < kRowsB; ++j) {
-                                if (row0 + j >= rows_here) continue;
-                                const int rr = rp * 256 + row0 + j;
-                                const float iw = 1.0f / wsum[j];
-                                const int i2 = rr / p.G, g2 = rr - i2 * p.G;
-                                __nv_bfloat16* op = p.out + ((static_cast<size_t>(f) * p.d + i2) * p.n_q_heads + h * p.G + g2) * D + lane * 4;
-                                const __nv_bfloat162 lo = __floats2bfloat162_rn(accv[j].x * iw, accv[j].y * iw);
-                                const __nv_bfloat162 hi = __floats2bfloat162_rn(accv[j].z * iw, accv[j].w * iw);
-                                *reinterpret_cast<uint2*>(op) = make_uint2(*reinterpret_cast<const uint32_t*>(&lo),
-                                                                           *reinterpret_cast<const uint32_t*>(&hi));
-                            }
-                        }
+                        if (!(M > -CUDART_INF_F)) M = 0.0f;
+                        const float iw = wsum > 0.0f ? 1.0f / wsum : 0.0f;
+                        __nv_bfloat16* op = p.out + ((static_cast<size_t>(f) * p.d + qi) * p.n_q_heads + h * p.G + qg) * D;
+                        if (n_pieces <= 2) merge_row<D, 16>(a.part_o, a.part_lse, slot_s, n_pieces, tid, M, iw, op);
+                        else if (n_pieces <= 4) merge_row<D, 8>(a.part_o, a.part_lse, slot_s, n_pieces, tid, M, iw, op);
+                        else merge_row<D, 4>(a.part_o, a.part_lse, slot_s, n_pieces, tid, M, iw, op);
                     }
                 }
             }
@@ -956,7 +969,8 @@ bool attention_tc_supported(const AttnProblem& a, int head_dim) {
     return tmap::encode_fn() != nullptr;
 }
 
-// Scratch of the split-unit merge: two partial slots (256 rows of D values + log-sum-exp) per CTA.
+// Scratch of the split-unit merge: two partial slots per CTA, each D / 4 float4 columns of 256 rows
+// plus the rows' log-sum-exps.
 size_t attention_ptc_workspace_bytes(int head_dim, int max_ctas) {
     return static_cast<size_t>(2) * max_ctas * 256 * (head_dim + 1) * sizeof(float);
 }
