@@ -8,8 +8,10 @@ generator.  The reading used by this repository: Philox4x32 with 10 rounds
 SC'11), keyed by the rollout's 64-bit seed, with the counter made of the
 vocabulary index, the position inside the block, the denoising step and the
 block index, so that a draw depends on nothing but (seed, block, step,
-position, vocabulary id).  Each uniform is assembled from two streams: an 8-bit
-coarse value (16 ids per Philox block) and 23 fine bits (4 ids per block).
+position, vocabulary id).  The draws are built as an "exponential race" over
+groups of 16 consecutive ids (see `exponential_row`): one 32-bit word per group
+fixes the group's smallest exponential variate and which id holds it, a second
+stream gives every id 23 bits of its own.
 
 Two implementations live here on purpose: a scalar one on Python integers that
 follows the published round function literally, and a numpy one used for whole
@@ -71,33 +73,25 @@ def philox4x32_vec(c0, c1, c2, c3, k0, k1, rounds=10):
 
 
 FINE_STREAM = 1 << 31   # added to the position word of the counter for the second stream
+GROUP = 16              # vocabulary ids per group
 
 
-def uniform_from_parts(coarse, fine):
-    """Map an 8-bit coarse value and a 23-bit fine value to the open interval (0, 1).
+def group_words(seed, block_idx, step, position, vocab):
+    """The 32-bit word R_j of every group j (ids 16 j .. 16 j + 15) of one row.
 
-    u = (coarse + (fine + 0.5) * 2**-23) / 256: the coarse byte picks one of 256
-    equal bins, the fine bits a point inside it, centred in its sub-bin.  u is a
-    multiple of 2**-32 in [2**-32, 1 - 2**-32], so -ln(-ln(u)) is always finite
-    (between -3.1 and 22.2).
+    Group j takes word (j // 256) % 4 of the Philox block with counter
+    ((j // 1024) * 256 + j % 256, position, step, block_idx): the four words of a block
+    belong to four groups that lie 256 groups (4096 ids) apart, so that one block
+    serves 64 ids of any run of 16 consecutive ids per 4096.
     """
-    coarse = np.asarray(coarse, dtype=np.float64)
-    fine = np.asarray(fine, dtype=np.float64)
-    return (coarse + (fine + 0.5) * (2.0 ** -23)) / 256.0
-
-
-def coarse_bytes(seed, block_idx, step, position, vocab):
-    """The coarse byte of every vocabulary id of one row: id v takes byte v % 16
-    (little-endian inside the four output words) of the Philox block with
-    counter (v // 16, position, step, block_idx)."""
     seed = int(seed) & 0xFFFFFFFFFFFFFFFF
-    nctr = (vocab + 15) // 16
-    ctr = np.arange(nctr, dtype=np.uint64)
+    ngroups = (vocab + GROUP - 1) // GROUP
+    j = np.arange(ngroups, dtype=np.uint64)
+    ctr = (j >> np.uint64(10)) * np.uint64(256) + (j & np.uint64(255))
     w = philox4x32_vec(ctr, np.uint64(position), np.uint64(step), np.uint64(block_idx),
                        seed & MASK32, seed >> 32)
-    words = np.stack(w, axis=1).reshape(-1)                       # word k of block c at 4 c + k
-    shifts = np.array([0, 8, 16, 24], dtype=np.uint64)
-    return ((words[:, None] >> shifts[None, :]) & np.uint64(0xFF)).reshape(-1)[:vocab]
+    words = np.stack(w, axis=1)                                    # [group, 4]
+    return words[np.arange(ngroups), ((j >> np.uint64(8)) & np.uint64(3)).astype(np.int64)]
 
 
 def fine_bits(seed, block_idx, step, position, vocab):
@@ -114,15 +108,51 @@ def fine_bits(seed, block_idx, step, position, vocab):
     return words >> np.uint64(9)
 
 
-def gumbel_row(seed, block_idx, step, position, vocab):
-    """Standard Gumbel noise g[v] = -ln(-ln(u[v])) for one row of a block, with
-    u[v] = uniform_from_parts(coarse byte of v, fine bits of v).  A draw depends
-    on nothing but (seed, block, step, position, vocabulary id).
+def leader_exponential(word, fine):
+    """The smallest exponential variate of a group, from the group's word and the
+    fine bits of the id that holds it.
 
-    The uniform is split in two so that an implementation can bound a draw from
-    its coarse byte alone (one Philox block per 16 ids) and spend the second
-    Philox block only on the few ids whose bound can still win the arg-max.
+    U = (h + (f + 0.5) 2**-23) / 2**28 with h = word >> 4 is uniform on (0, 1) in
+    steps of 2**-51; the minimum of 16 independent Exp(1) variates is Exp(1) / 16,
+    so E = -ln(U) / 16.  Written through 1 - U, which fp64 holds exactly, so that
+    the tail U -> 1 (the large Gumbel draws) loses nothing.
     """
-    u = uniform_from_parts(coarse_bytes(seed, block_idx, step, position, vocab),
-                           fine_bits(seed, block_idx, step, position, vocab))
-    return -np.log(-np.log(u))
+    h = (np.asarray(word, dtype=np.uint64) >> np.uint64(4)).astype(np.float64)
+    f = np.asarray(fine, dtype=np.float64)
+    one_minus_u = ((2.0 ** 28 - h) - (f + 0.5) * (2.0 ** -23)) * (2.0 ** -28)
+    return -np.log1p(-one_minus_u) / GROUP
+
+
+def exponential_row(seed, block_idx, step, position, vocab):
+    """E[v], independent Exp(1) variates for the ids of one row, as an exponential race
+    per group of 16 ids:
+
+      * the group's word R picks the id that holds the group's minimum, the
+        "leader" 16 j + R % 16, and with the leader's fine bits the minimum itself
+        (`leader_exponential`);
+      * every other id of the group gets the minimum plus a fresh Exp(1) variate
+        -ln((f + 0.5) 2**-23) from its own fine bits.
+
+    By the memorylessness of the exponential distribution this is exactly a family
+    of independent Exp(1) variates: the minimum of 16 of them is Exp(1) / 16, it sits
+    at a uniformly random place, and the others exceed it by independent Exp(1)
+    amounts.  What it buys an implementation: the word of a group alone bounds all
+    16 draws of the group from below, so the per-id stream is needed only for the few
+    ids that can still win an arg-max.
+    """
+    ngroups = (vocab + GROUP - 1) // GROUP
+    padded = ngroups * GROUP                        # the leader of the last group may lie beyond vocab
+    words = group_words(seed, block_idx, step, position, vocab)
+    fine = fine_bits(seed, block_idx, step, position, padded).astype(np.float64)
+    leader = np.arange(ngroups) * GROUP + (words & np.uint64(15)).astype(np.int64)
+    e_min = leader_exponential(words, fine[leader])
+    e = np.repeat(e_min, GROUP) - np.log((fine + 0.5) * (2.0 ** -23))
+    e[leader] = e_min
+    return e[:vocab]
+
+
+def gumbel_row(seed, block_idx, step, position, vocab):
+    """Standard Gumbel noise g[v] = -ln(E[v]) for one row of a block (E from
+    `exponential_row`: -ln of an Exp(1) variate is a standard Gumbel variate).  A draw
+    depends on nothing but (seed, block, step, position, vocabulary id)."""
+    return -np.log(exponential_row(seed, block_idx, step, position, vocab))

@@ -7,8 +7,8 @@ import numpy as np
 import pytest
 
 from oracle import MASKED, COMMITTED, SCAFFOLD
-from oracle.philox import (coarse_bytes, fine_bits, gumbel_row, philox4x32_scalar, philox4x32_vec,
-                           uniform_from_parts)
+from oracle.philox import (exponential_row, fine_bits, group_words, gumbel_row, leader_exponential,
+                           philox4x32_scalar, philox4x32_vec)
 from oracle.unmask import unmask_step
 
 GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
@@ -45,54 +45,84 @@ def test_philox_vectorised_equals_scalar():
         assert [int(o[0]) for o in out] == expect
 
 
-def test_uniform_map_is_open_interval_and_monotone():
-    c = np.array([0, 0, 0, 1, 127, 128, 255, 255])
-    f = np.array([0, 1, 2 ** 23 - 1, 0, 2 ** 23 - 1, 0, 0, 2 ** 23 - 1])
-    u = uniform_from_parts(c, f)
-    assert u[0] == 2.0 ** -32 and u[-1] == 1.0 - 2.0 ** -32
-    assert np.all(np.diff(u) > 0)                      # ordered by (coarse, fine)
-    assert u[3] - u[2] == 2.0 ** -31                   # bins tile (0, 1) without gap or overlap
-    assert np.all(u * 2.0 ** 32 == np.round(u * 2.0 ** 32))
-    g = -np.log(-np.log(u))
-    assert np.all(np.isfinite(g)) and -3.1 < g[0] and g[-1] < 22.2
+def test_leader_map_is_open_interval_and_monotone():
+    # U = (h + (f + 0.5) 2^-23) / 2^28 tiles (0, 1) in steps of 2^-51; E = -ln(U) / 16 falls as U grows
+    top = 2 ** 28 - 1
+    words = np.array([0, 0, 0, 1, top // 2, top, top], dtype=np.uint64) << np.uint64(4)
+    f = np.array([0, 1, 2 ** 23 - 1, 0, 5, 0, 2 ** 23 - 1])
+    e = leader_exponential(words, f)
+    assert np.all(np.diff(e) < 0) and np.all(e > 0) and np.all(np.isfinite(e))
+    assert e[0] == -math.log(2.0 ** -52) / 16                      # smallest U = 2^-52
+    assert abs(e[-1] - 2.0 ** -52 / 16) < 1e-30                    # largest U = 1 - 2^-52: E = 2^-52 / 16 + O(2^-104)
+    # the low four bits of the word (the leader's place) do not enter
+    assert np.array_equal(leader_exponential(words + np.uint64(9), f), e)
+    g = -np.log(e)
+    assert -1.0 < g[0] and g[-1] < 38.9
 
 
 def test_gumbel_row_layout_and_independence_from_vocab_size():
     seed = 0xDEADBEEFCAFEF00D
-    a = gumbel_row(seed, 3, 2, 5, 37)
-    b = gumbel_row(seed, 3, 2, 5, 64)
-    np.testing.assert_array_equal(a, b[:37])
+    V = 16 * 1024 + 40                                  # reaches the second run of 1024 groups
+    a = gumbel_row(seed, 3, 2, 5, V)
+    b = gumbel_row(seed, 3, 2, 5, V + 23)
+    np.testing.assert_array_equal(a, b[:V])
+    np.testing.assert_array_equal(gumbel_row(seed, 3, 2, 5, 37), a[:37])    # a cut group included
     key = (seed & 0xFFFFFFFF, seed >> 32)
-    # coarse: byte v % 16 of counter (v // 16, pos, step, block); fine: top 23 bits of word v % 4 of
-    # counter (v // 4, pos + 2^31, step, block); both under key (lo, hi)
-    for v in (0, 5, 18, 36):
-        cw = philox4x32_scalar((v // 16, 5, 2, 3), key)[(v % 16) // 4]
-        c = (cw >> (8 * (v % 4))) & 0xFF
-        f = philox4x32_scalar((v // 4, 5 + 2 ** 31, 2, 3), key)[v % 4] >> 9
-        u = (c + (f + 0.5) * 2.0 ** -23) / 256.0
-        assert a[v] == -math.log(-math.log(u))
-        assert coarse_bytes(seed, 3, 2, 5, 37)[v] == c and fine_bits(seed, 3, 2, 5, 37)[v] == f
+    words = group_words(seed, 3, 2, 5, V)
+    fb = fine_bits(seed, 3, 2, 5, V + 16)
+    # group j: word (j // 256) % 4 of counter ((j // 1024) * 256 + j % 256, pos, step, block); fine: top 23
+    # bits of word v % 4 of counter (v // 4, pos + 2^31, step, block); both under key (lo, hi)
+    seen_leader = seen_other = 0
+    for v in (0, 5, 18, 255 * 16 + 3, 256 * 16 + 1, 700 * 16 + 15, 1023 * 16, 1024 * 16 + 7, V - 1) + tuple(range(32, 64)):
+        j = v // 16
+        R = philox4x32_scalar(((j // 1024) * 256 + j % 256, 5, 2, 3), key)[(j // 256) % 4]
+        assert int(words[j]) == R
+        lead = 16 * j + R % 16
+        f_lead = philox4x32_scalar((lead // 4, 5 + 2 ** 31, 2, 3), key)[lead % 4] >> 9
+        assert int(fb[lead]) == f_lead
+        U = ((R >> 4) + (f_lead + 0.5) * 2.0 ** -23) * 2.0 ** -28
+        e = -math.log(U) / 16
+        if v != lead:
+            f_v = philox4x32_scalar((v // 4, 5 + 2 ** 31, 2, 3), key)[v % 4] >> 9
+            e += -math.log((f_v + 0.5) * 2.0 ** -23)
+            seen_other += 1
+        else:
+            seen_leader += 1
+        assert abs(a[v] + math.log(e)) <= 1e-12 * max(1.0, abs(a[v]))
+    assert seen_leader >= 2 and seen_other >= 20
     # every counter field and the seed matter
     for other in (gumbel_row(seed + 1, 3, 2, 5, 37), gumbel_row(seed, 4, 2, 5, 37),
                   gumbel_row(seed, 3, 1, 5, 37), gumbel_row(seed, 3, 2, 6, 37),
                   gumbel_row(seed ^ (1 << 40), 3, 2, 5, 37)):
-        assert not np.array_equal(a, other)
+        assert not np.array_equal(a[:37], other)
 
 
-def test_coarse_byte_bounds_the_draw():
-    # what lets an implementation skip the second stream: g < -ln(-ln((c + 1) / 256)) for c < 255
-    g = gumbel_row(777, 1, 4, 9, 50000)
-    c = coarse_bytes(777, 1, 4, 9, 50000).astype(np.float64)
-    low = c < 255
-    with np.errstate(divide="ignore"):
-        upper = -np.log(-np.log((c + 1.0) / 256.0))
-        lower = -np.log(-np.log(c / 256.0))
-    assert np.all(g[low] < upper[low]) and np.all(g[c > 0] > lower[c > 0])
-    # the two streams are not the same numbers: coarse bytes are uncorrelated with the fine bits
-    f = fine_bits(777, 1, 4, 9, 50000).astype(np.float64)
-    assert abs(np.corrcoef(c, f)[0, 1]) < 0.02
-    counts = np.bincount(c.astype(int), minlength=256)
-    assert counts.min() > 120 and counts.max() < 280    # 50000 / 256 = 195 expected per bin
+def test_group_word_bounds_every_draw_of_the_group():
+    # what lets an implementation skip the per-id stream: the word of a group alone bounds the 16
+    # draws of the group, E[v] >= -ln((h + 1) / 2^28) / 16 with h = word >> 4, and a word below
+    # 0xFF000000 (255 of 256 groups) caps them at g < 8.3158
+    V = 50000
+    e = exponential_row(777, 1, 4, 9, V)
+    words = group_words(777, 1, 4, 9, V)
+    h = (words >> np.uint64(4)).astype(np.float64)
+    floor = np.repeat(-np.log((h + 1.0) * 2.0 ** -28) / 16, 16)[:V]
+    ceil_leader = np.repeat(-np.log(np.maximum(h, 0.5) * 2.0 ** -28) / 16, 16)[:V]
+    assert np.all(e >= floor)
+    grp_min = np.minimum.reduceat(e, np.arange(0, V, 16))
+    lead = np.arange(len(words)) * 16 + (words & np.uint64(15)).astype(np.int64)
+    inside = lead < V
+    np.testing.assert_array_equal(grp_min[inside], e[lead[inside]])           # the leader holds the minimum
+    assert np.all(e[lead[inside]] <= ceil_leader[lead[inside]])
+    plain = np.repeat(words < np.uint64(0xFF000000), 16)[:V]
+    g = -np.log(e)
+    assert np.all(g[plain] < 8.3158)
+    assert 0.5 / 256 < 1.0 - plain.mean() < 2.0 / 256
+    # the leader's place is uniform over the 16 ids and unrelated to the minimum
+    places = (words & np.uint64(15)).astype(int)
+    counts = np.bincount(places, minlength=16)
+    chi2 = float(((counts - len(places) / 16) ** 2 / (len(places) / 16)).sum())
+    assert chi2 < 37.7                                   # chi-square(15) 0.1 % critical value
+    assert abs(np.corrcoef(places, h)[0, 1]) < 0.05
 
 
 def test_gumbel_uniformity_ks():
@@ -102,6 +132,26 @@ def test_gumbel_uniformity_ks():
     n = len(u)
     dist = np.max(np.abs(u - (np.arange(n) + 0.5) / n))
     assert dist < 1.63 / math.sqrt(n)          # 1 % critical value
+
+
+def test_draws_inside_a_group_are_independent_exponentials():
+    # the race construction must not show: group minima are Exp(1) / 16, neighbours inside a group are
+    # uncorrelated, and so are a group's minimum and the excess of its other ids
+    V = 320000
+    e = exponential_row(4242, 2, 1, 3, V).reshape(-1, 16)
+    m = np.sort(e.min(axis=1) * 16)
+    n = len(m)
+    cdf = 1.0 - np.exp(-m)
+    assert np.max(np.abs(cdf - (np.arange(n) + 0.5) / n)) < 1.63 / math.sqrt(n)
+    u = np.exp(-e)
+    for a_, b_ in ((0, 1), (3, 12), (7, 8), (14, 15)):
+        assert abs(np.corrcoef(u[:, a_], u[:, b_])[0, 1]) < 0.02
+    second = np.sort(e, axis=1)[:, 1] - e.min(axis=1)              # gap to the runner-up: Exp(1) / 15
+    s2 = np.sort(second * 15)
+    assert np.max(np.abs(1.0 - np.exp(-s2) - (np.arange(n) + 0.5) / n)) < 1.63 / math.sqrt(n)
+    assert abs(np.corrcoef(e.min(axis=1), second)[0, 1]) < 0.02
+    # every id alone is Exp(1), leader or not: mean 1, variance 1 per column
+    assert np.all(np.abs(e.mean(axis=0) - 1.0) < 0.03) and np.all(np.abs(e.var(axis=0) - 1.0) < 0.08)
 
 
 def _mk(N, d, V, seed, scaffold=()):
