@@ -172,11 +172,16 @@ fdd_status fdd_block_attn_gated(fdd_ctx* ctx, fdd_forkset* const* sets, int n_se
  * For every rollout f and every position i with state MASKED:
  *   tok  = argmax_v (logit[v] + temperature * g[v])            lowest v on ties
  *   conf = softmax(logit)[tok]                                  noise-free probability
- * where g[v] = -ln(-ln(u)), u = (c + (f + 0.5) * 2^-23) / 256 is assembled from two
- * Philox4x32-10 streams under key = the rollout's seed (low, high word):
- *   c = byte v % 16 (little-endian in the four output words) of counter (v / 16, i, step, block_idx)
- *   f = top 23 bits of output word v % 4 of counter (v / 4, i + 2^31, step, block_idx)
- * (the coarse byte bounds a draw, which lets the kernel skip the second stream for almost
+ * where g[v] = -ln(E[v]) and the E[v] are independent Exp(1) variates built as a race over
+ * groups of 16 consecutive ids from two Philox4x32-10 streams under key = the rollout's seed
+ * (low, high word).  Group j = v / 16 has the word
+ *   R = output word (j / 256) % 4 of counter ((j / 1024) * 256 + j % 256, i, step, block_idx),
+ * every id the fine bits
+ *   f[v] = top 23 bits of output word v % 4 of counter (v / 4, i + 2^31, step, block_idx).
+ * The id 16 j + R % 16 (the group's leader) holds the group's minimum,
+ *   E = -ln(U) / 16,  U = ((R >> 4) + (f + 0.5) * 2^-23) / 2^28,
+ * every other id of the group E[v] = E_leader - ln((f[v] + 0.5) * 2^-23)
+ * (the word of a group bounds its 16 draws, which lets the kernel skip the second stream for almost
  * every v); temperature == 0 uses no noise.  Positions with
  * conf > threshold are committed (token written, state -> COMMITTED); if a rollout has
  * MASKED positions and none passes, its single most confident one (lowest i on ties)

@@ -7,15 +7,19 @@
 // per thread and load) and keeps running soft-max statistics; nothing but the few logits that can
 // win the arg-max is looked at twice.  Rows that are not MASKED are never read.
 //
-// Noise (temperature > 0).  The uniform behind every Gumbel draw has two parts: a coarse byte c
-// (one Philox block serves 16 vocabulary ids) and 23 fine bits (one block per 4 ids).  The byte
-// alone bounds the draw, g < -ln(-ln((c + 1) / 256)) for c < 255, which is what makes the
-// kernel cheap: every id gets its coarse byte, but the second Philox block and the two
+// Noise (temperature > 0).  The Gumbel draws are g = -ln(E) with E an exponential race over groups
+// of 16 consecutive ids: one 32-bit word R per group (a Philox block serves the four groups that a
+// thread meets in four consecutive iterations) fixes the "leader" 16 j + R % 16, which holds the
+// group's smallest E = -ln(U) / 16, U = ((R >> 4) + (f + 0.5) 2^-23) / 2^28; every other id of the
+// group has E = E_leader - ln((f + 0.5) 2^-23) with 23 fine bits f of its own (second Philox
+// stream, one block per 4 ids).  The word alone bounds all 16 draws, which is what makes the
+// kernel cheap: the streaming pass tests one word per 16 logits, and the second stream and the
 // logarithms are spent only on
-//   (1) the ids with c = 255 (one in 256), whose best exact score L is a lower bound of the
+//   (1) the leaders of the groups whose word lies in the top 2^-b of its range (b = 2..6, so that
+//       a segment has 128 to 256 such groups), whose best exact score L is a lower bound of the
 //       segment's best score, and
-//   (2) the ids of threads whose largest logit could still beat L with the largest draw a
-//       byte below 255 allows (g < 5.5433), filtered once more by their own byte's bound.
+//   (2) the ids of threads whose largest logit could still beat L with the largest draw any other
+//       group allows (g < 6.9237 for b = 6), filtered once more by their own group's bound.
 // Any id left out cannot reach L, so the arg-max (lowest id on ties) is exact.
 //
 // Kernel 2 (unmask_finalize_kernel): one CTA per rollout merges the segment records of its
@@ -28,10 +32,16 @@ namespace {
 
 constexpr int kThreads = 256;
 constexpr int kGroup = 16;                            // consecutive entries per load and per coarse Philox block
-constexpr int kSegQuantum = kThreads * kGroup;        // segment lengths are multiples of this (4096)
-constexpr int kMaxCand = 1536;                        // c = 255 ids kept per segment (594 expected for a 152k row)
+constexpr int kSegQuantum = kThreads * kGroup;        // ids a CTA covers per iteration (4096); segment lengths are multiples of it
+constexpr int kMaxCand = 512;                         // groups with a top word kept per segment (148 expected for a 152k row)
 constexpr int kMaxRows = kUnmaskMaxRows;              // rows whose state fits the CTA's compaction buffer
-constexpr float kGumbelBelow255 = 5.5440f;            // > -ln(-ln(255/256)) = 5.54322, with rounding slack
+// "Top" words: the upper 2^-b of the word range, b chosen per launch so that a segment has 128 to
+// 256 top-word groups (b = 6 for whole rows of 152k ids, b = 2 for 8192-id segments).  Every draw
+// of the other groups lies below kGumbelPlain[b] > -ln(-ln(1 - 2^-b) / 16).
+constexpr int kTopBitsMin = 2, kTopBitsMax = 6;
+__device__ __forceinline__ float gumbel_plain(int b) {
+    return b == 2 ? 4.0195f : (b == 3 ? 4.7870f : (b == 4 ? 5.5140f : (b == 5 ? 6.2235f : 6.9245f)));
+}
 constexpr float kLog2e = 1.4426950408889634f;
 
 constexpr uint32_t kPhiloxM0 = 0xD2511F53u, kPhiloxM1 = 0xCD9E8D57u;
@@ -53,24 +63,34 @@ __device__ __forceinline__ uint4 philox4x32_10(uint4 c, uint2 k) {
     return c;
 }
 
-// g = -ln(-ln(u)), u = (c + (f + 0.5) 2^-23) / 256.  Near u = 1 the inner logarithm goes through
-// 1 - u, which fp32 holds almost exactly there.
-__device__ __forceinline__ float gumbel_exact(uint32_t c, uint32_t f23) {
-    float inner;                                        // -ln(u) > 0
-    if (c >= 128u) {
-        const float y = (static_cast<float>(255u - c) + (8388608.0f - static_cast<float>(f23) - 0.5f) * 1.1920928955078125e-07f)
-                        * 0.00390625f;                  // 1 - u
-        inner = -log1pf(-y);
-    } else {
-        const float a = static_cast<float>(c) + (static_cast<float>(f23) + 0.5f) * 1.1920928955078125e-07f;   // 256 u
-        inner = 5.545177444479562f - logf(a);
-    }
-    return -logf(inner);
+// Philox block and word of group j (16 ids): the four words of a block go to groups 256 apart.
+__device__ __forceinline__ uint32_t group_counter(int j) { return static_cast<uint32_t>((j >> 10) * 256 + (j & 255)); }
+__device__ __forceinline__ uint32_t pick_word(const uint4& r, int k) {
+    return k == 0 ? r.x : (k == 1 ? r.y : (k == 2 ? r.z : r.w));
 }
 
-// Upper bound of the draws with coarse byte c < 255 (c = 255 has no useful bound).
-__device__ __forceinline__ float gumbel_bound(uint32_t c) {
-    return -logf(-logf(static_cast<float>(c + 1u) * 0.00390625f)) + 1e-3f;
+// E of a group's leader: -ln(U) / 16, U = (h + (f + 0.5) 2^-23) / 2^28, h = R >> 4.  In the upper
+// half the logarithm goes through 1 - U, which fp32 holds almost exactly there.
+__device__ __forceinline__ float leader_exponential(uint32_t R, uint32_t f23) {
+    const uint32_t h = R >> 4;
+    const float frac = (static_cast<float>(f23) + 0.5f) * 1.1920928955078125e-07f;
+    float nl;                                               // -ln(U)
+    if (h >= (1u << 27)) {
+        const float y = (static_cast<float>((1u << 28) - h) - frac) * 3.7252902984619140625e-09f;   // 1 - U
+        nl = -log1pf(-y);
+    } else {
+        nl = 19.408121055678468f - logf(static_cast<float>(h) + frac);                              // 28 ln 2 - ln(2^28 U)
+    }
+    return nl * 0.0625f;
+}
+// Lower bound of the leader's E (so of every E of the group) from the word alone.
+__device__ __forceinline__ float group_floor(uint32_t R) {
+    const float hp = static_cast<float>((R >> 4) + 1u);     // rounds to nearest: the slack below covers it
+    return fmaxf(19.408121055678468f - logf(hp), 0.0f) * 0.0625f * 0.999f;
+}
+// E of an id that is not its group's leader: the leader's plus -ln((f + 0.5) 2^-23).
+__device__ __forceinline__ float follower_exponential(float e_leader, uint32_t f23) {
+    return e_leader + (15.942385152878742f - logf(static_cast<float>(f23) + 0.5f));                 // 23 ln 2 - ln(f + 0.5)
 }
 
 __device__ __forceinline__ float ex2_fast(float x) {
@@ -184,7 +204,9 @@ unmask_partial_kernel(const T* __restrict__ logits, const uint8_t* __restrict__ 
     __shared__ uint16_t s_rows[kMaxRows];               // the selected rows (MASKED, or DRAFT for the verifier), ascending
     __shared__ int s_n_rows;
     __shared__ int s_warp_count[kThreads / 32];
-    __shared__ int s_cand[kMaxCand];                    // vocabulary ids with coarse byte 255
+    __shared__ int s_cand[kMaxCand];                    // groups with a top word: first id of the group ...
+    __shared__ uint32_t s_cand_word[kMaxCand];          // ... the word ...
+    __shared__ float s_cand_e[kMaxCand];                // ... and its leader's E, once known
     __shared__ int s_n_cand;
     __shared__ uint16_t s_redo[kThreads];               // threads whose groups pass 2 goes over again
     __shared__ int s_n_redo;
@@ -221,6 +243,9 @@ unmask_partial_kernel(const T* __restrict__ logits, const uint8_t* __restrict__ 
     const int seg_len = ((vocab + segs - 1) / segs + kSegQuantum - 1) / kSegQuantum * kSegQuantum;
     segs = (vocab + seg_len - 1) / seg_len;
     const int n_items = n_rows * segs;
+    int top_bits = kTopBitsMin;                          // 2^-top_bits of the groups get their leader scored at once
+    while (top_bits < kTopBitsMax && (seg_len >> 4) >> (top_bits + 1) >= 128) ++top_bits;
+    const uint32_t top_word = 0xFFFFFFFFu << (32 - top_bits);
 
     for (int item = blockIdx.x; item < n_items; item += gridDim.x) {
         const int row = s_rows[item / segs];
@@ -242,7 +267,7 @@ unmask_partial_kernel(const T* __restrict__ logits, const uint8_t* __restrict__ 
         float m = -CUDART_INF_F, s = 0.0f;             // thread's running max and sum exp(l - m)
         Best best{-CUDART_INF_F, -CUDART_INF_F, 0x7FFFFFFF};
         // One group: `w` holds its raw words if it could be fetched with the wide loads.
-        auto process = [&](int v0, const uint32_t (&w)[Logit<T>::kWords]) {
+        auto process = [&](int v0, const uint32_t (&w)[Logit<T>::kWords], uint32_t R) {
             float val[kGroup];
             if (vec_ok && v0 + kGroup <= vocab) {
                 Logit<T>::widen(w, val);
@@ -280,47 +305,54 @@ unmask_partial_kernel(const T* __restrict__ logits, const uint8_t* __restrict__ 
                 s = s * ex2_fast((m - mn) * kLog2e) + (sa + sb);
                 m = mn;
             }
-            if (noisy) {
-                const uint4 r = philox4x32_10(make_uint4(static_cast<uint32_t>(v0 >> 4), pos, step, block_idx), keys);
-                const uint32_t cw[4] = {r.x, r.y, r.z, r.w};
-                // Does any of the 16 bytes equal 255?  (~w - 0x01010101) & w & 0x80808080 is non-zero
-                // exactly when the word has such a byte (a borrow can mark a byte above a real one
-                // too, so the places are found again, exactly, on the rare path).
-                uint32_t any = 0;
-#pragma unroll
-                for (int k = 0; k < 4; ++k) any |= (0xFEFEFEFEu - cw[k]) & cw[k] & 0x80808080u;
-                if (any) {
-#pragma unroll
-                    for (int k = 0; k < 4; ++k) {
-                        const uint32_t z = ~cw[k];
-                        uint32_t h = ~(((z & 0x7F7F7F7Fu) + 0x7F7F7F7Fu) | z | 0x7F7F7F7Fu);   // 0x80 where the byte is 255
-                        while (h) {
-                            const int j = (__ffs(h) - 1) >> 3;
-                            h &= h - 1;
-                            const int v = v0 + k * 4 + j;
-                            if (v < vocab) {
-                                const int slot = atomicAdd(&s_n_cand, 1);
-                                if (slot < kMaxCand) s_cand[slot] = v;
-                            }
-                        }
-                    }
-                }
+            if (noisy && R >= top_word && v0 < vocab) {
+                const int slot = atomicAdd(&s_n_cand, 1);
+                if (slot < kMaxCand) { s_cand[slot] = v0; s_cand_word[slot] = R; }
             }
         };
         auto fetch = [&](int v0, uint32_t (&w)[Logit<T>::kWords]) {
             if (vec_ok && v0 < seg_end && v0 + kGroup <= vocab) Logit<T>::fetch(row_ptr + v0, w);
         };
-        if (noisy || sizeof(T) == 4) {
-            // two register buffers take turns: the next group's load is in flight while this one is reduced
+        if (noisy) {
+            // Four iterations (four groups 4096 ids apart) share one Philox block; two register buffers
+            // take turns, so the next group's load is in flight while this one is reduced.
+            constexpr int Q = kSegQuantum;
+            uint32_t wa[Logit<T>::kWords], wb[Logit<T>::kWords];
+            int v0 = seg_begin + tid * kGroup;
+            const int k0 = (v0 >> 12) & 3;              // word index of the first group inside its Philox block
+            fetch(v0, wa);
+            if (k0 != 0 && v0 < seg_end) {
+                // a segment that starts inside a run of four: finish the run (one to three groups)
+                const uint4 rq = philox4x32_10(make_uint4(group_counter(v0 >> 4), pos, step, block_idx), keys);
+                if (k0 < 3) fetch(v0 + Q, wb);
+                process(v0, wa, pick_word(rq, k0));
+                if (k0 < 3 && v0 + Q < seg_end) {
+                    if (k0 < 2) fetch(v0 + 2 * Q, wa);
+                    process(v0 + Q, wb, pick_word(rq, k0 + 1));
+                    if (k0 < 2 && v0 + 2 * Q < seg_end) process(v0 + 2 * Q, wa, rq.w);
+                }
+                v0 += (4 - k0) * Q;
+                fetch(v0, wa);
+            }
+            while (v0 < seg_end) {
+                const uint4 rq = philox4x32_10(make_uint4(group_counter(v0 >> 4), pos, step, block_idx), keys);
+                fetch(v0 + Q, wb);
+                process(v0, wa, rq.x);
+                if (v0 + Q < seg_end) { fetch(v0 + 2 * Q, wa); process(v0 + Q, wb, rq.y); }
+                if (v0 + 2 * Q < seg_end) { fetch(v0 + 3 * Q, wb); process(v0 + 2 * Q, wa, rq.z); }
+                if (v0 + 3 * Q < seg_end) { fetch(v0 + 4 * Q, wa); process(v0 + 3 * Q, wb, rq.w); }
+                v0 += 4 * Q;
+            }
+        } else if (sizeof(T) == 4) {
             uint32_t wa[Logit<T>::kWords], wb[Logit<T>::kWords];
             int v0 = seg_begin + tid * kGroup;
             fetch(v0, wa);
             while (v0 < seg_end) {
                 fetch(v0 + kSegQuantum, wb);
-                process(v0, wa);
+                process(v0, wa, 0u);
                 if (v0 + kSegQuantum < seg_end) {
                     fetch(v0 + 2 * kSegQuantum, wa);
-                    process(v0 + kSegQuantum, wb);
+                    process(v0 + kSegQuantum, wb, 0u);
                 }
                 v0 += 2 * kSegQuantum;
             }
@@ -334,27 +366,33 @@ unmask_partial_kernel(const T* __restrict__ logits, const uint8_t* __restrict__ 
             fetch(v0 + 2 * kSegQuantum, wc);
             while (v0 < seg_end) {
                 fetch(v0 + 3 * kSegQuantum, wd);
-                process(v0, wa);
-                if (v0 + kSegQuantum < seg_end) { fetch(v0 + 4 * kSegQuantum, wa); process(v0 + kSegQuantum, wb); }
-                if (v0 + 2 * kSegQuantum < seg_end) { fetch(v0 + 5 * kSegQuantum, wb); process(v0 + 2 * kSegQuantum, wc); }
-                if (v0 + 3 * kSegQuantum < seg_end) { fetch(v0 + 6 * kSegQuantum, wc); process(v0 + 3 * kSegQuantum, wd); }
+                process(v0, wa, 0u);
+                if (v0 + kSegQuantum < seg_end) { fetch(v0 + 4 * kSegQuantum, wa); process(v0 + kSegQuantum, wb, 0u); }
+                if (v0 + 2 * kSegQuantum < seg_end) { fetch(v0 + 5 * kSegQuantum, wb); process(v0 + 2 * kSegQuantum, wc, 0u); }
+                if (v0 + 3 * kSegQuantum < seg_end) { fetch(v0 + 6 * kSegQuantum, wc); process(v0 + 3 * kSegQuantum, wd, 0u); }
                 v0 += 4 * kSegQuantum;
             }
         }
 
         if (noisy) {
             __syncthreads();
-            // ---- exact scores of the candidates: their best is a lower bound L of the segment's best
+            // Exact score of an id of group v0 whose word is R; e_leader < 0: not computed yet.
+            auto fine23 = [&](int v) {
+                const uint4 r = philox4x32_10(make_uint4(static_cast<uint32_t>(v >> 2), pos | kFineStream, step, block_idx), keys);
+                return pick_word(r, v & 3) >> 9;
+            };
+            // ---- exact scores of the leaders of the top-word groups: their best is a lower bound L of
+            // the segment's best
             const int n_cand = s_n_cand;
-            const bool overflow = n_cand > kMaxCand;    // (never for random bytes) then nothing is pruned
+            const bool overflow = n_cand > kMaxCand;    // (never for random words) then nothing is pruned
             if (!overflow) {
                 for (int c = tid; c < n_cand; c += kThreads) {
-                    const int v = s_cand[c];
+                    const int v = s_cand[c] + static_cast<int>(s_cand_word[c] & 15u);
+                    const float e = leader_exponential(s_cand_word[c], fine23(v));
+                    s_cand_e[c] = e;
+                    if (v >= vocab) continue;           // the leader of a cut last group may lie beyond the row
                     const float l = Logit<T>::load1(row_ptr + v);
-                    const uint4 r = philox4x32_10(make_uint4(static_cast<uint32_t>(v >> 2), pos | kFineStream, step, block_idx), keys);
-                    const uint32_t w4[4] = {r.x, r.y, r.z, r.w};
-                    const float sc = fmaf(temperature, gumbel_exact(255u, w4[v & 3] >> 9), l);
-                    best = better(best, Best{sc, l, v});
+                    best = better(best, Best{fmaf(temperature, -logf(e), l), l, v});
                 }
             }
             float lb = best.score;
@@ -366,9 +404,11 @@ unmask_partial_kernel(const T* __restrict__ logits, const uint8_t* __restrict__ 
 #pragma unroll
             for (int w2 = 1; w2 < kThreads / 32; ++w2) lb = fmaxf(lb, red_score[w2]);
             if (overflow) lb = -CUDART_INF_F;
-            // ---- pass 2: the groups of every thread whose largest logit can still reach L are gone over
-            // again, by the whole CTA (one group per thread), not by that thread alone
-            const float reach = lb - temperature * kGumbelBelow255 - 1e-3f;
+            // ---- pass 2: every id that can still reach L is scored exactly.  Two kinds of groups are
+            // gone over again, by the whole CTA (one group per thread): all groups of the threads whose
+            // largest logit can reach L with the largest draw a plain group allows, and the top-word
+            // groups (their other 15 ids are bounded by their leader's draw only).
+            const float reach = lb - temperature * gumbel_plain(top_bits) - 1e-3f;
             if (m >= reach) {
                 const int slot = atomicAdd(&s_n_redo, 1);
                 if (slot < kThreads) s_redo[slot] = static_cast<uint16_t>(tid);
@@ -376,32 +416,54 @@ unmask_partial_kernel(const T* __restrict__ logits, const uint8_t* __restrict__ 
             __syncthreads();
             const int n_redo = min(s_n_redo, kThreads);
             const int groups_per_thread = (seg_end - seg_begin + kSegQuantum - 1) / kSegQuantum;
-            for (int w = tid; w < n_redo * groups_per_thread; w += kThreads) {
-                const int owner = s_redo[w / groups_per_thread];
-                const int v0 = seg_begin + owner * kGroup + (w % groups_per_thread) * kSegQuantum;
-                if (v0 >= seg_end) continue;
+            const int n_plain = n_redo * groups_per_thread;
+            const int n_top = overflow ? 0 : n_cand;
+            for (int w = tid; w < n_plain + n_top; w += kThreads) {
+                int v0;
+                uint32_t R;
+                bool top;
+                if (w < n_plain) {
+                    const int owner = s_redo[w / groups_per_thread];
+                    v0 = seg_begin + owner * kGroup + (w % groups_per_thread) * kSegQuantum;
+                    if (v0 >= seg_end) continue;
+                } else {
+                    v0 = s_cand[w - n_plain];
+                }
                 float val[kGroup];
                 load_group(row_ptr, v0, vocab, vec_ok, val);
-                bool some = false;
+                float e_lead = -1.0f;                   // < 0: not known yet
+                if (w < n_plain) {
+                    bool some = false;
 #pragma unroll
-                for (int i = 0; i < kGroup; ++i) some = some || (val[i] >= reach && val[i] > -CUDART_INF_F);
-                if (!some) continue;
-                const uint4 rc = philox4x32_10(make_uint4(static_cast<uint32_t>(v0 >> 4), pos, step, block_idx), keys);
-                const uint32_t cw[4] = {rc.x, rc.y, rc.z, rc.w};
-                for (int i = 0; i < kGroup; ++i) {
-                    float l = -CUDART_INF_F;
-                    uint32_t word = 0;
+                    for (int i = 0; i < kGroup; ++i) some = some || (val[i] >= reach && val[i] > -CUDART_INF_F);
+                    if (!some) continue;
+                    const int j = v0 >> 4;
+                    R = pick_word(philox4x32_10(make_uint4(group_counter(j), pos, step, block_idx), keys), (j >> 8) & 3);
+                    top = R >= top_word;
+                    if (top && !overflow) continue;     // comes again as a top-word group
+                } else {
+                    R = s_cand_word[w - n_plain];
+                    e_lead = s_cand_e[w - n_plain];
+                    top = true;
+                }
+                // the bound every draw of the group obeys: exact for a top-word group, from the word
+                // alone otherwise (the leader's fine bits are fetched only if some id passes it)
+                const int lead = v0 + static_cast<int>(R & 15u);
+                if (top && e_lead < 0.0f) e_lead = leader_exponential(R, fine23(lead));
+                const float bar = lb - 1e-3f - temperature * -logf(top ? e_lead * 0.999f : group_floor(R));
+                uint32_t pass = 0;                      // ids whose logit clears the bar
 #pragma unroll
-                    for (int x = 0; x < kGroup; ++x) if (x == i) { l = val[x]; word = cw[x >> 2]; }
-                    if (!(l >= reach) || l == -CUDART_INF_F) continue;
-                    const uint32_t c = (word >> ((i & 3) * 8)) & 0xFFu;
-                    if (c == 255u && !overflow) continue;                  // handled as a candidate
-                    if (c < 255u && fmaf(temperature, gumbel_bound(c), l) < lb) continue;
+                for (int i = 0; i < kGroup; ++i) pass |= (val[i] >= bar && val[i] > -CUDART_INF_F) ? (1u << i) : 0u;
+                while (pass) {
+                    const int i = __ffs(pass) - 1;
+                    pass &= pass - 1;
+                    float l = val[0];
+#pragma unroll
+                    for (int x = 1; x < kGroup; ++x) if (x == i) l = val[x];
                     const int v = v0 + i;
-                    const uint4 r = philox4x32_10(make_uint4(static_cast<uint32_t>(v >> 2), pos | kFineStream, step, block_idx), keys);
-                    const uint32_t w4[4] = {r.x, r.y, r.z, r.w};
-                    const float sc = fmaf(temperature, gumbel_exact(c, w4[v & 3] >> 9), l);
-                    best = better(best, Best{sc, l, v});
+                    if (e_lead < 0.0f) e_lead = leader_exponential(R, fine23(lead));
+                    const float e = v == lead ? e_lead : follower_exponential(e_lead, fine23(v));
+                    best = better(best, Best{fmaf(temperature, -logf(e), l), l, v});
                 }
             }
         }

@@ -99,8 +99,8 @@ def test_gumbel_row_layout_and_independence_from_vocab_size():
 
 def test_group_word_bounds_every_draw_of_the_group():
     # what lets an implementation skip the per-id stream: the word of a group alone bounds the 16
-    # draws of the group, E[v] >= -ln((h + 1) / 2^28) / 16 with h = word >> 4, and a word below
-    # 0xFF000000 (255 of 256 groups) caps them at g < 8.3158
+    # draws of the group, E[v] >= -ln((h + 1) / 2^28) / 16 with h = word >> 4; a word below 0xFF000000
+    # (255 of 256 groups) caps them at g < 8.3158, one below 0xFC000000 (63 of 64) at g < 6.9237
     V = 50000
     e = exponential_row(777, 1, 4, 9, V)
     words = group_words(777, 1, 4, 9, V)
@@ -113,10 +113,11 @@ def test_group_word_bounds_every_draw_of_the_group():
     inside = lead < V
     np.testing.assert_array_equal(grp_min[inside], e[lead[inside]])           # the leader holds the minimum
     assert np.all(e[lead[inside]] <= ceil_leader[lead[inside]])
-    plain = np.repeat(words < np.uint64(0xFF000000), 16)[:V]
     g = -np.log(e)
-    assert np.all(g[plain] < 8.3158)
-    assert 0.5 / 256 < 1.0 - plain.mean() < 2.0 / 256
+    for top_word, cap, share in ((0xFF000000, 8.3158, 256), (0xFC000000, 6.9237, 64)):
+        plain = np.repeat(words < np.uint64(top_word), 16)[:V]
+        assert np.all(g[plain] < cap)
+        assert 0.6 / share < 1.0 - plain.mean() < 1.6 / share
     # the leader's place is uniform over the 16 ids and unrelated to the minimum
     places = (words & np.uint64(15)).astype(int)
     counts = np.bincount(places, minlength=16)
