@@ -39,6 +39,10 @@ constexpr int kMaxRows = kUnmaskMaxRows;              // rows whose state fits t
 // 256 top-word groups (b = 6 for whole rows of 152k ids, b = 2 for 8192-id segments).  Every draw
 // of the other groups lies below kGumbelPlain[b] > -ln(-ln(1 - 2^-b) / 16).
 constexpr int kTopBitsMin = 2, kTopBitsMax = 6;
+#ifndef FDD_UM_NOISY_CTAS
+#define FDD_UM_NOISY_CTAS 3
+#endif
+constexpr int kNoisyCtasPerSm = FDD_UM_NOISY_CTAS;   // noisy kernel: CTAs per SM (2: four load buffers per thread, 3: two)
 __device__ __forceinline__ float gumbel_plain(int b) {
     return b == 2 ? 4.0195f : (b == 3 ? 4.7870f : (b == 4 ? 5.5140f : (b == 5 ? 6.2235f : 6.9245f)));
 }
@@ -195,7 +199,7 @@ __device__ __forceinline__ Best warp_best(Best b) {
 }
 
 template <typename T, bool NOISY>
-__global__ void __launch_bounds__(kThreads, 3)
+__global__ void __launch_bounds__(kThreads, NOISY ? kNoisyCtasPerSm : 3)
 unmask_partial_kernel(const T* __restrict__ logits, const uint8_t* __restrict__ state,
                       const __grid_constant__ UnmaskSets sets, UnmaskPartial* __restrict__ partial,
                       int vocab, int n_chunks, float temperature,
@@ -236,23 +240,34 @@ unmask_partial_kernel(const T* __restrict__ logits, const uint8_t* __restrict__ 
     }
     const int n_rows = s_n_rows;
     if (n_rows == 0) return;
-    // Segments per row: one when there are plenty of rows, more (up to n_chunks) when the rows
-    // alone would leave SMs idle.  Every CTA derives the same numbers.
-    int segs = (2 * static_cast<int>(gridDim.x) + n_rows - 1) / n_rows;
-    segs = max(1, min(segs, n_chunks));
-    const int seg_len = ((vocab + segs - 1) / segs + kSegQuantum - 1) / kSegQuantum * kSegQuantum;
-    segs = (vocab + seg_len - 1) / seg_len;
-    const int n_items = n_rows * segs;
-    int top_bits = kTopBitsMin;                          // 2^-top_bits of the groups get their leader scored at once
-    while (top_bits < kTopBitsMax && (seg_len >> 4) >> (top_bits + 1) >= 128) ++top_bits;
-    const uint32_t top_word = 0xFFFFFFFFu << (32 - top_bits);
+    // The selected rows, cut into chunks of 8192 ids and laid end to end, are split into equal
+    // contiguous ranges, one per CTA: a CTA's range is the tail of one row, some whole rows and the
+    // head of another, and every (row, CTA) pair leaves one record (at most n_chunks per row).  With
+    // few rows every chunk gets its own CTA.  Every CTA derives the same numbers.
+    const long long W = static_cast<long long>(n_rows) * n_chunks;
+    const long long G = min(static_cast<long long>(gridDim.x), W);
+    if (blockIdx.x >= G) return;
+    const long long range_begin = W * blockIdx.x / G, range_end = W * (blockIdx.x + 1) / G;
 
-    for (int item = blockIdx.x; item < n_items; item += gridDim.x) {
-        const int row = s_rows[item / segs];
-        const int seg = item - (item / segs) * segs;
+    for (long long at = range_begin; at < range_end;) {
+        const int ri = static_cast<int>(at / n_chunks);
+        const int chunk0 = static_cast<int>(at - static_cast<long long>(ri) * n_chunks);
+        const int chunk1 = static_cast<int>(min(static_cast<long long>(n_chunks), chunk0 + (range_end - at)));
+        at += chunk1 - chunk0;
+        const int row = s_rows[ri];
+        const int seg_begin = chunk0 * kUnmaskChunk;
+        const int seg_end = min(vocab, chunk1 * kUnmaskChunk);
+        // which of the row's records this is, and how many there are (CTA c owns chunks [W c / G, W (c + 1) / G))
+        const long long row_first = static_cast<long long>(ri) * n_chunks;
+        const int cta_first = static_cast<int>(((row_first + 1) * G + W - 1) / W) - 1;
+        const int cta_last = static_cast<int>(((row_first + n_chunks) * G + W - 1) / W) - 1;
+        const int seg = static_cast<int>(blockIdx.x) - cta_first;
+        const int segs = cta_last - cta_first + 1;
+        // 2^-top_bits of the groups get their leader scored at once: 128 to 256 groups of this piece
+        int top_bits = kTopBitsMin;
+        while (top_bits < kTopBitsMax && ((seg_end - seg_begin) >> 4) >> (top_bits + 1) >= 128) ++top_bits;
+        const uint32_t top_word = 0xFFFFFFFFu << (32 - top_bits);
         const T* row_ptr = logits + static_cast<size_t>(row) * vocab;
-        const int seg_begin = seg * seg_len;
-        const int seg_end = min(vocab, seg_begin + seg_len);
         int set = 0;
         while (set + 1 < sets.n_sets && row >= sets.row_off[set + 1]) ++set;
         const int local = row - sets.row_off[set];
@@ -334,14 +349,30 @@ unmask_partial_kernel(const T* __restrict__ logits, const uint8_t* __restrict__ 
                 v0 += (4 - k0) * Q;
                 fetch(v0, wa);
             }
-            while (v0 < seg_end) {
-                const uint4 rq = philox4x32_10(make_uint4(group_counter(v0 >> 4), pos, step, block_idx), keys);
+            if (kNoisyCtasPerSm >= 3) {
+                while (v0 < seg_end) {
+                    const uint4 rq = philox4x32_10(make_uint4(group_counter(v0 >> 4), pos, step, block_idx), keys);
+                    fetch(v0 + Q, wb);
+                    process(v0, wa, rq.x);
+                    if (v0 + Q < seg_end) { fetch(v0 + 2 * Q, wa); process(v0 + Q, wb, rq.y); }
+                    if (v0 + 2 * Q < seg_end) { fetch(v0 + 3 * Q, wb); process(v0 + 2 * Q, wa, rq.z); }
+                    if (v0 + 3 * Q < seg_end) { fetch(v0 + 4 * Q, wa); process(v0 + 3 * Q, wb, rq.w); }
+                    v0 += 4 * Q;
+                }
+            } else {
+                // four buffers, three loads in flight
+                uint32_t wc[Logit<T>::kWords], wd[Logit<T>::kWords];
                 fetch(v0 + Q, wb);
-                process(v0, wa, rq.x);
-                if (v0 + Q < seg_end) { fetch(v0 + 2 * Q, wa); process(v0 + Q, wb, rq.y); }
-                if (v0 + 2 * Q < seg_end) { fetch(v0 + 3 * Q, wb); process(v0 + 2 * Q, wa, rq.z); }
-                if (v0 + 3 * Q < seg_end) { fetch(v0 + 4 * Q, wa); process(v0 + 3 * Q, wb, rq.w); }
-                v0 += 4 * Q;
+                fetch(v0 + 2 * Q, wc);
+                while (v0 < seg_end) {
+                    const uint4 rq = philox4x32_10(make_uint4(group_counter(v0 >> 4), pos, step, block_idx), keys);
+                    fetch(v0 + 3 * Q, wd);
+                    process(v0, wa, rq.x);
+                    if (v0 + Q < seg_end) { fetch(v0 + 4 * Q, wa); process(v0 + Q, wb, rq.y); }
+                    if (v0 + 2 * Q < seg_end) { fetch(v0 + 5 * Q, wb); process(v0 + 2 * Q, wc, rq.z); }
+                    if (v0 + 3 * Q < seg_end) { fetch(v0 + 6 * Q, wc); process(v0 + 3 * Q, wd, rq.w); }
+                    v0 += 4 * Q;
+                }
             }
         } else if (sizeof(T) == 4) {
             uint32_t wa[Logit<T>::kWords], wb[Logit<T>::kWords];
@@ -642,7 +673,7 @@ cudaError_t launch_unmask_kernels(const UnmaskProblem& p, UnmaskPartial* partial
             cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sm_count <= 0)
             sm_count = 148;
     }
-    const long long ctas = static_cast<long long>(sm_count) * 3;      // persistent: as many CTAs as fit on the SMs
+    const long long ctas = static_cast<long long>(sm_count) * (p.temperature != 0.0f ? kNoisyCtasPerSm : 3);   // persistent: as many CTAs as fit on the SMs
     const dim3 grid(static_cast<unsigned>(ctas));
     if (p.logits_dtype == FDD_LOGITS_BF16) {
         const int vec_ok = (p.vocab % 16 == 0) && (reinterpret_cast<uintptr_t>(p.logits) % 32 == 0);
