@@ -133,6 +133,20 @@ __device__ __forceinline__ void load32(const void* p, uint32_t (&r)[8]) {
                  : "l"(p));
 }
 
+// Asynchronous 16-byte copies global -> shared (the thread that issues them also waits for them).
+__device__ __forceinline__ void cp_async16(void* smem_dst, const void* gsrc) {
+    const uint32_t d = static_cast<uint32_t>(__cvta_generic_to_shared(smem_dst));
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(d), "l"(gsrc) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
+// Ring of bf16 groups in shared memory: every thread owns 32 bytes per stage, fills them with
+// asynchronous copies several groups ahead and reads only what it copied itself (no barrier).
+constexpr int kRingStages = 4;
+constexpr int kRingStageBytes = kThreads * kGroup * 2;
+
 // A group = 16 consecutive logits.  fetch() starts the 32-byte loads of a group into raw words,
 // widen() turns the words into fp32 once they are needed (so several groups can be in flight).
 template <typename T> struct Logit;
@@ -328,7 +342,48 @@ unmask_partial_kernel(const T* __restrict__ logits, const uint8_t* __restrict__ 
         auto fetch = [&](int v0, uint32_t (&w)[Logit<T>::kWords]) {
             if (vec_ok && v0 < seg_end && v0 + kGroup <= vocab) Logit<T>::fetch(row_ptr + v0, w);
         };
-        if (noisy) {
+        if (NOISY && sizeof(T) == 2 && vec_ok) {
+            // noisy step on bf16 rows that allow 16-byte copies: the groups travel through the thread's
+            // slots of the ring (three copies in flight without holding registers); four consecutive
+            // groups of a thread (4096 ids apart) share one Philox block.
+            constexpr int S = kRingStages;
+            extern __shared__ __align__(16) unsigned char s_ring[];
+            const int v_first = seg_begin + tid * kGroup;
+            const int n_g = v_first < seg_end ? (seg_end - v_first + kSegQuantum - 1) / kSegQuantum : 0;
+            const int k0 = (v_first >> 12) & 3;         // word index of the first group inside its Philox block
+            auto issue = [&](int g) {
+                const int v = v_first + g * kSegQuantum;
+                if (g < n_g && v + kGroup <= vocab) {
+                    unsigned char* dst = s_ring + (g % S) * kRingStageBytes + tid * 32;
+                    const unsigned char* src = reinterpret_cast<const unsigned char*>(row_ptr + v);
+                    cp_async16(dst, src);
+                    cp_async16(dst + 16, src + 16);
+                }
+                cp_async_commit();                      // an empty group keeps the count uniform
+            };
+#pragma unroll
+            for (int g = 0; g < S - 1; ++g) issue(g);
+            uint4 rq = make_uint4(0u, 0u, 0u, 0u);
+#pragma unroll 4
+            for (int g = 0; g < n_g; ++g) {
+                issue(g + S - 1);                       // into the slot that was consumed one iteration ago
+                cp_async_wait<S - 1>();                 // group g has landed
+                const int v = v_first + g * kSegQuantum;
+                uint32_t R = 0u;
+                if (noisy) {
+                    const int k = (k0 + g) & 3;
+                    if (g == 0 || k == 0) rq = philox4x32_10(make_uint4(group_counter(v >> 4), pos, step, block_idx), keys);
+                    R = pick_word(rq, k);
+                }
+                uint32_t w[Logit<T>::kWords];
+                const uint4* slot = reinterpret_cast<const uint4*>(s_ring + (g % S) * kRingStageBytes + tid * 32);
+                const uint4 lo = slot[0], hi = slot[1];
+                w[0] = lo.x; w[1] = lo.y; w[2] = lo.z; w[3] = lo.w;
+                w[Logit<T>::kWords - 4] = hi.x; w[Logit<T>::kWords - 3] = hi.y; w[Logit<T>::kWords - 2] = hi.z; w[Logit<T>::kWords - 1] = hi.w;
+                process(v, w, R);
+            }
+            cp_async_wait<0>();
+        } else if (noisy) {
             // Four iterations (four groups 4096 ids apart) share one Philox block; two register buffers
             // take turns, so the next group's load is in flight while this one is reduced.
             constexpr int Q = kSegQuantum;
@@ -677,12 +732,22 @@ cudaError_t launch_unmask_kernels(const UnmaskProblem& p, UnmaskPartial* partial
     const dim3 grid(static_cast<unsigned>(ctas));
     if (p.logits_dtype == FDD_LOGITS_BF16) {
         const int vec_ok = (p.vocab % 16 == 0) && (reinterpret_cast<uintptr_t>(p.logits) % 32 == 0);
+        // the noisy bf16 kernel streams through a ring in dynamic shared memory (more than the 48 KB a
+        // kernel gets without asking, together with its static arrays)
+        constexpr int kRingNoisy = kRingStages * kRingStageBytes, kRingGreedy = 0;
+        static bool configured = false;
+        if (!configured) {
+            cudaError_t ea = cudaFuncSetAttribute(unmask_partial_kernel<__nv_bfloat16, true>,
+                                                  cudaFuncAttributeMaxDynamicSharedMemorySize, kRingNoisy);
+            if (ea != cudaSuccess) return ea;
+            configured = true;
+        }
         if (p.temperature != 0.0f)
-            unmask_partial_kernel<__nv_bfloat16, true><<<grid, kThreads, 0, st>>>(
+            unmask_partial_kernel<__nv_bfloat16, true><<<grid, kThreads, kRingNoisy, st>>>(
                 static_cast<const __nv_bfloat16*>(p.logits), p.state, p.sets, partial, p.vocab,
                 n_chunks, p.temperature, p.block_idx, p.step, vec_ok, select_state);
         else
-            unmask_partial_kernel<__nv_bfloat16, false><<<grid, kThreads, 0, st>>>(
+            unmask_partial_kernel<__nv_bfloat16, false><<<grid, kThreads, kRingGreedy, st>>>(
                 static_cast<const __nv_bfloat16*>(p.logits), p.state, p.sets, partial, p.vocab,
                 n_chunks, p.temperature, p.block_idx, p.step, vec_ok, select_state);
     } else {
