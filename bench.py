@@ -28,7 +28,7 @@ METRIC = "committed tokens/s per denoise step (N forks, shared prefix)"
 UNIT = "tokens/s"
 # DRAM bytes (read + write) of one attention launch at the long_prefix workload, from the ncu capture
 # summarised in profiles/attn_ptc_long_prefix.md; None for other workloads or once the kernel changed.
-ATTN_DRAM_BYTES_PER_LAUNCH = {}
+ATTN_DRAM_BYTES_PER_LAUNCH = {"long_prefix": 180.0e6}
 LOOKAHEAD = True   # enqueue step t + 1 before the host has read the counts of step t (--no-lookahead)
 PRE_STEPS = 6      # distinct per-step input sets kept resident; later steps cycle through them (--pre-steps)
 

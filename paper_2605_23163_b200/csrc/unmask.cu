@@ -1,11 +1,12 @@
 // Confidence-threshold parallel unmasking: vocabulary-wide soft-max statistics and
 // (Gumbel-perturbed) arg-max per MASKED row, then the per-rollout commit rule.
 //
-// Kernel 1 (unmask_partial_kernel): a persistent grid walks the (MASKED row, segment) pairs of the
-// call; with many MASKED rows a segment is a whole row, with few the rows are cut so that every
-// SM has work.  A CTA streams its segment from HBM once with 32-byte loads (16 consecutive logits
-// per thread and load) and keeps running soft-max statistics; nothing but the few logits that can
-// win the arg-max is looked at twice.  Rows that are not MASKED are never read.
+// Kernel 1 (unmask_partial_kernel): persistent grid.  The MASKED rows of the call, cut into chunks
+// of 8192 ids and laid end to end, are split into equal contiguous ranges, one per CTA (with few
+// rows every chunk gets a CTA of its own).  A CTA streams each of its pieces from HBM once, 16
+// consecutive logits per thread and step (32-byte loads, or 16-byte asynchronous copies through a
+// per-thread ring in shared memory), and keeps running soft-max statistics; nothing but the few
+// logits that can win the arg-max is looked at twice.  Rows that are not MASKED are never read.
 //
 // Noise (temperature > 0).  The Gumbel draws are g = -ln(E) with E an exponential race over groups
 // of 16 consecutive ids: one 32-bit word R per group (a Philox block serves the four groups that a
