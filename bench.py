@@ -29,6 +29,7 @@ UNIT = "tokens/s"
 # DRAM bytes (read + write) of one attention launch at the long_prefix workload, from the ncu capture
 # summarised in profiles/attn_ptc_long_prefix.md; None for other workloads or once the kernel changed.
 ATTN_DRAM_BYTES_PER_LAUNCH = {"long_prefix": 180.0e6}
+COUNT_STREAM = None  # copy the per-rollout counts to the host on a stream of their own (None: for large steps only)
 LOOKAHEAD = True   # enqueue step t + 1 before the host has read the counts of step t (--no-lookahead)
 PRE_STEPS = 6      # distinct per-step input sets kept resident; later steps cycle through them (--pre-steps)
 
@@ -173,6 +174,15 @@ def run_ours(args):
                   g.prefix_capacity, g.sc.n_forks, fdd.u64_array(g.seeds), fdd.ptr_array(g.suffix_k),
                   fdd.ptr_array(g.suffix_v), g.suffix_capacity) for g in gscenes]
     step_done = [torch.cuda.Event(), torch.cuda.Event()]
+    # The counts go to the host on a stream of their own, so that the next attention call does not
+    # queue behind the copy; unmask writes them to two device buffers in turn (step t + 2 reuses the
+    # buffer of step t, whose copy the host has waited for by then).
+    count_stream = torch.cuda.Stream()
+    # (worth it when a step's kernels are long; a latency-bound step loses more to the second stream's
+    # event than the copy costs in line)
+    use_count_stream = COUNT_STREAM if COUNT_STREAM is not None else all_tokens >= 1024
+    unmask_done = [torch.cuda.Event(), torch.cuda.Event()]
+    n_left_d = [n_left, torch.zeros_like(n_left)]
 
     attn_events = []            # [start, end, rollouts still decoding] of every timed attention call
     unmask_events = []          # [start, end, MASKED rows on entry] of every timed unmask call
@@ -188,19 +198,19 @@ def run_ours(args):
         fs = fdd.ptr_array(fs_list)
         tokens.copy_(tokens0_d, non_blocking=True)
         state.copy_(state0_d, non_blocking=True)
-        n_left.copy_(n_left0_d, non_blocking=True)
         kv_of = [None, None]
         pending = [None, None]      # the event records of a step, completed once its entry counts are known
 
         def enqueue(t):
             q, k, v, lg = inputs(t)
             kv_of[t % 2] = (k, v)
+            gate = n_left0_d if t == 0 else n_left_d[(t - 1) % 2]     # who still decodes: the counts of the step before
             recs = []
             for layer in range(L):
                 if timed_attn:
                     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
                     e0.record(stream)
-                fdd.fdd_block_attn_gated(ctx, fs, layer, q, k, v, out, ds_c, scale, 0, n_left)
+                fdd.fdd_block_attn_gated(ctx, fs, layer, q, k, v, out, ds_c, scale, 0, gate)
                 if timed_attn:
                     e1.record(stream)
                     recs.append([e0, e1, None])
@@ -208,13 +218,20 @@ def run_ours(args):
             if timed_attn:
                 u0, u1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
                 u0.record(stream)
-            fdd.fdd_unmask(ctx, fs, lg, tokens, state, ds_c, w.threshold, w.temperature, 0, t, n_comm, n_left)
+            fdd.fdd_unmask(ctx, fs, lg, tokens, state, ds_c, w.threshold, w.temperature, 0, t, n_comm, n_left_d[t % 2])
             if timed_attn:
                 u1.record(stream)
                 recs.append([u0, u1, None])
                 unmask_events.append(recs[-1])
-            n_left_hosts[t % 2].copy_(n_left, non_blocking=True)
-            step_done[t % 2].record(stream)
+            if use_count_stream:
+                unmask_done[t % 2].record(stream)
+                count_stream.wait_event(unmask_done[t % 2])
+                with torch.cuda.stream(count_stream):
+                    n_left_hosts[t % 2].copy_(n_left_d[t % 2], non_blocking=True)
+                    step_done[t % 2].record(count_stream)
+            else:
+                n_left_hosts[t % 2].copy_(n_left_d[t % 2], non_blocking=True)
+                step_done[t % 2].record(stream)
             pending[t % 2] = recs
 
         def entry_counts(t, rollouts, rows):
@@ -356,6 +373,7 @@ def run_ours(args):
                    "l2": "per-step inputs (logits) larger than L2",
                    "step_pipeline": ("attention gated by n_left; step t+1 enqueued before the host reads step t"
                                      if LOOKAHEAD else "attention gated by n_left; one step in flight"),
+                   "count_copy": "own stream" if use_count_stream else "compute stream",
                    "rollouts_decoding_per_attention_call": float(np.mean([n for _, n in attn_all])) if attn_all else None,
                    "replicas": "independent scene per GPU, no collective"},
         "clocks": sampler.summary(),
@@ -474,7 +492,7 @@ def run_reference(args):
 
 
 def main():
-    global PRE_STEPS, LOOKAHEAD
+    global PRE_STEPS, LOOKAHEAD, COUNT_STREAM
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=40)
@@ -489,11 +507,14 @@ def main():
     ap.add_argument("--cpu-budget", type=float, default=20.0)
     ap.add_argument("--no-lookahead", action="store_true",
                     help="enqueue a denoising step only after the host has read the counts of the one before")
+    ap.add_argument("--counts", choices=["auto", "in-line", "own-stream"], default="auto",
+                    help="where the per-rollout counts are copied to the host: on the compute stream or on a stream of their own")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     PRE_STEPS = max(1, args.pre_steps)
     LOOKAHEAD = not args.no_lookahead
+    COUNT_STREAM = {"auto": None, "in-line": False, "own-stream": True}[args.counts]
     if args.impl == "reference":
         run_reference(args)
     else:
