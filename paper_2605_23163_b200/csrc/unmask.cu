@@ -235,22 +235,34 @@ unmask_partial_kernel(const T* __restrict__ logits, const uint8_t* __restrict__ 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     constexpr bool noisy = NOISY;                       // temperature > 0
 
-    // Every CTA compacts the list of MASKED rows for itself (the state array is a few KB).
+    // Every CTA compacts the list of MASKED rows for itself (the state array is a few KB): a thread
+    // takes a run of consecutive rows, one block-wide prefix sum places the runs.
     {
-        int base = 0;
-        for (int r0 = 0; r0 < rows; r0 += kThreads) {
-            const int r = r0 + tid;
-            const bool m = r < rows && state[r] == select_state;
-            const unsigned bal = __ballot_sync(0xFFFFFFFFu, m);
-            if (lane == 0) s_warp_count[warp] = __popc(bal);
-            __syncthreads();
-            int before = base;
-            for (int w2 = 0; w2 < warp; ++w2) before += s_warp_count[w2];
-            if (m) s_rows[before + __popc(bal & ((1u << lane) - 1u))] = static_cast<uint16_t>(r);
-            for (int w2 = 0; w2 < kThreads / 32; ++w2) base += s_warp_count[w2];
-            __syncthreads();
+        const int per = (rows + kThreads - 1) / kThreads;          // <= 32 (rows <= 8192)
+        const int r_begin = min(rows, tid * per), r_end = min(rows, r_begin + per);
+        uint32_t mine = 0;                                         // bit k: row r_begin + k is selected
+        for (int r = r_begin; r < r_end; ++r) mine |= (state[r] == select_state ? 1u : 0u) << (r - r_begin);
+        const int cnt = __popc(mine);
+        int incl = cnt;                                            // inclusive prefix sum inside the warp
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+            const int up = __shfl_up_sync(0xFFFFFFFFu, incl, off);
+            if (lane >= off) incl += up;
         }
-        if (tid == 0) { s_n_rows = base; s_n_cand = 0; s_n_redo = 0; }
+        if (lane == 31) s_warp_count[warp] = incl;
+        __syncthreads();
+        int before = incl - cnt, total = 0;
+#pragma unroll
+        for (int w2 = 0; w2 < kThreads / 32; ++w2) {
+            if (w2 < warp) before += s_warp_count[w2];
+            total += s_warp_count[w2];
+        }
+        while (mine) {
+            const int k = __ffs(mine) - 1;
+            mine &= mine - 1;
+            s_rows[before++] = static_cast<uint16_t>(r_begin + k);
+        }
+        if (tid == 0) { s_n_rows = total; s_n_cand = 0; s_n_redo = 0; }
         __syncthreads();
     }
     const int n_rows = s_n_rows;
