@@ -74,6 +74,36 @@ def test_attention_long_prefix_sampled_forks():
     _attention_case(synth.workload("long_prefix"), forks_checked=[0, 13, 31])
 
 
+def test_attention_long_prefix_two_rollouts_left_units_cut_into_many_pieces():
+    # late in a block only a few rollouts still decode: at the largest configuration two live
+    # rollouts make 16 units of 129 key tiles on 148 CTAs, so every unit is cut into about ten
+    # pieces (more than the merge folds in at once); causal and bidirectional
+    w = synth.workload("long_prefix")
+    sc = w.scenes[0]
+    ctx = harness.create_context(w)
+    try:
+        scene = harness.GpuScene(ctx, w, 0)
+        pk, pv = synth.make_prefix(w, 0)
+        empty = ([np.zeros((0, w.n_kv_heads, w.head_dim), dtype=np.uint16)] * sc.n_forks,) * 2
+        q, k, v = synth.make_qkv(w, 0, 0, 0, 3)
+        qd, kd, vd = harness.bf16_tensor(q), harness.bf16_tensor(k), harness.bf16_tensor(v)
+        live = [5, 30]
+        gate = torch.zeros(sc.n_forks, dtype=torch.int32, device="cuda")
+        gate[live] = 2
+        for causal in (False, True):
+            out = torch.full_like(qd, float("nan"))
+            fdd.fdd_block_attn_gated(ctx, [scene.forkset], 0, qd, kd, vd, out, [sc.block_len],
+                                     1.0 / np.sqrt(w.head_dim), int(causal), gate)
+            fdd.fdd_poll_status(ctx)
+            got = out.float().cpu().numpy().astype(np.float64).reshape(q.shape)
+            ref = pu.attention_oracle(w, (pk, pv), empty, q, k, v, causal=causal, forks=live)
+            pu.assert_attention_close(got[live], ref)
+            rest = np.setdiff1d(np.arange(sc.n_forks), live)
+            assert np.all(np.isnan(got[rest]))
+    finally:
+        fdd.fdd_destroy(ctx)
+
+
 def test_attention_no_prefix_and_single_position():
     w = synth.workload("tiny")
     sc = synth.Scene(prefix_len=0, n_forks=2, block_len=1, n_scaffold=0, n_blocks=2)
