@@ -11,6 +11,7 @@
  *   fdd_plan_blocks      section-aligned blocks of the output template         (Sec. 3.2)
  *   fdd_kv_commit        append the finished block to each private cache (Sec. 3.3 cache reuse; Sec. 3.4 fork)
  *   fdd_average_rollouts equal-weight mean of N trajectories            (Sec. 3.4, trajectory averaging)
+ *   fdd_average_rollouts_jmt  the same after jerk-minimising interpolation  (Sec. 3.4)
  *
  * Conventions
  *   - Every tensor is caller-owned.  "device" pointers are CUDA device memory of the
@@ -247,6 +248,21 @@ fdd_status fdd_kv_commit(fdd_ctx* ctx, fdd_forkset* const* sets, int n_sets, int
  */
 fdd_status fdd_average_rollouts(fdd_ctx* ctx, const float* traj, int n, int w, float* out,
                                 void* stream);
+
+/*
+ * fdd_average_rollouts_jmt -- Sec. 3.4: every rollout's trajectory is interpolated to w_out
+ * waypoints by jerk-minimising fitting, then the interpolants are averaged with equal weights.
+ * The paper gives no formula; this library's reading: per coordinate, the curve through the
+ * origin of the vehicle frame at t = 0 and waypoint k at t = k + 1 that minimises the integral
+ * of the squared jerk (the natural quintic spline), sampled at t_j = (j + 1) * w / w_out.
+ *   traj  device fp32 [n][w][2];  out  device fp32 [w_out][2];  n >= 1, 2 <= w <= 32,
+ *   1 <= w_out <= 256 (FDD_ERR_CAPACITY beyond; w = 1 is FDD_ERR_UNSUPPORTED: every curve of
+ *   constant acceleration through two knots has zero jerk, so there is no single minimiser).
+ * The first call for a pair (w, w_out) builds the interpolation matrix on the host, allocates
+ * w_out * w doubles on the device for it and waits for their upload; later calls only launch.
+ */
+fdd_status fdd_average_rollouts_jmt(fdd_ctx* ctx, const float* traj, int n, int w, int w_out,
+                                    float* out, void* stream);
 
 /*
  * fdd_unmask_static -- the unmasking step of fdd_unmask for callers that cannot allocate device

@@ -149,6 +149,7 @@ void fdd_destroy(fdd_ctx* ctx) {
         delete s;
     }
     for (const fdd_ctx::SeedBuf& b : ctx->seed_pool) cudaFree(b.ptr);
+    for (const fdd_ctx::JmtWeights& j : ctx->jmt_weights) cudaFree(j.d_weights);
     if (ctx->d_status) cudaFree(ctx->d_status);
     if (ctx->h_status) cudaFreeHost(ctx->h_status);
     if (ctx->ws_unmask) cudaFree(ctx->ws_unmask);
@@ -471,6 +472,37 @@ fdd_status fdd_average_rollouts(fdd_ctx* ctx, const float* traj, int n, int w, f
     cudaError_t e = launch_average(traj, n, w, out, static_cast<cudaStream_t>(stream));
     ctx->launches += 1;
     if (e != cudaSuccess) return cuda_fail(ctx, e, "fdd_average_rollouts launch");
+    return FDD_OK;
+}
+
+fdd_status fdd_average_rollouts_jmt(fdd_ctx* ctx, const float* traj, int n, int w, int w_out, float* out,
+                                    void* stream) {
+    if (!ctx) return FDD_ERR_INVALID_ARG;
+    if (!traj || !out) return fail(ctx, FDD_ERR_INVALID_ARG, "traj/out is NULL");
+    if (n < 1 || w < 1 || w_out < 1) return fail(ctx, FDD_ERR_INVALID_ARG, "n, w and w_out must be >= 1");
+    if (w < 2) return fail(ctx, FDD_ERR_UNSUPPORTED, "w = 1: two knots do not fix a jerk-minimising curve");
+    if (w > kJmtMaxWaypoints || w_out > kJmtMaxOutputs)
+        return fail(ctx, FDD_ERR_CAPACITY, "w = %d / w_out = %d beyond %d / %d", w, w_out, kJmtMaxWaypoints, kJmtMaxOutputs);
+    const double* d_weights = nullptr;
+    for (const fdd_ctx::JmtWeights& j : ctx->jmt_weights)
+        if (j.w == w && j.w_out == w_out) d_weights = j.d_weights;
+    if (!d_weights) {
+        // first call for this pair of sizes: build the matrix on the host and keep it on the device
+        std::vector<double> weights;
+        if (!jmt_weights(w, w_out, &weights)) return fail(ctx, FDD_ERR_UNSUPPORTED, "spline system is singular");
+        double* d = nullptr;
+        cudaError_t e = cudaMalloc(&d, weights.size() * sizeof(double));
+        if (e == cudaSuccess) e = cudaMemcpy(d, weights.data(), weights.size() * sizeof(double), cudaMemcpyHostToDevice);
+        if (e != cudaSuccess) {
+            if (d) cudaFree(d);
+            return cuda_fail(ctx, e, "fdd_average_rollouts_jmt weights");
+        }
+        ctx->jmt_weights.push_back({w, w_out, d});
+        d_weights = d;
+    }
+    cudaError_t e = launch_average_jmt(traj, n, w, w_out, d_weights, out, static_cast<cudaStream_t>(stream));
+    ctx->launches += 1;
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "fdd_average_rollouts_jmt launch");
     return FDD_OK;
 }
 

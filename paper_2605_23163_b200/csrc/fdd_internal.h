@@ -58,6 +58,8 @@ struct fdd_ctx {
     struct SeedBuf { uint64_t* ptr; int cap; };
     std::vector<SeedBuf> seed_pool;   // device seed buffers of freed fork sets, kept for the next fork
     std::vector<TcMapPoolEntry> map_pool;
+    struct JmtWeights { int w, w_out; double* d_weights; };
+    std::vector<JmtWeights> jmt_weights;   // interpolation matrices built so far (device, fp64 [w_out][w])
 };
 
 struct fdd_forkset {
@@ -96,6 +98,8 @@ struct AttnProblem {
     const int32_t* gate;           // device [N], 0 = leave the rollout out; nullptr = all take part
 };
 
+constexpr int kJmtMaxWaypoints = 32;        // decoded waypoints per rollout the interpolation takes
+constexpr int kJmtMaxOutputs = 256;         // interpolated waypoints
 constexpr int kAttnMaxGatedForks = 2048;    // rollouts of one fdd_block_attn_gated call
 constexpr int kUnmaskMaxSets = 16;          // scenes per unmask launch
 
@@ -146,3 +150,6 @@ cudaError_t launch_kv_commit(const __nv_bfloat16* k_blk, const __nv_bfloat16* v_
                              int n_forks, int d, int n_kv_heads, int head_dim,
                              int suffix_len, int suffix_capacity, cudaStream_t st);
 cudaError_t launch_average(const float* traj, int n, int w, float* out, cudaStream_t st);
+bool jmt_weights(int w, int w_out, std::vector<double>* weights);
+cudaError_t launch_average_jmt(const float* traj, int n, int w, int w_out, const double* d_weights, float* out,
+                               cudaStream_t st);

@@ -20,7 +20,7 @@ FDD_LOGITS_F32, FDD_LOGITS_BF16 = 0, 1
 
 EXPORTS = (
     "fdd_create", "fdd_destroy", "fdd_last_error", "fdd_launch_count", "fdd_fork",
-    "fdd_forkset_free", "fdd_forkset_suffix_len", "fdd_forkset_reset", "fdd_block_attn", "fdd_block_attn_gated",
+    "fdd_forkset_free", "fdd_forkset_suffix_len", "fdd_forkset_reset", "fdd_block_attn", "fdd_block_attn_gated", "fdd_average_rollouts_jmt",
     "fdd_unmask", "fdd_ss_draft", "fdd_ss_accept", "fdd_kv_commit", "fdd_average_rollouts", "fdd_poll_status", "fdd_unmask_static", "fdd_plan_blocks", "fdd_upload_masked_rows",
 )
 FDD_UNMASK_STATIC_MAX_RECORDS = 65536
@@ -83,6 +83,8 @@ def lib():
     L.fdd_kv_commit.restype = i32
     L.fdd_average_rollouts.argtypes = [vp, vp, i32, i32, vp, vp]
     L.fdd_average_rollouts.restype = i32
+    L.fdd_average_rollouts_jmt.argtypes = [vp, vp, i32, i32, i32, vp, vp]
+    L.fdd_average_rollouts_jmt.restype = i32
     L.fdd_poll_status.argtypes = [vp, vp]
     L.fdd_poll_status.restype = i32
     L.fdd_unmask_static.argtypes = [vp, i32, i32, i32, i32, vp, vp, vp, f32, f32, u32, u32, vp, vp, vp, vp,
@@ -243,6 +245,11 @@ def fdd_kv_commit(ctx, sets, layer, k_blk, v_blk, block_len, advance, stream=Non
     return _check(ctx, lib().fdd_kv_commit(
         ctx, _ptr_array(sets), len(sets), int(layer), _ptr(k_blk), _ptr(v_blk),
         _i32_array(block_len), int(advance), _stream(stream)))
+
+
+def fdd_average_rollouts_jmt(ctx, traj, n, w, w_out, out, stream=None):
+    return _check(ctx, lib().fdd_average_rollouts_jmt(ctx, _ptr(traj), int(n), int(w), int(w_out), _ptr(out),
+                                                       _stream(stream)))
 
 
 def fdd_average_rollouts(ctx, traj, n, w, out, stream=None):

@@ -859,6 +859,33 @@ def test_average_cancellation_and_single_rollout():
         fdd.fdd_destroy(ctx)
 
 
+def test_average_after_jerk_minimising_interpolation():
+    # fdd_average_rollouts_jmt against the oracle (every rollout interpolated by the library spline,
+    # then averaged): the paper's 5 waypoints -> 20, the benchmark's 10 -> 40, odd sizes, one rollout,
+    # rollouts that cancel, and the same call twice (the interpolation matrix is built once)
+    from oracle.jmt import average_rollouts_jmt
+    ctx = fdd.fdd_create(4, 1, 64, 64)
+    try:
+        g = np.random.default_rng(21)
+        for n, w, w_out in ((4, 5, 20), (32, 10, 40), (1, 5, 20), (7, 2, 9), (3, 32, 256), (6, 10, 10), (4, 5, 20)):
+            traj = np.cumsum(g.normal([4.0, 0.3], [1.5, 0.8], size=(n, w, 2)), axis=1).astype(np.float32)
+            if n == 6:
+                traj[3:] = -traj[:3] + np.float32(1e-3)            # cancellation: the mean is tiny
+            out = torch.full((w_out, 2), float("nan"), dtype=torch.float32, device="cuda")
+            fdd.fdd_average_rollouts_jmt(ctx, torch.from_numpy(traj).cuda(), n, w, w_out, out)
+            fdd.fdd_poll_status(ctx)
+            got = out.cpu().numpy().astype(np.float64)
+            ref = average_rollouts_jmt(traj, w_out)
+            scale = max(np.abs(ref).max(), 1e-30)
+            assert np.all(np.abs(got - ref) <= 1e-5 * np.maximum(np.abs(ref), 1e-2 * scale)), (n, w, w_out)
+        for bad in ((1, 1, 4), (1, 33, 4), (1, 5, 257)):
+            with pytest.raises(fdd.FddError):
+                fdd.fdd_average_rollouts_jmt(ctx, torch.zeros((bad[0], bad[1], 2), device="cuda"), bad[0], bad[1], bad[2],
+                                             torch.zeros((bad[2], 2), device="cuda"))
+    finally:
+        fdd.fdd_destroy(ctx)
+
+
 def test_upload_masked_rows_copies_exactly_the_rows_that_are_read():
     w = synth.small_variant(synth.workload("tts"), prefix_len=64, vocab=4096, n_forks=3, n_blocks=1)
     sc = w.scenes[0]
