@@ -204,6 +204,24 @@ fdd_status fdd_unmask(fdd_ctx* ctx, fdd_forkset* const* sets, int n_sets, const 
                       int32_t* n_committed, int32_t* n_left, float* conf, void* stream);
 
 /*
+ * fdd_unmask_counted -- fdd_unmask with the denoising step counted on the device.  The step
+ * index enters the noise, so a caller that records one step as a CUDA graph and replays it
+ * (Sec. 4.3 credits part of the deployed speed-up to CUDA graphs) cannot pass it by value.
+ *   step_counter  device uint32: read by the kernels when they run (the step index of this call),
+ *                 incremented by one when the call's work is done.  Set it to 0 at the start of
+ *                 a block (cudaMemsetAsync on the same stream).
+ * Everything else as fdd_unmask with step = *step_counter.  The library's calls allocate nothing
+ * and never synchronise on the paths a step takes (fdd_block_attn[_gated], fdd_unmask[_counted])
+ * once each has run before with the same shapes, so they can be issued while a stream is being
+ * captured.
+ */
+fdd_status fdd_unmask_counted(fdd_ctx* ctx, fdd_forkset* const* sets, int n_sets, const void* logits,
+                              int32_t* tokens, uint8_t* state, const int32_t* block_len,
+                              float threshold, float temperature, uint32_t block_idx,
+                              uint32_t* step_counter, int32_t* n_committed, int32_t* n_left,
+                              float* conf, void* stream);
+
+/*
  * fdd_ss_draft, fdd_ss_accept -- Scaffold Speculative Decoding (Sec. 3.3, Algorithm steps 1-3).
  * Scaffold positions are accepted as they are (step 1: they are never read or written).
  *

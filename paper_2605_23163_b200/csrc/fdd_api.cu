@@ -346,7 +346,8 @@ fdd_status fdd_block_attn_gated(fdd_ctx* ctx, fdd_forkset* const* sets, int n_se
 static fdd_status unmask_like(fdd_ctx* ctx, fdd_forkset* const* sets, int n_sets, const void* logits,
                               int32_t* tokens, uint8_t* state, const int32_t* block_len,
                               float threshold, float temperature, uint32_t block_idx, uint32_t step,
-                              int32_t* n_committed, int32_t* n_left, float* conf, void* stream, int mode) {
+                              int32_t* n_committed, int32_t* n_left, float* conf, void* stream, int mode,
+                              uint32_t* step_counter = nullptr) {
     if (!ctx) return FDD_ERR_INVALID_ARG;
     int total = 0;
     fdd_status st = check_sets(ctx, sets, n_sets, block_len, &total);
@@ -397,6 +398,8 @@ static fdd_status unmask_like(fdd_ctx* ctx, fdd_forkset* const* sets, int n_sets
         p.temperature = temperature;
         p.block_idx = block_idx;
         p.step = step;
+        p.step_counter = step_counter;
+        p.bump_counter = (step_counter != nullptr && s == n_sets) ? 1 : 0;      // the last group of the call advances it
         int n_launches = 0;
         cudaError_t e = launch_unmask(ctx, p, static_cast<cudaStream_t>(stream), &n_launches, mode);
         ctx->launches += n_launches;
@@ -413,6 +416,15 @@ fdd_status fdd_unmask(fdd_ctx* ctx, fdd_forkset* const* sets, int n_sets, const 
                       int32_t* n_committed, int32_t* n_left, float* conf, void* stream) {
     return unmask_like(ctx, sets, n_sets, logits, tokens, state, block_len, threshold, temperature, block_idx, step,
                        n_committed, n_left, conf, stream, 0);
+}
+
+fdd_status fdd_unmask_counted(fdd_ctx* ctx, fdd_forkset* const* sets, int n_sets, const void* logits,
+                              int32_t* tokens, uint8_t* state, const int32_t* block_len,
+                              float threshold, float temperature, uint32_t block_idx, uint32_t* step_counter,
+                              int32_t* n_committed, int32_t* n_left, float* conf, void* stream) {
+    if (ctx && !step_counter) return fail(ctx, FDD_ERR_INVALID_ARG, "step_counter is NULL");
+    return unmask_like(ctx, sets, n_sets, logits, tokens, state, block_len, threshold, temperature, block_idx, 0u,
+                       n_committed, n_left, conf, stream, 0, step_counter);
 }
 
 fdd_status fdd_ss_draft(fdd_ctx* ctx, fdd_forkset* const* sets, int n_sets, const void* logits,

@@ -123,6 +123,8 @@ struct UnmaskProblem {
     int vocab, logits_dtype;
     float threshold, temperature;
     uint32_t block_idx, step;
+    uint32_t* step_counter = nullptr;   // device or nullptr: its value is added to `step` when the kernels run
+    int bump_counter = 0;               // increment it once this launch pair is done
 };
 
 // Unmask scratch: one record per (row, chunk).

@@ -218,7 +218,9 @@ __global__ void __launch_bounds__(kThreads, NOISY ? kNoisyCtasPerSm : 3)
 unmask_partial_kernel(const T* __restrict__ logits, const uint8_t* __restrict__ state,
                       const __grid_constant__ UnmaskSets sets, UnmaskPartial* __restrict__ partial,
                       int vocab, int n_chunks, float temperature,
-                      uint32_t block_idx, uint32_t step, int vec_ok, int select_state) {
+                      uint32_t block_idx, uint32_t step, int vec_ok, int select_state,
+                      const uint32_t* __restrict__ step_counter) {
+    if (step_counter != nullptr) step += *step_counter;    // the denoising step as counted on the device
     const int rows = sets.row_off[sets.n_sets];
     __shared__ uint16_t s_rows[kMaxRows];               // the selected rows (MASKED, or DRAFT for the verifier), ascending
     __shared__ int s_n_rows;
@@ -605,7 +607,10 @@ __global__ void __launch_bounds__(128)
 unmask_finalize_kernel(const UnmaskPartial* __restrict__ partial, int32_t* __restrict__ tokens,
                        uint8_t* __restrict__ state, int32_t* __restrict__ n_committed,
                        int32_t* __restrict__ n_left, float* __restrict__ conf_out,
-                       const __grid_constant__ UnmaskSets sets, int n_chunks, float threshold, int commit_state) {
+                       const __grid_constant__ UnmaskSets sets, int n_chunks, float threshold, int commit_state,
+                       uint32_t* __restrict__ step_bump) {
+    // (the streaming kernel of this call has read the counter; the next call sees it advanced)
+    if (step_bump != nullptr && blockIdx.x == 0 && threadIdx.x == 0) *step_bump += 1u;
     const int fork = blockIdx.x;                        // rollout index over all sets of the call
     const int i = threadIdx.x;
     int set = 0;
@@ -758,21 +763,21 @@ cudaError_t launch_unmask_kernels(const UnmaskProblem& p, UnmaskPartial* partial
         if (p.temperature != 0.0f)
             unmask_partial_kernel<__nv_bfloat16, true><<<grid, kThreads, kRingNoisy, st>>>(
                 static_cast<const __nv_bfloat16*>(p.logits), p.state, p.sets, partial, p.vocab,
-                n_chunks, p.temperature, p.block_idx, p.step, vec_ok, select_state);
+                n_chunks, p.temperature, p.block_idx, p.step, vec_ok, select_state, p.step_counter);
         else
             unmask_partial_kernel<__nv_bfloat16, false><<<grid, kThreads, kRingGreedy, st>>>(
                 static_cast<const __nv_bfloat16*>(p.logits), p.state, p.sets, partial, p.vocab,
-                n_chunks, p.temperature, p.block_idx, p.step, vec_ok, select_state);
+                n_chunks, p.temperature, p.block_idx, p.step, vec_ok, select_state, p.step_counter);
     } else {
         const int vec_ok = (p.vocab % 8 == 0) && (reinterpret_cast<uintptr_t>(p.logits) % 32 == 0);
         if (p.temperature != 0.0f)
             unmask_partial_kernel<float, true><<<grid, kThreads, 0, st>>>(
                 static_cast<const float*>(p.logits), p.state, p.sets, partial, p.vocab,
-                n_chunks, p.temperature, p.block_idx, p.step, vec_ok, select_state);
+                n_chunks, p.temperature, p.block_idx, p.step, vec_ok, select_state, p.step_counter);
         else
             unmask_partial_kernel<float, false><<<grid, kThreads, 0, st>>>(
                 static_cast<const float*>(p.logits), p.state, p.sets, partial, p.vocab,
-                n_chunks, p.temperature, p.block_idx, p.step, vec_ok, select_state);
+                n_chunks, p.temperature, p.block_idx, p.step, vec_ok, select_state, p.step_counter);
     }
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
@@ -780,7 +785,8 @@ cudaError_t launch_unmask_kernels(const UnmaskProblem& p, UnmaskPartial* partial
         ss_accept_kernel<<<forks, 128, 0, st>>>(partial, p.tokens, p.state, p.n_committed, p.n_left, p.sets, n_chunks);
     else
         unmask_finalize_kernel<<<forks, 128, 0, st>>>(partial, p.tokens, p.state, p.n_committed, p.n_left, p.conf,
-                                                     p.sets, n_chunks, p.threshold, mode == 1 ? FDD_DRAFT : FDD_COMMITTED);
+                                                     p.sets, n_chunks, p.threshold, mode == 1 ? FDD_DRAFT : FDD_COMMITTED,
+                                                     p.bump_counter ? p.step_counter : nullptr);
     return cudaGetLastError();
 }
 

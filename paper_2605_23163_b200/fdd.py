@@ -20,7 +20,7 @@ FDD_LOGITS_F32, FDD_LOGITS_BF16 = 0, 1
 
 EXPORTS = (
     "fdd_create", "fdd_destroy", "fdd_last_error", "fdd_launch_count", "fdd_fork",
-    "fdd_forkset_free", "fdd_forkset_suffix_len", "fdd_forkset_reset", "fdd_block_attn", "fdd_block_attn_gated", "fdd_average_rollouts_jmt",
+    "fdd_forkset_free", "fdd_forkset_suffix_len", "fdd_forkset_reset", "fdd_block_attn", "fdd_block_attn_gated", "fdd_average_rollouts_jmt", "fdd_unmask_counted",
     "fdd_unmask", "fdd_ss_draft", "fdd_ss_accept", "fdd_kv_commit", "fdd_average_rollouts", "fdd_poll_status", "fdd_unmask_static", "fdd_plan_blocks", "fdd_upload_masked_rows",
 )
 FDD_UNMASK_STATIC_MAX_RECORDS = 65536
@@ -76,6 +76,8 @@ def lib():
     L.fdd_block_attn_gated.restype = i32
     L.fdd_unmask.argtypes = [vp, vpp, i32, vp, vp, vp, ip, f32, f32, u32, u32, vp, vp, vp, vp]
     L.fdd_unmask.restype = i32
+    L.fdd_unmask_counted.argtypes = [vp, vpp, i32, vp, vp, vp, ip, f32, f32, u32, vp, vp, vp, vp, vp]
+    L.fdd_unmask_counted.restype = i32
     for fn in (L.fdd_ss_draft, L.fdd_ss_accept):
         fn.argtypes = [vp, vpp, i32, vp, vp, vp, ip, f32, u32, u32, vp, vp, vp]
         fn.restype = i32
@@ -224,6 +226,14 @@ def fdd_unmask(ctx, sets, logits, tokens, state, block_len, threshold, temperatu
     return _check(ctx, lib().fdd_unmask(
         ctx, _ptr_array(sets), len(sets), _ptr(logits), _ptr(tokens), _ptr(state),
         _i32_array(block_len), float(threshold), float(temperature), int(block_idx), int(step),
+        _ptr(n_committed), _ptr(n_left), _ptr(conf), _stream(stream)))
+
+
+def fdd_unmask_counted(ctx, sets, logits, tokens, state, block_len, threshold, temperature, block_idx,
+                       step_counter, n_committed, n_left, conf=None, stream=None):
+    return _check(ctx, lib().fdd_unmask_counted(
+        ctx, _ptr_array(sets), len(sets), _ptr(logits), _ptr(tokens), _ptr(state),
+        _i32_array(block_len), float(threshold), float(temperature), int(block_idx), _ptr(step_counter),
         _ptr(n_committed), _ptr(n_left), _ptr(conf), _stream(stream)))
 
 

@@ -800,6 +800,73 @@ def test_pipelined_block_loop_gated_attention_one_step_ahead():
         fdd.fdd_destroy(ctx)
 
 
+def test_step_recorded_as_a_cuda_graph_replays_the_block_loop():
+    # One denoising step (gated attention, unmask with the step counted on the device, copy of the
+    # counts) is recorded once as a CUDA graph and replayed until the block is complete; the result
+    # must be what the same calls give when issued one by one with the step passed by value.
+    w = synth.small_variant(synth.workload("tts"), prefix_len=300, vocab=4096, n_forks=5)
+    sc = w.scenes[0]
+    N, d = sc.n_forks, sc.block_len
+    ctx = harness.create_context(w)
+    try:
+        scene = harness.GpuScene(ctx, w, 0)
+        tokens0, state0 = synth.make_block_template(w, 0, 0)
+        q, k, v = (harness.bf16_tensor(x) for x in synth.make_qkv(w, 0, 0, 0, 0))
+        lg = harness.logits_tensor(w, synth.make_logits(w, 0, 0, 0, rows="all"))   # the same inputs every step
+        scale = 1.0 / np.sqrt(w.head_dim)
+        n_left0 = torch.from_numpy((state0 == MASKED).sum(axis=1).astype(np.int32)).cuda()
+
+        def eager():
+            tokens, state = torch.from_numpy(tokens0).cuda(), torch.from_numpy(state0).cuda()
+            n_left, n_comm = n_left0.clone(), torch.zeros(N, dtype=torch.int32, device="cuda")
+            out = torch.zeros_like(q)
+            trace = []
+            for t in range(d):
+                fdd.fdd_block_attn_gated(ctx, [scene.forkset], 0, q, k, v, out, [d], scale, 0, n_left)
+                fdd.fdd_unmask(ctx, [scene.forkset], lg, tokens, state, [d], w.threshold, w.temperature, 0, t, n_comm, n_left)
+                trace.append((tokens.cpu().numpy(), state.cpu().numpy(), n_left.cpu().numpy(), out.float().cpu().numpy()))
+                if int(n_left.sum()) == 0:
+                    break
+            return trace
+
+        ref = eager()
+        assert 2 <= len(ref) < d
+        # the graph: static buffers, the step index lives in `counter`
+        tokens, state = torch.from_numpy(tokens0).cuda(), torch.from_numpy(state0).cuda()
+        n_left, n_comm = n_left0.clone(), torch.zeros(N, dtype=torch.int32, device="cuda")
+        out = torch.zeros_like(q)
+        counter = torch.zeros(1, dtype=torch.int32, device="cuda")
+        left_host = torch.zeros(N, dtype=torch.int32).pin_memory()
+        fset, dlen = fdd.ptr_array([scene.forkset]), fdd.i32_array([d])
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(side):
+            with torch.cuda.graph(graph, stream=side):
+                fdd.fdd_block_attn_gated(ctx, fset, 0, q, k, v, out, dlen, scale, 0, n_left)
+                fdd.fdd_unmask_counted(ctx, fset, lg, tokens, state, dlen, w.threshold, w.temperature, 0, counter,
+                                       n_comm, n_left)
+                left_host.copy_(n_left, non_blocking=True)
+        torch.cuda.current_stream().wait_stream(side)
+        # capture launches nothing: reset what the block starts from and replay
+        tokens.copy_(torch.from_numpy(tokens0)); state.copy_(torch.from_numpy(state0)); n_left.copy_(n_left0)
+        counter.zero_()
+        for t in range(len(ref)):
+            graph.replay()
+            torch.cuda.synchronize()
+            r_tok, r_st, r_left, r_out = ref[t]
+            assert np.array_equal(tokens.cpu().numpy(), r_tok) and np.array_equal(state.cpu().numpy(), r_st), t
+            assert np.array_equal(left_host.numpy(), r_left) and np.array_equal(n_left.cpu().numpy(), r_left), t
+            live = np.nonzero(ref[t - 1][2] if t else np.ones(N))[0]
+            got_out = out.float().cpu().numpy().reshape(N, -1)
+            assert np.array_equal(got_out[live], r_out.reshape(N, -1)[live]), t
+            assert int(counter.item()) == t + 1
+        assert int(left_host.sum()) == 0
+        fdd.fdd_poll_status(ctx)
+    finally:
+        fdd.fdd_destroy(ctx)
+
+
 def test_tts_full_size_block_loop_sampled_rollouts():
     # the test-time-scaling configuration at full size (8 rollouts, 4096-token prefix, vocabulary
     # 151936, Gumbel noise): the whole loop of one block runs on the GPU; every step the oracle
