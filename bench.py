@@ -30,6 +30,7 @@ UNIT = "tokens/s"
 # summarised in profiles/attn_ptc_long_prefix.md; None for other workloads or once the kernel changed.
 ATTN_DRAM_BYTES_PER_LAUNCH = {"long_prefix": 180.0e6}
 COUNT_STREAM = None  # copy the per-rollout counts to the host on a stream of their own (None: for large steps only)
+GRAPH = False       # replay every denoising step from a CUDA graph (--graph)
 TIME_EVERY = 4      # blocks between two blocks whose kernels are timed one by one
 LOOKAHEAD = True   # enqueue step t + 1 before the host has read the counts of step t (--no-lookahead)
 PRE_STEPS = 6      # distinct per-step input sets kept resident; later steps cycle through them (--pre-steps)
@@ -269,6 +270,69 @@ def run_ours(args):
 
     resident = lambda t: dev_steps[t % PRE_STEPS]
 
+    # ---- the same loop with every denoising step replayed from a CUDA graph (--graph).  A graph holds
+    # the L gated attention calls, the unmask call with the step counted on the device and the copy
+    # of the counts; there is one graph per resident input set (their addresses are part of it).
+    # The fork sets are made once and start every block with fdd_forkset_reset.
+    g_graphs = {}
+    g_period = PRE_STEPS if PRE_STEPS % 2 == 0 else 2 * PRE_STEPS      # input set and host count buffer of step t
+    g_n_left = torch.zeros_like(n_left)
+    g_counter = torch.zeros(1, dtype=torch.int32, device="cuda")
+    g_sets = {"list": None, "arr": None}
+    g_replays = [0]
+    capture_stream = torch.cuda.Stream()
+
+    def graph_of(t):
+        key = t % g_period
+        if key not in g_graphs:
+            q, k, v, lg = resident(t)
+            gph = torch.cuda.CUDAGraph()
+            capture_stream.wait_stream(stream)
+            with torch.cuda.stream(capture_stream):
+                with torch.cuda.graph(gph, stream=capture_stream):
+                    for layer in range(L):
+                        fdd.fdd_block_attn_gated(ctx, g_sets["arr"], layer, q, k, v, out, ds_c, scale, 0, g_n_left)
+                    fdd.fdd_unmask_counted(ctx, g_sets["arr"], lg, tokens, state, ds_c, w.threshold, w.temperature, 0,
+                                           g_counter, n_comm, g_n_left)
+                    n_left_hosts[t % 2].copy_(g_n_left, non_blocking=True)
+            stream.wait_stream(capture_stream)
+            g_graphs[key] = gph
+        return g_graphs[key]
+
+    def decode_block_graph():
+        if g_sets["list"] is None:
+            g_sets["list"] = [fdd.fdd_fork(ctx, *fa) for fa in fork_args]
+            g_sets["arr"] = fdd.ptr_array(g_sets["list"])
+        else:
+            for f_ in g_sets["list"]:
+                fdd.fdd_forkset_reset(ctx, f_)
+        tokens.copy_(tokens0_d, non_blocking=True)
+        state.copy_(state0_d, non_blocking=True)
+        g_n_left.copy_(n_left0_d, non_blocking=True)
+        g_counter.zero_()
+
+        def replay(t):
+            graph_of(t).replay()
+            step_done[t % 2].record(stream)
+            g_replays[0] += 1
+
+        replay(0)
+        t = 0
+        while True:
+            if t + 1 < d:
+                replay(t + 1)
+            step_done[t % 2].synchronize()
+            masked_rows = int(n_left_views[t % 2].sum())
+            t += 1
+            if masked_rows == 0 or t >= d:
+                break
+        _, k, v, _ = resident(t - 1)
+        for layer in range(L):
+            fdd.fdd_kv_commit(ctx, g_sets["arr"], layer, k, v, ds_c, 1 if layer == L - 1 else 0)
+        for i in range(n_scenes):
+            fdd.fdd_average_rollouts(ctx, trajs[i], Ns[i], w.waypoints, traj_out[i])
+        return t
+
     def barrier():
         if dist is not None:
             dist.barrier()
@@ -276,10 +340,14 @@ def run_ours(args):
 
     for _ in range(args.warmup):
         n_denoise = decode_block(resident, False, LOOKAHEAD)
+    if GRAPH:
+        for _ in range(2):                   # records the graphs of the steps a block usually takes
+            decode_block_graph()
     barrier()
     sampler = ClockSampler(local)
     sampler.start()
     launches0 = fdd.fdd_launch_count(ctx)
+    replays0 = g_replays[0]
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     ev0.record(stream)
     denoise_steps = 0
@@ -289,10 +357,15 @@ def run_ours(args):
     for b_ in range(args.steps):
         per_kernel = b_ % TIME_EVERY == 0
         timed_blocks += per_kernel
-        denoise_steps += decode_block(resident, per_kernel, LOOKAHEAD)
+        if GRAPH and not per_kernel:
+            denoise_steps += decode_block_graph()
+        else:
+            denoise_steps += decode_block(resident, per_kernel, LOOKAHEAD)
     ev1.record(stream)
     barrier()
     launches = fdd.fdd_launch_count(ctx) - launches0
+    replays_timed = g_replays[0] - replays0
+    launches += replays_timed * (L + 2)          # a replayed step launches L attention kernels and the unmask pair
     sampler.stop_flag = True
     sampler.join(timeout=2)
     ms = ev0.elapsed_time(ev1)
@@ -379,6 +452,7 @@ def run_ours(args):
                    "l2": "per-step inputs (logits) larger than L2",
                    "step_pipeline": ("attention gated by n_left; step t+1 enqueued before the host reads step t"
                                      if LOOKAHEAD else "attention gated by n_left; one step in flight"),
+                   "steps_from_cuda_graph": bool(GRAPH),
                    "count_copy": "own stream" if use_count_stream else "compute stream",
                    "rollouts_decoding_per_attention_call": float(np.mean([n for _, n in attn_all])) if attn_all else None,
                    "replicas": "independent scene per GPU, no collective"},
@@ -499,7 +573,7 @@ def run_reference(args):
 
 
 def main():
-    global PRE_STEPS, LOOKAHEAD, COUNT_STREAM
+    global PRE_STEPS, LOOKAHEAD, COUNT_STREAM, GRAPH
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=40)
@@ -516,11 +590,14 @@ def main():
                     help="enqueue a denoising step only after the host has read the counts of the one before")
     ap.add_argument("--counts", choices=["auto", "in-line", "own-stream"], default="auto",
                     help="where the per-rollout counts are copied to the host: on the compute stream or on a stream of their own")
+    ap.add_argument("--graph", action="store_true",
+                    help="replay every denoising step from a CUDA graph (blocks whose kernels are timed one by one still run call by call)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     PRE_STEPS = max(1, args.pre_steps)
     LOOKAHEAD = not args.no_lookahead
+    GRAPH = args.graph
     COUNT_STREAM = {"auto": None, "in-line": False, "own-stream": True}[args.counts]
     if args.impl == "reference":
         run_reference(args)
