@@ -111,7 +111,8 @@ struct TcShape {
 // Issue the TMA loads of one 128-key tile of K or V into `dst` (layout [chunk][128 rows][128 B]).
 template <int D>
 __device__ __forceinline__ void load_kv_tile(const SetParams& p, const CUtensorMap* seg_map, const CUtensorMap* tail_map,
-                                             const TileInfo& t, uint32_t dst, uint32_t bar, int h, int f) {
+                                             const TileInfo& t, uint32_t dst, uint32_t bar, int h, int f,
+                                             const int (&pages)[2]) {
     constexpr int kChunks = TcShape<D>::kChunks;
 #pragma unroll
     for (int rh = 0; rh < 2; ++rh) {
@@ -123,15 +124,12 @@ __device__ __forceinline__ void load_kv_tile(const SetParams& p, const CUtensorM
                 if (p.page_tokens == 0) {
                     tc::tma_load_3d(d_addr, seg_map, bar, ch * 64, row0, h);
                 } else {
+                    // pages[rh]: physical page of this half tile, looked up by the caller ahead of time
+                    // (n_phys_pages, one past the pool, for a half tile beyond the prefix: zeros)
                     const int lp = row0 / 64;
                     const int n_pages = (p.prefix_len + 63) / 64;
-                    if (lp < n_pages) {
-                        const int page = p.page_table[lp];
-                        const bool tail = (lp == n_pages - 1) && (p.prefix_len % 64 != 0);
-                        tc::tma_load_4d(d_addr, tail ? tail_map : seg_map, bar, ch * 64, 0, h, page);
-                    } else {
-                        tc::tma_load_4d(d_addr, seg_map, bar, ch * 64, 0, h, p.n_phys_pages);   // past the end: zeros
-                    }
+                    const bool tail = (lp == n_pages - 1) && (p.prefix_len % 64 != 0);
+                    tc::tma_load_4d(d_addr, tail ? tail_map : seg_map, bar, ch * 64, 0, h, pages[rh]);
                 }
             } else if (t.segment == 1) {
                 tc::tma_load_4d(d_addr, seg_map, bar, ch * 64, row0, h, f);
@@ -376,12 +374,23 @@ attn_ptc_kernel(const __grid_constant__ TcArgs<MAXSETS> a) {
                         const uint32_t ph = (n / kStages) & 1;
                         const CUtensorMap* mk = t.segment == 0 ? &maps.pk : (t.segment == 1 ? &maps.sk : &maps.bk);
                         const CUtensorMap* mv = t.segment == 0 ? &maps.pv : (t.segment == 1 ? &maps.sv : &maps.bv);
+                        // the page table is read before the wait for a free stage, so that the lookup
+                        // does not sit between a stage coming free and the copy into it
+                        int pages[2] = {0, 0};
+                        if (t.segment == 0 && p.page_tokens != 0) {
+                            const int n_pages = (p.prefix_len + 63) / 64;
+#pragma unroll
+                            for (int rh = 0; rh < 2; ++rh) {
+                                const int lp = t.index * 2 + rh;
+                                pages[rh] = lp < n_pages ? __ldg(p.page_table + lp) : p.n_phys_pages;
+                            }
+                        }
                         ok = tc::mbar_wait(tc::smem_u32(&bar_k_empty[s]), ph ^ 1, abort_flag, kWaitLimit);
                         ok = __shfl_sync(0xFFFFFFFFu, ok ? 1 : 0, 0) != 0;
                         if (!ok) break;
                         if (tc::elect_one()) {
                             tc::mbar_arrive_expect_tx(tc::smem_u32(&bar_k_full[s]), Shape::kTileBytes);
-                            load_kv_tile<D>(p, mk, &maps.pk_tail, t, k_s + s * Shape::kTileBytes, tc::smem_u32(&bar_k_full[s]), v.h, v.f);
+                            load_kv_tile<D>(p, mk, &maps.pk_tail, t, k_s + s * Shape::kTileBytes, tc::smem_u32(&bar_k_full[s]), v.h, v.f, pages);
                         }
                         __syncwarp();
                         ok = tc::mbar_wait(tc::smem_u32(&bar_v_empty[s]), ph ^ 1, abort_flag, kWaitLimit);
@@ -389,7 +398,7 @@ attn_ptc_kernel(const __grid_constant__ TcArgs<MAXSETS> a) {
                         if (!ok) break;
                         if (tc::elect_one()) {
                             tc::mbar_arrive_expect_tx(tc::smem_u32(&bar_v_full[s]), Shape::kTileBytes);
-                            load_kv_tile<D>(p, mv, &maps.pv_tail, t, v_s + s * Shape::kTileBytes, tc::smem_u32(&bar_v_full[s]), v.h, v.f);
+                            load_kv_tile<D>(p, mv, &maps.pv_tail, t, v_s + s * Shape::kTileBytes, tc::smem_u32(&bar_v_full[s]), v.h, v.f, pages);
                         }
                         __syncwarp();
                     }
