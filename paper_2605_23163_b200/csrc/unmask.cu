@@ -103,25 +103,6 @@ __device__ __forceinline__ float ex2_fast(float x) {
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
 }
-// two fp32 values in one 64-bit register for the packed fp32x2 instructions of sm_100
-__device__ __forceinline__ uint64_t pack2(float lo, float hi) {
-    uint64_t d;
-    asm("mov.b64 %0, {%1, %2};" : "=l"(d) : "f"(lo), "f"(hi));
-    return d;
-}
-__device__ __forceinline__ void unpack2(uint64_t v, float& lo, float& hi) {
-    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
-}
-__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
-    uint64_t d;
-    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
-    return d;
-}
-__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
-    uint64_t d;
-    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
-    return d;
-}
 __device__ __forceinline__ float max3f(float a, float b, float c) {
     float d;
     asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
@@ -334,16 +315,16 @@ unmask_partial_kernel(const T* __restrict__ logits, const uint8_t* __restrict__ 
                 }
                 const float mn = fmaxf(m, gm);
                 const float mnl = mn * kLog2e;
-                const uint64_t l2e2 = pack2(kLog2e, kLog2e), nm2 = pack2(-mnl, -mnl);
-                uint64_t s2[2] = {0ull, 0ull};
+                // packed fp32x2 arithmetic: one FMA and one add per two logits
+                const float2 l2e2 = make_float2(kLog2e, kLog2e), nm2 = make_float2(-mnl, -mnl);
+                float2 s2[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
 #pragma unroll
                 for (int i = 0; i < kGroup; i += 2) {
-                    float x0, x1;
-                    unpack2(fma2(pack2(val[i], val[i + 1]), l2e2, nm2), x0, x1);
-                    s2[(i >> 1) & 1] = add2(s2[(i >> 1) & 1], pack2(ex2_fast(x0), ex2_fast(x1)));
+                    const float2 x = __ffma2_rn(make_float2(val[i], val[i + 1]), l2e2, nm2);
+                    s2[(i >> 1) & 1] = __fadd2_rn(s2[(i >> 1) & 1], make_float2(ex2_fast(x.x), ex2_fast(x.y)));
                 }
-                float sa, sb;
-                unpack2(add2(s2[0], s2[1]), sa, sb);
+                const float2 s01 = __fadd2_rn(s2[0], s2[1]);
+                const float sa = s01.x, sb = s01.y;
                 // rescale by 2^((m - mn) log2e): exactly 1 while the maximum stands (the rounded mnl must
                 // not enter here, or a factor 1 + 1e-7 would compound over the groups)
                 s = s * ex2_fast((m - mn) * kLog2e) + (sa + sb);
