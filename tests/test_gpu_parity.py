@@ -104,6 +104,16 @@ def test_attention_long_prefix_two_rollouts_left_units_cut_into_many_pieces():
         fdd.fdd_destroy(ctx)
 
 
+@pytest.mark.parametrize("prefix_len", [2100, 4096, 10000])
+def test_attention_head_dim_64_single_unit_cut_into_pieces(prefix_len):
+    # head dimension 64 with one rollout and one KV head: a single unit of 18 / 33 / 80 key tiles,
+    # cut into 2 / 4 / 10 pieces, so each branch of the merge (by piece count) runs at D = 64 too
+    sc = synth.Scene(prefix_len=prefix_len, n_forks=1, block_len=16, n_scaffold=4, n_blocks=1)
+    w = synth.Workload("d64_split", 4, 1, 64, 256, "f32", "normal_sigma2", 0.9, 0.0, (sc,), qkv_sigma=0.35, seed=50 + prefix_len)
+    _attention_case(w)
+    _attention_case(w, causal=True)
+
+
 def test_attention_no_prefix_and_single_position():
     w = synth.workload("tiny")
     sc = synth.Scene(prefix_len=0, n_forks=2, block_len=1, n_scaffold=0, n_blocks=2)
