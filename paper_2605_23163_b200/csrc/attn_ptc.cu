@@ -9,8 +9,10 @@
 // tile steps that is cut into equal contiguous ranges, one per CTA.  A CTA walks its range item
 // by item (item = the part of one unit inside the range).  A unit that lies inside one range is
 // written directly; a unit cut by a range border leaves normalised fp32 partials plus their
-// log-sum-exp in scratch, and whichever CTA finishes its piece last (an atomic counter per unit,
-// nobody waits) merges the pieces and writes the bf16 rows.
+// log-sum-exp in scratch.  Once a CTA is through its range it takes its share of the merges of the
+// (at most two) cut units it holds a piece of: it waits until all pieces of the unit are written
+// (a counter per unit; the launch is cooperative, so the CTAs it waits for are running; the wait is
+// bounded) and merges an equal share of the unit's rows into the bf16 output.
 //
 // Warp roles (384 threads): warps 0-3 and 4-7 are the two soft-max groups (thread = one query
 // row = one TMEM lane), warp 8 lane 0 drives TMA, warps 9 and 10 issue the tcgen05.mma (one lane each:
@@ -43,7 +45,7 @@ constexpr int kTcThreads = 384;
 constexpr int kKeysPerTile = 128;
 constexpr long long kWaitLimit = 4000000000LL;   // about two seconds of SM clocks
 constexpr int kMaxGatedForks = kAttnMaxGatedForks;   // rollouts of one launch when any scene has a gate
-constexpr int kMinTilesPerCta = 8;               // do not cut the work finer than this (every cut costs a merge)
+constexpr int kMinTilesPerCta = 4;               // do not cut the work finer than this (every cut costs a piece to write and merge)
 // Registers per thread after the hand-over.  The CTA starts with 384 x 168; 8 soft-max warps x
 // kRegsSoftmax + 4 other warps x kRegsOther must not exceed that (2 * 208 + 88 = 3 * 168).
 constexpr int kRegsSoftmax = 208;
@@ -69,7 +71,8 @@ struct TcArgs {
     SetParams sets[MAXSETS];
     float* part_o;             // [2 * ctas][D / 4][256] float4: normalised partial outputs, column-major per slot
     float* part_lse;           // [2 * ctas][256] log2-domain log-sum-exp of the partial
-    int* unit_count;           // pieces finished per unit (self-resetting)
+    int* unit_count;           // [2][max_units]: pieces written per unit, CTAs done with the unit's merge (self-resetting)
+    int max_units;
     int* status;
     int min_tiles;             // do not cut the work into ranges shorter than this
     int n_sets;
@@ -173,52 +176,54 @@ constexpr float kPoly2 = 0.2426108568906784f * kPolyScale;
 constexpr float kPoly3 = 0.055171459913253784f * kPolyScale;
 constexpr float kRoundMagic = 12582912.0f;                    // 1.5 * 2^23: adding it rounds to an integer
 
-// Merge of a unit cut between CTAs, one output row:  out = sum_k w_k O_k,  w_k = 2^(lse_k - M) / sum.
-// Partials lie column-major in their slots ([D / 4][256 rows] float4).  CB columns x 32 / CB pieces
-// are read per round trip.
-template <int D, int CB>
-__device__ __forceinline__ void merge_row(const float* part_o, const float* part_lse, const int* slot_s, int n_pieces,
-                                          int row, float M, float inv_wsum, __nv_bfloat16* op) {
+// Merge of a unit cut between CTAs:  out = sum_k w_k O_k,  w_k = 2^(lse_k - M) / sum_j 2^(lse_j - M).
+// Every CTA that holds a piece merges an equal share of the unit's rows.  A thread takes CT float4
+// columns of one row: 32 / CT pieces are read per round trip, 32 independent 16-byte reads in flight.
+// Partials lie column-major in their slots ([D / 4][256 rows] float4).
+template <int D, int CT>
+__device__ __forceinline__ void merge_columns(const float* part_o, const float* part_lse, const int* slot_s, int n_pieces,
+                                              int row, int col0, float M, float inv_wsum, __nv_bfloat16* op) {
     constexpr int NC4 = D / 4;
-    constexpr int CBE = CB < NC4 ? CB : NC4;        // columns per batch
-    constexpr int PC = 32 / CBE;                    // pieces per chunk
+    constexpr int PC = 32 / CT;                     // pieces per chunk
     const float4* po4 = reinterpret_cast<const float4*>(part_o);
-    for (int c0 = 0; c0 < NC4; c0 += CBE) {
-        float4 acc[CBE];
+    float4 acc[CT];
 #pragma unroll
-        for (int c = 0; c < CBE; ++c) acc[c] = make_float4(0.f, 0.f, 0.f, 0.f);
-        for (int k0 = 0; k0 < n_pieces; k0 += PC) {
-            float ls[PC];
-            float4 ov[PC][CBE];
+    for (int c = 0; c < CT; ++c) acc[c] = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int k0 = 0; k0 < n_pieces; k0 += PC) {
+        float ls[PC];
+        float4 ov[PC][CT];
 #pragma unroll
-            for (int k = 0; k < PC; ++k) {
-                const bool live = k0 + k < n_pieces;
-                const size_t slot = slot_s[min(k0 + k, n_pieces - 1)];
-                ls[k] = live ? __ldcg(part_lse + slot * 256 + row) : -CUDART_INF_F;
+        for (int k = 0; k < PC; ++k) {
+            const bool live = k0 + k < n_pieces;
+            const size_t slot = slot_s[min(k0 + k, n_pieces - 1)];
+            ls[k] = live ? __ldcg(part_lse + slot * 256 + row) : -CUDART_INF_F;
 #pragma unroll
-                for (int c = 0; c < CBE; ++c)
-                    ov[k][c] = live ? __ldcg(po4 + (slot * NC4 + c0 + c) * 256 + row) : make_float4(0.f, 0.f, 0.f, 0.f);
-            }
-#pragma unroll
-            for (int k = 0; k < PC; ++k) {
-                const float wgt = exp2f(ls[k] - M) * inv_wsum;      // 0 for a piece that is not there
-#pragma unroll
-                for (int c = 0; c < CBE; ++c) {
-                    acc[c].x = fmaf(wgt, ov[k][c].x, acc[c].x); acc[c].y = fmaf(wgt, ov[k][c].y, acc[c].y);
-                    acc[c].z = fmaf(wgt, ov[k][c].z, acc[c].z); acc[c].w = fmaf(wgt, ov[k][c].w, acc[c].w);
-                }
-            }
+            for (int c = 0; c < CT; ++c)
+                ov[k][c] = live ? __ldcg(po4 + (slot * NC4 + col0 + c) * 256 + row) : make_float4(0.f, 0.f, 0.f, 0.f);
         }
 #pragma unroll
-        for (int c = 0; c < CBE; c += 2) {
-            const __nv_bfloat162 b0 = __floats2bfloat162_rn(acc[c].x, acc[c].y), b1 = __floats2bfloat162_rn(acc[c].z, acc[c].w);
-            const __nv_bfloat162 b2 = __floats2bfloat162_rn(acc[c + 1].x, acc[c + 1].y), b3 = __floats2bfloat162_rn(acc[c + 1].z, acc[c + 1].w);
-            *reinterpret_cast<uint4*>(op + (c0 + c) * 4) =
-                make_uint4(*reinterpret_cast<const uint32_t*>(&b0), *reinterpret_cast<const uint32_t*>(&b1),
-                           *reinterpret_cast<const uint32_t*>(&b2), *reinterpret_cast<const uint32_t*>(&b3));
+        for (int k = 0; k < PC; ++k) {
+            const float wgt = exp2f(ls[k] - M) * inv_wsum;          // 0 for a piece that is not there
+#pragma unroll
+            for (int c = 0; c < CT; ++c) {
+                acc[c].x = fmaf(wgt, ov[k][c].x, acc[c].x); acc[c].y = fmaf(wgt, ov[k][c].y, acc[c].y);
+                acc[c].z = fmaf(wgt, ov[k][c].z, acc[c].z); acc[c].w = fmaf(wgt, ov[k][c].w, acc[c].w);
+            }
         }
     }
+#pragma unroll
+    for (int c = 0; c < CT; ++c) {
+        const __nv_bfloat162 b0 = __floats2bfloat162_rn(acc[c].x, acc[c].y), b1 = __floats2bfloat162_rn(acc[c].z, acc[c].w);
+        *reinterpret_cast<uint2*>(op + (col0 + c) * 4) =
+            make_uint2(*reinterpret_cast<const uint32_t*>(&b0), *reinterpret_cast<const uint32_t*>(&b1));
+    }
 }
+
+// A unit whose merge this CTA takes part in once its range is done.
+struct Deferred {
+    int s, unit, f, rp, h, c_first, n_pieces, gu;
+    long long unit_begin;
+};
 
 template <int D, int MAXSETS, int EMU>
 __global__ void __launch_bounds__(kTcThreads, 1)
@@ -235,7 +240,8 @@ attn_ptc_kernel(const __grid_constant__ TcArgs<MAXSETS> a) {
     __shared__ __align__(8) unsigned long long bar_q_full, bar_k_full[kStages], bar_k_empty[kStages],
         bar_v_full[kStages], bar_v_empty[kStages], bar_s_full[2], bar_s_free[2], bar_p_full[2], bar_o_done[2], bar_item_done;
     __shared__ uint32_t tmem_base_s;
-    __shared__ int abort_s, last_s;
+    __shared__ int abort_s, n_deferred_s;
+    __shared__ Deferred deferred_s[2];                  // a range starts and ends inside at most one cut unit each
     constexpr int kMaxPieces = 160;                     // a unit is cut by CTA borders: at most one piece per CTA
     __shared__ int slot_s[kMaxPieces];                  // scratch slot of every piece of the unit being merged
     volatile int* abort_flag = &abort_s;
@@ -285,7 +291,7 @@ attn_ptc_kernel(const __grid_constant__ TcArgs<MAXSETS> a) {
 
     if (tid == 0) {
         abort_s = 0;
-        last_s = 0;
+        n_deferred_s = 0;
         tc::mbar_init(tc::smem_u32(&bar_q_full), 1);
         tc::mbar_init(tc::smem_u32(&bar_item_done), 1);
         for (int s = 0; s < kStages; ++s) {
@@ -738,52 +744,15 @@ attn_ptc_kernel(const __grid_constant__ TcArgs<MAXSETS> a) {
                 __threadfence();
                 tc::named_barrier(1, 256);
                 if (tid == 0) {
+                    // the piece is written: count it, and note the unit for this CTA's share of its
+                    // merge, which follows once the whole range is done (waiting here, in the middle
+                    // of the range, would chain every CTA behind its neighbour)
                     const int gu = unit_base_s[it.s] + it.unit;
-                    const int old = atomicAdd(a.unit_count + gu, 1);
-                    const int last = old == n_pieces - 1;
-                    if (last) a.unit_count[gu] = 0;          // every piece has arrived: ready for the next launch
-                    last_s = last;
-                }
-                tc::named_barrier(1, 256);
-                if (last_s) {
-                    // This CTA finished the unit's last outstanding piece: merge all of them.
-                    //   out = sum_s w_s O_s / sum_s w_s,  w_s = 2^(lse_s - max lse)
-                    __threadfence();
-                    // Thread = row, as in the writer (tid = q * 128 + row_local is the row inside the unit).
-                    // First the row's weights: M = max lse, 1 / sum 2^(lse - M), the log-sum-exps read eight
-                    // at a time.  Then the columns, in batches sized so that 32 independent 16-byte reads
-                    // are in flight per thread whatever the number of pieces.
-                    if (tid < n_pieces && tid < kMaxPieces) {
-                        const int pc = c_first + tid;
-                        slot_s[tid] = pc * 2 + (it.unit_begin <= T * pc / C ? 0 : 1);
-                    }
-                    tc::named_barrier(1, 256);
-                    if (row_ok) {
-                        float M = -CUDART_INF_F, wsum = 0.0f;
-                        for (int k0 = 0; k0 < n_pieces; k0 += 8) {
-                            float ls[8];
-#pragma unroll
-                            for (int k = 0; k < 8; ++k)
-                                ls[k] = k0 + k < n_pieces ? __ldcg(a.part_lse + static_cast<size_t>(slot_s[min(k0 + k, n_pieces - 1)]) * 256 + tid)
-                                                          : -CUDART_INF_F;
-                            float mc = ls[0];
-#pragma unroll
-                            for (int k = 1; k < 8; ++k) mc = fmaxf(mc, ls[k]);
-                            const float mn = fmaxf(M, mc);
-                            if (mn > -CUDART_INF_F) {
-                                wsum *= exp2f(M - mn);                  // 0 the first time (M = -inf)
-#pragma unroll
-                                for (int k = 0; k < 8; ++k) wsum += exp2f(ls[k] - mn);
-                                M = mn;
-                            }
-                        }
-                        if (!(M > -CUDART_INF_F)) M = 0.0f;
-                        const float iw = wsum > 0.0f ? 1.0f / wsum : 0.0f;
-                        __nv_bfloat16* op = p.out + ((static_cast<size_t>(f) * p.d + qi) * p.n_q_heads + h * p.G + qg) * D;
-                        if (n_pieces <= 2) merge_row<D, 16>(a.part_o, a.part_lse, slot_s, n_pieces, tid, M, iw, op);
-                        else if (n_pieces <= 4) merge_row<D, 8>(a.part_o, a.part_lse, slot_s, n_pieces, tid, M, iw, op);
-                        else merge_row<D, 4>(a.part_o, a.part_lse, slot_s, n_pieces, tid, M, iw, op);
-                    }
+                    atomicAdd(a.unit_count + gu, 1);
+                    Deferred& dfr = deferred_s[n_deferred_s++];
+                    dfr.s = it.s; dfr.unit = it.unit; dfr.f = f; dfr.rp = rp; dfr.h = h;
+                    dfr.c_first = c_first; dfr.n_pieces = n_pieces; dfr.gu = gu;
+                    dfr.unit_begin = it.unit_begin;
                 }
             }
             if (!ok) {
@@ -794,6 +763,89 @@ attn_ptc_kernel(const __grid_constant__ TcArgs<MAXSETS> a) {
             ++item_cnt;
             pos += nt;
             if (!end_of_item()) break;
+        }
+
+        // ------------------------------------------------------------ merges of the cut units
+        // Every CTA that holds a piece of a unit merges an equal share of the unit's rows, once all
+        // pieces are there.  (All CTAs of the launch are resident at once: the wait is for CTAs
+        // that are running, and it is bounded like every other wait.)
+        tc::named_barrier(1, 256);
+        const int n_deferred = *abort_flag ? 0 : n_deferred_s;
+        for (int e = 0; e < n_deferred; ++e) {
+            const Deferred dfr = deferred_s[e];
+            const SetParams& p = a.sets[dfr.s];
+            const int n_pieces = dfr.n_pieces;
+            if (tid == 0) {
+                const long long t0 = clock64();
+                volatile int* arrived = a.unit_count + dfr.gu;
+                while (*arrived < n_pieces) {
+                    if (clock64() - t0 > kWaitLimit) {
+                        atomicCAS(a.status, 0, FDD_ERR_DEVICE_TIMEOUT);
+                        *abort_flag = 1;
+                        break;
+                    }
+                }
+            }
+            if (tid < n_pieces && tid < kMaxPieces) {
+                const int pc = dfr.c_first + tid;
+                slot_s[tid] = pc * 2 + (dfr.unit_begin <= T * pc / C ? 0 : 1);
+            }
+            tc::named_barrier(1, 256);
+            if (*abort_flag) break;
+            __threadfence();
+            // this CTA's share of the rows; a row is split between `col_groups` threads
+            const int rows_here = min(256, p.R - dfr.rp * 256);
+            const int mine = static_cast<int>(blockIdx.x) - dfr.c_first;
+            const int row_lo = rows_here * mine / n_pieces, row_hi = rows_here * (mine + 1) / n_pieces;
+            const int share = row_hi - row_lo;
+            int col_groups = 1;                                   // a power of two, share * col_groups <= 256
+            while (col_groups < D / 4 && share * col_groups * 2 <= 256) col_groups *= 2;
+            const int ct = (D / 4) / col_groups;                  // float4 columns per thread
+            const int row_in_share = tid / col_groups, cg = tid - row_in_share * col_groups;
+            if (share > 0 && row_in_share < share) {
+                const int rowu = row_lo + row_in_share;
+                float M = -CUDART_INF_F, wsum = 0.0f;
+                for (int k0 = 0; k0 < n_pieces; k0 += 8) {
+                    float ls[8];
+#pragma unroll
+                    for (int k = 0; k < 8; ++k)
+                        ls[k] = k0 + k < n_pieces ? __ldcg(a.part_lse + static_cast<size_t>(slot_s[min(k0 + k, n_pieces - 1)]) * 256 + rowu)
+                                                  : -CUDART_INF_F;
+                    float mc = ls[0];
+#pragma unroll
+                    for (int k = 1; k < 8; ++k) mc = fmaxf(mc, ls[k]);
+                    const float mn = fmaxf(M, mc);
+                    if (mn > -CUDART_INF_F) {
+                        wsum *= exp2f(M - mn);                  // 0 the first time (M = -inf)
+#pragma unroll
+                        for (int k = 0; k < 8; ++k) wsum += exp2f(ls[k] - mn);
+                        M = mn;
+                    }
+                }
+                if (!(M > -CUDART_INF_F)) M = 0.0f;
+                const float iw = wsum > 0.0f ? 1.0f / wsum : 0.0f;
+                const int r = dfr.rp * 256 + rowu;
+                const int qi2 = r / p.G, qg2 = r - qi2 * p.G;
+                __nv_bfloat16* op = p.out + ((static_cast<size_t>(dfr.f) * p.d + qi2) * p.n_q_heads + dfr.h * p.G + qg2) * D;
+                const int col0 = cg * ct;
+                switch (ct) {
+                    case 1: merge_columns<D, 1>(a.part_o, a.part_lse, slot_s, n_pieces, rowu, col0, M, iw, op); break;
+                    case 2: merge_columns<D, 2>(a.part_o, a.part_lse, slot_s, n_pieces, rowu, col0, M, iw, op); break;
+                    case 4: merge_columns<D, 4>(a.part_o, a.part_lse, slot_s, n_pieces, rowu, col0, M, iw, op); break;
+                    case 8: merge_columns<D, 8>(a.part_o, a.part_lse, slot_s, n_pieces, rowu, col0, M, iw, op); break;
+                    case 16: merge_columns<D, 16>(a.part_o, a.part_lse, slot_s, n_pieces, rowu, col0, M, iw, op); break;
+                    default: merge_columns<D, 32>(a.part_o, a.part_lse, slot_s, n_pieces, rowu, col0, M, iw, op); break;
+                }
+            }
+            tc::named_barrier(1, 256);
+            if (tid == 0) {
+                // the last CTA to finish its share leaves both counters at zero for the next launch
+                int* done = a.unit_count + a.max_units + dfr.gu;
+                if (atomicAdd(done, 1) == n_pieces - 1) {
+                    *done = 0;
+                    a.unit_count[dfr.gu] = 0;
+                }
+            }
         }
     }
 
@@ -900,8 +952,11 @@ cudaError_t launch_one(const TcArgs<MAXSETS>& args, unsigned ctas, cudaStream_t 
         if (e != cudaSuccess) return e;
         configured = true;
     }
-    attn_ptc_kernel<D, MAXSETS, EMU><<<ctas, kTcThreads, smem, st>>>(args);
-    return cudaGetLastError();
+    // The CTAs wait for one another's pieces at the end: a cooperative launch makes the runtime
+    // guarantee that all of them are resident at once (or fail the launch).
+    void* params[] = {const_cast<TcArgs<MAXSETS>*>(&args)};
+    return cudaLaunchCooperativeKernel(reinterpret_cast<const void*>(&attn_ptc_kernel<D, MAXSETS, EMU>), dim3(ctas),
+                                       dim3(kTcThreads), params, static_cast<size_t>(smem), st);
 }
 
 template <int MAXSETS>
@@ -960,6 +1015,7 @@ cudaError_t launch_group(fdd_ctx* ctx, const AttnProblem* probs, TcMapCache* con
     args.part_o = static_cast<float*>(ctx->ws_attn);
     args.part_lse = args.part_o + static_cast<size_t>(2) * ctx->attn_max_ctas * 256 * head_dim;
     args.unit_count = ctx->attn_unit_count;
+    args.max_units = ctx->attn_max_units;
     args.status = ctx->d_status;
     args.min_tiles = min_tiles;
     args.n_sets = n;

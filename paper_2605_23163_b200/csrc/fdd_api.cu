@@ -131,8 +131,9 @@ fdd_status fdd_create(const fdd_config* cfg, fdd_ctx** out) {
         const int G = cfg->n_q_heads / cfg->n_kv_heads;
         const int row_pairs = (cfg->max_block * G + 255) / 256;
         ctx->attn_max_units = cfg->n_kv_heads * row_pairs * cfg->max_forks;
-        e = cudaMalloc(&ctx->attn_unit_count, sizeof(int) * ctx->attn_max_units);
-        if (e == cudaSuccess) e = cudaMemset(ctx->attn_unit_count, 0, sizeof(int) * ctx->attn_max_units);
+        // two counters per unit: pieces written, CTAs done with their share of the merge
+        e = cudaMalloc(&ctx->attn_unit_count, sizeof(int) * 2 * ctx->attn_max_units);
+        if (e == cudaSuccess) e = cudaMemset(ctx->attn_unit_count, 0, sizeof(int) * 2 * ctx->attn_max_units);
     }
     if (e != cudaSuccess) {
         fdd_destroy(ctx);
@@ -553,7 +554,7 @@ fdd_status fdd_poll_status(fdd_ctx* ctx, void* stream) {
     const int code = *ctx->h_status;
     if (code != FDD_OK) {
         // a kernel that gave up may have left piece counters of the attention merge half counted
-        cudaMemsetAsync(ctx->attn_unit_count, 0, sizeof(int) * ctx->attn_max_units, st);
+        cudaMemsetAsync(ctx->attn_unit_count, 0, sizeof(int) * 2 * ctx->attn_max_units, st);
         cudaStreamSynchronize(st);
         return fail(ctx, code, "a kernel recorded device status %d", code);
     }

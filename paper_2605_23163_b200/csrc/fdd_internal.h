@@ -49,7 +49,7 @@ struct fdd_ctx {
     size_t ws_unmask_bytes = 0;
     void* ws_attn = nullptr;          // partial outputs of attention units cut between CTAs
     size_t ws_attn_bytes = 0;
-    int* attn_unit_count = nullptr;   // device [attn_max_units]: finished pieces per unit (self-resetting)
+    int* attn_unit_count = nullptr;   // device [2][attn_max_units]: pieces written / merge shares done per unit (self-resetting)
     int attn_max_units = 0;
     int attn_max_ctas = 0;
     uint64_t launches = 0;
