@@ -137,6 +137,9 @@ fdd_status fdd_forkset_reset(fdd_ctx* ctx, fdd_forkset* set);
  *   out            device bf16, same packing and shape as q.
  *   block_len      host int32 [n_sets]: d_s, 1 <= d_s <= cfg.max_block.
  *   scale          soft-max scale (1/sqrt(D) by convention), the same for every set of the call.
+ * The tensor-core kernel is launched cooperatively (its CTAs wait, with a bound, for one another's
+ * partial results): it needs as many free SMs as it has CTAs, and the launch fails with
+ * FDD_ERR_CUDA where the device cannot give them (an MPS share of the SMs, for instance).
  * All sets of a call go into one launch (groups of 16 sets).  Rollouts with equal inputs agree
  * up to the rounding of the bf16 output, not bit for bit: where a unit of work is cut between
  * CTAs depends on its place in the call.

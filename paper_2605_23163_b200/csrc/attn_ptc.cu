@@ -9,10 +9,11 @@
 // tile steps that is cut into equal contiguous ranges, one per CTA.  A CTA walks its range item
 // by item (item = the part of one unit inside the range).  A unit that lies inside one range is
 // written directly; a unit cut by a range border leaves normalised fp32 partials plus their
-// log-sum-exp in scratch.  Once a CTA is through its range it takes its share of the merges of the
-// (at most two) cut units it holds a piece of: it waits until all pieces of the unit are written
-// (a counter per unit; the launch is cooperative, so the CTAs it waits for are running; the wait is
-// bounded) and merges an equal share of the unit's rows into the bf16 output.
+// log-sum-exp in scratch.  A unit in two pieces is merged at once by whichever CTA writes its piece
+// second (a counter per unit, nobody waits).  A unit in more pieces is merged by all its piece
+// holders together: once a CTA is through its range it waits until all pieces of the unit are
+// written (the launch is cooperative, so the CTAs it waits for are running; the wait is bounded)
+// and merges an equal share of the unit's rows into the bf16 output.
 //
 // Warp roles (384 threads): warps 0-3 and 4-7 are the two soft-max groups (thread = one query
 // row = one TMEM lane), warp 8 lane 0 drives TMA, warps 9 and 10 issue the tcgen05.mma (one lane each:
@@ -240,7 +241,7 @@ attn_ptc_kernel(const __grid_constant__ TcArgs<MAXSETS> a) {
     __shared__ __align__(8) unsigned long long bar_q_full, bar_k_full[kStages], bar_k_empty[kStages],
         bar_v_full[kStages], bar_v_empty[kStages], bar_s_full[2], bar_s_free[2], bar_p_full[2], bar_o_done[2], bar_item_done;
     __shared__ uint32_t tmem_base_s;
-    __shared__ int abort_s, n_deferred_s;
+    __shared__ int abort_s, n_deferred_s, last_s;
     __shared__ Deferred deferred_s[2];                  // a range starts and ends inside at most one cut unit each
     constexpr int kMaxPieces = 160;                     // a unit is cut by CTA borders: at most one piece per CTA
     __shared__ int slot_s[kMaxPieces];                  // scratch slot of every piece of the unit being merged
@@ -743,10 +744,38 @@ attn_ptc_kernel(const __grid_constant__ TcArgs<MAXSETS> a) {
                 }
                 __threadfence();
                 tc::named_barrier(1, 256);
-                if (tid == 0) {
-                    // the piece is written: count it, and note the unit for this CTA's share of its
-                    // merge, which follows once the whole range is done (waiting here, in the middle
-                    // of the range, would chain every CTA behind its neighbour)
+                if (n_pieces == 2) {
+                    // Two pieces: whichever of the two CTAs writes its piece second merges the unit
+                    // at once; nobody waits.
+                    if (tid == 0) {
+                        const int gu = unit_base_s[it.s] + it.unit;
+                        const int last = atomicAdd(a.unit_count + gu, 1) == 1;
+                        if (last) a.unit_count[gu] = 0;          // both pieces are there: ready for the next launch
+                        last_s = last;
+                        slot_s[0] = c_first * 2 + (it.unit_begin <= T * c_first / C ? 0 : 1);
+                        slot_s[1] = (c_first + 1) * 2;           // the second piece starts its CTA's range
+                    }
+                    tc::named_barrier(1, 256);
+                    if (last_s) {
+                        __threadfence();
+                        if (row_ok) {                            // thread = row
+                            const float l0 = __ldcg(a.part_lse + static_cast<size_t>(slot_s[0]) * 256 + tid);
+                            const float l1 = __ldcg(a.part_lse + static_cast<size_t>(slot_s[1]) * 256 + tid);
+                            float M = fmaxf(l0, l1);
+                            if (!(M > -CUDART_INF_F)) M = 0.0f;
+                            const float wsum = exp2f(l0 - M) + exp2f(l1 - M);
+                            const float iw = wsum > 0.0f ? 1.0f / wsum : 0.0f;
+                            __nv_bfloat16* op = p.out + ((static_cast<size_t>(f) * p.d + qi) * p.n_q_heads + h * p.G + qg) * D;
+#pragma unroll
+                            for (int col0 = 0; col0 < D / 4; col0 += 16)
+                                merge_columns<D, 16>(a.part_o, a.part_lse, slot_s, 2, tid, col0, M, iw, op);
+                        }
+                    }
+                    tc::named_barrier(1, 256);                   // slot_s is free again
+                } else if (tid == 0) {
+                    // More pieces: count this one, and note the unit for this CTA's share of its merge,
+                    // which follows once the whole range is done (waiting here, in the middle of the
+                    // range, would chain every CTA behind its neighbour).
                     const int gu = unit_base_s[it.s] + it.unit;
                     atomicAdd(a.unit_count + gu, 1);
                     Deferred& dfr = deferred_s[n_deferred_s++];
