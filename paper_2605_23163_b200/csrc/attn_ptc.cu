@@ -244,7 +244,8 @@ attn_ptc_kernel(const __grid_constant__ TcArgs<MAXSETS> a) {
     __shared__ int abort_s, n_deferred_s, last_s;
     __shared__ Deferred deferred_s[2];                  // a range starts and ends inside at most one cut unit each
     constexpr int kMaxPieces = 160;                     // a unit is cut by CTA borders: at most one piece per CTA
-    __shared__ int slot_s[kMaxPieces];                  // scratch slot of every piece of the unit being merged
+    __shared__ int slot2_s[2][kMaxPieces];              // scratch slot of every piece of the (up to two) units being merged
+    int* const slot_s = slot2_s[0];
     volatile int* abort_flag = &abort_s;
 
     // The rollouts that take part (gate != 0), scene after scene, and the layout of the work that
@@ -795,84 +796,93 @@ attn_ptc_kernel(const __grid_constant__ TcArgs<MAXSETS> a) {
         }
 
         // ------------------------------------------------------------ merges of the cut units
-        // Every CTA that holds a piece of a unit merges an equal share of the unit's rows, once all
-        // pieces are there.  (All CTAs of the launch are resident at once: the wait is for CTAs
-        // that are running, and it is bounded like every other wait.)
+        // Every CTA that holds a piece of a unit (in more than two pieces) merges an equal share of
+        // the unit's rows, once all pieces are there.  (All CTAs of the launch are resident at once:
+        // the wait is for CTAs that are running, and it is bounded like every other wait.)  A CTA
+        // with two such units gives half of its threads to each.
         tc::named_barrier(1, 256);
         const int n_deferred = *abort_flag ? 0 : n_deferred_s;
-        for (int e = 0; e < n_deferred; ++e) {
-            const Deferred dfr = deferred_s[e];
-            const SetParams& p = a.sets[dfr.s];
-            const int n_pieces = dfr.n_pieces;
+        if (n_deferred > 0) {
             if (tid == 0) {
                 const long long t0 = clock64();
-                volatile int* arrived = a.unit_count + dfr.gu;
-                while (*arrived < n_pieces) {
-                    if (clock64() - t0 > kWaitLimit) {
-                        atomicCAS(a.status, 0, FDD_ERR_DEVICE_TIMEOUT);
-                        *abort_flag = 1;
-                        break;
+                for (int e = 0; e < n_deferred; ++e) {
+                    volatile int* arrived = a.unit_count + deferred_s[e].gu;
+                    while (*arrived < deferred_s[e].n_pieces) {
+                        if (clock64() - t0 > kWaitLimit) {
+                            atomicCAS(a.status, 0, FDD_ERR_DEVICE_TIMEOUT);
+                            *abort_flag = 1;
+                            break;
+                        }
                     }
                 }
             }
-            if (tid < n_pieces && tid < kMaxPieces) {
-                const int pc = dfr.c_first + tid;
-                slot_s[tid] = pc * 2 + (dfr.unit_begin <= T * pc / C ? 0 : 1);
-            }
+            for (int e = 0; e < n_deferred; ++e)
+                if (tid < deferred_s[e].n_pieces && tid < kMaxPieces) {
+                    const int pc = deferred_s[e].c_first + tid;
+                    slot2_s[e][tid] = pc * 2 + (deferred_s[e].unit_begin <= T * pc / C ? 0 : 1);
+                }
             tc::named_barrier(1, 256);
-            if (*abort_flag) break;
-            __threadfence();
-            // this CTA's share of the rows; a row is split between `col_groups` threads
-            const int rows_here = min(256, p.R - dfr.rp * 256);
-            const int mine = static_cast<int>(blockIdx.x) - dfr.c_first;
-            const int row_lo = rows_here * mine / n_pieces, row_hi = rows_here * (mine + 1) / n_pieces;
-            const int share = row_hi - row_lo;
-            int col_groups = 1;                                   // a power of two, share * col_groups <= 256
-            while (col_groups < D / 4 && share * col_groups * 2 <= 256) col_groups *= 2;
-            const int ct = (D / 4) / col_groups;                  // float4 columns per thread
-            const int row_in_share = tid / col_groups, cg = tid - row_in_share * col_groups;
-            if (share > 0 && row_in_share < share) {
-                const int rowu = row_lo + row_in_share;
-                float M = -CUDART_INF_F, wsum = 0.0f;
-                for (int k0 = 0; k0 < n_pieces; k0 += 8) {
-                    float ls[8];
+            if (*abort_flag == 0) {
+                __threadfence();
+                const int threads_e = 256 / n_deferred;               // threads per unit
+                const int e = tid / threads_e, lt = tid - e * threads_e;
+                const Deferred dfr = deferred_s[e];
+                const SetParams& p = a.sets[dfr.s];
+                const int n_pieces = dfr.n_pieces;
+                const int* slots = slot2_s[e];
+                // this CTA's share of the rows; a row is split between `col_groups` threads
+                const int rows_here = min(256, p.R - dfr.rp * 256);
+                const int mine = static_cast<int>(blockIdx.x) - dfr.c_first;
+                const int row_lo = rows_here * mine / n_pieces, row_hi = rows_here * (mine + 1) / n_pieces;
+                const int share = row_hi - row_lo;                    // <= 86 (three pieces or more)
+                int col_groups = 1;                                   // a power of two, share * col_groups <= threads_e
+                while (col_groups < D / 4 && share * col_groups * 2 <= threads_e) col_groups *= 2;
+                const int ct = (D / 4) / col_groups;                  // float4 columns per thread
+                const int row_in_share = lt / col_groups, cg = lt - row_in_share * col_groups;
+                if (share > 0 && row_in_share < share) {
+                    const int rowu = row_lo + row_in_share;
+                    float M = -CUDART_INF_F, wsum = 0.0f;
+                    for (int k0 = 0; k0 < n_pieces; k0 += 8) {
+                        float ls[8];
 #pragma unroll
-                    for (int k = 0; k < 8; ++k)
-                        ls[k] = k0 + k < n_pieces ? __ldcg(a.part_lse + static_cast<size_t>(slot_s[min(k0 + k, n_pieces - 1)]) * 256 + rowu)
-                                                  : -CUDART_INF_F;
-                    float mc = ls[0];
+                        for (int k = 0; k < 8; ++k)
+                            ls[k] = k0 + k < n_pieces ? __ldcg(a.part_lse + static_cast<size_t>(slots[min(k0 + k, n_pieces - 1)]) * 256 + rowu)
+                                                      : -CUDART_INF_F;
+                        float mc = ls[0];
 #pragma unroll
-                    for (int k = 1; k < 8; ++k) mc = fmaxf(mc, ls[k]);
-                    const float mn = fmaxf(M, mc);
-                    if (mn > -CUDART_INF_F) {
-                        wsum *= exp2f(M - mn);                  // 0 the first time (M = -inf)
+                        for (int k = 1; k < 8; ++k) mc = fmaxf(mc, ls[k]);
+                        const float mn = fmaxf(M, mc);
+                        if (mn > -CUDART_INF_F) {
+                            wsum *= exp2f(M - mn);                  // 0 the first time (M = -inf)
 #pragma unroll
-                        for (int k = 0; k < 8; ++k) wsum += exp2f(ls[k] - mn);
-                        M = mn;
+                            for (int k = 0; k < 8; ++k) wsum += exp2f(ls[k] - mn);
+                            M = mn;
+                        }
+                    }
+                    if (!(M > -CUDART_INF_F)) M = 0.0f;
+                    const float iw = wsum > 0.0f ? 1.0f / wsum : 0.0f;
+                    const int r = dfr.rp * 256 + rowu;
+                    const int qi2 = r / p.G, qg2 = r - qi2 * p.G;
+                    __nv_bfloat16* op = p.out + ((static_cast<size_t>(dfr.f) * p.d + qi2) * p.n_q_heads + dfr.h * p.G + qg2) * D;
+                    const int col0 = cg * ct;
+                    switch (ct) {
+                        case 1: merge_columns<D, 1>(a.part_o, a.part_lse, slots, n_pieces, rowu, col0, M, iw, op); break;
+                        case 2: merge_columns<D, 2>(a.part_o, a.part_lse, slots, n_pieces, rowu, col0, M, iw, op); break;
+                        case 4: merge_columns<D, 4>(a.part_o, a.part_lse, slots, n_pieces, rowu, col0, M, iw, op); break;
+                        case 8: merge_columns<D, 8>(a.part_o, a.part_lse, slots, n_pieces, rowu, col0, M, iw, op); break;
+                        case 16: merge_columns<D, 16>(a.part_o, a.part_lse, slots, n_pieces, rowu, col0, M, iw, op); break;
+                        default: merge_columns<D, 32>(a.part_o, a.part_lse, slots, n_pieces, rowu, col0, M, iw, op); break;
                     }
                 }
-                if (!(M > -CUDART_INF_F)) M = 0.0f;
-                const float iw = wsum > 0.0f ? 1.0f / wsum : 0.0f;
-                const int r = dfr.rp * 256 + rowu;
-                const int qi2 = r / p.G, qg2 = r - qi2 * p.G;
-                __nv_bfloat16* op = p.out + ((static_cast<size_t>(dfr.f) * p.d + qi2) * p.n_q_heads + dfr.h * p.G + qg2) * D;
-                const int col0 = cg * ct;
-                switch (ct) {
-                    case 1: merge_columns<D, 1>(a.part_o, a.part_lse, slot_s, n_pieces, rowu, col0, M, iw, op); break;
-                    case 2: merge_columns<D, 2>(a.part_o, a.part_lse, slot_s, n_pieces, rowu, col0, M, iw, op); break;
-                    case 4: merge_columns<D, 4>(a.part_o, a.part_lse, slot_s, n_pieces, rowu, col0, M, iw, op); break;
-                    case 8: merge_columns<D, 8>(a.part_o, a.part_lse, slot_s, n_pieces, rowu, col0, M, iw, op); break;
-                    case 16: merge_columns<D, 16>(a.part_o, a.part_lse, slot_s, n_pieces, rowu, col0, M, iw, op); break;
-                    default: merge_columns<D, 32>(a.part_o, a.part_lse, slot_s, n_pieces, rowu, col0, M, iw, op); break;
-                }
-            }
-            tc::named_barrier(1, 256);
-            if (tid == 0) {
-                // the last CTA to finish its share leaves both counters at zero for the next launch
-                int* done = a.unit_count + a.max_units + dfr.gu;
-                if (atomicAdd(done, 1) == n_pieces - 1) {
-                    *done = 0;
-                    a.unit_count[dfr.gu] = 0;
+                tc::named_barrier(1, 256);
+                if (tid < n_deferred) {
+                    // the last CTA to finish its share leaves both counters at zero for the next launch
+                    const Deferred& d2 = deferred_s[tid];
+                    int* done = a.unit_count + a.max_units + d2.gu;
+                    if (atomicAdd(done, 1) == d2.n_pieces - 1) {
+                        *done = 0;
+                        a.unit_count[d2.gu] = 0;
+                    }
                 }
             }
         }
