@@ -46,7 +46,7 @@ constexpr int kTcThreads = 384;
 constexpr int kKeysPerTile = 128;
 constexpr long long kWaitLimit = 4000000000LL;   // about two seconds of SM clocks
 constexpr int kMaxGatedForks = kAttnMaxGatedForks;   // rollouts of one launch when any scene has a gate
-constexpr int kMinTilesPerCta = 4;               // do not cut the work finer than this (every cut costs a piece to write and merge)
+constexpr int kMinTilesPerCta = 3;               // do not cut the work finer than this (every cut costs a piece to write and merge)
 // Registers per thread after the hand-over.  The CTA starts with 384 x 168; 8 soft-max warps x
 // kRegsSoftmax + 4 other warps x kRegsOther must not exceed that (2 * 208 + 88 = 3 * 168).
 constexpr int kRegsSoftmax = 208;
