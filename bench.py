@@ -28,7 +28,7 @@ METRIC = "committed tokens/s per denoise step (N forks, shared prefix)"
 UNIT = "tokens/s"
 # DRAM bytes (read + write) of one attention launch at the long_prefix workload, from the ncu capture
 # summarised in profiles/attn_ptc_long_prefix.md; None for other workloads or once the kernel changed.
-ATTN_DRAM_BYTES_PER_LAUNCH = {"long_prefix": 167.3e6}
+ATTN_DRAM_BYTES_PER_LAUNCH = {"long_prefix": 168.6e6}
 COUNT_STREAM = None  # copy the per-rollout counts to the host on a stream of their own (None: for large steps only)
 GRAPH = False       # replay every denoising step from a CUDA graph (--graph)
 TIME_EVERY = 4      # blocks between two blocks whose kernels are timed one by one
