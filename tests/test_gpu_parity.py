@@ -449,6 +449,43 @@ def test_more_scenes_and_rows_than_one_launch_takes():
         fdd.fdd_destroy(ctx)
 
 
+def test_unmask_counted_matches_unmask_with_the_step_passed_by_value():
+    # 18 scenes (two groups of launches inside one call): the device-side step counter must advance
+    # once per call, not once per group, and give the same draws as the step passed by value
+    scenes = tuple(synth.Scene(prefix_len=40, n_forks=1 + i % 2, block_len=16, n_scaffold=4, n_blocks=1) for i in range(18))
+    w = synth.Workload("counted", 8, 2, 64, 512, "f32", "peaked", 0.95, 0.8, scenes, seed=77)
+    ctx = harness.create_context(w)
+    try:
+        gs = [harness.GpuScene(ctx, w, i) for i in range(18)]
+        sets = [g.forkset for g in gs]
+        flat = lambda xs: np.concatenate([x.reshape(-1) for x in xs])
+        toks, sts = zip(*[synth.make_block_template(w, i, 0) for i in range(18)])
+        nf = sum(sc.n_forks for sc in scenes)
+        results = []
+        for counted in (False, True):
+            tok_d, st_d = torch.from_numpy(flat(toks)).cuda(), torch.from_numpy(flat(sts)).cuda()
+            n_c = torch.zeros(nf, dtype=torch.int32, device="cuda"); n_l = torch.zeros(nf, dtype=torch.int32, device="cuda")
+            counter = torch.zeros(1, dtype=torch.int32, device="cuda")
+            trace = []
+            for step in range(3):
+                lg = torch.from_numpy(flat([synth.make_logits(w, i, 0, step, rows="all") for i in range(18)])).cuda()
+                if counted:
+                    fdd.fdd_unmask_counted(ctx, sets, lg, tok_d, st_d, [16] * 18, w.threshold, w.temperature, 0, counter, n_c, n_l)
+                else:
+                    fdd.fdd_unmask(ctx, sets, lg, tok_d, st_d, [16] * 18, w.threshold, w.temperature, 0, step, n_c, n_l)
+                trace.append((tok_d.cpu().numpy(), st_d.cpu().numpy(), n_c.cpu().numpy(), n_l.cpu().numpy()))
+            fdd.fdd_poll_status(ctx)
+            if counted:
+                assert int(counter.item()) == 3
+            results.append(trace)
+        for a_, b_ in zip(*results):
+            for x, y in zip(a_, b_):
+                assert np.array_equal(x, y)
+        assert results[0][0][2].sum() > 0 and not np.array_equal(results[0][0][0], results[0][2][0])
+    finally:
+        fdd.fdd_destroy(ctx)
+
+
 def test_prefix_is_never_written_and_forks_with_equal_inputs_agree():
     w = synth.small_variant(synth.workload("tts"), prefix_len=512, vocab=512, n_forks=4, n_blocks=1)
     ctx = harness.create_context(w)
