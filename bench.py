@@ -186,6 +186,7 @@ def run_ours(args):
     unmask_done = [torch.cuda.Event(), torch.cuda.Event()]
     n_left_d = [n_left, torch.zeros_like(n_left)]
 
+    prepared, retired = [], []  # fork sets made ahead for the next block / of the last block, to be freed
     attn_events = []            # [start, end, rollouts still decoding] of every timed attention call
     unmask_events = []          # [start, end, MASKED rows on entry] of every timed unmask call
 
@@ -196,7 +197,10 @@ def run_ours(args):
         `lookahead` step t + 1 is enqueued before the host has seen the result of step t (once
         every rollout is done its kernels return at once), which keeps the GPU busy while the host
         reads the counts."""
-        fs_list = [fdd.fdd_fork(ctx, *fa) for fa in fork_args]
+        # The fork sets of this block were made while the block before was running (fdd_fork is host
+        # work only), and the sets of the block before are freed once this block's first step is
+        # enqueued: neither sits between two blocks, where the GPU would wait for the host.
+        fs_list = prepared.pop() if prepared else [fdd.fdd_fork(ctx, *fa) for fa in fork_args]
         fs = fdd.ptr_array(fs_list)
         tokens.copy_(tokens0_d, non_blocking=True)
         state.copy_(state0_d, non_blocking=True)
@@ -244,10 +248,15 @@ def run_ours(args):
 
         enqueue(0)
         entry_counts(0, N, value_tokens)
+        while retired:
+            for f_ in retired.pop():
+                fdd.fdd_forkset_free(ctx, f_)
         t = 0
         while True:
             if lookahead and t + 1 < d:
                 enqueue(t + 1)
+            if t == 0:
+                prepared.append([fdd.fdd_fork(ctx, *fa) for fa in fork_args])     # for the next block
             step_done[t % 2].synchronize()
             left = n_left_views[t % 2]
             masked_rows = int(left.sum())
@@ -264,8 +273,7 @@ def run_ours(args):
             fdd.fdd_kv_commit(ctx, fs, layer, k, v, ds_c, 1 if layer == L - 1 else 0)
         for i in range(n_scenes):
             fdd.fdd_average_rollouts(ctx, trajs[i], Ns[i], w.waypoints, traj_out[i])
-        for f_ in fs_list:
-            fdd.fdd_forkset_free(ctx, f_)
+        retired.append(fs_list)
         return t
 
     resident = lambda t: dev_steps[t % PRE_STEPS]
