@@ -179,7 +179,7 @@ fdd_status fdd_block_attn_gated(fdd_ctx* ctx, fdd_forkset* const* sets, int n_se
  * where g[v] = -ln(E[v]) and the E[v] are independent Exp(1) variates built as a race over
  * groups of 16 consecutive ids from two Philox4x32-10 streams under key = the rollout's seed
  * (low, high word).  Group j = v / 16 has the word
- *   R = output word (j / 256) % 4 of counter ((j / 1024) * 256 + j % 256, i, step, block_idx),
+ *   R = output word j % 4 of counter (j / 4, i, step, block_idx),
  * every id the fine bits
  *   f[v] = top 23 bits of output word v % 4 of counter (v / 4, i + 2^31, step, block_idx).
  * The id 16 j + R % 16 (the group's leader) holds the group's minimum,

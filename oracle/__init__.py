@@ -19,7 +19,9 @@ it.  It shares no code with the CUDA library and never imports it.
 Parity pins (see tests/test_oracle_*.py): every function here is pinned by
 closed forms, brute force on tiny inputs, library special cases or published
 known-answer values.  The jerk-minimising interpolation mentioned in Sec. 3.4
-is not implemented anywhere in this repository (the paper gives no formula).
+has no formula in the paper: `jmt.py` implements this repository's reading of it
+and is pinned to that reading's variational definition only (parity with the
+paper unpinned).
 """
 
 MASKED = 0

@@ -8,16 +8,36 @@ generator.  The reading used by this repository: Philox4x32 with 10 rounds
 SC'11), keyed by the rollout's 64-bit seed, with the counter made of the
 vocabulary index, the position inside the block, the denoising step and the
 block index, so that a draw depends on nothing but (seed, block, step,
-position, vocabulary id).  The draws are built as an "exponential race" over
-groups of 16 consecutive ids (see `exponential_row`): one 32-bit word per group
-fixes the group's smallest exponential variate and which id holds it, a second
-stream gives every id 23 bits of its own.
+position, vocabulary id).
 
-Two implementations live here on purpose: a scalar one on Python integers that
-follows the published round function literally, and a numpy one used for whole
-rows.  The tests pin the scalar one to the published known-answer values and
-the vectorised one to the scalar one.
+The definition, for vocabulary id v of one row (`exponential_scalar` is this
+paragraph on Python integers, nothing else):
+
+    group j = v // 16 has the 32-bit word
+        R_j  = output word j % 4 of Philox(counter (j // 4, position, step, block))
+    every id has 23 bits of its own
+        f_v  = top 23 bits of output word v % 4 of
+               Philox(counter (v // 4, position + 2**31, step, block))
+    the id 16 j + R_j % 16 is the group's leader and holds the group's minimum
+        E    = -ln(U) / 16,   U = ((R_j >> 4) + (f_leader + 0.5) 2**-23) / 2**28
+    every other id of the group has
+        E_v  = E_leader - ln((f_v + 0.5) 2**-23)
+    and the noise is g_v = -ln(E_v).
+
+The counters are the plain running indices of groups and ids: nothing in them
+knows how an implementation walks through a row.  That the E_v are independent
+Exp(1) variates (so that the g_v are independent standard Gumbel variates) is
+the memorylessness of the exponential distribution, see `exponential_row`.
+
+Three implementations live here on purpose: Philox on Python integers that
+follows the published round function literally, `exponential_scalar` (the
+definition above, one id at a time) and numpy versions for whole rows.  The
+tests pin the scalar Philox to the published known-answer values, the
+vectorised functions to the scalar ones, and the distribution of the draws to
+what the construction promises.
 """
+import math
+
 import numpy as np
 
 PHILOX_M0 = 0xD2511F53
@@ -76,22 +96,35 @@ FINE_STREAM = 1 << 31   # added to the position word of the counter for the seco
 GROUP = 16              # vocabulary ids per group
 
 
-def group_words(seed, block_idx, step, position, vocab):
-    """The 32-bit word R_j of every group j (ids 16 j .. 16 j + 15) of one row.
+def exponential_scalar(seed, block_idx, step, position, v):
+    """E[v] of a single vocabulary id on Python integers and math.log: the definition in
+    the module docstring, line by line."""
+    seed = int(seed) & 0xFFFFFFFFFFFFFFFF
+    key = (seed & MASK32, seed >> 32)
 
-    Group j takes word (j // 256) % 4 of the Philox block with counter
-    ((j // 1024) * 256 + j % 256, position, step, block_idx): the four words of a block
-    belong to four groups that lie 256 groups (4096 ids) apart, so that one block
-    serves 64 ids of any run of 16 consecutive ids per 4096.
-    """
+    def fine(u):
+        return philox4x32_scalar((u // 4, position + FINE_STREAM, step, block_idx), key)[u % 4] >> 9
+
+    j = v // GROUP
+    R = philox4x32_scalar((j // 4, position, step, block_idx), key)[j % 4]
+    leader = GROUP * j + R % GROUP
+    U = ((R >> 4) + (fine(leader) + 0.5) * 2.0 ** -23) * 2.0 ** -28      # exact in fp64 (51 bits)
+    e = -math.log(U) / GROUP
+    if v != leader:
+        e += -math.log((fine(v) + 0.5) * 2.0 ** -23)
+    return e
+
+
+def group_words(seed, block_idx, step, position, vocab):
+    """The 32-bit word R_j of every group j (ids 16 j .. 16 j + 15) of one row:
+    output word j % 4 of the Philox block with counter (j // 4, position, step,
+    block_idx), i.e. the blocks 0, 1, 2, ... of the stream read word by word."""
     seed = int(seed) & 0xFFFFFFFFFFFFFFFF
     ngroups = (vocab + GROUP - 1) // GROUP
-    j = np.arange(ngroups, dtype=np.uint64)
-    ctr = (j >> np.uint64(10)) * np.uint64(256) + (j & np.uint64(255))
+    ctr = np.arange((ngroups + 3) // 4, dtype=np.uint64)
     w = philox4x32_vec(ctr, np.uint64(position), np.uint64(step), np.uint64(block_idx),
                        seed & MASK32, seed >> 32)
-    words = np.stack(w, axis=1)                                    # [group, 4]
-    return words[np.arange(ngroups), ((j >> np.uint64(8)) & np.uint64(3)).astype(np.int64)]
+    return np.stack(w, axis=1).reshape(-1)[:ngroups]
 
 
 def fine_bits(seed, block_idx, step, position, vocab):

@@ -7,8 +7,8 @@ import numpy as np
 import pytest
 
 from oracle import MASKED, COMMITTED, SCAFFOLD
-from oracle.philox import (exponential_row, fine_bits, group_words, gumbel_row, leader_exponential,
-                           philox4x32_scalar, philox4x32_vec)
+from oracle.philox import (exponential_row, exponential_scalar, fine_bits, group_words, gumbel_row,
+                           leader_exponential, philox4x32_scalar, philox4x32_vec)
 from oracle.unmask import unmask_step
 
 GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
@@ -62,7 +62,7 @@ def test_leader_map_is_open_interval_and_monotone():
 
 def test_gumbel_row_layout_and_independence_from_vocab_size():
     seed = 0xDEADBEEFCAFEF00D
-    V = 16 * 1024 + 40                                  # reaches the second run of 1024 groups
+    V = 16 * 1024 + 40
     a = gumbel_row(seed, 3, 2, 5, V)
     b = gumbel_row(seed, 3, 2, 5, V + 23)
     np.testing.assert_array_equal(a, b[:V])
@@ -70,12 +70,13 @@ def test_gumbel_row_layout_and_independence_from_vocab_size():
     key = (seed & 0xFFFFFFFF, seed >> 32)
     words = group_words(seed, 3, 2, 5, V)
     fb = fine_bits(seed, 3, 2, 5, V + 16)
-    # group j: word (j // 256) % 4 of counter ((j // 1024) * 256 + j % 256, pos, step, block); fine: top 23
-    # bits of word v % 4 of counter (v // 4, pos + 2^31, step, block); both under key (lo, hi)
+    # group j: word j % 4 of counter (j // 4, pos, step, block); fine: top 23 bits of word v % 4 of
+    # counter (v // 4, pos + 2^31, step, block); both under key (lo, hi).  Spelled out here once more
+    # on Python integers, and compared with the one-id-at-a-time definition of the oracle.
     seen_leader = seen_other = 0
-    for v in (0, 5, 18, 255 * 16 + 3, 256 * 16 + 1, 700 * 16 + 15, 1023 * 16, 1024 * 16 + 7, V - 1) + tuple(range(32, 64)):
+    for v in (0, 5, 18, 63, 64, 255 * 16 + 3, 256 * 16 + 1, 700 * 16 + 15, 1023 * 16, 1024 * 16 + 7, V - 1) + tuple(range(32, 64)):
         j = v // 16
-        R = philox4x32_scalar(((j // 1024) * 256 + j % 256, 5, 2, 3), key)[(j // 256) % 4]
+        R = philox4x32_scalar((j // 4, 5, 2, 3), key)[j % 4]
         assert int(words[j]) == R
         lead = 16 * j + R % 16
         f_lead = philox4x32_scalar((lead // 4, 5 + 2 ** 31, 2, 3), key)[lead % 4] >> 9
@@ -89,12 +90,38 @@ def test_gumbel_row_layout_and_independence_from_vocab_size():
         else:
             seen_leader += 1
         assert abs(a[v] + math.log(e)) <= 1e-12 * max(1.0, abs(a[v]))
+        assert e == exponential_scalar(seed, 3, 2, 5, v)
     assert seen_leader >= 2 and seen_other >= 20
     # every counter field and the seed matter
     for other in (gumbel_row(seed + 1, 3, 2, 5, 37), gumbel_row(seed, 4, 2, 5, 37),
                   gumbel_row(seed, 3, 1, 5, 37), gumbel_row(seed, 3, 2, 6, 37),
                   gumbel_row(seed ^ (1 << 40), 3, 2, 5, 37)):
         assert not np.array_equal(a[:37], other)
+
+
+def test_row_function_equals_the_scalar_definition_everywhere():
+    # the vectorised row against the one-id-at-a-time definition on every id of a short row and on
+    # random ids of a long one (both rows cut their last group)
+    for seed, blk, step, pos, V, ids in ((7, 0, 0, 0, 100, range(100)),
+                                         (2 ** 63 + 11, 5, 9, 127, 151936 - 3,
+                                          np.random.default_rng(3).integers(0, 151936 - 3, 300))):
+        e = exponential_row(seed, blk, step, pos, V)
+        for v in ids:
+            ref = exponential_scalar(seed, blk, step, pos, int(v))
+            assert abs(e[v] - ref) <= 1e-13 * ref
+
+
+def test_words_are_the_stream_in_order_and_streams_do_not_overlap():
+    # the group words are the Philox blocks 0, 1, 2, ... of (position, step, block) read word by
+    # word; the fine bits come from the blocks of (position + 2^31, step, block): no counter is
+    # used by both, whatever the position (positions stay far below 2^31)
+    seed, key = 99, (99, 0)
+    words = group_words(seed, 1, 2, 3, 16 * 12)
+    flat = [x for c in range(3) for x in philox4x32_scalar((c, 3, 2, 1), key)]
+    assert [int(x) for x in words] == flat
+    fb = fine_bits(seed, 1, 2, 3, 12)
+    flat_f = [x >> 9 for c in range(3) for x in philox4x32_scalar((c, 3 + 2 ** 31, 2, 1), key)]
+    assert [int(x) for x in fb] == flat_f
 
 
 def test_group_word_bounds_every_draw_of_the_group():
@@ -310,6 +337,54 @@ def test_gumbel_max_samples_softmax_of_scaled_logits():
     # confidence reported is the noise-free probability of the *chosen* token
     sm = np.exp(l) / np.exp(l).sum()
     np.testing.assert_allclose(r["conf"][0], sm[r["tokens"][0]], rtol=1e-13)
+
+
+def _winner_counts(l, T, n, seed0):
+    """argmax(l + T g) over n independent rows (positions x seeds) through unmask_step."""
+    V = len(l)
+    rows = 50
+    logits = np.tile(np.asarray(l, dtype=np.float64), (1, rows, 1))
+    tokens = np.zeros((1, rows), dtype=np.int32)
+    state = np.zeros((1, rows), dtype=np.uint8)
+    counts = np.zeros(V)
+    lead_wins = 0
+    for s in range(n // rows):
+        r = unmask_step(logits, tokens, state, [seed0 + s], threshold=-1.0, temperature=T, block_idx=2, step=s % 7)
+        counts += np.bincount(r["tokens"][0], minlength=V)
+        for i in range(rows):
+            w = group_words(seed0 + s, 2, s % 7, i, V)
+            t = int(r["tokens"][0, i])
+            lead_wins += int(16 * (t // 16) + int(w[t // 16]) % 16 == t)
+    return counts, lead_wins
+
+
+def test_gumbel_max_over_several_groups_leaders_and_followers_win():
+    # V = 48: three groups of 16.  The race construction gives every group one id (its leader) a
+    # head start; the frequencies must still be softmax(l / T), whether the winner is a leader or
+    # not.  chi-square(47): 0.1 % critical value 82.7
+    V, T, n = 48, 0.7, 20000
+    g = np.random.default_rng(11)
+    l = g.standard_normal(V) * 1.2
+    p = np.exp(l / T) / np.exp(l / T).sum()
+    counts, lead_wins = _winner_counts(l, T, n, 5000)
+    chi2 = float(((counts - n * p) ** 2 / (n * p)).sum())
+    assert chi2 < 82.7
+    # P(winner is its group's leader) = sum_v p_v P(v leads | v wins); a leader is the smallest of 16
+    # draws, so it wins far more often than 1 / 16 of the time, yet not always
+    assert 0.25 * n < lead_wins < 0.95 * n
+    # per group: the group's total mass
+    grp = counts.reshape(3, 16).sum(axis=1)
+    pg = p.reshape(3, 16).sum(axis=1)
+    assert float(((grp - n * pg) ** 2 / (n * pg)).sum()) < 13.8       # chi-square(2) 0.1 %
+
+
+def test_equal_logits_give_a_uniform_winner():
+    # all logits equal: the noise alone decides, every id of every group equally often
+    V, n = 48, 14400
+    counts, lead_wins = _winner_counts(np.full(V, 1.5), 1.0, n, 9000)
+    chi2 = float(((counts - n / V) ** 2 / (n / V)).sum())
+    assert chi2 < 82.7
+    assert lead_wins == n          # with equal logits the winner is the id with the smallest E: a leader
 
 
 def test_planted_mistakes_are_caught():
