@@ -193,8 +193,9 @@ fdd_status fdd_block_attn_gated(fdd_ctx* ctx, fdd_forkset* const* sets, int n_se
  *
  *   logits        device, packed like q: [N_s][d_s][V], fp32 or bf16 per cfg.logits_dtype.
  *                 Only rows of MASKED positions are read.  N_s * d_s <= 8192 per set
- *                 (FDD_ERR_CAPACITY otherwise); the wide loads need V % 16 == 0 (bf16) or
- *                 V % 8 == 0 (fp32) and a 32-byte aligned base, else a slower path runs.
+ *                 (FDD_ERR_CAPACITY otherwise); the bulk copies need 16-byte aligned rows
+ *                 (V % 8 == 0 for bf16, V % 4 == 0 for fp32, 16-byte aligned base), else a
+ *                 slower path runs.
  *   tokens        device int32 [N_s][d_s], in/out.     state: device uint8, in/out.
  *   n_committed   device int32 [sum N_s]: commits of this step per rollout (written).
  *   n_left        device int32 [sum N_s]: MASKED positions remaining per rollout (written).
@@ -304,9 +305,10 @@ fdd_status fdd_average_rollouts_jmt(fdd_ctx* ctx, const float* traj, int n, int 
  *   seeds         device uint64 [n_forks] (the caller keeps them on the device)
  *   n_committed, n_left  device int32 [n_forks] (written);  conf: device fp32 [n_forks][block_len] or NULL
  *   err, err_len  optional host buffer that receives the error text (may be NULL / 0)
- * Limits: block_len <= 128 and n_forks * block_len * ceil(vocab / 8192) <= FDD_UNMASK_STATIC_MAX_RECORDS;
- * anything larger is rejected with FDD_ERR_CAPACITY before any launch (e.g. vocab 151936 has 19
- * chunks, so up to 3449 rows: 32 rollouts x 64 positions fit).
+ * Limits: block_len <= 128, n_forks * block_len <= 8192 rows, and
+ * n_forks * block_len * ceil(vocab / 8192) <= FDD_UNMASK_STATIC_MAX_RECORDS; anything larger is
+ * rejected with FDD_ERR_CAPACITY before any launch (e.g. vocab 151936 has 19 record slots per row,
+ * so up to 3449 rows: 32 rollouts x 64 positions fit).
  * Set-up: the first call on each device (with that device current) asks the runtime for the
  * device address of the array (cudaGetSymbolAddress) and caches it; make that first call before
  * any stream capture begins.  Later calls do no set-up.

@@ -118,7 +118,8 @@ fdd_status fdd_create(const fdd_config* cfg, fdd_ctx** out) {
     if (e == cudaSuccess) e = cudaMemset(ctx->d_status, 0, sizeof(int));
     if (e == cudaSuccess) e = cudaMallocHost(&ctx->h_status, sizeof(int));
     if (e == cudaSuccess) {
-        ctx->ws_unmask_bytes = static_cast<size_t>(cfg->max_forks) * cfg->max_block * unmask_chunks(cfg->vocab) * sizeof(UnmaskPartial);
+        const long long max_rows = static_cast<long long>(cfg->max_forks) * cfg->max_block;
+        ctx->ws_unmask_bytes = unmask_workspace_bytes(cfg->vocab, static_cast<int>(std::min<long long>(max_rows, kUnmaskMaxRows)));
         e = cudaMalloc(&ctx->ws_unmask, ctx->ws_unmask_bytes);
     }
     if (e == cudaSuccess) {

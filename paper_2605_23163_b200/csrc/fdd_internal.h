@@ -45,7 +45,7 @@ struct fdd_ctx {
     int sm_count = 0;
     int* d_status = nullptr;          // device status word (first error wins)
     int* h_status = nullptr;          // pinned mirror
-    void* ws_unmask = nullptr;        // per (row, chunk) partial reductions
+    void* ws_unmask = nullptr;        // per (row, tile) partial reductions
     size_t ws_unmask_bytes = 0;
     void* ws_attn = nullptr;          // partial outputs of attention units cut between CTAs
     size_t ws_attn_bytes = 0;
@@ -137,9 +137,15 @@ struct UnmaskPartial {
     int pad[3];
 };
 
-static constexpr int kUnmaskChunk = 8192;   // vocabulary entries per work item
+static constexpr int kUnmaskTile = 2048;    // vocabulary entries per tile of the streaming kernel (one bulk copy)
+static constexpr int kUnmaskChunk = 8192;   // vocabulary entries per record slot of fdd_unmask_static
 static constexpr int kUnmaskMaxRows = 8192; // rollouts x positions of one launch (the kernel compacts them in shared memory)
-static inline int unmask_chunks(int vocab) { return (vocab + kUnmaskChunk - 1) / kUnmaskChunk; }
+// Record slots per row when tiles_per_item tiles share a slot.
+static inline int unmask_items_per_row(int vocab, int tiles_per_item) {
+    const int tiles = (vocab + kUnmaskTile - 1) / kUnmaskTile;
+    return (tiles + tiles_per_item - 1) / tiles_per_item;
+}
+size_t unmask_workspace_bytes(int vocab, int max_rows);
 
 cudaError_t launch_attention_simple(const AttnProblem& p, int head_dim, cudaStream_t st);
 bool attention_tc_supported(const AttnProblem& a, int head_dim);

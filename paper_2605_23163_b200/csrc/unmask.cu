@@ -1,53 +1,59 @@
 // Confidence-threshold parallel unmasking: vocabulary-wide soft-max statistics and
 // (Gumbel-perturbed) arg-max per MASKED row, then the per-rollout commit rule.
 //
-// Kernel 1 (unmask_partial_kernel): persistent grid.  The MASKED rows of the call, cut into chunks
-// of 8192 ids and laid end to end, are split into equal contiguous ranges, one per CTA (with few
-// rows every chunk gets a CTA of its own).  A CTA streams each of its pieces from HBM once, 16
-// consecutive logits per thread and step (32-byte loads, or 16-byte asynchronous copies through a
-// per-thread ring in shared memory), and keeps running soft-max statistics; nothing but the few
-// logits that can win the arg-max is looked at twice.  Rows that are not MASKED are never read.
+// Kernel 1 (unmask_stream_kernel): persistent grid, every warp on its own.  The MASKED rows of the
+// call, cut into tiles of 2048 ids and laid end to end, are split into equal contiguous ranges, one
+// per warp (tail of a row, whole rows, head of the next; one record per (row, warp), merged by the
+// second kernel).  A warp streams its tiles from HBM once, through a ring of bulk asynchronous
+// copies (cp.async.bulk, completion on an mbarrier, no multicast) into its own part of shared
+// memory, three tiles deep; a lane takes 64 consecutive ids of a tile (16-byte reads, chunk order
+// rotated by the lane so that the banks do not collide) and keeps running soft-max statistics.
+// There is no CTA-wide barrier after the set-up, and nothing but the few logits that can win the
+// arg-max is looked at twice.  Rows that are not MASKED are never read.
 //
 // Noise (temperature > 0).  The Gumbel draws are g = -ln(E) with E an exponential race over groups
-// of 16 consecutive ids: one 32-bit word R per group (a Philox block serves the four groups that a
-// thread meets in four consecutive iterations) fixes the "leader" 16 j + R % 16, which holds the
-// group's smallest E = -ln(U) / 16, U = ((R >> 4) + (f + 0.5) 2^-23) / 2^28; every other id of the
-// group has E = E_leader - ln((f + 0.5) 2^-23) with 23 fine bits f of its own (second Philox
-// stream, one block per 4 ids).  The word alone bounds all 16 draws, which is what makes the
-// kernel cheap: the streaming pass tests one word per 16 logits, and the second stream and the
-// logarithms are spent only on
-//   (1) the leaders of the groups whose word lies in the top 2^-b of its range (b = 2..6, so that
-//       a segment has 128 to 256 such groups), whose best exact score L is a lower bound of the
-//       segment's best score, and
-//   (2) the ids of threads whose largest logit could still beat L with the largest draw any other
-//       group allows (g < 6.9237 for b = 6), filtered once more by their own group's bound.
+// of 16 consecutive ids: group j has the 32-bit word R = word j % 4 of Philox block j / 4 (so the 64
+// ids of a lane share one block), which fixes the "leader" 16 j + R % 16 holding the group's
+// smallest E = -ln(U) / 16, U = ((R >> 4) + (f + 0.5) 2^-23) / 2^28; every other id of the group has
+// E = E_leader - ln((f + 0.5) 2^-23) with 23 fine bits f of its own (second Philox stream, one block
+// per 4 ids).  The word alone bounds all 16 draws from above, g < 32 ln 2 - ln(2^28 - 1 - (R >> 4)),
+// and the leader's draw from below, which is what makes the kernel cheap.  While a lane's 64 ids
+// are in shared memory the streaming pass takes the largest of their four words and forms
+//   an upper bound of every score of the block: its largest logit + T * (bound of that word), and
+//   a lower bound of one score: the logit of that word's leader + T * (lower bound of its draw);
+// the warp keeps the largest lower bound so far, L (also: the largest logit so far with the smallest
+// draw there is), and notes the blocks whose upper bound reaches it in a short list in shared
+// memory.  After the piece L is a lower bound of the piece's best score, and only the noted blocks
+// that still reach it (a handful) are read again, from L2, and scored exactly with the second
+// stream, one group of 16 ids per lane.
 // Any id left out cannot reach L, so the arg-max (lowest id on ties) is exact.
 //
-// Kernel 2 (unmask_finalize_kernel): one CTA per rollout merges the segment records of its
-// rows, forms the confidences and applies the threshold / at-least-one rule.
+// Kernel 2 (unmask_finalize_kernel): one CTA per rollout merges the records of its rows, forms the
+// confidences and applies the threshold / at-least-one rule.
 #include "fdd_internal.h"
+#include "tc_ptx.cuh"
 
 #include <math_constants.h>
 
+#include <atomic>
+
 namespace {
 
-constexpr int kThreads = 256;
-constexpr int kGroup = 16;                            // consecutive entries per load and per coarse Philox block
-constexpr int kSegQuantum = kThreads * kGroup;        // ids a CTA covers per iteration (4096); segment lengths are multiples of it
-constexpr int kMaxCand = 512;                         // groups with a top word kept per segment (148 expected for a 152k row)
-constexpr int kMaxRows = kUnmaskMaxRows;              // rows whose state fits the CTA's compaction buffer
-// "Top" words: the upper 2^-b of the word range, b chosen per launch so that a segment has 128 to
-// 256 top-word groups (b = 6 for whole rows of 152k ids, b = 2 for 8192-id segments).  Every draw
-// of the other groups lies below kGumbelPlain[b] > -ln(-ln(1 - 2^-b) / 16).
-constexpr int kTopBitsMin = 2, kTopBitsMax = 6;
-#ifndef FDD_UM_NOISY_CTAS
-#define FDD_UM_NOISY_CTAS 3
-#endif
-constexpr int kNoisyCtasPerSm = FDD_UM_NOISY_CTAS;   // noisy kernel: CTAs per SM (2: four load buffers per thread, 3: two)
-__device__ __forceinline__ float gumbel_plain(int b) {
-    return b == 2 ? 4.0195f : (b == 3 ? 4.7870f : (b == 4 ? 5.5140f : (b == 5 ? 6.2235f : 6.9245f)));
-}
+constexpr int kWarps = 8;                             // per CTA; every warp works alone
+constexpr int kThreads = kWarps * 32;
+constexpr int kGroup = 16;                            // ids per group of the noise construction
+constexpr int kLaneIds = 64;                          // consecutive ids a lane takes per tile: one Philox block of group words
+constexpr int kTile = kUnmaskTile;                    // ids per tile (one bulk copy, one warp)
+constexpr int kStages = 3;                            // tiles a warp holds in shared memory (two in flight while one is reduced)
+constexpr int kMaxRows = kUnmaskMaxRows;              // rows of one launch (32 per thread in the set-up)
+constexpr int kMaxList = 224;                         // blocks in reach of the running lower bound kept per piece (a few dozen expected)
+constexpr long long kCopyWaitLimit = 4000000000LL;    // SM clocks a warp waits for one of its own copies (about two seconds)
+static_assert(kTile == 32 * kLaneIds, "a tile is 64 ids for each of 32 lanes");
+static_assert(kMaxRows <= kThreads * 32, "the set-up gives every thread at most 32 rows");
+
 constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kLn2 = 0.6931471805599453f;
+constexpr float kGumbelMin = -2.95f;                  // no draw is smaller: E <= 36 / 16 + 23 ln 2 + ln 2 < e^2.95
 
 constexpr uint32_t kPhiloxM0 = 0xD2511F53u, kPhiloxM1 = 0xCD9E8D57u;
 constexpr uint32_t kPhiloxW0 = 0x9E3779B9u, kPhiloxW1 = 0xBB67AE85u;
@@ -67,106 +73,63 @@ __device__ __forceinline__ uint4 philox4x32_10(uint4 c, uint2 k) {
     }
     return c;
 }
-
-// Philox block and word of group j (16 ids): the four words of a block go to groups 256 apart.
-__device__ __forceinline__ uint32_t group_counter(int j) { return static_cast<uint32_t>((j >> 10) * 256 + (j & 255)); }
 __device__ __forceinline__ uint32_t pick_word(const uint4& r, int k) {
     return k == 0 ? r.x : (k == 1 ? r.y : (k == 2 ? r.z : r.w));
 }
 
-// E of a group's leader: -ln(U) / 16, U = (h + (f + 0.5) 2^-23) / 2^28, h = R >> 4.  In the upper
-// half the logarithm goes through 1 - U, which fp32 holds almost exactly there.
-__device__ __forceinline__ float leader_exponential(uint32_t R, uint32_t f23) {
-    const uint32_t h = R >> 4;
-    const float frac = (static_cast<float>(f23) + 0.5f) * 1.1920928955078125e-07f;
-    float nl;                                               // -ln(U)
-    if (h >= (1u << 27)) {
-        const float y = (static_cast<float>((1u << 28) - h) - frac) * 3.7252902984619140625e-09f;   // 1 - U
-        nl = -log1pf(-y);
-    } else {
-        nl = 19.408121055678468f - logf(static_cast<float>(h) + frac);                              // 28 ln 2 - ln(2^28 U)
-    }
-    return nl * 0.0625f;
-}
-// Lower bound of the leader's E (so of every E of the group) from the word alone.
-__device__ __forceinline__ float group_floor(uint32_t R) {
-    const float hp = static_cast<float>((R >> 4) + 1u);     // rounds to nearest: the slack below covers it
-    return fmaxf(19.408121055678468f - logf(hp), 0.0f) * 0.0625f * 0.999f;
-}
-// E of an id that is not its group's leader: the leader's plus -ln((f + 0.5) 2^-23).
-__device__ __forceinline__ float follower_exponential(float e_leader, uint32_t f23) {
-    return e_leader + (15.942385152878742f - logf(static_cast<float>(f23) + 0.5f));                 // 23 ln 2 - ln(f + 0.5)
+// One bulk asynchronous copy global -> shared of this CTA; `bytes` and both addresses are multiples
+// of 16.  Completion is counted in bytes on the mbarrier.
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar)
+                 : "memory");
 }
 
-__device__ __forceinline__ float ex2_fast(float x) {
-    float y;
-    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-    return y;
+// Wait for one of the warp's own copies; false once the time limit has run out.
+__device__ __forceinline__ bool wait_copy(uint32_t bar, uint32_t parity) {
+    if (tc::mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    while (!tc::mbar_try_wait(bar, parity))
+        if (clock64() - t0 > kCopyWaitLimit) return false;
+    return true;
 }
-__device__ __forceinline__ float max3f(float a, float b, float c) {
-    float d;
-    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
-    return d;
-}
-
-__device__ __forceinline__ void load32(const void* p, uint32_t (&r)[8]) {
-    asm volatile("ld.global.L1::no_allocate.v8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
-                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
-                 : "l"(p));
+// Position of the (k + 1)-th set bit of mask (k < popc(mask)).
+__device__ __forceinline__ int nth_set_bit(uint32_t mask, int k) {
+    for (; k > 0; --k) mask &= mask - 1;
+    return __ffs(mask) - 1;
 }
 
-// Asynchronous 16-byte copies global -> shared (the thread that issues them also waits for them).
-__device__ __forceinline__ void cp_async16(void* smem_dst, const void* gsrc) {
-    const uint32_t d = static_cast<uint32_t>(__cvta_generic_to_shared(smem_dst));
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(d), "l"(gsrc) : "memory");
-}
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
-template <int N>
-__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
-
-// Ring of bf16 groups in shared memory: every thread owns 32 bytes per stage, fills them with
-// asynchronous copies several groups ahead and reads only what it copied itself (no barrier).
-constexpr int kRingStages = 4;
-constexpr int kRingStageBytes = kThreads * kGroup * 2;
-
-// A group = 16 consecutive logits.  fetch() starts the 32-byte loads of a group into raw words,
-// widen() turns the words into fp32 once they are needed (so several groups can be in flight).
 template <typename T> struct Logit;
 template <> struct Logit<__nv_bfloat16> {
-    static constexpr int kWords = 8;
-    __device__ static void fetch(const __nv_bfloat16* p, uint32_t (&w)[kWords]) { load32(p, w); }
-    __device__ static void widen(const uint32_t (&w)[kWords], float* out) {
+    static constexpr int kPerChunk = 8;                  // logits per 16-byte chunk
+    __device__ static float load1(const __nv_bfloat16* p) { return __bfloat162float(*p); }
+    __device__ static __nv_bfloat16 minus_inf() { return __ushort_as_bfloat16(0xFF80u); }
+    __device__ static void widen(const uint4& w, float* out) {
+        const uint32_t x[4] = {w.x, w.y, w.z, w.w};
 #pragma unroll
-        for (int i = 0; i < 8; ++i) {
-            out[2 * i] = __uint_as_float(w[i] << 16);
-            out[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u);
+        for (int i = 0; i < 4; ++i) {
+            out[2 * i] = __uint_as_float(x[i] << 16);
+            out[2 * i + 1] = __uint_as_float(x[i] & 0xFFFF0000u);
         }
     }
-    __device__ static float load1(const __nv_bfloat16* p) { return __bfloat162float(*p); }
 };
 template <> struct Logit<float> {
-    static constexpr int kWords = 16;
-    __device__ static void fetch(const float* p, uint32_t (&w)[kWords]) {
-        uint32_t a[8], b[8];
-        load32(p, a);
-        load32(p + 8, b);
-#pragma unroll
-        for (int i = 0; i < 8; ++i) { w[i] = a[i]; w[8 + i] = b[i]; }
-    }
-    __device__ static void widen(const uint32_t (&w)[kWords], float* out) {
-#pragma unroll
-        for (int i = 0; i < 16; ++i) out[i] = __uint_as_float(w[i]);
-    }
+    static constexpr int kPerChunk = 4;
     __device__ static float load1(const float* p) { return *p; }
+    __device__ static float minus_inf() { return -CUDART_INF_F; }
+    __device__ static void widen(const uint4& w, float* out) {
+        out[0] = __uint_as_float(w.x); out[1] = __uint_as_float(w.y);
+        out[2] = __uint_as_float(w.z); out[3] = __uint_as_float(w.w);
+    }
 };
 
-// 16 logits starting at vocabulary id v0 (a multiple of 16); ids >= vocab read as -inf.
+// 16 logits starting at vocabulary id v0 (a multiple of 16), from global memory; ids >= vocab read as -inf.
 template <typename T>
 __device__ __forceinline__ void load_group(const T* row_ptr, int v0, int vocab, int vec_ok, float* val) {
     if (vec_ok && v0 + kGroup <= vocab) {
-        uint32_t w[Logit<T>::kWords];
-        Logit<T>::fetch(row_ptr + v0, w);
-        Logit<T>::widen(w, val);
+        const uint4* p = reinterpret_cast<const uint4*>(row_ptr + v0);
+#pragma unroll
+        for (int c = 0; c < kGroup / Logit<T>::kPerChunk; ++c) Logit<T>::widen(p[c], val + c * Logit<T>::kPerChunk);
     } else {
 #pragma unroll
         for (int j = 0; j < kGroup; ++j) val[j] = (v0 + j < vocab) ? Logit<T>::load1(row_ptr + v0 + j) : -CUDART_INF_F;
@@ -194,393 +157,440 @@ __device__ __forceinline__ Best warp_best(Best b) {
     return b;
 }
 
+// ---- phase 2 of the noisy step: exact scores of the 16 ids of one group.
+struct RowNoise {                                       // what fixes the draws of one row
+    uint2 keys;                                         // the rollout's seed
+    uint32_t pos, step, block_idx;
+};
+// Upper bound of every draw of a group from its word alone: U < (h + 1) / 2^28 = 1 - d / 2^28 with
+// d = 2^28 - 1 - h, so -ln U > d / 2^28, E > d / 2^32 and g < 32 ln 2 - ln d (no bound for d = 0).
+__device__ __forceinline__ float word_gumbel_bound(uint32_t R) {
+    const uint32_t d = 0x0FFFFFFFu - (R >> 4);
+    return d == 0u ? CUDART_INF_F : 22.18070977791825f - __logf(static_cast<float>(d)) + 1e-3f;
+}
+// E of a group's leader, -ln(U) / 16 with U = (h + (f + 0.5) 2^-23) / 2^28, h = R >> 4, on the fast
+// logarithm (absolute error 4e-7 on [0.5, 2], 3 ulp elsewhere).  In the upper half of the range the
+// logarithm goes through y = 1 - U, which fp32 holds almost exactly there: a series below 2^-6, where
+// the fast logarithm of a number next to 1 would lose the leading digits of -ln U.
+__device__ __forceinline__ float leader_exponential(uint32_t R, uint32_t f23) {
+    const uint32_t h = R >> 4;
+    const float frac = (static_cast<float>(f23) + 0.5f) * 1.1920928955078125e-07f;
+    float nl;                                               // -ln(U)
+    if (h >= (1u << 27)) {
+        const float y = (static_cast<float>((1u << 28) - h) - frac) * 3.7252902984619140625e-09f;   // 1 - U
+        nl = y < 0.015625f ? y * fmaf(y, fmaf(y, fmaf(y, 0.25f, 0.33333334f), 0.5f), 1.0f) : -__logf(1.0f - y);
+    } else {
+        nl = 19.408121055678468f - __logf(static_cast<float>(h) + frac);                            // 28 ln 2 - ln(2^28 U)
+    }
+    return nl * 0.0625f;
+}
+struct ScoreArgs {
+    float lb, temperature;
+    int vocab, vec_ok;
+};
+// The best exact score among the 16 ids of group v0 (score -inf if the group cannot reach the lower
+// bound a.lb, or has no finite logit).  One Philox block for the group's word and four for the fine
+// bits of its ids, all independent of each other and of the load; every id is then scored, without a
+// branch: E = E_leader for the leader, E_leader - ln((f + 0.5) 2^-23) for the others, g = -ln E.
+template <typename T>
+__device__ __noinline__ Best score_group(const T* row_ptr, int v0, ScoreArgs a, RowNoise n) {
+    Best best{-CUDART_INF_F, -CUDART_INF_F, 0x7FFFFFFF};
+    float val[kGroup];
+    load_group(row_ptr, v0, a.vocab, a.vec_ok, val);
+    const int j = v0 >> 4;
+    const uint32_t R = pick_word(philox4x32_10(make_uint4(static_cast<uint32_t>(j >> 2), n.pos, n.step, n.block_idx), n.keys), j & 3);
+    uint32_t f[kGroup];
+#pragma unroll
+    for (int k = 0; k < kGroup / 4; ++k) {
+        const uint4 r = philox4x32_10(make_uint4(static_cast<uint32_t>((v0 >> 2) + k), n.pos | kFineStream, n.step, n.block_idx), n.keys);
+        f[4 * k] = r.x >> 9; f[4 * k + 1] = r.y >> 9; f[4 * k + 2] = r.z >> 9; f[4 * k + 3] = r.w >> 9;
+    }
+    float gmax = val[0];
+#pragma unroll
+    for (int i = 1; i < kGroup; ++i) gmax = fmaxf(gmax, val[i]);
+    if (!(fmaf(a.temperature, word_gumbel_bound(R), gmax) >= a.lb - 1e-3f)) return best;
+    const int li = static_cast<int>(R & 15u);
+    uint32_t f_lead = f[0];
+#pragma unroll
+    for (int i = 1; i < kGroup; ++i) if (i == li) f_lead = f[i];
+    const float e_lead = leader_exponential(R, f_lead);
+#pragma unroll
+    for (int i = kGroup - 1; i >= 0; --i) {             // downwards: equal scores keep the lower id
+        const float e = i == li ? e_lead : e_lead + (15.942385152878742f - __logf(static_cast<float>(f[i]) + 0.5f));   // 23 ln 2 - ln(f + 0.5)
+        const float sc = fmaf(a.temperature, -__logf(e), val[i]);
+        if (val[i] > -CUDART_INF_F && sc >= best.score) best = Best{sc, val[i], v0 + i};
+    }
+    return best;
+}
+
+// The ri-th selected row (ascending) from the set-up's per-thread runs: thread t owns rows
+// [t * per, (t + 1) * per), s_before[t] selected rows lie before its run, bit k of s_mask[t] says
+// that row t * per + k is selected.
+__device__ __forceinline__ int nth_selected_row(const int* s_before, const uint32_t* s_mask, int per, int ri) {
+    int lo = 0, hi = kThreads - 1;
+    while (lo < hi) {                                    // the last thread with s_before <= ri (its run is not empty)
+        const int mid = (lo + hi + 1) >> 1;
+        if (s_before[mid] <= ri) lo = mid; else hi = mid - 1;
+    }
+    return lo * per + nth_set_bit(s_mask[lo], ri - s_before[lo]);
+}
+
+// A block (the 64 ids of one lane in one tile) whose upper bound reached the running lower bound.
+struct Reach {
+    float ub;            // upper bound of the block's scores
+    uint16_t tile;       // tile inside the piece
+    uint16_t lane;
+};
+static_assert(sizeof(Reach) == 8, "eight bytes per kept block");
+
+// Shared memory of the streaming kernel beyond its static arrays: the rings, the lists of kept blocks, the barriers.
+template <typename T>
+constexpr int stream_smem_bytes() {
+    return kWarps * kStages * kTile * static_cast<int>(sizeof(T)) + kWarps * kMaxList * 8 + kWarps * kStages * 8;
+}
+
 template <typename T, bool NOISY>
-__global__ void __launch_bounds__(kThreads, NOISY ? kNoisyCtasPerSm : 3)
-unmask_partial_kernel(const T* __restrict__ logits, const uint8_t* __restrict__ state,
-                      const __grid_constant__ UnmaskSets sets, UnmaskPartial* __restrict__ partial,
-                      int vocab, int n_chunks, float temperature,
-                      uint32_t block_idx, uint32_t step, int vec_ok, int select_state,
-                      const uint32_t* __restrict__ step_counter) {
+__global__ void __launch_bounds__(kThreads, sizeof(T) == 2 ? 2 : 1)
+unmask_stream_kernel(const T* __restrict__ logits, const uint8_t* __restrict__ state,
+                     const __grid_constant__ UnmaskSets sets, UnmaskPartial* __restrict__ partial,
+                     int vocab, int tiles_per_item, float temperature,
+                     uint32_t block_idx, uint32_t step, int bulk_ok, int select_state,
+                     const uint32_t* __restrict__ step_counter, int* __restrict__ status) {
     if (step_counter != nullptr) step += *step_counter;    // the denoising step as counted on the device
     const int rows = sets.row_off[sets.n_sets];
-    __shared__ uint16_t s_rows[kMaxRows];               // the selected rows (MASKED, or DRAFT for the verifier), ascending
-    __shared__ int s_n_rows;
-    __shared__ int s_warp_count[kThreads / 32];
-    __shared__ int s_cand[kMaxCand];                    // groups with a top word: first id of the group ...
-    __shared__ uint32_t s_cand_word[kMaxCand];          // ... the word ...
-    __shared__ float s_cand_e[kMaxCand];                // ... and its leader's E, once known
-    __shared__ int s_n_cand;
-    __shared__ uint16_t s_redo[kThreads];               // threads whose groups pass 2 goes over again
-    __shared__ int s_n_redo;
-    __shared__ float red_max[kThreads / 32], red_sum[kThreads / 32], red_score[kThreads / 32];
-    __shared__ Best red_best[kThreads / 32];
+    __shared__ int s_before[kThreads];                  // selected rows before the thread's run
+    __shared__ uint32_t s_mask[kThreads];               // which rows of the thread's run are selected (MASKED, or DRAFT for the verifier)
+    __shared__ int s_warp_count[kWarps];
+    __shared__ int s_n_list[kWarps];
+    extern __shared__ __align__(128) unsigned char s_dyn[];
+    constexpr int kStageBytes = kTile * static_cast<int>(sizeof(T));
+    constexpr int kPerChunk = Logit<T>::kPerChunk;
+    constexpr int kLaneChunks = kLaneIds / kPerChunk;   // 16-byte chunks of a lane's 64 ids: 8 (bf16) or 16 (fp32)
+    constexpr int kLaneGroups = kLaneIds / kGroup;      // groups of a lane's 64 ids
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    constexpr bool noisy = NOISY;                       // temperature > 0
+    unsigned char* ring = s_dyn + warp * (kStages * kStageBytes);
+    Reach* list = reinterpret_cast<Reach*>(s_dyn + kWarps * kStages * kStageBytes) + warp * kMaxList;
+    uint64_t* bars = reinterpret_cast<uint64_t*>(s_dyn + kWarps * kStages * kStageBytes + kWarps * kMaxList * 8) + warp * kStages;
 
-    // Every CTA compacts the list of MASKED rows for itself (the state array is a few KB): a thread
-    // takes a run of consecutive rows, one block-wide prefix sum places the runs.
+    // ---- set-up (the only CTA-wide part): which rows are selected.  A thread takes a run of
+    // consecutive rows, one block-wide prefix sum places the runs.
+    const int per = (rows + kThreads - 1) / kThreads;              // <= 32 (rows <= 8192)
+    int n_rows;
     {
-        const int per = (rows + kThreads - 1) / kThreads;          // <= 32 (rows <= 8192)
         const int r_begin = min(rows, tid * per), r_end = min(rows, r_begin + per);
-        uint32_t mine = 0;                                         // bit k: row r_begin + k is selected
+        uint32_t mine = 0;
         for (int r = r_begin; r < r_end; ++r) mine |= (state[r] == select_state ? 1u : 0u) << (r - r_begin);
         const int cnt = __popc(mine);
-        int incl = cnt;                                            // inclusive prefix sum inside the warp
+        int incl = cnt;
 #pragma unroll
         for (int off = 1; off < 32; off <<= 1) {
             const int up = __shfl_up_sync(0xFFFFFFFFu, incl, off);
             if (lane >= off) incl += up;
         }
         if (lane == 31) s_warp_count[warp] = incl;
+        if (lane == 0) {
+            s_n_list[warp] = 0;
+            if (bulk_ok) {
+                for (int s = 0; s < kStages; ++s) tc::mbar_init(tc::smem_u32(&bars[s]), 1);
+                tc::fence_barrier_init();
+            }
+        }
         __syncthreads();
         int before = incl - cnt, total = 0;
 #pragma unroll
-        for (int w2 = 0; w2 < kThreads / 32; ++w2) {
+        for (int w2 = 0; w2 < kWarps; ++w2) {
             if (w2 < warp) before += s_warp_count[w2];
             total += s_warp_count[w2];
         }
-        while (mine) {
-            const int k = __ffs(mine) - 1;
-            mine &= mine - 1;
-            s_rows[before++] = static_cast<uint16_t>(r_begin + k);
-        }
-        if (tid == 0) { s_n_rows = total; s_n_cand = 0; s_n_redo = 0; }
+        s_before[tid] = before;
+        s_mask[tid] = mine;
+        n_rows = total;
         __syncthreads();
     }
-    const int n_rows = s_n_rows;
     if (n_rows == 0) return;
-    // The selected rows, cut into chunks of 8192 ids and laid end to end, are split into equal
-    // contiguous ranges, one per CTA: a CTA's range is the tail of one row, some whole rows and the
-    // head of another, and every (row, CTA) pair leaves one record (at most n_chunks per row).  With
-    // few rows every chunk gets its own CTA.  Every CTA derives the same numbers.
-    const long long W = static_cast<long long>(n_rows) * n_chunks;
-    const long long G = min(static_cast<long long>(gridDim.x), W);
-    if (blockIdx.x >= G) return;
-    const long long range_begin = W * blockIdx.x / G, range_end = W * (blockIdx.x + 1) / G;
 
-    for (long long at = range_begin; at < range_end;) {
-        const int ri = static_cast<int>(at / n_chunks);
-        const int chunk0 = static_cast<int>(at - static_cast<long long>(ri) * n_chunks);
-        const int chunk1 = static_cast<int>(min(static_cast<long long>(n_chunks), chunk0 + (range_end - at)));
+    // ---- this warp's range of work items.  An item is tiles_per_item consecutive tiles of a row
+    // (the last item of a row may be shorter); a row has items_per_row of them and as many record
+    // slots.  Warp c (of the G that get work) owns items [W c / G, W (c + 1) / G).
+    const int tiles_per_row = (vocab + kTile - 1) / kTile;
+    const int ipr = (tiles_per_row + tiles_per_item - 1) / tiles_per_item;
+    const long long W = static_cast<long long>(n_rows) * ipr;
+    const long long G = min(static_cast<long long>(gridDim.x) * kWarps, W);
+    const long long gw = static_cast<long long>(warp) * gridDim.x + blockIdx.x;   // warps of a CTA lie a grid apart: few items spread over all SMs
+    if (gw >= G) return;
+    const long long range_begin = W * gw / G, range_end = W * (gw + 1) / G;
+
+    const uint32_t full = 0xFFFFFFFFu;
+    const int sw = lane & 7;                            // rotation of the chunk order (bank conflicts)
+    bool alive = true;                                  // false once a wait for a copy ran out
+
+    // ---- producer side (lane 0 issues, every lane keeps the same cursor): tile p_k of the warp's
+    // sequence goes to stage p_k % kStages
+    long long p_at = range_begin;                       // next item to open
+    int p_tile = 0, p_tile_end = 0;
+    const T* p_row_ptr = nullptr;
+    uint32_t p_k = 0;
+    auto produce_one = [&]() {
+        if (!bulk_ok) return;
+        if (p_tile == p_tile_end) {
+            if (p_at >= range_end) return;
+            const int ri = static_cast<int>(p_at / ipr);
+            const int c0 = static_cast<int>(p_at - static_cast<long long>(ri) * ipr);
+            const int c1 = static_cast<int>(min(static_cast<long long>(ipr), c0 + (range_end - p_at)));
+            p_at += c1 - c0;
+            p_tile = c0 * tiles_per_item;
+            p_tile_end = min(tiles_per_row, c1 * tiles_per_item);
+            p_row_ptr = logits + static_cast<size_t>(nth_selected_row(s_before, s_mask, per, ri)) * vocab;
+        }
+        if (lane == 0) {
+            const int v0 = p_tile * kTile;
+            const uint32_t bytes = static_cast<uint32_t>(min(kTile, vocab - v0)) * sizeof(T);
+            const uint32_t bar = tc::smem_u32(&bars[p_k % kStages]);
+            tc::mbar_arrive_expect_tx(bar, bytes);
+            bulk_load(tc::smem_u32(ring + (p_k % kStages) * kStageBytes), p_row_ptr + v0, bytes, bar);
+        }
+        ++p_tile;
+        ++p_k;
+    };
+    for (int s = 0; s < kStages; ++s) produce_one();
+
+    uint32_t c_k = 0;                                   // tiles consumed so far
+    for (long long at = range_begin; at < range_end && alive;) {
+        // ---- open the piece: items [at, at + n) of one row
+        const int ri = static_cast<int>(at / ipr);
+        const int chunk0 = static_cast<int>(at - static_cast<long long>(ri) * ipr);
+        const int chunk1 = static_cast<int>(min(static_cast<long long>(ipr), chunk0 + (range_end - at)));
         at += chunk1 - chunk0;
-        const int row = s_rows[ri];
-        const int seg_begin = chunk0 * kUnmaskChunk;
-        const int seg_end = min(vocab, chunk1 * kUnmaskChunk);
-        // which of the row's records this is, and how many there are (CTA c owns chunks [W c / G, W (c + 1) / G))
-        const long long row_first = static_cast<long long>(ri) * n_chunks;
-        const int cta_first = static_cast<int>(((row_first + 1) * G + W - 1) / W) - 1;
-        const int cta_last = static_cast<int>(((row_first + n_chunks) * G + W - 1) / W) - 1;
-        const int seg = static_cast<int>(blockIdx.x) - cta_first;
-        const int segs = cta_last - cta_first + 1;
-        // 2^-top_bits of the groups get their leader scored at once: 128 to 256 groups of this piece
-        int top_bits = kTopBitsMin;
-        while (top_bits < kTopBitsMax && ((seg_end - seg_begin) >> 4) >> (top_bits + 1) >= 128) ++top_bits;
-        const uint32_t top_word = 0xFFFFFFFFu << (32 - top_bits);
+        const int tile0 = chunk0 * tiles_per_item, tile1 = min(tiles_per_row, chunk1 * tiles_per_item);
+        const int row = nth_selected_row(s_before, s_mask, per, ri);
+        const int seg_end = min(vocab, tile1 * kTile);
+        // which of the row's records this is, and how many there are
+        const long long row_first = static_cast<long long>(ri) * ipr;
+        const int w_first = static_cast<int>(((row_first + 1) * G + W - 1) / W) - 1;
+        const int w_last = static_cast<int>(((row_first + ipr) * G + W - 1) / W) - 1;
+        const int seg = static_cast<int>(gw) - w_first;
+        const int segs = w_last - w_first + 1;
         const T* row_ptr = logits + static_cast<size_t>(row) * vocab;
         int set = 0;
         while (set + 1 < sets.n_sets && row >= sets.row_off[set + 1]) ++set;
         const int local = row - sets.row_off[set];
         const int fork = local / sets.d[set], pos = local - fork * sets.d[set];   // rollout inside its set
         uint2 keys = make_uint2(0u, 0u);
-        if (noisy) {
+        if (NOISY) {
             const uint64_t seed = sets.seeds[set][fork];
             keys = make_uint2(static_cast<uint32_t>(seed), static_cast<uint32_t>(seed >> 32));
         }
 
-        // ---- pass 1: stream the segment; running soft-max statistics, coarse bytes, candidates
-        float m = -CUDART_INF_F, s = 0.0f;             // thread's running max and sum exp(l - m)
+        // ---- pass 1: stream the piece; per lane the running maximum m and sum exp(l - m).  The greedy
+        // step also keeps the first tile t1 that showed m (u1 = m there); the noisy step keeps the warp's
+        // running lower bound lb of the piece's best score and lists the blocks that reach it.
+        float m = -CUDART_INF_F, s = 0.0f, nml = 0.0f;  // nml = -m log2(e) once m is finite
+        float u1 = -CUDART_INF_F, lb = -CUDART_INF_F;
+        int t1 = tile0;
         Best best{-CUDART_INF_F, -CUDART_INF_F, 0x7FFFFFFF};
-        // One group: `w` holds its raw words if it could be fetched with the wide loads.
-        auto process = [&](int v0, const uint32_t (&w)[Logit<T>::kWords], uint32_t R) {
-            float val[kGroup];
-            if (vec_ok && v0 + kGroup <= vocab) {
-                Logit<T>::widen(w, val);
+        for (int tile = tile0; tile < tile1; ++tile) {
+            const int stage = c_k % kStages;
+            unsigned char* buf = ring + stage * kStageBytes;
+            const int tile_base = tile * kTile;
+            if (bulk_ok) {
+                if (!wait_copy(tc::smem_u32(&bars[stage]), (c_k / kStages) & 1u)) alive = false;
+                alive = __all_sync(full, alive);
+                if (!alive) break;
             } else {
-#pragma unroll
-                for (int j = 0; j < kGroup; ++j) val[j] = (v0 + j < vocab) ? Logit<T>::load1(row_ptr + v0 + j) : -CUDART_INF_F;
+                // rows that bulk copies cannot address (odd vocabulary, unaligned base): the warp fills the stage itself
+                T* dst = reinterpret_cast<T*>(buf);
+                for (int i = lane; i < kTile; i += 32)
+                    dst[i] = (tile_base + i < vocab) ? row_ptr[tile_base + i] : Logit<T>::minus_inf();
+                __syncwarp();
             }
-            float g4[4];
+            const int vb = tile_base + lane * kLaneIds;  // first id of the lane's 64
+            const uint4* sp = reinterpret_cast<const uint4*>(buf) + lane * kLaneChunks;
+            const T* lp = reinterpret_cast<const T*>(buf) + lane * kLaneIds;
+            float bm64 = -CUDART_INF_F;
+            const bool whole = tile_base + kTile <= seg_end;
+            if (whole) {
+                // whole tile: two halves of 32 logits, chunk c of the lane read from place c ^ sw (the
+                // eight lanes of a quarter warp then touch eight different 16-byte columns of the banks)
 #pragma unroll
-            for (int u = 0; u < 4; ++u) g4[u] = max3f(val[4 * u], val[4 * u + 1], fmaxf(val[4 * u + 2], val[4 * u + 3]));
-            const float gm = fmaxf(fmaxf(g4[0], g4[1]), fmaxf(g4[2], g4[3]));
-            if (gm > -CUDART_INF_F) {
-                if (!noisy && gm > m) {
-                    // greedy: the arg-max so far moves into this group; find its first place
-                    int at = kGroup;
+                for (int h = 0; h < 2; ++h) {
+                    float v[32];
+#pragma unroll
+                    for (int c = 0; c < kLaneChunks / 2; ++c)
+                        Logit<T>::widen(sp[(h * (kLaneChunks / 2) + c) ^ sw], v + c * kPerChunk);
+                    float g8[8];
+#pragma unroll
+                    for (int u = 0; u < 8; ++u) g8[u] = tc::max3(v[4 * u], v[4 * u + 1], fmaxf(v[4 * u + 2], v[4 * u + 3]));
+                    const float bm = tc::max3(tc::max3(g8[0], g8[1], g8[2]), tc::max3(g8[3], g8[4], g8[5]), fmaxf(g8[6], g8[7]));
+                    bm64 = fmaxf(bm64, bm);
+                    if (bm > m) {
+                        // rescale by 2^((m - bm) log2 e); the rounded nml must not enter here
+                        s *= tc::ex2((m - bm) * kLog2e);
+                        m = bm;
+                        nml = -bm * kLog2e;
+                    }
+                    // packed fp32x2 arithmetic: one FMA and one add per two logits
+                    const uint64_t l2e2 = tc::pack2(kLog2e, kLog2e), nm2 = tc::pack2(nml, nml);
+                    uint64_t acc[2] = {tc::pack2(0.f, 0.f), tc::pack2(0.f, 0.f)};
+#pragma unroll
+                    for (int i = 0; i < 32; i += 2) {
+                        float x0, x1;
+                        tc::unpack2(tc::fma2(tc::pack2(v[i], v[i + 1]), l2e2, nm2), x0, x1);
+                        acc[(i >> 1) & 1] = tc::add2(acc[(i >> 1) & 1], tc::pack2(tc::ex2(x0), tc::ex2(x1)));
+                    }
+                    float a0, a1;
+                    tc::unpack2(tc::add2(acc[0], acc[1]), a0, a1);
+                    s += a0 + a1;
+                }
+            } else {
+                // the row's last tile: ids from seg_end on do not exist
+                for (int e = 0; e < kLaneIds; ++e)
+                    if (vb + e < seg_end) bm64 = fmaxf(bm64, Logit<T>::load1(lp + e));
+                if (bm64 > m) {
+                    s *= tc::ex2((m - bm64) * kLog2e);
+                    m = bm64;
+                    nml = -bm64 * kLog2e;
+                }
+                float add = 0.0f;
+                for (int e = 0; e < kLaneIds; ++e)
+                    if (vb + e < seg_end) add += tc::ex2(fmaf(Logit<T>::load1(lp + e), kLog2e, nml));
+                s += add;
+            }
+            if (!NOISY) {
+                if (bm64 > u1) { u1 = bm64; t1 = tile; }   // strictly: t1 is the first tile that holds the lane's maximum
+            } else {
+                // The block's four words: the largest one bounds every draw of the block, and its group's
+                // leader gives a score that exists.  d = 2^28 - 1 - (R >> 4), cut to 23 bits (d5 = d / 32,
+                // rounded down) so that it turns into a float exactly; both bounds stay on the safe side.
+                const uint4 rq = philox4x32_10(make_uint4(static_cast<uint32_t>(vb >> 6), pos, step, block_idx), keys);
+                uint32_t rmax;
+                int gp;                                 // the group (of the block's four) that holds rmax
+                if (whole) {
+                    const uint32_t r01 = max(rq.x, rq.y), r23 = max(rq.z, rq.w);
+                    rmax = max(r01, r23);
+                    gp = rmax == rq.x ? 0 : (rmax == rq.y ? 1 : (rmax == rq.z ? 2 : 3));
+                } else {
+                    rmax = rq.x;                        // (group 0 exists: the block does)
+                    gp = 0;
+#pragma unroll
+                    for (int g = 1; g < kLaneGroups; ++g)
+                        if (vb + g * kGroup < seg_end && pick_word(rq, g) > rmax) { rmax = pick_word(rq, g); gp = g; }
+                }
+                const uint32_t d5 = (0x0FFFFFFFu - (rmax >> 4)) >> 5;
+                const float fd5 = __uint_as_float(0x4B000000u | d5) - 8388608.0f;          // d5 as a float, exactly
+                // g < 32 ln 2 - ln d <= 27 ln 2 - ln d5
+                const float g_hi = d5 == 0u ? CUDART_INF_F : fmaf(-kLn2, __log2f(fd5), 18.71497388f + 2e-3f);
+                // g_leader >= 32 ln 2 - ln((d + 1) (1 + y)), y = (d + 1) / 2^28 <= 1 / 2; d + 1 <= 32 (d5 + 1)
+                const float y = (fd5 + 1.0f) * 1.1920928955078125e-07f;                     // >= (d + 1) / 2^28
+                const float g_lo = y <= 0.5f ? fmaf(-kLn2, __log2f(fd5 + 1.0f), 18.71497388f - 2e-3f) - y : kGumbelMin;
+                const int li = gp * kGroup + static_cast<int>(rmax & 15u);
+                // a score that exists in this block: that leader's, or the largest logit's with the smallest draw there is
+                float lo = bm64 > -CUDART_INF_F ? fmaf(temperature, kGumbelMin, bm64) : -CUDART_INF_F;
+                if (vb + li < seg_end) lo = fmaxf(lo, fmaf(temperature, g_lo, Logit<T>::load1(lp + li)));
+#pragma unroll
+                for (int off = 16; off > 0; off >>= 1) lo = fmaxf(lo, __shfl_xor_sync(full, lo, off));
+                lb = fmaxf(lb, lo);
+                const float ub = fmaf(temperature, g_hi, bm64);
+                if (bm64 > -CUDART_INF_F && ub >= lb - 1e-3f) {
+                    const int slot = atomicAdd(&s_n_list[warp], 1);
+                    if (slot < kMaxList) list[slot] = Reach{ub, static_cast<uint16_t>(tile - tile0), static_cast<uint16_t>(lane)};
+                }
+            }
+            __syncwarp();                               // every lane is done with the stage
+            produce_one();                              // tile c_k + kStages goes into it
+            ++c_k;
+        }
+        if (!alive) break;
+
+        if (NOISY) {
+            // ---- pass 2: lb is now a lower bound of the piece's best score.  The listed blocks that still
+            // reach it are read again (the piece has just gone through L2) and scored exactly, group by
+            // group: a turn deals out eight blocks, one group per lane, so that the loads are in flight
+            // together.  (A list that ran over, or a piece of more than 65536 tiles: every block.)
+            __syncwarp();
+            const RowNoise noise{keys, static_cast<uint32_t>(pos), step, block_idx};
+            const ScoreArgs sargs{lb, temperature, vocab, bulk_ok};
+            const float cut = lb - 1e-3f;
+            const int n_seen = *reinterpret_cast<volatile int*>(&s_n_list[warp]);
+            const bool every = n_seen > kMaxList || tile1 - tile0 > 65536;
+            int n_blocks = 0;
+            if (every) {
+                n_blocks = (tile1 - tile0) * 32;
+            } else {
+                // keep the blocks that reach the final bound, in place
+                for (int c0 = 0; c0 < n_seen; c0 += 32) {
+                    const int c = c0 + lane;
+                    Reach r{-CUDART_INF_F, 0, 0};
+                    if (c < n_seen) r = list[c];
+                    const bool keep = r.ub >= cut;
+                    const uint32_t km = __ballot_sync(full, keep);
+                    if (keep) list[n_blocks + __popc(km & ((1u << lane) - 1u))] = r;
+                    n_blocks += __popc(km);
+                    __syncwarp();
+                }
+            }
+            for (int b0 = 0; b0 < n_blocks; b0 += 32 / kLaneGroups) {
+                const int blk = b0 + lane / kLaneGroups;
+                if (blk < n_blocks) {
+                    const int tl = every ? blk / 32 : list[blk].tile, fl = every ? blk % 32 : list[blk].lane;
+                    const int v0 = (tile0 + tl) * kTile + fl * kLaneIds + (lane % kLaneGroups) * kGroup;
+                    if (v0 < seg_end) best = better(best, score_group<T>(row_ptr, v0, sargs, noise));
+                }
+                __syncwarp();
+            }
+            if (lane == 0) s_n_list[warp] = 0;          // the list is empty again for the next piece
+        } else {
+            // ---- greedy: the piece's maximum and its first place.  The lanes that hold the maximum look
+            // for it in the 64 ids of the first tile that showed it (equal values in later tiles have
+            // higher ids).
+            float pm = u1;
+#pragma unroll
+            for (int off = 16; off > 0; off >>= 1) pm = fmaxf(pm, __shfl_xor_sync(full, pm, off));
+            if (pm > -CUDART_INF_F && u1 == pm) {
+                int at_e = 0x7FFFFFFF;
+                const int vb = t1 * kTile + lane * kLaneIds;
+#pragma unroll
+                for (int g = kLaneGroups - 1; g >= 0; --g) {
+                    float val[kGroup];
+                    load_group(row_ptr, vb + g * kGroup, vocab, bulk_ok, val);
 #pragma unroll
                     for (int i = kGroup - 1; i >= 0; --i)
-                        if (val[i] == gm) at = i;
-                    best = Best{gm, gm, v0 + at};
+                        if (val[i] == pm) at_e = vb + g * kGroup + i;
                 }
-                const float mn = fmaxf(m, gm);
-                const float mnl = mn * kLog2e;
-                // packed fp32x2 arithmetic: one FMA and one add per two logits
-                const float2 l2e2 = make_float2(kLog2e, kLog2e), nm2 = make_float2(-mnl, -mnl);
-                float2 s2[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
-#pragma unroll
-                for (int i = 0; i < kGroup; i += 2) {
-                    const float2 x = __ffma2_rn(make_float2(val[i], val[i + 1]), l2e2, nm2);
-                    s2[(i >> 1) & 1] = __fadd2_rn(s2[(i >> 1) & 1], make_float2(ex2_fast(x.x), ex2_fast(x.y)));
-                }
-                const float2 s01 = __fadd2_rn(s2[0], s2[1]);
-                const float sa = s01.x, sb = s01.y;
-                // rescale by 2^((m - mn) log2e): exactly 1 while the maximum stands (the rounded mnl must
-                // not enter here, or a factor 1 + 1e-7 would compound over the groups)
-                s = s * ex2_fast((m - mn) * kLog2e) + (sa + sb);
-                m = mn;
-            }
-            if (noisy && R >= top_word && v0 < vocab) {
-                const int slot = atomicAdd(&s_n_cand, 1);
-                if (slot < kMaxCand) { s_cand[slot] = v0; s_cand_word[slot] = R; }
-            }
-        };
-        auto fetch = [&](int v0, uint32_t (&w)[Logit<T>::kWords]) {
-            if (vec_ok && v0 < seg_end && v0 + kGroup <= vocab) Logit<T>::fetch(row_ptr + v0, w);
-        };
-        if (NOISY && sizeof(T) == 2 && vec_ok) {
-            // noisy step on bf16 rows that allow 16-byte copies: the groups travel through the thread's
-            // slots of the ring (three copies in flight without holding registers); four consecutive
-            // groups of a thread (4096 ids apart) share one Philox block.
-            constexpr int S = kRingStages;
-            extern __shared__ __align__(16) unsigned char s_ring[];
-            const int v_first = seg_begin + tid * kGroup;
-            const int n_g = v_first < seg_end ? (seg_end - v_first + kSegQuantum - 1) / kSegQuantum : 0;
-            const int k0 = (v_first >> 12) & 3;         // word index of the first group inside its Philox block
-            auto issue = [&](int g) {
-                const int v = v_first + g * kSegQuantum;
-                if (g < n_g && v + kGroup <= vocab) {
-                    unsigned char* dst = s_ring + (g % S) * kRingStageBytes + tid * 32;
-                    const unsigned char* src = reinterpret_cast<const unsigned char*>(row_ptr + v);
-                    cp_async16(dst, src);
-                    cp_async16(dst + 16, src + 16);
-                }
-                cp_async_commit();                      // an empty group keeps the count uniform
-            };
-#pragma unroll
-            for (int g = 0; g < S - 1; ++g) issue(g);
-            uint4 rq = make_uint4(0u, 0u, 0u, 0u);
-#pragma unroll 4
-            for (int g = 0; g < n_g; ++g) {
-                issue(g + S - 1);                       // into the slot that was consumed one iteration ago
-                cp_async_wait<S - 1>();                 // group g has landed
-                const int v = v_first + g * kSegQuantum;
-                uint32_t R = 0u;
-                if (noisy) {
-                    const int k = (k0 + g) & 3;
-                    if (g == 0 || k == 0) rq = philox4x32_10(make_uint4(group_counter(v >> 4), pos, step, block_idx), keys);
-                    R = pick_word(rq, k);
-                }
-                uint32_t w[Logit<T>::kWords];
-                const uint4* slot = reinterpret_cast<const uint4*>(s_ring + (g % S) * kRingStageBytes + tid * 32);
-                const uint4 lo = slot[0], hi = slot[1];
-                w[0] = lo.x; w[1] = lo.y; w[2] = lo.z; w[3] = lo.w;
-                w[Logit<T>::kWords - 4] = hi.x; w[Logit<T>::kWords - 3] = hi.y; w[Logit<T>::kWords - 2] = hi.z; w[Logit<T>::kWords - 1] = hi.w;
-                process(v, w, R);
-            }
-            cp_async_wait<0>();
-        } else if (noisy) {
-            // Four iterations (four groups 4096 ids apart) share one Philox block; two register buffers
-            // take turns, so the next group's load is in flight while this one is reduced.
-            constexpr int Q = kSegQuantum;
-            uint32_t wa[Logit<T>::kWords], wb[Logit<T>::kWords];
-            int v0 = seg_begin + tid * kGroup;
-            const int k0 = (v0 >> 12) & 3;              // word index of the first group inside its Philox block
-            fetch(v0, wa);
-            if (k0 != 0 && v0 < seg_end) {
-                // a segment that starts inside a run of four: finish the run (one to three groups)
-                const uint4 rq = philox4x32_10(make_uint4(group_counter(v0 >> 4), pos, step, block_idx), keys);
-                if (k0 < 3) fetch(v0 + Q, wb);
-                process(v0, wa, pick_word(rq, k0));
-                if (k0 < 3 && v0 + Q < seg_end) {
-                    if (k0 < 2) fetch(v0 + 2 * Q, wa);
-                    process(v0 + Q, wb, pick_word(rq, k0 + 1));
-                    if (k0 < 2 && v0 + 2 * Q < seg_end) process(v0 + 2 * Q, wa, rq.w);
-                }
-                v0 += (4 - k0) * Q;
-                fetch(v0, wa);
-            }
-            if (kNoisyCtasPerSm >= 3) {
-                while (v0 < seg_end) {
-                    const uint4 rq = philox4x32_10(make_uint4(group_counter(v0 >> 4), pos, step, block_idx), keys);
-                    fetch(v0 + Q, wb);
-                    process(v0, wa, rq.x);
-                    if (v0 + Q < seg_end) { fetch(v0 + 2 * Q, wa); process(v0 + Q, wb, rq.y); }
-                    if (v0 + 2 * Q < seg_end) { fetch(v0 + 3 * Q, wb); process(v0 + 2 * Q, wa, rq.z); }
-                    if (v0 + 3 * Q < seg_end) { fetch(v0 + 4 * Q, wa); process(v0 + 3 * Q, wb, rq.w); }
-                    v0 += 4 * Q;
-                }
-            } else {
-                // four buffers, three loads in flight
-                uint32_t wc[Logit<T>::kWords], wd[Logit<T>::kWords];
-                fetch(v0 + Q, wb);
-                fetch(v0 + 2 * Q, wc);
-                while (v0 < seg_end) {
-                    const uint4 rq = philox4x32_10(make_uint4(group_counter(v0 >> 4), pos, step, block_idx), keys);
-                    fetch(v0 + 3 * Q, wd);
-                    process(v0, wa, rq.x);
-                    if (v0 + Q < seg_end) { fetch(v0 + 4 * Q, wa); process(v0 + Q, wb, rq.y); }
-                    if (v0 + 2 * Q < seg_end) { fetch(v0 + 5 * Q, wb); process(v0 + 2 * Q, wc, rq.z); }
-                    if (v0 + 3 * Q < seg_end) { fetch(v0 + 6 * Q, wc); process(v0 + 3 * Q, wd, rq.w); }
-                    v0 += 4 * Q;
-                }
-            }
-        } else if (sizeof(T) == 4) {
-            uint32_t wa[Logit<T>::kWords], wb[Logit<T>::kWords];
-            int v0 = seg_begin + tid * kGroup;
-            fetch(v0, wa);
-            while (v0 < seg_end) {
-                fetch(v0 + kSegQuantum, wb);
-                process(v0, wa, 0u);
-                if (v0 + kSegQuantum < seg_end) {
-                    fetch(v0 + 2 * kSegQuantum, wa);
-                    process(v0 + kSegQuantum, wb, 0u);
-                }
-                v0 += 2 * kSegQuantum;
-            }
-        } else {
-            // the greedy step has little arithmetic per logit to hide the memory latency behind: four
-            // buffers, three loads in flight
-            uint32_t wa[Logit<T>::kWords], wb[Logit<T>::kWords], wc[Logit<T>::kWords], wd[Logit<T>::kWords];
-            int v0 = seg_begin + tid * kGroup;
-            fetch(v0, wa);
-            fetch(v0 + kSegQuantum, wb);
-            fetch(v0 + 2 * kSegQuantum, wc);
-            while (v0 < seg_end) {
-                fetch(v0 + 3 * kSegQuantum, wd);
-                process(v0, wa, 0u);
-                if (v0 + kSegQuantum < seg_end) { fetch(v0 + 4 * kSegQuantum, wa); process(v0 + kSegQuantum, wb, 0u); }
-                if (v0 + 2 * kSegQuantum < seg_end) { fetch(v0 + 5 * kSegQuantum, wb); process(v0 + 2 * kSegQuantum, wc, 0u); }
-                if (v0 + 3 * kSegQuantum < seg_end) { fetch(v0 + 6 * kSegQuantum, wc); process(v0 + 3 * kSegQuantum, wd, 0u); }
-                v0 += 4 * kSegQuantum;
+                best = Best{pm, pm, at_e};
             }
         }
 
-        if (noisy) {
-            __syncthreads();
-            // Exact score of an id of group v0 whose word is R; e_leader < 0: not computed yet.
-            auto fine23 = [&](int v) {
-                const uint4 r = philox4x32_10(make_uint4(static_cast<uint32_t>(v >> 2), pos | kFineStream, step, block_idx), keys);
-                return pick_word(r, v & 3) >> 9;
-            };
-            // ---- exact scores of the leaders of the top-word groups: their best is a lower bound L of
-            // the segment's best
-            const int n_cand = s_n_cand;
-            const bool overflow = n_cand > kMaxCand;    // (never for random words) then nothing is pruned
-            if (!overflow) {
-                for (int c = tid; c < n_cand; c += kThreads) {
-                    const int v = s_cand[c] + static_cast<int>(s_cand_word[c] & 15u);
-                    const float e = leader_exponential(s_cand_word[c], fine23(v));
-                    s_cand_e[c] = e;
-                    if (v >= vocab) continue;           // the leader of a cut last group may lie beyond the row
-                    const float l = Logit<T>::load1(row_ptr + v);
-                    best = better(best, Best{fmaf(temperature, -logf(e), l), l, v});
-                }
-            }
-            float lb = best.score;
-#pragma unroll
-            for (int off = 16; off > 0; off >>= 1) lb = fmaxf(lb, __shfl_xor_sync(0xFFFFFFFFu, lb, off));
-            if (lane == 0) red_score[warp] = lb;
-            __syncthreads();
-            lb = red_score[0];
-#pragma unroll
-            for (int w2 = 1; w2 < kThreads / 32; ++w2) lb = fmaxf(lb, red_score[w2]);
-            if (overflow) lb = -CUDART_INF_F;
-            // ---- pass 2: every id that can still reach L is scored exactly.  Two kinds of groups are
-            // gone over again, by the whole CTA (one group per thread): all groups of the threads whose
-            // largest logit can reach L with the largest draw a plain group allows, and the top-word
-            // groups (their other 15 ids are bounded by their leader's draw only).
-            const float reach = lb - temperature * gumbel_plain(top_bits) - 1e-3f;
-            if (m >= reach) {
-                const int slot = atomicAdd(&s_n_redo, 1);
-                if (slot < kThreads) s_redo[slot] = static_cast<uint16_t>(tid);
-            }
-            __syncthreads();
-            const int n_redo = min(s_n_redo, kThreads);
-            const int groups_per_thread = (seg_end - seg_begin + kSegQuantum - 1) / kSegQuantum;
-            const int n_plain = n_redo * groups_per_thread;
-            const int n_top = overflow ? 0 : n_cand;
-            for (int w = tid; w < n_plain + n_top; w += kThreads) {
-                int v0;
-                uint32_t R;
-                bool top;
-                if (w < n_plain) {
-                    const int owner = s_redo[w / groups_per_thread];
-                    v0 = seg_begin + owner * kGroup + (w % groups_per_thread) * kSegQuantum;
-                    if (v0 >= seg_end) continue;
-                } else {
-                    v0 = s_cand[w - n_plain];
-                }
-                float val[kGroup];
-                load_group(row_ptr, v0, vocab, vec_ok, val);
-                float e_lead = -1.0f;                   // < 0: not known yet
-                if (w < n_plain) {
-                    bool some = false;
-#pragma unroll
-                    for (int i = 0; i < kGroup; ++i) some = some || (val[i] >= reach && val[i] > -CUDART_INF_F);
-                    if (!some) continue;
-                    const int j = v0 >> 4;
-                    R = pick_word(philox4x32_10(make_uint4(group_counter(j), pos, step, block_idx), keys), (j >> 8) & 3);
-                    top = R >= top_word;
-                    if (top && !overflow) continue;     // comes again as a top-word group
-                } else {
-                    R = s_cand_word[w - n_plain];
-                    e_lead = s_cand_e[w - n_plain];
-                    top = true;
-                }
-                // the bound every draw of the group obeys: exact for a top-word group, from the word
-                // alone otherwise (the leader's fine bits are fetched only if some id passes it)
-                const int lead = v0 + static_cast<int>(R & 15u);
-                if (top && e_lead < 0.0f) e_lead = leader_exponential(R, fine23(lead));
-                const float bar = lb - 1e-3f - temperature * -logf(top ? e_lead * 0.999f : group_floor(R));
-                uint32_t pass = 0;                      // ids whose logit clears the bar
-#pragma unroll
-                for (int i = 0; i < kGroup; ++i) pass |= (val[i] >= bar && val[i] > -CUDART_INF_F) ? (1u << i) : 0u;
-                while (pass) {
-                    const int i = __ffs(pass) - 1;
-                    pass &= pass - 1;
-                    float l = val[0];
-#pragma unroll
-                    for (int x = 1; x < kGroup; ++x) if (x == i) l = val[x];
-                    const int v = v0 + i;
-                    if (e_lead < 0.0f) e_lead = leader_exponential(R, fine23(lead));
-                    const float e = v == lead ? e_lead : follower_exponential(e_lead, fine23(v));
-                    best = better(best, Best{fmaf(temperature, -logf(e), l), l, v});
-                }
-            }
-        }
-
-        // ---- block reduction
+        // ---- the piece's record
 #pragma unroll
         for (int off = 16; off > 0; off >>= 1) {
-            const float m2 = __shfl_xor_sync(0xFFFFFFFFu, m, off);
-            const float s2 = __shfl_xor_sync(0xFFFFFFFFu, s, off);
-            const float mn = fmaxf(m, m2);
-            if (mn > -CUDART_INF_F) s = s * __expf(m - mn) + s2 * __expf(m2 - mn);
+            const float mx = __shfl_xor_sync(full, m, off);
+            const float sx = __shfl_xor_sync(full, s, off);
+            const float mn = fmaxf(m, mx);
+            if (mn > -CUDART_INF_F) s = s * __expf(m - mn) + sx * __expf(mx - mn);
             m = mn;
         }
         best = warp_best(best);
-        if (lane == 0) { red_max[warp] = m; red_sum[warp] = s; red_best[warp] = best; }
-        __syncthreads();
-        if (tid == 0) {
-            float M = red_max[0], S = red_sum[0];
-            Best B = red_best[0];
-            for (int w2 = 1; w2 < kThreads / 32; ++w2) {
-                const float mn = fmaxf(M, red_max[w2]);
-                if (mn > -CUDART_INF_F) S = S * __expf(M - mn) + red_sum[w2] * __expf(red_max[w2] - mn);
-                M = mn;
-                B = better(B, red_best[w2]);
-            }
+        if (lane == 0) {
             UnmaskPartial out;
-            out.row_max = M; out.sum_exp = S; out.best_score = B.score; out.best_logit = B.logit;
-            out.best_index = B.index;
+            out.row_max = m; out.sum_exp = s; out.best_score = best.score; out.best_logit = best.logit;
+            out.best_index = best.index;
             out.pad[0] = segs;                          // how many records this row has (read from record 0)
             out.pad[1] = out.pad[2] = 0;
-            partial[static_cast<size_t>(row) * n_chunks + seg] = out;
-            s_n_cand = 0;
-            s_n_redo = 0;
+            partial[static_cast<size_t>(row) * ipr + seg] = out;
         }
-        __syncthreads();                                // red_* and the candidate list are reused by the next item
+        __syncwarp();
+    }
+
+    if (!alive) {
+        // A copy did not arrive in time: say so, then give the copies still in flight one more bounded
+        // wait each before the shared memory they write to is handed back.
+        if (lane == 0 && status != nullptr) atomicCAS(status, 0, FDD_ERR_DEVICE_TIMEOUT);
+        for (uint32_t k = c_k; k < p_k; ++k) {
+            const long long t0 = clock64();
+            while (!tc::mbar_try_wait(tc::smem_u32(&bars[k % kStages]), (k / kStages) & 1u))
+                if (clock64() - t0 > kCopyWaitLimit) break;
+        }
     }
 }
 
@@ -588,7 +598,7 @@ __global__ void __launch_bounds__(128)
 unmask_finalize_kernel(const UnmaskPartial* __restrict__ partial, int32_t* __restrict__ tokens,
                        uint8_t* __restrict__ state, int32_t* __restrict__ n_committed,
                        int32_t* __restrict__ n_left, float* __restrict__ conf_out,
-                       const __grid_constant__ UnmaskSets sets, int n_chunks, float threshold, int commit_state,
+                       const __grid_constant__ UnmaskSets sets, int items_per_row, float threshold, int commit_state,
                        uint32_t* __restrict__ step_bump) {
     // (the streaming kernel of this call has read the counter; the next call sees it advanced)
     if (step_bump != nullptr && blockIdx.x == 0 && threadIdx.x == 0) *step_bump += 1u;
@@ -610,7 +620,7 @@ unmask_finalize_kernel(const UnmaskPartial* __restrict__ partial, int32_t* __res
     if (i < d) {
         masked = state[row] == FDD_MASKED;
         if (masked) {
-            const UnmaskPartial* p = partial + static_cast<size_t>(row) * n_chunks;
+            const UnmaskPartial* p = partial + static_cast<size_t>(row) * items_per_row;
             const int n_rec = p[0].pad[0];              // records the first kernel wrote for this row
             float M = -CUDART_INF_F;
             for (int c = 0; c < n_rec; ++c) M = fmaxf(M, p[c].row_max);
@@ -661,7 +671,7 @@ unmask_finalize_kernel(const UnmaskPartial* __restrict__ partial, int32_t* __res
 __global__ void __launch_bounds__(128)
 ss_accept_kernel(const UnmaskPartial* __restrict__ partial, int32_t* __restrict__ tokens,
                  uint8_t* __restrict__ state, int32_t* __restrict__ n_accepted, int32_t* __restrict__ n_left,
-                 const __grid_constant__ UnmaskSets sets, int n_chunks) {
+                 const __grid_constant__ UnmaskSets sets, int items_per_row) {
     const int fork = blockIdx.x;
     const int i = threadIdx.x;
     int set = 0;
@@ -677,7 +687,7 @@ ss_accept_kernel(const UnmaskPartial* __restrict__ partial, int32_t* __restrict_
         st = state[row];
         draft = st == FDD_DRAFT;
         if (draft) {
-            const UnmaskPartial* p = partial + static_cast<size_t>(row) * n_chunks;
+            const UnmaskPartial* p = partial + static_cast<size_t>(row) * items_per_row;
             const int n_rec = p[0].pad[0];
             Best B{-CUDART_INF_F, -CUDART_INF_F, 0x7FFFFFFF};
             for (int c = 0; c < n_rec; ++c) B = better(B, Best{p[c].best_score, p[c].best_logit, p[c].best_index});
@@ -711,71 +721,105 @@ ss_accept_kernel(const UnmaskPartial* __restrict__ partial, int32_t* __restrict_
 
 namespace {
 
+// Per-device set-up of the streaming kernels (they need more dynamic shared memory than a kernel
+// gets without asking) and the device's SM count, done by the first launch on each device.
+constexpr int kMaxDevices = 64;
+std::atomic<int> g_device_ready[kMaxDevices];
+int g_device_sms[kMaxDevices];
+int g_device_ctas[kMaxDevices][4];          // resident CTAs per SM of each instantiation: [bf16 noisy, bf16 greedy, fp32 noisy, fp32 greedy]
+
+template <typename T, bool NOISY>
+cudaError_t setup_one(int* ctas_per_sm) {
+    auto kernel = unmask_stream_kernel<T, NOISY>;
+    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, stream_smem_bytes<T>());
+    // all of the SM's configurable memory as shared memory: two CTAs of the bf16 kernel need 215 KB
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
+    if (e == cudaSuccess) e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(ctas_per_sm, kernel, kThreads, stream_smem_bytes<T>());
+    if (e == cudaSuccess && *ctas_per_sm < 1) e = cudaErrorLaunchOutOfResources;
+    return e;
+}
+
+cudaError_t device_setup(int dev, int* sm_count, const int** ctas_per_sm) {
+    if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+    if (!g_device_ready[dev].load(std::memory_order_acquire)) {
+        int* c = g_device_ctas[dev];
+        cudaError_t e = setup_one<__nv_bfloat16, true>(c + 0);
+        if (e == cudaSuccess) e = setup_one<__nv_bfloat16, false>(c + 1);
+        if (e == cudaSuccess) e = setup_one<float, true>(c + 2);
+        if (e == cudaSuccess) e = setup_one<float, false>(c + 3);
+        int sms = 0;
+        if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+        if (e != cudaSuccess) return e;
+        g_device_sms[dev] = sms > 0 ? sms : 148;
+        g_device_ready[dev].store(1, std::memory_order_release);
+    }
+    *sm_count = g_device_sms[dev];
+    *ctas_per_sm = g_device_ctas[dev];
+    return cudaSuccess;
+}
+
+template <typename T, bool NOISY>
+void launch_stream(const UnmaskProblem& p, UnmaskPartial* partial, int tiles_per_item, int bulk_ok, int select_state,
+                   int* status, int resident_ctas, cudaStream_t st) {
+    const int rows = p.sets.row_off[p.sets.n_sets];
+    const int tiles_per_row = (p.vocab + kTile - 1) / kTile;
+    const long long items = static_cast<long long>(rows) * ((tiles_per_row + tiles_per_item - 1) / tiles_per_item);
+    // persistent: as many CTAs as fit on the SMs, fewer when there is not an item for every warp
+    const long long fit = resident_ctas;
+    const long long need = (items + kWarps - 1) / kWarps;
+    const unsigned grid = static_cast<unsigned>(need < fit ? (need < 1 ? 1 : need) : fit);
+    unmask_stream_kernel<T, NOISY><<<grid, kThreads, stream_smem_bytes<T>(), st>>>(
+        static_cast<const T*>(p.logits), p.state, p.sets, partial, p.vocab, tiles_per_item, p.temperature,
+        p.block_idx, p.step, bulk_ok, select_state, p.step_counter, status);
+}
+
 // Both entry points launch the same two kernels; only the home of the records differs.
 // mode 0: unmasking step; 1: draft of Scaffold Speculative Decoding (every MASKED row becomes DRAFT);
 // 2: its accept scan (rows in state DRAFT are read, then the scan runs).
-cudaError_t launch_unmask_kernels(const UnmaskProblem& p, UnmaskPartial* partial, cudaStream_t st, int mode = 0) {
+// tiles_per_item: how many 2048-id tiles share one record slot (a row has ceil(tiles / tiles_per_item) slots).
+cudaError_t launch_unmask_kernels(const UnmaskProblem& p, UnmaskPartial* partial, int tiles_per_item, int dev,
+                                  int* status, cudaStream_t st, int mode = 0) {
     const int select_state = mode == 2 ? FDD_DRAFT : FDD_MASKED;
     const int rows = p.sets.row_off[p.sets.n_sets];
     const int forks = p.sets.fork_off[p.sets.n_sets];
     if (rows > kMaxRows) return cudaErrorInvalidValue;
-    const int n_chunks = unmask_chunks(p.vocab);
-    static int sm_count = 0;
-    if (sm_count == 0) {
-        int dev = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess ||
-            cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sm_count <= 0)
-            sm_count = 148;
-    }
-    const long long ctas = static_cast<long long>(sm_count) * (p.temperature != 0.0f ? kNoisyCtasPerSm : 3);   // persistent: as many CTAs as fit on the SMs
-    const dim3 grid(static_cast<unsigned>(ctas));
+    int sm_count = 0;
+    const int* per_sm = nullptr;
+    cudaError_t e = device_setup(dev, &sm_count, &per_sm);
+    if (e != cudaSuccess) return e;
+    const int items_per_row = unmask_items_per_row(p.vocab, tiles_per_item);
+    const bool noisy = p.temperature != 0.0f;
+    // bulk copies need 16-byte aligned rows: base and row pitch
     if (p.logits_dtype == FDD_LOGITS_BF16) {
-        const int vec_ok = (p.vocab % 16 == 0) && (reinterpret_cast<uintptr_t>(p.logits) % 32 == 0);
-        // the noisy bf16 kernel streams through a ring in dynamic shared memory (more than the 48 KB a
-        // kernel gets without asking, together with its static arrays)
-        constexpr int kRingNoisy = kRingStages * kRingStageBytes, kRingGreedy = 0;
-        static bool configured = false;
-        if (!configured) {
-            cudaError_t ea = cudaFuncSetAttribute(unmask_partial_kernel<__nv_bfloat16, true>,
-                                                  cudaFuncAttributeMaxDynamicSharedMemorySize, kRingNoisy);
-            if (ea != cudaSuccess) return ea;
-            configured = true;
-        }
-        if (p.temperature != 0.0f)
-            unmask_partial_kernel<__nv_bfloat16, true><<<grid, kThreads, kRingNoisy, st>>>(
-                static_cast<const __nv_bfloat16*>(p.logits), p.state, p.sets, partial, p.vocab,
-                n_chunks, p.temperature, p.block_idx, p.step, vec_ok, select_state, p.step_counter);
-        else
-            unmask_partial_kernel<__nv_bfloat16, false><<<grid, kThreads, kRingGreedy, st>>>(
-                static_cast<const __nv_bfloat16*>(p.logits), p.state, p.sets, partial, p.vocab,
-                n_chunks, p.temperature, p.block_idx, p.step, vec_ok, select_state, p.step_counter);
+        const int bulk_ok = (p.vocab % 8 == 0) && (reinterpret_cast<uintptr_t>(p.logits) % 16 == 0);
+        if (noisy) launch_stream<__nv_bfloat16, true>(p, partial, tiles_per_item, bulk_ok, select_state, status, sm_count * per_sm[0], st);
+        else launch_stream<__nv_bfloat16, false>(p, partial, tiles_per_item, bulk_ok, select_state, status, sm_count * per_sm[1], st);
     } else {
-        const int vec_ok = (p.vocab % 8 == 0) && (reinterpret_cast<uintptr_t>(p.logits) % 32 == 0);
-        if (p.temperature != 0.0f)
-            unmask_partial_kernel<float, true><<<grid, kThreads, 0, st>>>(
-                static_cast<const float*>(p.logits), p.state, p.sets, partial, p.vocab,
-                n_chunks, p.temperature, p.block_idx, p.step, vec_ok, select_state, p.step_counter);
-        else
-            unmask_partial_kernel<float, false><<<grid, kThreads, 0, st>>>(
-                static_cast<const float*>(p.logits), p.state, p.sets, partial, p.vocab,
-                n_chunks, p.temperature, p.block_idx, p.step, vec_ok, select_state, p.step_counter);
+        const int bulk_ok = (p.vocab % 4 == 0) && (reinterpret_cast<uintptr_t>(p.logits) % 16 == 0);
+        if (noisy) launch_stream<float, true>(p, partial, tiles_per_item, bulk_ok, select_state, status, sm_count * per_sm[2], st);
+        else launch_stream<float, false>(p, partial, tiles_per_item, bulk_ok, select_state, status, sm_count * per_sm[3], st);
     }
-    cudaError_t e = cudaGetLastError();
+    e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     if (mode == 2)
-        ss_accept_kernel<<<forks, 128, 0, st>>>(partial, p.tokens, p.state, p.n_committed, p.n_left, p.sets, n_chunks);
+        ss_accept_kernel<<<forks, 128, 0, st>>>(partial, p.tokens, p.state, p.n_committed, p.n_left, p.sets, items_per_row);
     else
         unmask_finalize_kernel<<<forks, 128, 0, st>>>(partial, p.tokens, p.state, p.n_committed, p.n_left, p.conf,
-                                                     p.sets, n_chunks, p.threshold, mode == 1 ? FDD_DRAFT : FDD_COMMITTED,
+                                                     p.sets, items_per_row, p.threshold, mode == 1 ? FDD_DRAFT : FDD_COMMITTED,
                                                      p.bump_counter ? p.step_counter : nullptr);
     return cudaGetLastError();
 }
 
 }  // namespace
 
+size_t unmask_workspace_bytes(int vocab, int max_rows) {
+    const int rows = max_rows < kMaxRows ? max_rows : kMaxRows;      // a launch takes at most kMaxRows rows
+    return static_cast<size_t>(rows) * unmask_items_per_row(vocab, 1) * sizeof(UnmaskPartial);
+}
+
 cudaError_t launch_unmask(fdd_ctx* ctx, const UnmaskProblem& p, cudaStream_t st, int* n_launches, int mode) {
     *n_launches += 2;
-    return launch_unmask_kernels(p, static_cast<UnmaskPartial*>(ctx->ws_unmask), st, mode);
+    return launch_unmask_kernels(p, static_cast<UnmaskPartial*>(ctx->ws_unmask), 1, ctx->device, ctx->d_status, st, mode);
 }
 
 // -------------------------------------------------------------------------------------------------
@@ -787,15 +831,15 @@ cudaError_t launch_unmask(fdd_ctx* ctx, const UnmaskProblem& p, cudaStream_t st,
 namespace {
 
 constexpr int kStaticMaxRecords = FDD_UNMASK_STATIC_MAX_RECORDS;
-constexpr int kStaticMaxDevices = 64;
+constexpr int kStaticTilesPerItem = kUnmaskChunk / kUnmaskTile;    // one record slot per 8192 ids
 
 // Held by every GPU that loads the library until the process exits (2 MiB).
 static __device__ __align__(256) UnmaskPartial g_static_partials[kStaticMaxRecords];
 
 // Device address of g_static_partials per device ordinal, resolved on first use.  In host code the
 // array's name is only a handle for the runtime; the address a kernel can use must be asked for.
-UnmaskPartial* g_static_ptr[kStaticMaxDevices];
-bool g_static_ready[kStaticMaxDevices];
+UnmaskPartial* g_static_ptr[kMaxDevices];
+bool g_static_ready[kMaxDevices];
 
 void put_error(char* err, size_t err_len, const char* text) {
     if (err && err_len) snprintf(err, err_len, "%s", text);
@@ -824,7 +868,14 @@ extern "C" fdd_status fdd_unmask_static(const void* logits, int logits_dtype, in
         put_error(err, err_len, "fdd_unmask_static: block_len above 128 is not supported");
         return FDD_ERR_UNSUPPORTED;
     }
-    const long long records = static_cast<long long>(n_forks) * block_len * unmask_chunks(vocab);
+    const long long n_rows = static_cast<long long>(n_forks) * block_len;
+    if (n_rows > kUnmaskMaxRows) {
+        if (err && err_len)
+            snprintf(err, err_len, "fdd_unmask_static: n_forks * block_len = %lld exceeds the %d rows one call takes",
+                     n_rows, kUnmaskMaxRows);
+        return FDD_ERR_CAPACITY;
+    }
+    const long long records = n_rows * unmask_items_per_row(vocab, kStaticTilesPerItem);
     if (records > kStaticMaxRecords) {
         if (err && err_len)
             snprintf(err, err_len,
@@ -834,7 +885,7 @@ extern "C" fdd_status fdd_unmask_static(const void* logits, int logits_dtype, in
     }
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
-    if (e != cudaSuccess || dev < 0 || dev >= kStaticMaxDevices) {
+    if (e != cudaSuccess || dev < 0 || dev >= kMaxDevices) {
         put_error(err, err_len, "fdd_unmask_static: no usable current CUDA device");
         return FDD_ERR_CUDA;
     }
@@ -858,7 +909,7 @@ extern "C" fdd_status fdd_unmask_static(const void* logits, int logits_dtype, in
     p.sets.d[0] = block_len; p.sets.seeds[0] = seeds;
     p.vocab = vocab; p.logits_dtype = logits_dtype;
     p.threshold = threshold; p.temperature = temperature; p.block_idx = block_idx; p.step = step;
-    e = launch_unmask_kernels(p, g_static_ptr[dev], static_cast<cudaStream_t>(stream));
+    e = launch_unmask_kernels(p, g_static_ptr[dev], kStaticTilesPerItem, dev, nullptr, static_cast<cudaStream_t>(stream));
     if (e != cudaSuccess) {
         if (err && err_len) snprintf(err, err_len, "fdd_unmask_static: launch failed: %s", cudaGetErrorString(e));
         return FDD_ERR_CUDA;

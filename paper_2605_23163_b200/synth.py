@@ -42,7 +42,7 @@ class Workload:
     head_dim: int
     vocab: int
     logits_dtype: str        # "f32" or "bf16"
-    logit_recipe: str        # "normal_sigma2" or "peaked"
+    logit_recipe: str        # "normal_sigma2", "peaked" or "constant"
     threshold: float
     temperature: float
     scenes: tuple
@@ -178,6 +178,8 @@ def make_logits_row(w, scene_idx, block, step, fork, pos):
     the at-least-one rule).  "peaked": iid N(0, 1) with one seeded entry raised
     to logsumexp(rest) + m, m ~ U(0, 6), so the soft-max maximum is sigmoid(m)
     in [0.5, 0.9975] and a threshold of 0.8-0.9 is reached by most rows.
+    "constant": every entry of the row has the same seeded value (the degenerate
+    case in which sampling noise alone decides the token).
     Returns fp32 values ("f32") or bf16 bits ("bf16").
     """
     g = _rng(w, "logits", scene_idx, block, step, fork, pos)
@@ -194,6 +196,8 @@ def make_logits_row(w, scene_idx, block, step, fork, pos):
         mx = float(np.max(r64))
         lse = mx + float(np.log(np.sum(np.exp(r64 - mx))))
         row[t] = np.float32(lse + m)
+    elif w.logit_recipe == "constant":
+        row = np.full(w.vocab, np.float32(g.uniform(-3.0, 3.0)), dtype=np.float32)
     else:
         raise ValueError(w.logit_recipe)
     if w.logits_dtype == "bf16":

@@ -611,6 +611,33 @@ def test_unmask_odd_vocab_and_partial_state():
     assert not info["ambiguous_forks"]
 
 
+@pytest.mark.parametrize("recipe,dtype,vocab,temperature", [
+    ("normal_sigma2", "bf16", 151936, 1.0),
+    ("normal_sigma2", "bf16", 151936, 0.05),
+    ("normal_sigma2", "bf16", 151936, 2.0),
+    ("normal_sigma2", "f32", 8192 * 2 + 1237, 1.0),      # rows that bulk copies cannot address
+    ("normal_sigma2", "f32", 50000, 0.05),
+    ("constant", "bf16", 151936, 1.0),
+    ("constant", "f32", 4099, 0.7),
+])
+def test_unmask_noise_decides_on_flat_and_equal_rows(recipe, dtype, vocab, temperature):
+    # The hard case of the sampled trajectory section: no id towers over the rest, so the noise
+    # decides the arg-max and the pruning of the kernel has to keep every id that can still win.
+    # Threshold below any probability: every MASKED row commits, and every row's token is compared.
+    sc = synth.Scene(prefix_len=16, n_forks=2, block_len=8, n_scaffold=2, n_blocks=1)
+    w = synth.Workload("flat", 4, 1, 64, vocab, dtype, recipe, -1.0, temperature, (sc,), seed=31)
+    for step in (0, 3):
+        info, got, ref = _unmask_step_case(w, step=step)
+        assert info["rows"] == 2 * 6 and not info["ambiguous_forks"] or info["low_margin_rows"] > 0
+        masked = ref["choice"] >= 0
+        clear = masked & (ref["score_margin"] > pu.SCORE_MARGIN)
+        assert clear.sum() >= 2 * 6 - 2
+        assert np.array_equal(got["tokens"][clear], ref["choice"][clear])
+        assert np.all(got["state"][masked] == COMMITTED)
+        if recipe == "constant":
+            assert len(set(got["tokens"][masked].tolist())) >= 8        # the winners are spread over the vocabulary
+
+
 def test_unmask_threshold_extremes():
     w = synth.small_variant(synth.workload("tts"), prefix_len=64, vocab=4096, n_forks=2, n_blocks=1)
     info, got, ref = _unmask_step_case(w, threshold=1.5)          # nothing passes: one commit each

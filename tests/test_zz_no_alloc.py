@@ -5,7 +5,8 @@ pre-allocated buffers, cannot go through fdd_create / fdd_fork, because both all
 memory.  fdd_unmask_static needs neither: its scratch is a fixed array inside the library.  This
 test calls it through the C ABI twice in a row (the second call sees the first call's leftovers in
 the shared scratch) and requires exactly the results of the regular entry point: identical tokens,
-states and counters, confidences within the tolerance the other unmask tests use.
+states and counters, confidences within the tolerance the other unmask tests use.  Both calls are
+also held against the CPU oracle, under the same rules as every other unmask parity test.
 
 Collected last on purpose, so that a run that stops at the first failure has already run every
 other test; it also passes when run on its own in a fresh process.
@@ -14,11 +15,11 @@ import numpy as np
 import pytest
 import torch
 
+from oracle.unmask import unmask_step
 from paper_2605_23163_b200 import fdd, harness, synth
+from parity_utils import CONF_TOL, compare_unmask, widen_logits
 
 pytestmark = pytest.mark.gpu
-
-CONF_TOL = 2e-5
 
 
 def _regular(w, logits, tokens, state, seeds, step):
@@ -61,6 +62,13 @@ def _same(a, b):
     assert np.nanmax(np.abs(a[4] - b[4])) <= CONF_TOL
 
 
+def _matches_oracle(w, got, logits, tokens, state, seeds, step):
+    ref = unmask_step(widen_logits(w, logits), tokens, state, seeds, w.threshold, w.temperature, 0, step)
+    res = compare_unmask(dict(tokens=got[0], state=got[1], n_committed=got[2], n_left=got[3], conf=got[4]),
+                         ref, tokens, state, w.threshold)
+    assert len(res["ambiguous_forks"]) <= 1
+
+
 def test_static_entry_matches_regular_entry_twice():
     assert torch.cuda.is_available()
     # first call: several chunks per row, noisy arg-max, 4 rollouts
@@ -68,14 +76,18 @@ def test_static_entry_matches_regular_entry_twice():
     tokens, state = synth.make_block_template(w1, 0, 0)
     seeds = synth.fork_seeds(w1, 0)
     logits = synth.make_logits(w1, 0, 0, 0, rows="all")
-    _same(_static(w1, logits, tokens, state, seeds, 0), _regular(w1, logits, tokens, state, seeds, 0))
+    got = _static(w1, logits, tokens, state, seeds, 0)
+    _same(got, _regular(w1, logits, tokens, state, seeds, 0))
+    _matches_oracle(w1, got, logits, tokens, state, seeds, 0)
     # second call right after, different shape and dtype: the shared scratch still holds the first
     # call's records, which must not leak into this result
     w2 = synth.workload("tiny")
     tokens, state = synth.make_block_template(w2, 0, 0)
     seeds = synth.fork_seeds(w2, 0)
     logits = synth.make_logits(w2, 0, 0, 3, rows="all")
-    _same(_static(w2, logits, tokens, state, seeds, 3), _regular(w2, logits, tokens, state, seeds, 3))
+    got = _static(w2, logits, tokens, state, seeds, 3)
+    _same(got, _regular(w2, logits, tokens, state, seeds, 3))
+    _matches_oracle(w2, got, logits, tokens, state, seeds, 3)
 
 
 def test_static_entry_rejects_oversize_and_bad_arguments():
@@ -84,6 +96,9 @@ def test_static_entry_rejects_oversize_and_bad_arguments():
     with pytest.raises(fdd.FddError) as ei:      # 64 * 128 rows x 19 chunks > 65536 records
         fdd.fdd_unmask_static(t, fdd.FDD_LOGITS_BF16, 64, 128, 151936, t, t, t, 0.9, 0.0, 0, 0, t, t)
     assert ei.value.status == fdd.FDD_ERR_CAPACITY and "exceeds the fixed scratch" in str(ei.value)
+    with pytest.raises(fdd.FddError) as ei:      # 128 x 128 rows: few records (vocab 4096), but more rows than one call takes
+        fdd.fdd_unmask_static(t, fdd.FDD_LOGITS_F32, 128, 128, 4096, t, t, t, 0.9, 0.0, 0, 0, t, t)
+    assert ei.value.status == fdd.FDD_ERR_CAPACITY and "8192 rows" in str(ei.value)
     with pytest.raises(fdd.FddError) as ei:
         fdd.fdd_unmask_static(None, fdd.FDD_LOGITS_BF16, 1, 16, 64, t, t, t, 0.9, 0.0, 0, 0, t, t)
     assert ei.value.status == fdd.FDD_ERR_INVALID_ARG
