@@ -10,6 +10,7 @@
  *   fdd_ss_draft/_accept draft and accept scan of Scaffold Speculative Decoding (Sec. 3.3, Algorithm)
  *   fdd_plan_blocks      section-aligned blocks of the output template         (Sec. 3.2)
  *   fdd_kv_commit        append the finished block to each private cache (Sec. 3.3 cache reuse; Sec. 3.4 fork)
+ *   fdd_prefix_extend    append a deterministic block to the shared cache before the fork (Sec. 3.4)
  *   fdd_average_rollouts equal-weight mean of N trajectories            (Sec. 3.4, trajectory averaging)
  *   fdd_average_rollouts_jmt  the same after jerk-minimising interpolation  (Sec. 3.4)
  *
@@ -96,8 +97,9 @@ uint64_t fdd_launch_count(const fdd_ctx* ctx);
  *   prefix_k, prefix_v  host arrays [L] of device pointers, one cache per layer, bf16.
  *                       contiguous (cfg.page_tokens == 0): [Hkv][prefix_capacity][D]
  *                       paged:                             [prefix_capacity pages][Hkv][page_tokens][D]
- *                       Read-only for the library; must stay valid and unmodified while
- *                       the fork set lives.
+ *                       Read-only for the library except for fdd_prefix_extend; must stay valid
+ *                       while the fork set lives, and the caller does not write the first
+ *                       prefix_len tokens.
  *   page_table          device int32 [ceil(prefix_len / page_tokens)] physical page of each
  *                       logical page (paged layout), NULL for the contiguous layout.  Every
  *                       entry must be in [0, prefix_capacity); entries are read on the device.
@@ -265,6 +267,29 @@ fdd_status fdd_kv_commit(fdd_ctx* ctx, fdd_forkset* const* sets, int n_sets, int
                          int advance, void* stream);
 
 /*
+ * fdd_prefix_extend -- Sec. 3.4 "Shared prefix": the first three sections are deterministic, so
+ * they are decoded once, by a fork set of ONE rollout, and the N rollouts of the trajectory section
+ * are forked from the cache that holds them.  This call is that set's commit: its block's K/V
+ * ([1][d_s][Hkv][D], packed like fdd_block_attn) go to positions [P, P + d_s) of the shared prefix
+ * cache of `layer` itself (P = the set's current prefix length), bit for bit, in the cache's own
+ * layout (paged: through the page table, whose entries for the touched pages the caller has filled
+ * in).  With advance != 0 the set's prefix length grows by d_s afterwards (pass it on the last
+ * layer).  A later fdd_fork over the same cache buffers with prefix_len = fdd_forkset_prefix_len(set)
+ * gives N rollouts that share everything decoded so far; nothing is copied or re-laid.
+ * This is the only call that writes a prefix cache.  It writes beyond the current prefix length
+ * only, so fork sets that already read the same buffers with a shorter length are not disturbed.
+ * FDD_ERR_STATE if a set has more than one rollout or has committed a private suffix;
+ * FDD_ERR_CAPACITY if P + d_s exceeds prefix_capacity (nothing is launched).  A page table entry
+ * outside [0, prefix_capacity) is not followed: the rows are dropped and the device status word
+ * gets FDD_ERR_INVALID_ARG (see fdd_poll_status).
+ */
+fdd_status fdd_prefix_extend(fdd_ctx* ctx, fdd_forkset* const* sets, int n_sets, int layer,
+                             const void* k_blk, const void* v_blk, const int32_t* block_len,
+                             int advance, void* stream);
+/* Tokens of the shared prefix the set currently reads; < 0 on error. */
+int fdd_forkset_prefix_len(const fdd_forkset* set);
+
+/*
  * fdd_average_rollouts -- Sec. 3.4: tau_out = (1/N) sum_i tau_i.
  *   traj  device fp32 [n][w][2];  out  device fp32 [w][2];  n >= 1, w >= 1.
  */
@@ -354,8 +379,18 @@ fdd_status fdd_plan_blocks(const uint8_t* editable, const int32_t* section_end, 
 fdd_status fdd_upload_masked_rows(fdd_ctx* ctx, const void* host_logits, void* dev_logits,
                                   const uint8_t* host_state, int rows, size_t* bytes_copied, void* stream);
 
+/*
+ * fdd_set_merge_wait_limit -- how long a CTA of fdd_block_attn waits for the partial results of the
+ * other CTAs that share a unit of work with it, in SM clocks (default 4e9, about two seconds).  When
+ * the limit runs out the CTA records FDD_ERR_DEVICE_TIMEOUT in the device status word and returns
+ * without writing its share of the output; the launch itself always ends.  fdd_poll_status then
+ * reports the error and puts the context's counters back in order, and the next call is valid.
+ * Meant for deployments that want a tighter bound than the default, and for testing the error path
+ */
+fdd_status fdd_set_merge_wait_limit(fdd_ctx* ctx, long long sm_clocks);
+
 /* Synchronise `stream` and return the device status word: FDD_OK, or the first error a
- * kernel recorded (FDD_ERR_DEVICE_TIMEOUT).  Reading clears it. */
+ * kernel recorded (FDD_ERR_DEVICE_TIMEOUT, FDD_ERR_INVALID_ARG).  Reading clears it. */
 fdd_status fdd_poll_status(fdd_ctx* ctx, void* stream);
 
 #ifdef __cplusplus

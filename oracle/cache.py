@@ -7,6 +7,11 @@ finished blocks stay in the cache and are reused without recomputation.
 A fork shares the prefix arrays by reference (they are never written) and owns
 an initially empty suffix per layer.  Committing a block appends that rollout's
 block K/V rows, bit for bit, to its suffix.
+
+The scene-level order of Sec. 3.4: a set of ONE rollout decodes the first three
+(deterministic) sections; each of its finished blocks is appended to the shared
+prefix itself (`extend_prefix`); then `fork` makes N rollouts over that longer
+prefix, each with an empty suffix and a seed of its own.
 """
 import numpy as np
 
@@ -41,3 +46,20 @@ class ForkSet:
         for f in range(self.n_forks):
             self.suffix_k[layer][f] = np.concatenate([self.suffix_k[layer][f], k_blk[f]], axis=0)
             self.suffix_v[layer][f] = np.concatenate([self.suffix_v[layer][f], v_blk[f]], axis=0)
+
+    def extend_prefix(self, layer, k_blk, v_blk):
+        """The one rollout of a deterministic set commits a block to the shared prefix:
+        k_blk, v_blk [1, d, Hkv, D] are appended to the prefix of `layer` (a new array:
+        whoever forked from the shorter prefix keeps reading that one)."""
+        assert self.n_forks == 1, "only a set of one rollout extends its prefix"
+        assert self.suffix_len(0) == 0, "the prefix stays in front of every private suffix"
+        k_blk = np.asarray(k_blk)
+        v_blk = np.asarray(v_blk)
+        assert k_blk.shape[0] == 1 and v_blk.shape[0] == 1
+        self.prefix_k[layer] = np.concatenate([self.prefix_k[layer], k_blk[0]], axis=0)
+        self.prefix_v[layer] = np.concatenate([self.prefix_v[layer], v_blk[0]], axis=0)
+
+    def fork(self, n_forks, seeds):
+        """N rollouts over this set's current prefix (shared by reference), empty suffixes."""
+        assert self.suffix_len(0) == 0
+        return ForkSet(self.prefix_k, self.prefix_v, n_forks, seeds)

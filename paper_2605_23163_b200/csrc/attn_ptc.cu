@@ -38,6 +38,7 @@
 
 #include <math_constants.h>
 
+#include <atomic>
 #include <cstdlib>
 
 namespace {
@@ -78,6 +79,7 @@ struct TcArgs {
     int min_tiles;             // do not cut the work into ranges shorter than this
     int n_sets;
     float scale_log2;
+    long long merge_wait_limit; // SM clocks a CTA waits for the other pieces of a cut unit before it gives up
 };
 
 struct TileInfo {
@@ -808,7 +810,7 @@ attn_ptc_kernel(const __grid_constant__ TcArgs<MAXSETS> a) {
                 for (int e = 0; e < n_deferred; ++e) {
                     volatile int* arrived = a.unit_count + deferred_s[e].gu;
                     while (*arrived < deferred_s[e].n_pieces) {
-                        if (clock64() - t0 > kWaitLimit) {
+                        if (clock64() - t0 > a.merge_wait_limit) {
                             atomicCAS(a.status, 0, FDD_ERR_DEVICE_TIMEOUT);
                             *abort_flag = 1;
                             break;
@@ -955,7 +957,7 @@ bool make_cache_maps(const AttnProblem& a, int D, TcSetMaps* m) {
 const TcSetMaps* maps_for(const AttnProblem& a, int D, TcMapCache* cache) {
     const bool call_same = cache->valid && cache->q == a.q && cache->k_blk == a.k_blk && cache->v_blk == a.v_blk &&
                            cache->d == a.d;
-    const bool cache_same = cache->valid && cache->suffix_len == a.suffix_len;
+    const bool cache_same = cache->valid && cache->suffix_len == a.suffix_len && cache->prefix_len == a.prefix_len;
     if (call_same && cache_same) return &cache->maps;
     if (!call_same) {
         if (!make_call_maps(a, D, &cache->maps)) { cache->valid = false; return nullptr; }
@@ -964,6 +966,7 @@ const TcSetMaps* maps_for(const AttnProblem& a, int D, TcMapCache* cache) {
     if (!make_cache_maps(a, D, &cache->maps)) { cache->valid = false; return nullptr; }
     cache->q = a.q; cache->k_blk = a.k_blk; cache->v_blk = a.v_blk; cache->d = a.d;
     cache->suffix_len = a.suffix_len;
+    cache->prefix_len = a.prefix_len;
     cache->valid = true;
     return &cache->maps;
 }
@@ -983,13 +986,16 @@ int emulated_exponentials() {
 }
 
 template <int D, int MAXSETS, int EMU>
-cudaError_t launch_one(const TcArgs<MAXSETS>& args, unsigned ctas, cudaStream_t st) {
+cudaError_t launch_one(const TcArgs<MAXSETS>& args, unsigned ctas, int device, cudaStream_t st) {
     const int smem = TcShape<D>::kSmemBytes;
-    static bool configured = false;
-    if (!configured) {
+    // the kernel's shared-memory size is a per-device attribute: set on the first launch on each device
+    constexpr int kMaxDevices = 64;
+    static std::atomic<bool> configured[kMaxDevices];
+    if (device < 0 || device >= kMaxDevices) return cudaErrorInvalidDevice;
+    if (!configured[device].load(std::memory_order_acquire)) {
         cudaError_t e = cudaFuncSetAttribute(attn_ptc_kernel<D, MAXSETS, EMU>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
         if (e != cudaSuccess) return e;
-        configured = true;
+        configured[device].store(true, std::memory_order_release);
     }
     // The CTAs wait for one another's pieces at the end: a cooperative launch makes the runtime
     // guarantee that all of them are resident at once (or fail the launch).
@@ -999,19 +1005,21 @@ cudaError_t launch_one(const TcArgs<MAXSETS>& args, unsigned ctas, cudaStream_t 
 }
 
 template <int MAXSETS>
-cudaError_t launch_emu(const TcArgs<MAXSETS>& args, int head_dim, unsigned ctas, cudaStream_t st) {
-    if (head_dim == 64) return launch_one<64, MAXSETS, 0>(args, ctas, st);
+cudaError_t launch_emu(const TcArgs<MAXSETS>& args, int head_dim, unsigned ctas, int device, cudaStream_t st) {
+    if (head_dim == 64) return launch_one<64, MAXSETS, 0>(args, ctas, device, st);
     switch (emulated_exponentials()) {
-        case 16: return launch_one<128, MAXSETS, 16>(args, ctas, st);
-        case 32: return launch_one<128, MAXSETS, 32>(args, ctas, st);
-        default: return launch_one<128, MAXSETS, 0>(args, ctas, st);
+        case 16: return launch_one<128, MAXSETS, 16>(args, ctas, device, st);
+        case 32: return launch_one<128, MAXSETS, 32>(args, ctas, device, st);
+        default: return launch_one<128, MAXSETS, 0>(args, ctas, device, st);
     }
 }
 
 template <int MAXSETS>
 cudaError_t launch_group(fdd_ctx* ctx, const AttnProblem* probs, TcMapCache* const* caches, int n, int head_dim,
                          cudaStream_t st) {
-    static TcArgs<MAXSETS> args;     // 1-20 KB, kept off the stack (a context is used by one host thread at a time)
+    // 1-20 KB, kept off the stack in the context's own buffer (a context is used by one host thread at a time)
+    if (ctx->attn_args.size() * sizeof(uint64_t) < sizeof(TcArgs<MAXSETS>)) ctx->attn_args.resize((sizeof(TcArgs<MAXSETS>) + 7) / 8);
+    TcArgs<MAXSETS>& args = *reinterpret_cast<TcArgs<MAXSETS>*>(ctx->attn_args.data());
     long long steps = 0;
     int units = 0, forks = 0;
     bool gated = false;
@@ -1059,7 +1067,8 @@ cudaError_t launch_group(fdd_ctx* ctx, const AttnProblem* probs, TcMapCache* con
     args.min_tiles = min_tiles;
     args.n_sets = n;
     args.scale_log2 = probs[0].scale * 1.4426950408889634f;
-    return launch_emu<MAXSETS>(args, head_dim, static_cast<unsigned>(ctas), st);
+    args.merge_wait_limit = ctx->attn_merge_wait_limit;
+    return launch_emu<MAXSETS>(args, head_dim, static_cast<unsigned>(ctas), ctx->device, st);
 }
 
 }  // namespace

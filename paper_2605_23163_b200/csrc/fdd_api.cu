@@ -44,7 +44,7 @@ __global__ void seed_store_kernel(const __grid_constant__ SeedChunk c) {
 
 // Store the seeds of every set of the call that has not been used for sampling yet.
 cudaError_t ensure_seeds(fdd_ctx* ctx, fdd_forkset* const* sets, int n_sets, cudaStream_t st) {
-    static SeedChunk chunk;        // 4 KB, kept off the stack (a context is used by one host thread at a time)
+    SeedChunk& chunk = *static_cast<SeedChunk*>(ctx->seed_chunk);   // 4 KB, kept off the stack, one per context
     chunk.n = 0;
     auto flush = [&]() -> cudaError_t {
         if (chunk.n == 0) return cudaSuccess;
@@ -117,6 +117,8 @@ fdd_status fdd_create(const fdd_config* cfg, fdd_ctx** out) {
     if (e == cudaSuccess) e = cudaMalloc(&ctx->d_status, sizeof(int));
     if (e == cudaSuccess) e = cudaMemset(ctx->d_status, 0, sizeof(int));
     if (e == cudaSuccess) e = cudaMallocHost(&ctx->h_status, sizeof(int));
+    ctx->seed_chunk = new (std::nothrow) SeedChunk();
+    if (!ctx->seed_chunk && e == cudaSuccess) e = cudaErrorMemoryAllocation;
     if (e == cudaSuccess) {
         const long long max_rows = static_cast<long long>(cfg->max_forks) * cfg->max_block;
         ctx->ws_unmask_bytes = unmask_workspace_bytes(cfg->vocab, static_cast<int>(std::min<long long>(max_rows, kUnmaskMaxRows)));
@@ -157,6 +159,7 @@ void fdd_destroy(fdd_ctx* ctx) {
     if (ctx->ws_unmask) cudaFree(ctx->ws_unmask);
     if (ctx->ws_attn) cudaFree(ctx->ws_attn);
     if (ctx->attn_unit_count) cudaFree(ctx->attn_unit_count);
+    delete static_cast<SeedChunk*>(ctx->seed_chunk);
     delete ctx;
 }
 
@@ -446,9 +449,10 @@ fdd_status fdd_ss_accept(fdd_ctx* ctx, fdd_forkset* const* sets, int n_sets, con
                        n_accepted, n_left, nullptr, stream, 2);
 }
 
-fdd_status fdd_kv_commit(fdd_ctx* ctx, fdd_forkset* const* sets, int n_sets, int layer,
-                         const void* k_blk, const void* v_blk, const int32_t* block_len,
-                         int advance, void* stream) {
+// Common body of fdd_kv_commit (to_prefix = false) and fdd_prefix_extend (to_prefix = true).
+static fdd_status commit_like(fdd_ctx* ctx, fdd_forkset* const* sets, int n_sets, int layer,
+                              const void* k_blk, const void* v_blk, const int32_t* block_len,
+                              int advance, void* stream, bool to_prefix) {
     if (!ctx) return FDD_ERR_INVALID_ARG;
     int total = 0;
     fdd_status st = check_sets(ctx, sets, n_sets, block_len, &total);
@@ -456,28 +460,89 @@ fdd_status fdd_kv_commit(fdd_ctx* ctx, fdd_forkset* const* sets, int n_sets, int
     if (!k_blk || !v_blk) return fail(ctx, FDD_ERR_INVALID_ARG, "k_blk/v_blk is NULL");
     if (!aligned16(k_blk) || !aligned16(v_blk)) return fail(ctx, FDD_ERR_INVALID_ARG, "k_blk/v_blk must be 16-byte aligned");
     if (layer < 0 || layer >= ctx->cfg.n_layers) return fail(ctx, FDD_ERR_SHAPE, "layer %d outside [0, %d)", layer, ctx->cfg.n_layers);
-    for (int s = 0; s < n_sets; ++s)
-        if (sets[s]->suffix_len + block_len[s] > sets[s]->suffix_capacity)
-            return fail(ctx, FDD_ERR_CAPACITY, "set %d: suffix %d + block %d exceeds capacity %d", s,
-                        sets[s]->suffix_len, block_len[s], sets[s]->suffix_capacity);
     const fdd_config& c = ctx->cfg;
-    size_t kv_off = 0;
     for (int s = 0; s < n_sets; ++s) {
-        fdd_forkset* fs = sets[s];
-        cudaError_t e = launch_kv_commit(static_cast<const __nv_bfloat16*>(k_blk) + kv_off,
-                                         static_cast<const __nv_bfloat16*>(v_blk) + kv_off,
-                                         static_cast<__nv_bfloat16*>(fs->suffix_k[layer]),
-                                         static_cast<__nv_bfloat16*>(fs->suffix_v[layer]),
-                                         fs->n_forks, block_len[s], c.n_kv_heads, c.head_dim,
-                                         fs->suffix_len, fs->suffix_capacity, static_cast<cudaStream_t>(stream));
+        const fdd_forkset* fs = sets[s];
+        if (!to_prefix) {
+            if (fs->suffix_len + block_len[s] > fs->suffix_capacity)
+                return fail(ctx, FDD_ERR_CAPACITY, "set %d: suffix %d + block %d exceeds capacity %d", s,
+                            fs->suffix_len, block_len[s], fs->suffix_capacity);
+            continue;
+        }
+        if (fs->n_forks != 1)
+            return fail(ctx, FDD_ERR_STATE, "set %d has %d rollouts: only a set of one rollout extends its prefix", s, fs->n_forks);
+        if (fs->suffix_len != 0)
+            return fail(ctx, FDD_ERR_STATE, "set %d has a private suffix of %d tokens: the prefix must stay in front of it", s, fs->suffix_len);
+        const int need = fs->prefix_len + block_len[s];
+        const bool fits = c.page_tokens == 0 ? need <= fs->prefix_capacity
+                                             : (need + c.page_tokens - 1) / c.page_tokens <= fs->prefix_capacity;
+        if (!fits)
+            return fail(ctx, FDD_ERR_CAPACITY, "set %d: prefix %d + block %d exceeds the cache (%d %s)", s, fs->prefix_len,
+                        block_len[s], fs->prefix_capacity, c.page_tokens ? "pages" : "tokens");
+        if (c.page_tokens != 0 && !fs->page_table)
+            return fail(ctx, FDD_ERR_INVALID_ARG, "set %d: a paged prefix needs its page table", s);
+    }
+    size_t kv_off = 0;
+    for (int first = 0; first < n_sets; first += kCommitMaxSets) {
+        CommitArgs a;
+        a.n = std::min(kCommitMaxSets, n_sets - first);
+        a.n_kv_heads = c.n_kv_heads;
+        a.vec_per_row = c.head_dim / 8;
+        a.status = ctx->d_status;
+        a.total = 0;
+        for (int k = 0; k < a.n; ++k) {
+            fdd_forkset* fs = sets[first + k];
+            CommitSet& cs = a.set[k];
+            cs.k_src = static_cast<const __nv_bfloat16*>(k_blk) + kv_off;
+            cs.v_src = static_cast<const __nv_bfloat16*>(v_blk) + kv_off;
+            cs.n_forks = fs->n_forks;
+            cs.d = block_len[first + k];
+            cs.page_table = fs->page_table;
+            cs.page_tokens = c.page_tokens > 0 ? c.page_tokens : 1;
+            if (to_prefix) {
+                // the prefix caches are the caller's and read-only for every other call
+                cs.k_dst = const_cast<void*>(fs->prefix_k[layer]);
+                cs.v_dst = const_cast<void*>(fs->prefix_v[layer]);
+                cs.len = fs->prefix_len;
+                cs.cap = fs->prefix_capacity;
+                cs.mode = c.page_tokens == 0 ? kCommitPrefix : kCommitPagedPrefix;
+            } else {
+                cs.k_dst = fs->suffix_k[layer];
+                cs.v_dst = fs->suffix_v[layer];
+                cs.len = fs->suffix_len;
+                cs.cap = fs->suffix_capacity;
+                cs.mode = kCommitSuffix;
+            }
+            cs.vec_begin = a.total;
+            const size_t elems = static_cast<size_t>(fs->n_forks) * cs.d * c.n_kv_heads * c.head_dim;
+            a.total += static_cast<long long>(elems / 8);
+            kv_off += elems;
+        }
+        cudaError_t e = launch_kv_commit(a, ctx->sm_count, static_cast<cudaStream_t>(stream));
         ctx->launches += 1;
-        if (e != cudaSuccess) return cuda_fail(ctx, e, "fdd_kv_commit launch");
-        kv_off += static_cast<size_t>(fs->n_forks) * block_len[s] * c.n_kv_heads * c.head_dim;
+        if (e != cudaSuccess) return cuda_fail(ctx, e, to_prefix ? "fdd_prefix_extend launch" : "fdd_kv_commit launch");
     }
     if (advance)
-        for (int s = 0; s < n_sets; ++s) sets[s]->suffix_len += block_len[s];
+        for (int s = 0; s < n_sets; ++s) {
+            if (to_prefix) sets[s]->prefix_len += block_len[s];
+            else sets[s]->suffix_len += block_len[s];
+        }
     return FDD_OK;
 }
+
+fdd_status fdd_kv_commit(fdd_ctx* ctx, fdd_forkset* const* sets, int n_sets, int layer,
+                         const void* k_blk, const void* v_blk, const int32_t* block_len,
+                         int advance, void* stream) {
+    return commit_like(ctx, sets, n_sets, layer, k_blk, v_blk, block_len, advance, stream, false);
+}
+
+fdd_status fdd_prefix_extend(fdd_ctx* ctx, fdd_forkset* const* sets, int n_sets, int layer,
+                             const void* k_blk, const void* v_blk, const int32_t* block_len,
+                             int advance, void* stream) {
+    return commit_like(ctx, sets, n_sets, layer, k_blk, v_blk, block_len, advance, stream, true);
+}
+
+int fdd_forkset_prefix_len(const fdd_forkset* set) { return set ? set->prefix_len : FDD_ERR_INVALID_ARG; }
 
 fdd_status fdd_average_rollouts(fdd_ctx* ctx, const float* traj, int n, int w, float* out, void* stream) {
     if (!ctx) return FDD_ERR_INVALID_ARG;
@@ -542,6 +607,13 @@ fdd_status fdd_upload_masked_rows(fdd_ctx* ctx, const void* host_logits, void* d
         r = e;
     }
     if (bytes_copied) *bytes_copied = total;
+    return FDD_OK;
+}
+
+fdd_status fdd_set_merge_wait_limit(fdd_ctx* ctx, long long sm_clocks) {
+    if (!ctx) return FDD_ERR_INVALID_ARG;
+    if (sm_clocks < 1) return fail(ctx, FDD_ERR_INVALID_ARG, "the wait limit must be at least one clock");
+    ctx->attn_merge_wait_limit = sm_clocks;
     return FDD_OK;
 }
 

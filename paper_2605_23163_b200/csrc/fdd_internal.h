@@ -27,6 +27,7 @@ struct TcMapCache {
     const void* v_blk = nullptr;
     int d = 0;
     int suffix_len = -1;
+    int prefix_len = -1;
     TcSetMaps maps;
 };
 
@@ -52,6 +53,9 @@ struct fdd_ctx {
     int* attn_unit_count = nullptr;   // device [2][attn_max_units]: pieces written / merge shares done per unit (self-resetting)
     int attn_max_units = 0;
     int attn_max_ctas = 0;
+    std::vector<uint64_t> attn_args;  // host buffer for the attention kernel's argument block (8-byte aligned)
+    long long attn_merge_wait_limit = 4000000000LL;   // SM clocks (about two seconds): wait for the pieces of a cut unit
+    void* seed_chunk = nullptr;       // host staging of seeds on their way to the device as kernel arguments
     uint64_t launches = 0;
     std::string last_error;
     std::vector<fdd_forkset*> live_sets;
@@ -153,10 +157,26 @@ size_t attention_ptc_workspace_bytes(int head_dim, int max_ctas);
 cudaError_t launch_attention_ptc(fdd_ctx* ctx, const AttnProblem* probs, TcMapCache* const* caches, int n,
                                  int head_dim, cudaStream_t st, int* n_launches);
 cudaError_t launch_unmask(fdd_ctx* ctx, const UnmaskProblem& p, cudaStream_t st, int* n_launches, int mode = 0);
-cudaError_t launch_kv_commit(const __nv_bfloat16* k_blk, const __nv_bfloat16* v_blk,
-                             __nv_bfloat16* suffix_k, __nv_bfloat16* suffix_v,
-                             int n_forks, int d, int n_kv_heads, int head_dim,
-                             int suffix_len, int suffix_capacity, cudaStream_t st);
+// One scene's part of a cache append.
+constexpr int kCommitSuffix = 0, kCommitPrefix = 1, kCommitPagedPrefix = 2;
+constexpr int kCommitMaxSets = 16;          // scenes per append launch
+struct CommitSet {
+    const void* k_src;       // this scene's rows of k_blk / v_blk
+    const void* v_src;
+    void* k_dst;             // the layer's cache
+    void* v_dst;
+    const int32_t* page_table;
+    long long vec_begin;     // first 16-byte vector of this scene in the launch
+    int n_forks, d, len, cap, mode, page_tokens;
+};
+struct CommitArgs {
+    CommitSet set[kCommitMaxSets];
+    int n;
+    long long total;         // 16-byte vectors of all scenes
+    int n_kv_heads, vec_per_row;
+    int* status;             // device status word
+};
+cudaError_t launch_kv_commit(const CommitArgs& a, int sm_count, cudaStream_t st);
 cudaError_t launch_average(const float* traj, int n, int w, float* out, cudaStream_t st);
 bool jmt_weights(int w, int w_out, std::vector<double>* weights);
 cudaError_t launch_average_jmt(const float* traj, int n, int w, int w_out, const double* d_weights, float* out,

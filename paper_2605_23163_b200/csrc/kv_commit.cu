@@ -1,42 +1,52 @@
-// Append a finished block's K/V rows to each rollout's private suffix cache.
-// Source [N][d][Hkv][D] (token-major, as projected), destination [N][Hkv][cap][D]
-// (head-major, so that a key tile of one head is contiguous).  16-byte copies.
+// Append a finished block's K/V rows to a cache: every rollout's private suffix (fdd_kv_commit),
+// or the shared prefix itself when the one rollout that decodes the deterministic sections
+// commits a block (fdd_prefix_extend).  Source [N][d][Hkv][D] (token-major, as projected);
+// destination head-major, so that a key tile of one head is contiguous:
+//   private suffix    [N][Hkv][cap][D]
+//   contiguous prefix [Hkv][cap][D]
+//   paged prefix      [pages][Hkv][64][D], logical page -> physical page through the page table.
+// 16-byte copies; all scenes of a call go into one launch.
 #include "fdd_internal.h"
 
 namespace {
-__global__ void kv_commit_kernel(const uint4* __restrict__ k_blk, const uint4* __restrict__ v_blk,
-                                 uint4* __restrict__ suffix_k, uint4* __restrict__ suffix_v,
-                                 int n_forks, int d, int n_kv_heads, int vec_per_row,
-                                 int suffix_len, int suffix_capacity) {
-    const long long total = static_cast<long long>(n_forks) * d * n_kv_heads * vec_per_row;
-    for (long long idx = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x; idx < total;
+__global__ void kv_commit_kernel(const __grid_constant__ CommitArgs a) {
+    for (long long idx = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x; idx < a.total;
          idx += static_cast<long long>(gridDim.x) * blockDim.x) {
-        const int c = static_cast<int>(idx % vec_per_row);
-        long long t = idx / vec_per_row;
-        const int h = static_cast<int>(t % n_kv_heads); t /= n_kv_heads;
-        const int i = static_cast<int>(t % d);
-        const int f = static_cast<int>(t / d);
-        const long long dst = ((static_cast<long long>(f) * n_kv_heads + h) * suffix_capacity + suffix_len + i)
-                                  * vec_per_row + c;
-        suffix_k[dst] = k_blk[idx];
-        suffix_v[dst] = v_blk[idx];
+        int s = 0;
+        while (s + 1 < a.n && idx >= a.set[s + 1].vec_begin) ++s;
+        const CommitSet& cs = a.set[s];
+        const long long local = idx - cs.vec_begin;
+        const int c = static_cast<int>(local % a.vec_per_row);
+        long long t = local / a.vec_per_row;
+        const int h = static_cast<int>(t % a.n_kv_heads); t /= a.n_kv_heads;
+        const int i = static_cast<int>(t % cs.d);
+        const int f = static_cast<int>(t / cs.d);
+        const int tok = cs.len + i;
+        long long dst;
+        if (cs.mode == kCommitSuffix) {
+            dst = ((static_cast<long long>(f) * a.n_kv_heads + h) * cs.cap + tok) * a.vec_per_row + c;
+        } else if (cs.mode == kCommitPrefix) {
+            dst = (static_cast<long long>(h) * cs.cap + tok) * a.vec_per_row + c;
+        } else {
+            const long long page = cs.page_table[tok / cs.page_tokens];
+            if (page < 0 || page >= cs.cap) {           // a page table entry outside the pool: nothing is written
+                atomicCAS(a.status, 0, FDD_ERR_INVALID_ARG);
+                continue;
+            }
+            dst = ((page * a.n_kv_heads + h) * cs.page_tokens + tok % cs.page_tokens) * a.vec_per_row + c;
+        }
+        reinterpret_cast<uint4*>(cs.k_dst)[dst] = reinterpret_cast<const uint4*>(cs.k_src)[local];
+        reinterpret_cast<uint4*>(cs.v_dst)[dst] = reinterpret_cast<const uint4*>(cs.v_src)[local];
     }
 }
 }  // namespace
 
-cudaError_t launch_kv_commit(const __nv_bfloat16* k_blk, const __nv_bfloat16* v_blk,
-                             __nv_bfloat16* suffix_k, __nv_bfloat16* suffix_v,
-                             int n_forks, int d, int n_kv_heads, int head_dim,
-                             int suffix_len, int suffix_capacity, cudaStream_t st) {
-    const int vec_per_row = head_dim / 8;
-    const long long total = static_cast<long long>(n_forks) * d * n_kv_heads * vec_per_row;
+cudaError_t launch_kv_commit(const CommitArgs& a, int sm_count, cudaStream_t st) {
     const int threads = 256;
-    long long blocks = (total + threads - 1) / threads;
-    if (blocks > 148 * 8) blocks = 148 * 8;
+    long long blocks = (a.total + threads - 1) / threads;
+    const long long most = static_cast<long long>(sm_count > 0 ? sm_count : 148) * 8;
+    if (blocks > most) blocks = most;
     if (blocks < 1) blocks = 1;
-    kv_commit_kernel<<<static_cast<unsigned>(blocks), threads, 0, st>>>(
-        reinterpret_cast<const uint4*>(k_blk), reinterpret_cast<const uint4*>(v_blk),
-        reinterpret_cast<uint4*>(suffix_k), reinterpret_cast<uint4*>(suffix_v),
-        n_forks, d, n_kv_heads, vec_per_row, suffix_len, suffix_capacity);
+    kv_commit_kernel<<<static_cast<unsigned>(blocks), threads, 0, st>>>(a);
     return cudaGetLastError();
 }

@@ -22,6 +22,7 @@ EXPORTS = (
     "fdd_create", "fdd_destroy", "fdd_last_error", "fdd_launch_count", "fdd_fork",
     "fdd_forkset_free", "fdd_forkset_suffix_len", "fdd_forkset_reset", "fdd_block_attn", "fdd_block_attn_gated", "fdd_average_rollouts_jmt", "fdd_unmask_counted",
     "fdd_unmask", "fdd_ss_draft", "fdd_ss_accept", "fdd_kv_commit", "fdd_average_rollouts", "fdd_poll_status", "fdd_unmask_static", "fdd_plan_blocks", "fdd_upload_masked_rows",
+    "fdd_prefix_extend", "fdd_forkset_prefix_len", "fdd_set_merge_wait_limit",
 )
 FDD_UNMASK_STATIC_MAX_RECORDS = 65536
 
@@ -83,6 +84,12 @@ def lib():
         fn.restype = i32
     L.fdd_kv_commit.argtypes = [vp, vpp, i32, i32, vp, vp, ip, i32, vp]
     L.fdd_kv_commit.restype = i32
+    L.fdd_prefix_extend.argtypes = [vp, vpp, i32, i32, vp, vp, ip, i32, vp]
+    L.fdd_prefix_extend.restype = i32
+    L.fdd_forkset_prefix_len.argtypes = [vp]
+    L.fdd_forkset_prefix_len.restype = i32
+    L.fdd_set_merge_wait_limit.argtypes = [vp, ctypes.c_longlong]
+    L.fdd_set_merge_wait_limit.restype = i32
     L.fdd_average_rollouts.argtypes = [vp, vp, i32, i32, vp, vp]
     L.fdd_average_rollouts.restype = i32
     L.fdd_average_rollouts_jmt.argtypes = [vp, vp, i32, i32, i32, vp, vp]
@@ -255,6 +262,20 @@ def fdd_kv_commit(ctx, sets, layer, k_blk, v_blk, block_len, advance, stream=Non
     return _check(ctx, lib().fdd_kv_commit(
         ctx, _ptr_array(sets), len(sets), int(layer), _ptr(k_blk), _ptr(v_blk),
         _i32_array(block_len), int(advance), _stream(stream)))
+
+
+def fdd_prefix_extend(ctx, sets, layer, k_blk, v_blk, block_len, advance, stream=None):
+    return _check(ctx, lib().fdd_prefix_extend(
+        ctx, _ptr_array(sets), len(sets), int(layer), _ptr(k_blk), _ptr(v_blk),
+        _i32_array(block_len), int(advance), _stream(stream)))
+
+
+def fdd_forkset_prefix_len(fs):
+    return int(lib().fdd_forkset_prefix_len(fs))
+
+
+def fdd_set_merge_wait_limit(ctx, sm_clocks):
+    return _check(ctx, lib().fdd_set_merge_wait_limit(ctx, int(sm_clocks)))
 
 
 def fdd_average_rollouts_jmt(ctx, traj, n, w, w_out, out, stream=None):

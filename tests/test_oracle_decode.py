@@ -58,6 +58,48 @@ def test_attention_after_commit_equals_block_passed_as_suffix():
     np.testing.assert_array_equal(a, b)
 
 
+def test_fork_after_deterministic_blocks_equals_fork_from_a_longer_prefix():
+    # Sec. 3.4: decode the deterministic sections once (one rollout), then fork.  Forking after k
+    # blocks were appended to the prefix is the same thing, bit for bit, as forking from a prefix
+    # that contained them from the start; the rollouts' attention then equals attention over the
+    # short prefix with those blocks handed to every rollout as its suffix.
+    w = synth.small_variant(synth.workload("tts"), prefix_len=24, vocab=64, n_forks=3, n_blocks=4)
+    pk, pv = synth.make_prefix(w, 0)
+    one = ForkSet([pk], [pv], 1, [7])
+    blocks = []
+    for b in range(2):
+        _, kb, vb = synth.make_qkv(w, 0, 0, b, 0)
+        blocks.append((kb[:1], vb[:1]))
+        one.extend_prefix(0, kb[:1], vb[:1])
+    assert one.prefix_k[0].shape[0] == 24 + 2 * w.scenes[0].block_len
+    np.testing.assert_array_equal(one.prefix_k[0][:24], pk)                 # the old part is untouched
+    np.testing.assert_array_equal(one.prefix_k[0][24:24 + 32], blocks[0][0][0])
+    np.testing.assert_array_equal(one.prefix_v[0][24 + 32:], blocks[1][1][0])
+    assert pk.shape[0] == 24                                                 # the caller's array was not grown in place
+    forked = one.fork(3, [1, 2, 3])
+    long_k = np.concatenate([pk, blocks[0][0][0], blocks[1][0][0]], axis=0)
+    long_v = np.concatenate([pv, blocks[0][1][0], blocks[1][1][0]], axis=0)
+    direct = ForkSet([long_k], [long_v], 3, [1, 2, 3])
+    np.testing.assert_array_equal(forked.prefix_k[0], direct.prefix_k[0])
+    np.testing.assert_array_equal(forked.prefix_v[0], direct.prefix_v[0])
+    assert all(forked.suffix_len(f) == 0 for f in range(3)) and forked.seeds == [1, 2, 3]
+    q, k, v = synth.make_qkv(w, 0, 0, 2, 0)
+    W = bf16_bits_to_f64
+    none = [np.zeros((0, w.n_kv_heads, w.head_dim))] * 3
+    a = decode_block_attention(W(q), W(k), W(v), W(forked.prefix_k[0]), W(forked.prefix_v[0]), none, none, 0.1)
+    as_suffix_k = [W(np.concatenate([blocks[0][0][0], blocks[1][0][0]], axis=0))] * 3
+    as_suffix_v = [W(np.concatenate([blocks[0][1][0], blocks[1][1][0]], axis=0))] * 3
+    b_ = decode_block_attention(W(q), W(k), W(v), W(pk), W(pv), as_suffix_k, as_suffix_v, 0.1)
+    np.testing.assert_array_equal(a, b_)
+    # a set with several rollouts, or one that has a private suffix, cannot extend the prefix
+    import pytest
+    with pytest.raises(AssertionError):
+        forked.extend_prefix(0, k[:1], v[:1])
+    one.kv_commit(0, k[:1], v[:1])
+    with pytest.raises(AssertionError):
+        one.extend_prefix(0, k[:1], v[:1])
+
+
 def _run_block(w, block=0, identical_seeds=False, temperature=None):
     pk, pv = synth.make_prefix(w, 0)
     fs = ForkSet([pk], [pv], w.scenes[0].n_forks, synth.fork_seeds(w, 0, identical=identical_seeds))
