@@ -325,13 +325,14 @@ unmask_stream_kernel(const T* __restrict__ logits, const uint8_t* __restrict__ s
     const int sw = lane & 7;                            // rotation of the chunk order (bank conflicts)
     bool alive = true;                                  // false once a wait for a copy ran out
 
-    // ---- producer side (lane 0 issues, every lane keeps the same cursor): tile p_k of the warp's
-    // sequence goes to stage p_k % kStages
+    // ---- producer side (lane 0 issues, every lane keeps the same cursor): tile k of the warp's
+    // sequence goes to stage k % kStages, which is the stage the consumer has just left
+    const uint32_t ring_u32 = tc::smem_u32(ring), bars_u32 = tc::smem_u32(bars);
     long long p_at = range_begin;                       // next item to open
     int p_tile = 0, p_tile_end = 0;
     const T* p_row_ptr = nullptr;
     uint32_t p_k = 0;
-    auto produce_one = [&]() {
+    auto produce_one = [&](int stage) {
         if (!bulk_ok) return;
         if (p_tile == p_tile_end) {
             if (p_at >= range_end) return;
@@ -346,16 +347,18 @@ unmask_stream_kernel(const T* __restrict__ logits, const uint8_t* __restrict__ s
         if (lane == 0) {
             const int v0 = p_tile * kTile;
             const uint32_t bytes = static_cast<uint32_t>(min(kTile, vocab - v0)) * sizeof(T);
-            const uint32_t bar = tc::smem_u32(&bars[p_k % kStages]);
+            const uint32_t bar = bars_u32 + stage * 8;
             tc::mbar_arrive_expect_tx(bar, bytes);
-            bulk_load(tc::smem_u32(ring + (p_k % kStages) * kStageBytes), p_row_ptr + v0, bytes, bar);
+            bulk_load(ring_u32 + stage * kStageBytes, p_row_ptr + v0, bytes, bar);
         }
         ++p_tile;
         ++p_k;
     };
-    for (int s = 0; s < kStages; ++s) produce_one();
+    for (int s = 0; s < kStages; ++s) produce_one(s);
 
-    uint32_t c_k = 0;                                   // tiles consumed so far
+    uint32_t c_k = 0;                                   // tiles consumed so far: the next one sits in stage c_k % kStages
+    int stage = 0;
+    uint32_t phase = 0;                                 // parity of the stage's current use
     for (long long at = range_begin; at < range_end && alive;) {
         // ---- open the piece: items [at, at + n) of one row
         const int ri = static_cast<int>(at / ipr);
@@ -390,11 +393,10 @@ unmask_stream_kernel(const T* __restrict__ logits, const uint8_t* __restrict__ s
         int t1 = tile0;
         Best best{-CUDART_INF_F, -CUDART_INF_F, 0x7FFFFFFF};
         for (int tile = tile0; tile < tile1; ++tile) {
-            const int stage = c_k % kStages;
             unsigned char* buf = ring + stage * kStageBytes;
             const int tile_base = tile * kTile;
             if (bulk_ok) {
-                if (!wait_copy(tc::smem_u32(&bars[stage]), (c_k / kStages) & 1u)) alive = false;
+                if (!wait_copy(bars_u32 + stage * 8, phase)) alive = false;
                 alive = __all_sync(full, alive);
                 if (!alive) break;
             } else {
@@ -409,6 +411,8 @@ unmask_stream_kernel(const T* __restrict__ logits, const uint8_t* __restrict__ s
             const T* lp = reinterpret_cast<const T*>(buf) + lane * kLaneIds;
             float bm64 = -CUDART_INF_F;
             const bool whole = tile_base + kTile <= seg_end;
+            uint4 rq = make_uint4(0u, 0u, 0u, 0u);      // the words of the block's four groups
+            if (NOISY) rq = philox4x32_10(make_uint4(static_cast<uint32_t>(vb >> 6), pos, step, block_idx), keys);
             if (whole) {
                 // whole tile: two halves of 32 logits, chunk c of the lane read from place c ^ sw (the
                 // eight lanes of a quarter warp then touch eight different 16-byte columns of the banks)
@@ -423,11 +427,14 @@ unmask_stream_kernel(const T* __restrict__ logits, const uint8_t* __restrict__ s
                     for (int u = 0; u < 8; ++u) g8[u] = tc::max3(v[4 * u], v[4 * u + 1], fmaxf(v[4 * u + 2], v[4 * u + 3]));
                     const float bm = tc::max3(tc::max3(g8[0], g8[1], g8[2]), tc::max3(g8[3], g8[4], g8[5]), fmaxf(g8[6], g8[7]));
                     bm64 = fmaxf(bm64, bm);
-                    if (bm > m) {
-                        // rescale by 2^((m - bm) log2 e); the rounded nml must not enter here
-                        s *= tc::ex2((m - bm) * kLog2e);
-                        m = bm;
-                        nml = -bm * kLog2e;
+                    {
+                        // rescale by 2^((m - mn) log2 e): exactly 1 while the maximum stands (the rounded nml
+                        // must not enter here).  Without a branch, so that the tile step is one straight run of
+                        // instructions and the Philox rounds of the noisy step overlap the exponentials.
+                        const float mn = fmaxf(m, bm);
+                        s *= tc::ex2(mn == m ? 0.0f : (m - mn) * kLog2e);
+                        m = mn;
+                        nml = mn > -CUDART_INF_F ? -mn * kLog2e : 0.0f;
                     }
                     // packed fp32x2 arithmetic: one FMA and one add per two logits
                     const uint64_t l2e2 = tc::pack2(kLog2e, kLog2e), nm2 = tc::pack2(nml, nml);
@@ -457,12 +464,12 @@ unmask_stream_kernel(const T* __restrict__ logits, const uint8_t* __restrict__ s
                 s += add;
             }
             if (!NOISY) {
-                if (bm64 > u1) { u1 = bm64; t1 = tile; }   // strictly: t1 is the first tile that holds the lane's maximum
+                t1 = bm64 > u1 ? tile : t1;             // strictly: t1 is the first tile that holds the lane's maximum
+                u1 = fmaxf(u1, bm64);
             } else {
                 // The block's four words: the largest one bounds every draw of the block, and its group's
                 // leader gives a score that exists.  d = 2^28 - 1 - (R >> 4), cut to 23 bits (d5 = d / 32,
                 // rounded down) so that it turns into a float exactly; both bounds stay on the safe side.
-                const uint4 rq = philox4x32_10(make_uint4(static_cast<uint32_t>(vb >> 6), pos, step, block_idx), keys);
                 uint32_t rmax;
                 int gp;                                 // the group (of the block's four) that holds rmax
                 if (whole) {
@@ -497,8 +504,12 @@ unmask_stream_kernel(const T* __restrict__ logits, const uint8_t* __restrict__ s
                 }
             }
             __syncwarp();                               // every lane is done with the stage
-            produce_one();                              // tile c_k + kStages goes into it
+            produce_one(stage);                         // tile c_k + kStages goes into it
             ++c_k;
+            if (++stage == kStages) {
+                stage = 0;
+                phase ^= 1u;
+            }
         }
         if (!alive) break;
 
