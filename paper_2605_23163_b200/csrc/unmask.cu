@@ -382,7 +382,10 @@ unmask_stream_kernel(const T* __restrict__ logits, const uint8_t* __restrict__ s
         uint2 keys = make_uint2(0u, 0u);
         if (NOISY) {
             const uint64_t seed = sets.seeds[set][fork];
-            keys = make_uint2(static_cast<uint32_t>(seed), static_cast<uint32_t>(seed >> 32));
+            // (through a shuffle, which tells the compiler that the key is the same in every lane: the
+            // round keys of the Philox blocks then live in uniform registers)
+            keys = make_uint2(__shfl_sync(0xFFFFFFFFu, static_cast<uint32_t>(seed), 0),
+                              __shfl_sync(0xFFFFFFFFu, static_cast<uint32_t>(seed >> 32), 0));
         }
 
         // ---- pass 1: stream the piece; per lane the running maximum m and sum exp(l - m).  The greedy
@@ -487,20 +490,25 @@ unmask_stream_kernel(const T* __restrict__ logits, const uint8_t* __restrict__ s
                 const float fd5 = __uint_as_float(0x4B000000u | d5) - 8388608.0f;          // d5 as a float, exactly
                 // g < 32 ln 2 - ln d <= 27 ln 2 - ln d5
                 const float g_hi = d5 == 0u ? CUDART_INF_F : fmaf(-kLn2, __log2f(fd5), 18.71497388f + 2e-3f);
-                // g_leader >= 32 ln 2 - ln((d + 1) (1 + y)), y = (d + 1) / 2^28 <= 1 / 2; d + 1 <= 32 (d5 + 1)
-                const float y = (fd5 + 1.0f) * 1.1920928955078125e-07f;                     // >= (d + 1) / 2^28
-                const float g_lo = y <= 0.5f ? fmaf(-kLn2, __log2f(fd5 + 1.0f), 18.71497388f - 2e-3f) - y : kGumbelMin;
-                const int li = gp * kGroup + static_cast<int>(rmax & 15u);
-                // a score that exists in this block: that leader's, or the largest logit's with the smallest draw there is
-                float lo = bm64 > -CUDART_INF_F ? fmaf(temperature, kGumbelMin, bm64) : -CUDART_INF_F;
-                if (vb + li < seg_end) lo = fmaxf(lo, fmaf(temperature, g_lo, Logit<T>::load1(lp + li)));
-#pragma unroll
-                for (int off = 16; off > 0; off >>= 1) lo = fmaxf(lo, __shfl_xor_sync(full, lo, off));
-                lb = fmaxf(lb, lo);
                 const float ub = fmaf(temperature, g_hi, bm64);
-                if (bm64 > -CUDART_INF_F && ub >= lb - 1e-3f) {
-                    const int slot = atomicAdd(&s_n_list[warp], 1);
-                    if (slot < kMaxList) list[slot] = Reach{ub, static_cast<uint16_t>(tile - tile0), static_cast<uint16_t>(lane)};
+                const bool reaches = bm64 > -CUDART_INF_F && ub >= lb - 1e-3f;
+                // (no block in reach: no score of this tile step can raise the bound either, since the
+                // lower bounds below lie under the blocks' upper bounds)
+                if (__any_sync(full, reaches)) {
+                    // g_leader >= 32 ln 2 - ln((d + 1) (1 + y)), y = (d + 1) / 2^28 <= 1 / 2; d + 1 <= 32 (d5 + 1)
+                    const float y = (fd5 + 1.0f) * 1.1920928955078125e-07f;                 // >= (d + 1) / 2^28
+                    const float g_lo = y <= 0.5f ? fmaf(-kLn2, __log2f(fd5 + 1.0f), 18.71497388f - 2e-3f) - y : kGumbelMin;
+                    const int li = gp * kGroup + static_cast<int>(rmax & 15u);
+                    // a score that exists in this block: that leader's, or the largest logit's with the smallest draw there is
+                    float lo = bm64 > -CUDART_INF_F ? fmaf(temperature, kGumbelMin, bm64) : -CUDART_INF_F;
+                    if (vb + li < seg_end) lo = fmaxf(lo, fmaf(temperature, g_lo, Logit<T>::load1(lp + li)));
+#pragma unroll
+                    for (int off = 16; off > 0; off >>= 1) lo = fmaxf(lo, __shfl_xor_sync(full, lo, off));
+                    lb = fmaxf(lb, lo);
+                    if (reaches && ub >= lb - 1e-3f) {
+                        const int slot = atomicAdd(&s_n_list[warp], 1);
+                        if (slot < kMaxList) list[slot] = Reach{ub, static_cast<uint16_t>(tile - tile0), static_cast<uint16_t>(lane)};
+                    }
                 }
             }
             __syncwarp();                               // every lane is done with the stage
