@@ -47,3 +47,22 @@ def test_without_a_process_group_the_helpers_are_identities():
     w = synth.workload("tiny")
     assert replicas.replica_workload(w, 0) is w
     assert replicas.max_over_ranks(3.5) == 3.5 and replicas.sum_over_ranks(7) == 7.0
+
+
+def test_bench_gpus_flag_starts_the_ranks_itself():
+    # `python bench.py --gpus 2` without a launcher re-executes itself as two ranks; here the ranks only
+    # do the bookkeeping (gloo, no GPU): MAX of the times 10 and 11 ms, SUM of 2 x 12 x steps tokens
+    import json
+    import subprocess
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "WORLD_SIZE", "LOCAL_RANK", "MASTER_ADDR", "MASTER_PORT")}
+    res = subprocess.run([sys.executable, os.path.join(root, "bench.py"), "--gpus", "2", "--selftest-replicas",
+                          "--steps", "5", "--warmup", "3"], capture_output=True, text=True, env=env, timeout=300)
+    assert res.returncode == 0, res.stderr[-2000:]
+    lines = [json.loads(x) for x in res.stdout.splitlines() if x.startswith("{")]
+    assert len(lines) == 1                                    # rank 0 alone prints
+    line = lines[0]
+    assert line["n_gpus"] == 2 and line["steps"] == 5 and line["warmup"] == 3
+    assert abs(line["ms_per_step"] - 11.0 / 5) < 1e-12
+    assert abs(line["value"] - 120.0 / 11e-3) < 1e-6
