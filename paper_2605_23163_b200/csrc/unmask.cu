@@ -613,6 +613,13 @@ unmask_stream_kernel(const T* __restrict__ logits, const uint8_t* __restrict__ s
     }
 }
 
+// Soft-max statistics of a row spread over several records: (m, s) with s = sum exp(l - m).
+__device__ __forceinline__ void merge_stats(float& m, float& s, float m2, float s2) {
+    const float mn = fmaxf(m, m2);
+    if (mn > -CUDART_INF_F) s = s * __expf(m - mn) + s2 * __expf(m2 - mn);
+    m = mn;
+}
+
 __global__ void __launch_bounds__(128)
 unmask_finalize_kernel(const UnmaskPartial* __restrict__ partial, int32_t* __restrict__ tokens,
                        uint8_t* __restrict__ state, int32_t* __restrict__ n_committed,
@@ -622,44 +629,75 @@ unmask_finalize_kernel(const UnmaskPartial* __restrict__ partial, int32_t* __res
     // (the streaming kernel of this call has read the counter; the next call sees it advanced)
     if (step_bump != nullptr && blockIdx.x == 0 && threadIdx.x == 0) *step_bump += 1u;
     const int fork = blockIdx.x;                        // rollout index over all sets of the call
-    const int i = threadIdx.x;
+    const int i = threadIdx.x, warp = i >> 5, lane = i & 31;
     int set = 0;
     while (set + 1 < sets.n_sets && fork >= sets.fork_off[set + 1]) ++set;
     const int d = sets.d[set];
     const int row0 = sets.row_off[set] + (fork - sets.fork_off[set]) * d;
     __shared__ float s_conf[128];
-    __shared__ int s_masked, s_pass;
-    if (i == 0) { s_masked = 0; s_pass = 0; }
+    __shared__ int s_tok[128], s_nrec[128], s_rows[128];
+    __shared__ int s_masked, s_pass, s_max_rec;
+    if (i == 0) { s_masked = 0; s_pass = 0; s_max_rec = 1; }
     __syncthreads();
 
+    // ---- the MASKED positions of the rollout and how many records each has (one round trip each)
     const int row = row0 + i;
-    bool masked = false;
-    float conf = -1.0f;
-    int tok = 0;
-    if (i < d) {
-        masked = state[row] == FDD_MASKED;
-        if (masked) {
-            const UnmaskPartial* p = partial + static_cast<size_t>(row) * items_per_row;
-            const int n_rec = p[0].pad[0];              // records the first kernel wrote for this row
-            float M = -CUDART_INF_F;
-            for (int c = 0; c < n_rec; ++c) M = fmaxf(M, p[c].row_max);
-            float S = 0.0f;
-            Best B{-CUDART_INF_F, -CUDART_INF_F, 0x7FFFFFFF};
-            for (int c = 0; c < n_rec; ++c) {
-                S += p[c].sum_exp * expf(p[c].row_max - M);
-                B = better(B, Best{p[c].best_score, p[c].best_logit, p[c].best_index});
-            }
-            conf = expf(B.logit - M) / S;
-            tok = B.index;
-        }
-        if (conf_out) conf_out[row] = masked ? conf : CUDART_NAN_F;
+    const bool masked = i < d && state[row] == FDD_MASKED;
+    if (masked) {
+        // records the first kernel wrote for this row (never more than the row has slots)
+        const int n_rec = max(1, min(items_per_row, partial[static_cast<size_t>(row) * items_per_row].pad[0]));
+        s_nrec[i] = n_rec;
+        s_rows[atomicAdd(&s_masked, 1)] = i;
+        atomicMax(&s_max_rec, n_rec);
     }
-    s_conf[i] = masked ? conf : -1.0f;
+    s_conf[i] = -1.0f;
+    __syncthreads();
+    const int n_masked = s_masked;
+
+    // ---- merge the records: a group of w lanes per position (w = the largest record count, rounded up
+    // to a power of two, 32 at most), so that all records of 32 / w positions are fetched in one round
+    // trip per warp.  Early steps have many positions with two or three records, late steps a few
+    // positions with up to a record per tile.
+    int w = 1;
+    while (w < s_max_rec && w < 32) w <<= 1;
+    const int per = 32 / w, sub = lane / w, sl = lane - sub * w;
+    for (int base = warp * per; base < n_masked; base += 4 * per) {   // (warp-uniform bounds)
+        const int k = base + sub;
+        const bool valid = k < n_masked;
+        const int j = valid ? s_rows[k] : 0;
+        const int nr = valid ? s_nrec[j] : 0;
+        const UnmaskPartial* p = partial + static_cast<size_t>(row0 + j) * items_per_row;
+        float M = -CUDART_INF_F, S = 0.0f;
+        Best B{-CUDART_INF_F, -CUDART_INF_F, 0x7FFFFFFF};
+        for (int c = sl; c < nr; c += w) {
+            const float4 st4 = *reinterpret_cast<const float4*>(&p[c]);     // row_max, sum_exp, best_score, best_logit
+            const int idx = p[c].best_index;
+            merge_stats(M, S, st4.x, st4.y);
+            B = better(B, Best{st4.z, st4.w, idx});
+        }
+        for (int off = w >> 1; off > 0; off >>= 1) {
+            const float m2 = __shfl_xor_sync(0xFFFFFFFFu, M, off), s2 = __shfl_xor_sync(0xFFFFFFFFu, S, off);
+            Best o;
+            o.score = __shfl_xor_sync(0xFFFFFFFFu, B.score, off);
+            o.logit = __shfl_xor_sync(0xFFFFFFFFu, B.logit, off);
+            o.index = __shfl_xor_sync(0xFFFFFFFFu, B.index, off);
+            merge_stats(M, S, m2, s2);
+            B = better(B, o);
+        }
+        if (valid && sl == 0) {
+            s_conf[j] = expf(B.logit - M) / S;
+            s_tok[j] = B.index;
+        }
+    }
+    __syncthreads();
+
+    // ---- the commit rule of the rollout
+    const float conf = s_conf[i];
+    if (i < d && conf_out) conf_out[row] = masked ? conf : CUDART_NAN_F;
     const bool pass = masked && conf > threshold;
-    if (masked) atomicAdd(&s_masked, 1);
     if (pass) atomicAdd(&s_pass, 1);
     __syncthreads();
-    const int n_masked = s_masked, n_pass = s_pass;
+    const int n_pass = s_pass;
     bool commit = pass;
     if (n_masked > 0 && n_pass == 0) {
         // at-least-one rule: the most confident MASKED position, lowest index on ties
@@ -672,7 +710,7 @@ unmask_finalize_kernel(const UnmaskPartial* __restrict__ partial, int32_t* __res
         commit = (i == best_i);
     }
     if (commit && i < d) {
-        tokens[row] = tok;
+        tokens[row] = s_tok[i];
         state[row] = static_cast<uint8_t>(commit_state);
     }
     if (i == 0) {
