@@ -12,6 +12,7 @@ Under torchrun (N > 1) every rank decodes an independent scene replica (no data-
 collective); the time is the max over ranks and the value the sum of all ranks' tokens.
 """
 import argparse
+import ctypes
 import json
 import os
 import sys
@@ -29,7 +30,8 @@ UNIT = "tokens/s"
 TIMED_PASSES = 3    # the timed region (exactly --steps blocks) is run this often; the median pass is reported
 COUNT_STREAM = None  # copy the per-rollout counts to the host on a stream of their own (None: for large steps only)
 GRAPH = False       # replay every denoising step from a CUDA graph (--graph)
-TIME_EVERY = 4      # blocks between two blocks whose kernels are timed one by one
+TIME_EVERY = 10     # blocks between two blocks whose kernels are timed one by one
+NATIVE_LOOP = True  # the block loop is run by the library (fdd_decode_block); --loop python keeps it in this file
 LOOKAHEAD = True   # enqueue step t + 1 before the host has read the counts of step t (--no-lookahead)
 PRE_STEPS = 6      # distinct per-step input sets kept resident; later steps cycle through them (--pre-steps)
 
@@ -158,6 +160,7 @@ def run_ours(args):
     for g in gscenes:                      # the benchmark forks anew for every block
         g.free()
     stream = torch.cuda.current_stream()
+    stream_c = ctypes.c_void_p(stream.cuda_stream)
     scale = 1.0 / np.sqrt(w.head_dim)
     ds = [s_.block_len for s_ in w.scenes]
     Ns = [s_.n_forks for s_ in w.scenes]
@@ -365,6 +368,32 @@ def run_ours(args):
             fdd.fdd_average_rollouts(ctx, trajs[i], Ns[i], w.waypoints, traj_out[i])
         return t
 
+    # ---- the same loop run by the library (fdd_decode_block): the calls of a step are issued from
+    # native code, one step ahead of the counts, and the block's K/V are committed by the same call.
+    # The fork sets are made once and start every block with fdd_forkset_reset.
+    nat = {"list": None, "arr": None}
+    nat_q = fdd.ptr_array([dev_steps[t][0] for t in range(PRE_STEPS) for _ in range(L)])
+    nat_k = fdd.ptr_array([dev_steps[t][1] for t in range(PRE_STEPS) for _ in range(L)])
+    nat_v = fdd.ptr_array([dev_steps[t][2] for t in range(PRE_STEPS) for _ in range(L)])
+    nat_out = fdd.ptr_array([out for t in range(PRE_STEPS) for _ in range(L)])
+    nat_lg = fdd.ptr_array([dev_steps[t][3] for t in range(PRE_STEPS)])
+
+    def decode_block_native():
+        if nat["list"] is None:
+            nat["list"] = [fdd.fdd_fork(ctx, *fa) for fa in fork_args]
+            nat["arr"] = fdd.ptr_array(nat["list"])
+        else:
+            for f_ in nat["list"]:
+                fdd.fdd_forkset_reset(ctx, f_)
+        tokens.copy_(tokens0_d, non_blocking=True)
+        state.copy_(state0_d, non_blocking=True)
+        steps, left = fdd.fdd_decode_block(ctx, nat["arr"], L, d, nat_q, nat_k, nat_v, nat_out, nat_lg, tokens, state, ds_c,
+                                           scale, 0, w.threshold, w.temperature, 0, 1, n_comm, n_left, stream=stream_c)
+        assert left == 0
+        for i in range(n_scenes):
+            fdd.fdd_average_rollouts(ctx, trajs[i], Ns[i], w.waypoints, traj_out[i])
+        return steps
+
     def barrier():
         if dist is not None:
             dist.barrier()
@@ -375,6 +404,9 @@ def run_ours(args):
     if GRAPH:
         for _ in range(2):                   # records the graphs of the steps a block usually takes
             decode_block_graph()
+    if NATIVE_LOOP:
+        for _ in range(2):
+            decode_block_native()
     sampler = ClockSampler(local)
     sampler.start()
     # every TIME_EVERY-th block carries CUDA events around each of its kernels (the per-kernel
@@ -395,6 +427,8 @@ def run_ours(args):
             timed_blocks += per_kernel
             if GRAPH and not per_kernel:
                 denoise_steps += decode_block_graph()
+            elif NATIVE_LOOP and not per_kernel:
+                denoise_steps += decode_block_native()
             else:
                 denoise_steps += decode_block(resident, per_kernel, LOOKAHEAD)
         ev1.record(stream)
@@ -526,6 +560,7 @@ def run_ours(args):
                    "step_pipeline": ("attention gated by n_left; step t+1 enqueued before the host reads step t"
                                      if LOOKAHEAD else "attention gated by n_left; one step in flight"),
                    "steps_from_cuda_graph": bool(GRAPH),
+                   "block_loop": ("library (fdd_decode_block)" if NATIVE_LOOP and not GRAPH else "bench.py"),
                    "count_copy": "own stream" if use_count_stream else "compute stream",
                    "rollouts_decoding_per_attention_call": float(np.mean([n for _, n in attn_all])) if attn_all else None,
                    "replicas": "independent scene per GPU, no collective"},
@@ -740,7 +775,7 @@ def run_replica_selftest(args):
 
 
 def main():
-    global PRE_STEPS, LOOKAHEAD, COUNT_STREAM, GRAPH
+    global PRE_STEPS, LOOKAHEAD, COUNT_STREAM, GRAPH, NATIVE_LOOP
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=40)
@@ -757,6 +792,8 @@ def main():
                     help="enqueue a denoising step only after the host has read the counts of the one before")
     ap.add_argument("--counts", choices=["auto", "in-line", "own-stream"], default="auto",
                     help="where the per-rollout counts are copied to the host: on the compute stream or on a stream of their own")
+    ap.add_argument("--loop", choices=["library", "python"], default="library",
+                    help="who runs the block loop of the blocks that are not timed kernel by kernel: the library's fdd_decode_block or this file")
     ap.add_argument("--graph", action="store_true",
                     help="replay every denoising step from a CUDA graph (blocks whose kernels are timed one by one still run call by call)")
     ap.add_argument("--selftest-replicas", action="store_true",
@@ -767,6 +804,7 @@ def main():
     PRE_STEPS = max(1, args.pre_steps)
     LOOKAHEAD = not args.no_lookahead
     GRAPH = args.graph
+    NATIVE_LOOP = args.loop == "library" and not args.no_lookahead
     COUNT_STREAM = {"auto": None, "in-line": False, "own-stream": True}[args.counts]
     if args.impl == "reference":
         run_reference(args)

@@ -312,6 +312,47 @@ fdd_status fdd_average_rollouts_jmt(fdd_ctx* ctx, const float* traj, int n, int 
                                     float* out, void* stream);
 
 /*
+ * fdd_decode_block -- Sec. 3.3: the denoising loop of one block, run by the library.  "At every
+ * step the block attends to the cached context, the model scores the MASKED positions, the
+ * confident ones are committed, and the loop ends when no MASK is left; the finished block's
+ * K/V are then cached."  Equivalent to the caller doing, for t = 0, 1, ...:
+ *     for layer in [0, n_layers): fdd_block_attn_gated(layer, q, k_blk, v_blk -> out; gate = n_left of step t - 1,
+ *                                                      every rollout at t = 0)
+ *     fdd_unmask(logits, step = t) -> tokens, state, n_committed, n_left
+ *     stop when sum(n_left) == 0 (or after max_steps steps)
+ * and then, with commit_kv != 0 and the block complete, fdd_kv_commit for every layer with the K/V
+ * of the last step (advance on the last layer).  The loop lives here because on short steps (one
+ * scene, few rollouts) the kernels take less time than an interpreter needs to issue them: the
+ * library issues step t + 1 before it reads the counts of step t, so the GPU never waits for the
+ * host; if step t completed the block, the kernels of step t + 1 find every rollout gated off and
+ * no MASKED row and return at once (n_committed and n_left then hold that step's zeros).
+ *   q, k_blk, v_blk, out   host arrays [n_inputs][n_layers] of device pointers, each laid out as for
+ *                          fdd_block_attn; step t uses row t mod n_inputs (a caller whose model
+ *                          writes every step into the same buffers passes n_inputs = 1)
+ *   logits                 host array [n_inputs] of device pointers, laid out as for fdd_unmask
+ *   tokens, state, n_committed, n_left   device, as for fdd_unmask
+ *   steps_taken            host out: steps that found a MASKED position on entry
+ *   masked_left            host out or NULL: MASKED positions left (0 unless max_steps ran out)
+ *   before_step            NULL, or a function the library calls as before_step(user, t, stream)
+ *                          before it issues step t: the place where a caller enqueues, on `stream`,
+ *                          the model work that produces step t's q / k / v / logits
+ * The call returns when the counts of the last step have reached the host (it synchronises with
+ * events on `stream`, not with the device); the commits it issued may still be running.
+ * Errors as for the calls it makes; nothing is issued after the first failure.
+ */
+typedef void (*fdd_step_fn)(void* user, int step, void* stream);
+fdd_status fdd_decode_block(fdd_ctx* ctx, fdd_forkset* const* sets, int n_sets, int n_layers,
+                            int max_steps, int n_inputs,
+                            const void* const* q, const void* const* k_blk, const void* const* v_blk,
+                            void* const* out, const void* const* logits,
+                            int32_t* tokens, uint8_t* state, const int32_t* block_len,
+                            float scale, int causal_in_block, float threshold, float temperature,
+                            uint32_t block_idx, int commit_kv,
+                            int32_t* n_committed, int32_t* n_left,
+                            int* steps_taken, int* masked_left,
+                            fdd_step_fn before_step, void* user, void* stream);
+
+/*
  * fdd_unmask_static -- the unmasking step of fdd_unmask for callers that cannot allocate device
  * memory.  (The paper has no counterpart; this is a deployment variant of fdd_unmask.)
  *

@@ -257,6 +257,10 @@ attn_ptc_kernel(const __grid_constant__ TcArgs<MAXSETS> a) {
     __shared__ long long step_base_s[MAXSETS + 1];
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    // A kernel launched behind this one for an early start (the unmasking step's streaming kernel)
+    // may be made resident on SMs as their CTA of this launch exits; it waits for the whole of this
+    // launch before it reads anything.
+    tc::grid_launch_dependents();
 
     for (int s = warp; s < a.n_sets; s += kTcThreads / 32) {
         const SetParams& p = a.sets[s];

@@ -46,6 +46,10 @@ struct fdd_ctx {
     int sm_count = 0;
     int* d_status = nullptr;          // device status word (first error wins)
     int* h_status = nullptr;          // pinned mirror
+    int32_t* h_counts[2] = {nullptr, nullptr};     // pinned, [max_forks] each: the counts of two steps in flight (fdd_decode_block)
+    cudaEvent_t count_ready[2] = {nullptr, nullptr};   // recorded behind the unmask call of a step
+    int32_t* d_counts[2] = {nullptr, nullptr};         // the device's addresses of h_counts
+    int32_t* unmask_left_mirror = nullptr;             // set by fdd_decode_block around its fdd_unmask calls
     void* ws_unmask = nullptr;        // per (row, tile) partial reductions
     size_t ws_unmask_bytes = 0;
     void* ws_attn = nullptr;          // partial outputs of attention units cut between CTAs
@@ -129,6 +133,7 @@ struct UnmaskProblem {
     uint32_t block_idx, step;
     uint32_t* step_counter = nullptr;   // device or nullptr: its value is added to `step` when the kernels run
     int bump_counter = 0;               // increment it once this launch pair is done
+    int32_t* left_mirror = nullptr;     // host memory mapped for the device, [forks], or nullptr: n_left is written there too
 };
 
 // Unmask scratch: one record per (row, chunk).

@@ -264,4 +264,13 @@ __device__ __forceinline__ void named_barrier(int id, int count) {
     asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(count) : "memory");
 }
 
+
+// Programmatic dependent launch.  A kernel launched with the programmatic-serialization attribute may
+// be made resident while the kernel before it on the stream still runs; grid_dependency_wait blocks
+// until that kernel has completed and its writes are visible (it returns at once for a kernel that
+// was launched the ordinary way).  grid_launch_dependents lets the kernel after this one be made
+// resident early, once every CTA of this one has called it or has exited.
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 }  // namespace tc

@@ -256,6 +256,11 @@ unmask_stream_kernel(const T* __restrict__ logits, const uint8_t* __restrict__ s
                      int vocab, int tiles_per_item, float temperature,
                      uint32_t block_idx, uint32_t step, int bulk_ok, int select_state,
                      const uint32_t* __restrict__ step_counter, int* __restrict__ status) {
+    // The launch may have been made resident before the kernel ahead of it on the stream was done (its
+    // set-up then overlaps that kernel's tail); nothing is read before this wait.  The kernel behind
+    // this one (the per-rollout step) may come in as soon as every CTA here has started.
+    tc::grid_dependency_wait();
+    tc::grid_launch_dependents();
     if (step_counter != nullptr) step += *step_counter;    // the denoising step as counted on the device
     const int rows = sets.row_off[sets.n_sets];
     __shared__ int s_before[kThreads];                  // selected rows before the thread's run
@@ -620,12 +625,15 @@ __device__ __forceinline__ void merge_stats(float& m, float& s, float m2, float 
     m = mn;
 }
 
-__global__ void __launch_bounds__(128)
+constexpr int kFinalizeThreads = 512;               // the first 128 are the positions of the rollout; all of them merge records
+
+__global__ void __launch_bounds__(kFinalizeThreads)
 unmask_finalize_kernel(const UnmaskPartial* __restrict__ partial, int32_t* __restrict__ tokens,
                        uint8_t* __restrict__ state, int32_t* __restrict__ n_committed,
                        int32_t* __restrict__ n_left, float* __restrict__ conf_out,
                        const __grid_constant__ UnmaskSets sets, int items_per_row, float threshold, int commit_state,
-                       uint32_t* __restrict__ step_bump) {
+                       uint32_t* __restrict__ step_bump, int32_t* __restrict__ left_mirror) {
+    tc::grid_dependency_wait();                         // the streaming kernel's records are complete and visible
     // (the streaming kernel of this call has read the counter; the next call sees it advanced)
     if (step_bump != nullptr && blockIdx.x == 0 && threadIdx.x == 0) *step_bump += 1u;
     const int fork = blockIdx.x;                        // rollout index over all sets of the call
@@ -642,7 +650,7 @@ unmask_finalize_kernel(const UnmaskPartial* __restrict__ partial, int32_t* __res
 
     // ---- the MASKED positions of the rollout and how many records each has (one round trip each)
     const int row = row0 + i;
-    const bool masked = i < d && state[row] == FDD_MASKED;
+    const bool masked = i < d && state[row] == FDD_MASKED;     // (d <= 128: threads beyond it only help with the merge)
     if (masked) {
         // records the first kernel wrote for this row (never more than the row has slots)
         const int n_rec = max(1, min(items_per_row, partial[static_cast<size_t>(row) * items_per_row].pad[0]));
@@ -650,7 +658,7 @@ unmask_finalize_kernel(const UnmaskPartial* __restrict__ partial, int32_t* __res
         s_rows[atomicAdd(&s_masked, 1)] = i;
         atomicMax(&s_max_rec, n_rec);
     }
-    s_conf[i] = -1.0f;
+    if (i < 128) s_conf[i] = -1.0f;
     __syncthreads();
     const int n_masked = s_masked;
 
@@ -661,7 +669,7 @@ unmask_finalize_kernel(const UnmaskPartial* __restrict__ partial, int32_t* __res
     int w = 1;
     while (w < s_max_rec && w < 32) w <<= 1;
     const int per = 32 / w, sub = lane / w, sl = lane - sub * w;
-    for (int base = warp * per; base < n_masked; base += 4 * per) {   // (warp-uniform bounds)
+    for (int base = warp * per; base < n_masked; base += (kFinalizeThreads / 32) * per) {   // (warp-uniform bounds)
         const int k = base + sub;
         const bool valid = k < n_masked;
         const int j = valid ? s_rows[k] : 0;
@@ -692,7 +700,7 @@ unmask_finalize_kernel(const UnmaskPartial* __restrict__ partial, int32_t* __res
     __syncthreads();
 
     // ---- the commit rule of the rollout
-    const float conf = s_conf[i];
+    const float conf = i < 128 ? s_conf[i] : -1.0f;
     if (i < d && conf_out) conf_out[row] = masked ? conf : CUDART_NAN_F;
     const bool pass = masked && conf > threshold;
     if (pass) atomicAdd(&s_pass, 1);
@@ -717,6 +725,7 @@ unmask_finalize_kernel(const UnmaskPartial* __restrict__ partial, int32_t* __res
         const int nc = (n_masked == 0) ? 0 : (n_pass > 0 ? n_pass : 1);
         n_committed[fork] = nc;
         n_left[fork] = n_masked - nc;
+        if (left_mirror != nullptr) left_mirror[fork] = n_masked - nc;     // host memory the GPU can write: no copy needed
     }
 }
 
@@ -815,6 +824,17 @@ cudaError_t device_setup(int dev, int* sm_count, const int** ctas_per_sm) {
     return cudaSuccess;
 }
 
+// Launch attribute that lets a kernel be made resident while the kernel ahead of it on the stream
+// drains (the kernels here wait with grid_dependency_wait before they read anything).  Not used
+// while the stream is being captured into a graph.  Returns the number of attributes written.
+int overlap_launch_attribute(cudaStream_t st, cudaLaunchAttribute* attr) {
+    cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+    if (cudaStreamIsCapturing(st, &cap) != cudaSuccess || cap != cudaStreamCaptureStatusNone) return 0;
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    return 1;
+}
+
 template <typename T, bool NOISY>
 void launch_stream(const UnmaskProblem& p, UnmaskPartial* partial, int tiles_per_item, int bulk_ok, int select_state,
                    int* status, int resident_ctas, cudaStream_t st) {
@@ -825,9 +845,18 @@ void launch_stream(const UnmaskProblem& p, UnmaskPartial* partial, int tiles_per
     const long long fit = resident_ctas;
     const long long need = (items + kWarps - 1) / kWarps;
     const unsigned grid = static_cast<unsigned>(need < fit ? (need < 1 ? 1 : need) : fit);
-    unmask_stream_kernel<T, NOISY><<<grid, kThreads, stream_smem_bytes<T>(), st>>>(
-        static_cast<const T*>(p.logits), p.state, p.sets, partial, p.vocab, tiles_per_item, p.temperature,
-        p.block_idx, p.step, bulk_ok, select_state, p.step_counter, status);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = stream_smem_bytes<T>();
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    const int n_attr = overlap_launch_attribute(st, attr);
+    cfg.attrs = attr;
+    cfg.numAttrs = n_attr;
+    cudaLaunchKernelEx(&cfg, unmask_stream_kernel<T, NOISY>, static_cast<const T*>(p.logits), static_cast<const uint8_t*>(p.state),
+                       p.sets, partial, p.vocab, tiles_per_item, p.temperature, p.block_idx, p.step, bulk_ok, select_state,
+                       static_cast<const uint32_t*>(p.step_counter), status);
 }
 
 // Both entry points launch the same two kernels; only the home of the records differs.
@@ -861,9 +890,19 @@ cudaError_t launch_unmask_kernels(const UnmaskProblem& p, UnmaskPartial* partial
     if (mode == 2)
         ss_accept_kernel<<<forks, 128, 0, st>>>(partial, p.tokens, p.state, p.n_committed, p.n_left, p.sets, items_per_row);
     else
-        unmask_finalize_kernel<<<forks, 128, 0, st>>>(partial, p.tokens, p.state, p.n_committed, p.n_left, p.conf,
-                                                     p.sets, items_per_row, p.threshold, mode == 1 ? FDD_DRAFT : FDD_COMMITTED,
-                                                     p.bump_counter ? p.step_counter : nullptr);
+    {
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(forks);
+        cfg.blockDim = dim3(kFinalizeThreads);
+        cfg.stream = st;
+        cudaLaunchAttribute attr[1];
+        cfg.numAttrs = overlap_launch_attribute(st, attr);
+        cfg.attrs = attr;
+        cudaLaunchKernelEx(&cfg, unmask_finalize_kernel, static_cast<const UnmaskPartial*>(partial), p.tokens, p.state,
+                           p.n_committed, p.n_left, p.conf, p.sets, items_per_row, p.threshold,
+                           mode == 1 ? static_cast<int>(FDD_DRAFT) : static_cast<int>(FDD_COMMITTED),
+                           p.bump_counter ? p.step_counter : static_cast<uint32_t*>(nullptr), p.left_mirror);
+    }
     return cudaGetLastError();
 }
 

@@ -22,7 +22,7 @@ EXPORTS = (
     "fdd_create", "fdd_destroy", "fdd_last_error", "fdd_launch_count", "fdd_fork",
     "fdd_forkset_free", "fdd_forkset_suffix_len", "fdd_forkset_reset", "fdd_block_attn", "fdd_block_attn_gated", "fdd_average_rollouts_jmt", "fdd_unmask_counted",
     "fdd_unmask", "fdd_ss_draft", "fdd_ss_accept", "fdd_kv_commit", "fdd_average_rollouts", "fdd_poll_status", "fdd_unmask_static", "fdd_plan_blocks", "fdd_upload_masked_rows",
-    "fdd_prefix_extend", "fdd_forkset_prefix_len", "fdd_set_merge_wait_limit",
+    "fdd_prefix_extend", "fdd_forkset_prefix_len", "fdd_set_merge_wait_limit", "fdd_decode_block",
 )
 FDD_UNMASK_STATIC_MAX_RECORDS = 65536
 
@@ -99,6 +99,9 @@ def lib():
     L.fdd_unmask_static.argtypes = [vp, i32, i32, i32, i32, vp, vp, vp, f32, f32, u32, u32, vp, vp, vp, vp,
                                     ctypes.c_char_p, ctypes.c_size_t]
     L.fdd_unmask_static.restype = i32
+    L.fdd_decode_block.argtypes = [vp, vpp, i32, i32, i32, i32, vpp, vpp, vpp, vpp, vpp, vp, vp, ip, f32, i32, f32, f32, u32,
+                                   i32, vp, vp, ctypes.POINTER(ctypes.c_int), ctypes.POINTER(ctypes.c_int), vp, vp, vp]
+    L.fdd_decode_block.restype = i32
     _lib_handle = L
     return L
 
@@ -234,6 +237,26 @@ def fdd_unmask(ctx, sets, logits, tokens, state, block_len, threshold, temperatu
         ctx, _ptr_array(sets), len(sets), _ptr(logits), _ptr(tokens), _ptr(state),
         _i32_array(block_len), float(threshold), float(temperature), int(block_idx), int(step),
         _ptr(n_committed), _ptr(n_left), _ptr(conf), _stream(stream)))
+
+
+def fdd_decode_block(ctx, sets, n_layers, max_steps, q, k_blk, v_blk, out, logits, tokens, state, block_len, scale,
+                     causal_in_block, threshold, temperature, block_idx, commit_kv, n_committed, n_left, stream=None):
+    """The denoising loop of one block, run by the library.  q, k_blk, v_blk, out: per resident input
+    set a list of n_layers tensors (or arrays made by ptr_array over the flattened [set][layer] list);
+    logits: one tensor per input set.  Returns (steps_taken, masked_left)."""
+    n_inputs = len(logits)
+
+    def flat(x):
+        return x if isinstance(x, ctypes.Array) else _ptr_array([t for per_set in x for t in per_set])
+
+    steps, left = ctypes.c_int(0), ctypes.c_int(0)
+    _check(ctx, lib().fdd_decode_block(
+        ctx, _ptr_array(sets), len(sets), int(n_layers), int(max_steps), int(n_inputs),
+        flat(q), flat(k_blk), flat(v_blk), flat(out), _ptr_array(logits), _ptr(tokens), _ptr(state),
+        _i32_array(block_len), float(scale), int(causal_in_block), float(threshold), float(temperature),
+        int(block_idx), int(commit_kv), _ptr(n_committed), _ptr(n_left), ctypes.byref(steps), ctypes.byref(left),
+        None, None, _stream(stream)))
+    return steps.value, left.value
 
 
 def fdd_unmask_counted(ctx, sets, logits, tokens, state, block_len, threshold, temperature, block_idx,

@@ -228,3 +228,74 @@ def test_merge_wait_that_runs_out_is_reported_and_the_context_recovers():
             pu.assert_attention_close(got, _oracle_attn(w, ofs, 0, q, k, v))
     finally:
         fdd.fdd_destroy(ctx)
+
+
+def test_library_block_loop_matches_the_oracle_loop():
+    # Sec. 3.3: fdd_decode_block runs the denoising loop of a block by itself (gated attention on
+    # every layer, unmasking, counts to the host, one step ahead) and commits the block's K/V when no
+    # MASK is left.  Two layers with caches of their own, two blocks in a row (the second reads what
+    # the first committed).  The oracle runs its own loop on the same inputs: the number of steps,
+    # the final tokens and state, the attention output of every step for the rollouts that still
+    # decoded, and the committed bytes must agree; rollouts that had finished are never written.
+    from oracle.decode import decode_block
+    L = 2
+    w = synth.small_variant(synth.workload("tts"), prefix_len=300 + 11, vocab=2048, n_forks=5, n_blocks=2)
+    sc = w.scenes[0]
+    N, d = sc.n_forks, sc.block_len
+    scale = 1.0 / np.sqrt(w.head_dim)
+    ctx = harness.create_context(w, n_layers=L)
+    try:
+        scene = harness.GpuScene(ctx, w, 0, n_layers=L, suffix_capacity=2 * d)
+        prefixes = [synth.make_prefix(w, 0, layer) for layer in range(L)]
+        ofs = ForkSet([p[0] for p in prefixes], [p[1] for p in prefixes], N, scene.seeds)
+        for block in range(2):
+            tokens0, state0 = synth.make_block_template(w, 0, block)
+            steps_in = d                                   # a block never needs more steps than it has positions
+            host = [dict(qkv=[synth.make_qkv(w, 0, layer, block, t) for layer in range(L)],
+                         logits=synth.make_logits(w, 0, block, t, rows="all")) for t in range(steps_in)]
+            inputs = lambda t: dict(q=[x[0] for x in host[t]["qkv"]], k=[x[1] for x in host[t]["qkv"]],
+                                    v=[x[2] for x in host[t]["qkv"]], logits=host[t]["logits"])
+            ref = decode_block(ofs, inputs, tokens0, state0, w.threshold, w.temperature, block, scale)
+            dq = [[harness.bf16_tensor(x[0]) for x in h["qkv"]] for h in host]
+            dk = [[harness.bf16_tensor(x[1]) for x in h["qkv"]] for h in host]
+            dv = [[harness.bf16_tensor(x[2]) for x in h["qkv"]] for h in host]
+            dout = [[torch.full_like(q_, float("nan")) for q_ in per] for per in dq]
+            dlg = [harness.logits_tensor(w, h["logits"]) for h in host]
+            tokens = torch.from_numpy(tokens0).cuda()
+            state = torch.from_numpy(state0).cuda()
+            n_c = torch.zeros(N, dtype=torch.int32, device="cuda")
+            n_l = torch.zeros(N, dtype=torch.int32, device="cuda")
+            steps, left = fdd.fdd_decode_block(ctx, [scene.forkset], L, steps_in, dq, dk, dv, dout, dlg, tokens, state,
+                                               [d], scale, 0, w.threshold, w.temperature, block, 1, n_c, n_l)
+            fdd.fdd_poll_status(ctx)
+            assert left == 0 and steps == ref["steps"] and 2 <= steps < d
+            assert np.array_equal(state.cpu().numpy(), ref["state"]) and not np.any(ref["state"] == MASKED)
+            assert np.array_equal(tokens.cpu().numpy(), ref["tokens"])
+            assert fdd.fdd_forkset_suffix_len(scene.forkset) == (block + 1) * d
+            # attention of every step: who still decoded on entry follows from the oracle's commits
+            masked_left = (state0 == MASKED).sum(axis=1)
+            for t in range(steps + 1):                     # the step after the last one was issued ahead and must do nothing
+                decoding = np.nonzero(masked_left > 0)[0] if t < steps else np.zeros(0, dtype=int)
+                for layer in range(L):
+                    got = dout[t][layer].float().cpu().numpy().astype(np.float64).reshape(N, d, w.n_q_heads, w.head_dim)
+                    if t < steps:
+                        pu.assert_attention_close(got[decoding], ref["attn"][t][layer][decoding])
+                    idle = np.setdiff1d(np.arange(N), decoding)
+                    assert np.all(np.isnan(got[idle])), "attention wrote rows of a rollout that had finished"
+                if t < steps:
+                    masked_left = masked_left - ref["committed_per_step"][t]
+            for layer in range(L):                         # the committed bytes (the oracle's loop commits too)
+                sk = scene.suffix_k[layer].view(torch.int16).cpu().numpy().view(np.uint16)
+                for f in range(N):
+                    assert np.array_equal(sk[f, :, :(block + 1) * d].transpose(1, 0, 2), ofs.suffix_k[layer][f])
+        # a loop that is cut short says so and commits nothing
+        tokens0, state0 = synth.make_block_template(w, 0, 0)
+        tokens, state = torch.from_numpy(tokens0).cuda(), torch.from_numpy(state0).cuda()
+        before = fdd.fdd_forkset_suffix_len(scene.forkset)
+        steps, left = fdd.fdd_decode_block(ctx, [scene.forkset], L, 1, dq[:1], dk[:1], dv[:1], dout[:1], dlg[:1], tokens, state,
+                                           [d], scale, 0, w.threshold, w.temperature, 0, 1, n_c, n_l)
+        fdd.fdd_poll_status(ctx)
+        assert steps == 1 and left == int((state.cpu().numpy() == MASKED).sum()) > 0
+        assert fdd.fdd_forkset_suffix_len(scene.forkset) == before
+    finally:
+        fdd.fdd_destroy(ctx)
