@@ -336,8 +336,12 @@ fdd_status fdd_average_rollouts_jmt(fdd_ctx* ctx, const float* traj, int n, int 
  *   before_step            NULL, or a function the library calls as before_step(user, t, stream)
  *                          before it issues step t: the place where a caller enqueues, on `stream`,
  *                          the model work that produces step t's q / k / v / logits
- * The call returns when the counts of the last step have reached the host (it synchronises with
- * events on `stream`, not with the device); the commits it issued may still be running.
+ * The counts reach the host through pinned host memory that the unmasking step writes itself
+ * (count and a per-step stamp in one 8-byte store), which the call polls: no copy and no event sits
+ * between two steps on the stream.  The poll is bounded: it ends with FDD_ERR_CUDA if the stream
+ * reports an error or runs empty without the counts, and with FDD_ERR_DEVICE_TIMEOUT after 30 s.
+ * The call returns when the counts of the last step have reached the host; the commits it issued
+ * may still be running.
  * Errors as for the calls it makes; nothing is issued after the first failure.
  */
 typedef void (*fdd_step_fn)(void* user, int step, void* stream);

@@ -261,6 +261,8 @@ attn_ptc_kernel(const __grid_constant__ TcArgs<MAXSETS> a) {
     // may be made resident on SMs as their CTA of this launch exits; it waits for the whole of this
     // launch before it reads anything.
     tc::grid_launch_dependents();
+    // (and this launch may itself have started early: the gate below is written by the kernel ahead of it)
+    tc::grid_dependency_wait();
 
     for (int s = warp; s < a.n_sets; s += kTcThreads / 32) {
         const SetParams& p = a.sets[s];
@@ -1002,10 +1004,34 @@ cudaError_t launch_one(const TcArgs<MAXSETS>& args, unsigned ctas, int device, c
         configured[device].store(true, std::memory_order_release);
     }
     // The CTAs wait for one another's pieces at the end: a cooperative launch makes the runtime
-    // guarantee that all of them are resident at once (or fail the launch).
+    // guarantee that all of them are resident at once (or fail the launch).  The launch also asks for
+    // an early start behind the kernel ahead of it on the stream (the kernel waits before it reads
+    // anything); a runtime that does not take the two attributes together gets the first one alone.
     void* params[] = {const_cast<TcArgs<MAXSETS>*>(&args)};
-    return cudaLaunchCooperativeKernel(reinterpret_cast<const void*>(&attn_ptc_kernel<D, MAXSETS, EMU>), dim3(ctas),
-                                       dim3(kTcThreads), params, static_cast<size_t>(smem), st);
+    static std::atomic<int> early_start_refused[kMaxDevices];
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(ctas);
+    cfg.blockDim = dim3(kTcThreads);
+    cfg.dynamicSmemBytes = static_cast<size_t>(smem);
+    cfg.stream = st;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeCooperative;
+    attr[0].val.cooperative = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+    const bool capturing = cudaStreamIsCapturing(st, &cap) != cudaSuccess || cap != cudaStreamCaptureStatusNone;
+    const void* fn = reinterpret_cast<const void*>(&attn_ptc_kernel<D, MAXSETS, EMU>);
+    if (!capturing && !early_start_refused[device].load(std::memory_order_relaxed)) {
+        cfg.numAttrs = 2;
+        const cudaError_t e = cudaLaunchKernelExC(&cfg, fn, params);
+        if (e == cudaSuccess) return e;
+        (void)cudaGetLastError();                         // a refused configuration launches nothing and leaves no sticky error
+        early_start_refused[device].store(1, std::memory_order_relaxed);
+    }
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelExC(&cfg, fn, params);
 }
 
 template <int MAXSETS>

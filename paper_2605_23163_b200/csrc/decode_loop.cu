@@ -7,6 +7,58 @@
 // native code and runs one step ahead of the counts it reads.
 #include "fdd_internal.h"
 
+#include <chrono>
+
+namespace {
+
+// Wait until every rollout's (n_left, stamp) of the step with this stamp has reached the host; their
+// sum goes to *left.  The wait is bounded: it ends with an error if the stream reports one, if the
+// stream has run empty without the counts arriving, or after kCountWaitSeconds.
+constexpr double kCountWaitSeconds = 30.0;
+
+fdd_status wait_for_counts(fdd_ctx* ctx, int buf, int stamp, int forks, cudaStream_t st, int* left) {
+    const volatile long long* src = reinterpret_cast<const volatile long long*>(ctx->h_counts[buf]);
+    const auto t0 = std::chrono::steady_clock::now();
+    int f = 0, sum = 0;
+    unsigned spins = 0;
+    bool drained = false;
+    while (f < forks) {
+        const long long v = src[f];                      // one aligned 8-byte load: count in the low half, stamp in the high half
+        if (static_cast<int>(v >> 32) == stamp) {
+            sum += static_cast<int>(v & 0xFFFFFFFFLL);
+            ++f;
+            continue;
+        }
+        if ((++spins & 0x3FFu) == 0) {
+            const double waited = std::chrono::duration<double>(std::chrono::steady_clock::now() - t0).count();
+            if (waited > 200e-6) {
+                // a long wait: make sure the stream is still alive
+                if (drained) {
+                    ctx->last_error = "fdd_decode_block: the stream ran empty but the counts of a step never arrived";
+                    return FDD_ERR_CUDA;
+                }
+                const cudaError_t q = cudaStreamQuery(st);
+                if (q == cudaSuccess) drained = true;    // everything issued has completed: one more look at the counts, then give up
+                else if (q != cudaErrorNotReady) {
+                    ctx->last_error = std::string("fdd_decode_block: ") + cudaGetErrorString(q);
+                    return FDD_ERR_CUDA;
+                }
+            }
+            if (waited > kCountWaitSeconds) {
+                ctx->last_error = "fdd_decode_block: timed out waiting for the counts of a step";
+                return FDD_ERR_DEVICE_TIMEOUT;
+            }
+        }
+#if defined(__x86_64__) || defined(__i386__)
+        __builtin_ia32_pause();
+#endif
+    }
+    *left = sum;
+    return FDD_OK;
+}
+
+}  // namespace
+
 fdd_status fdd_decode_block(fdd_ctx* ctx, fdd_forkset* const* sets, int n_sets, int n_layers,
                             int max_steps, int n_inputs,
                             const void* const* q, const void* const* k_blk, const void* const* v_blk,
@@ -42,6 +94,7 @@ fdd_status fdd_decode_block(fdd_ctx* ctx, fdd_forkset* const* sets, int n_sets, 
     *steps_taken = 0;
     if (masked_left) *masked_left = 0;
 
+    int stamp_of[2] = {0, 0};
     // One denoising step on the stream.  From the second step on, attention skips the rollouts that
     // the step before left without a MASKED position (n_left is written by that step's unmask and
     // read by this step's attention, both on `st`).
@@ -54,18 +107,17 @@ fdd_status fdd_decode_block(fdd_ctx* ctx, fdd_forkset* const* sets, int n_sets, 
                                                        scale, causal_in_block, t == 0 ? nullptr : n_left, stream);
             if (rc != FDD_OK) return rc;
         }
-        // the unmasking step also writes its n_left into host memory that the device can address:
-        // the counts are on the host when the event behind the call has completed, without a copy
+        // the unmasking step also writes (n_left, stamp) of every rollout into host memory that the
+        // device can address: the host sees the counts the moment they land, without a copy and
+        // without an event on the stream (which would sit between this step and the next one's early start)
+        if (++ctx->count_stamp <= 0) ctx->count_stamp = 1;
+        stamp_of[t & 1] = ctx->count_stamp;
         ctx->unmask_left_mirror = ctx->d_counts[t & 1];
+        ctx->unmask_mirror_stamp = ctx->count_stamp;
         const fdd_status rc = fdd_unmask(ctx, sets, n_sets, logits[in], tokens, state, block_len, threshold, temperature,
                                          block_idx, static_cast<uint32_t>(t), n_committed, n_left, nullptr, stream);
         ctx->unmask_left_mirror = nullptr;
         if (rc != FDD_OK) return rc;
-        const cudaError_t e = cudaEventRecord(ctx->count_ready[t & 1], st);
-        if (e != cudaSuccess) {
-            ctx->last_error = std::string("fdd_decode_block: ") + cudaGetErrorString(e);
-            return FDD_ERR_CUDA;
-        }
         return FDD_OK;
     };
 
@@ -76,14 +128,8 @@ fdd_status fdd_decode_block(fdd_ctx* ctx, fdd_forkset* const* sets, int n_sets, 
         // complete, its kernels find every rollout gated off and no MASKED row, and return at once
         if (t + 1 < max_steps) rc = enqueue(t + 1);
         if (rc != FDD_OK) break;
-        const cudaError_t e = cudaEventSynchronize(ctx->count_ready[t & 1]);
-        if (e != cudaSuccess) {
-            ctx->last_error = std::string("fdd_decode_block: ") + cudaGetErrorString(e);
-            rc = FDD_ERR_CUDA;
-            break;
-        }
-        left = 0;
-        for (int f = 0; f < forks; ++f) left += ctx->h_counts[t & 1][f];
+        rc = wait_for_counts(ctx, t & 1, stamp_of[t & 1], forks, st, &left);
+        if (rc != FDD_OK) break;
         ++t;
         if (left == 0 || t >= max_steps) break;
     }

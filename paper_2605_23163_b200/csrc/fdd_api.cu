@@ -118,10 +118,12 @@ fdd_status fdd_create(const fdd_config* cfg, fdd_ctx** out) {
     if (e == cudaSuccess) e = cudaMemset(ctx->d_status, 0, sizeof(int));
     if (e == cudaSuccess) e = cudaMallocHost(&ctx->h_status, sizeof(int));
     for (int i = 0; i < 2 && e == cudaSuccess; ++i) {
-        e = cudaHostAlloc(&ctx->h_counts[i], sizeof(int32_t) * static_cast<size_t>(cfg->max_forks > 0 ? cfg->max_forks : 1),
-                          cudaHostAllocMapped);
-        if (e == cudaSuccess) e = cudaHostGetDevicePointer(&ctx->d_counts[i], ctx->h_counts[i], 0);
-        if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->count_ready[i], cudaEventDisableTiming);
+        const size_t bytes = sizeof(int2) * static_cast<size_t>(cfg->max_forks > 0 ? cfg->max_forks : 1);
+        e = cudaHostAlloc(&ctx->h_counts[i], bytes, cudaHostAllocMapped);
+        if (e == cudaSuccess) {
+            memset(ctx->h_counts[i], 0, bytes);
+            e = cudaHostGetDevicePointer(&ctx->d_counts[i], ctx->h_counts[i], 0);
+        }
     }
     ctx->seed_chunk = new (std::nothrow) SeedChunk();
     if (!ctx->seed_chunk && e == cudaSuccess) e = cudaErrorMemoryAllocation;
@@ -162,10 +164,8 @@ void fdd_destroy(fdd_ctx* ctx) {
     for (const fdd_ctx::JmtWeights& j : ctx->jmt_weights) cudaFree(j.d_weights);
     if (ctx->d_status) cudaFree(ctx->d_status);
     if (ctx->h_status) cudaFreeHost(ctx->h_status);
-    for (int i = 0; i < 2; ++i) {
+    for (int i = 0; i < 2; ++i)
         if (ctx->h_counts[i]) cudaFreeHost(ctx->h_counts[i]);
-        if (ctx->count_ready[i]) cudaEventDestroy(ctx->count_ready[i]);
-    }
     if (ctx->ws_unmask) cudaFree(ctx->ws_unmask);
     if (ctx->ws_attn) cudaFree(ctx->ws_attn);
     if (ctx->attn_unit_count) cudaFree(ctx->attn_unit_count);
@@ -416,6 +416,7 @@ static fdd_status unmask_like(fdd_ctx* ctx, fdd_forkset* const* sets, int n_sets
         p.step_counter = step_counter;
         p.bump_counter = (step_counter != nullptr && s == n_sets) ? 1 : 0;      // the last group of the call advances it
         p.left_mirror = (mode == 0 && ctx->unmask_left_mirror) ? ctx->unmask_left_mirror + fork_off : nullptr;
+        p.mirror_stamp = ctx->unmask_mirror_stamp;
         int n_launches = 0;
         cudaError_t e = launch_unmask(ctx, p, static_cast<cudaStream_t>(stream), &n_launches, mode);
         ctx->launches += n_launches;

@@ -46,10 +46,11 @@ struct fdd_ctx {
     int sm_count = 0;
     int* d_status = nullptr;          // device status word (first error wins)
     int* h_status = nullptr;          // pinned mirror
-    int32_t* h_counts[2] = {nullptr, nullptr};     // pinned, [max_forks] each: the counts of two steps in flight (fdd_decode_block)
-    cudaEvent_t count_ready[2] = {nullptr, nullptr};   // recorded behind the unmask call of a step
-    int32_t* d_counts[2] = {nullptr, nullptr};         // the device's addresses of h_counts
-    int32_t* unmask_left_mirror = nullptr;             // set by fdd_decode_block around its fdd_unmask calls
+    int2* h_counts[2] = {nullptr, nullptr};   // pinned and mapped, [max_forks] each: (n_left, stamp) of the two steps in flight (fdd_decode_block)
+    int2* d_counts[2] = {nullptr, nullptr};   // the device's addresses of h_counts
+    int2* unmask_left_mirror = nullptr;       // set by fdd_decode_block around its fdd_unmask calls
+    int unmask_mirror_stamp = 0;
+    int count_stamp = 0;                      // the stamp of the step issued last
     void* ws_unmask = nullptr;        // per (row, tile) partial reductions
     size_t ws_unmask_bytes = 0;
     void* ws_attn = nullptr;          // partial outputs of attention units cut between CTAs
@@ -133,7 +134,8 @@ struct UnmaskProblem {
     uint32_t block_idx, step;
     uint32_t* step_counter = nullptr;   // device or nullptr: its value is added to `step` when the kernels run
     int bump_counter = 0;               // increment it once this launch pair is done
-    int32_t* left_mirror = nullptr;     // host memory mapped for the device, [forks], or nullptr: n_left is written there too
+    int2* left_mirror = nullptr;        // host memory mapped for the device, [forks], or nullptr: (n_left, mirror_stamp) is written there too
+    int mirror_stamp = 0;
 };
 
 // Unmask scratch: one record per (row, chunk).

@@ -632,7 +632,8 @@ unmask_finalize_kernel(const UnmaskPartial* __restrict__ partial, int32_t* __res
                        uint8_t* __restrict__ state, int32_t* __restrict__ n_committed,
                        int32_t* __restrict__ n_left, float* __restrict__ conf_out,
                        const __grid_constant__ UnmaskSets sets, int items_per_row, float threshold, int commit_state,
-                       uint32_t* __restrict__ step_bump, int32_t* __restrict__ left_mirror) {
+                       uint32_t* __restrict__ step_bump, int2* __restrict__ left_mirror, int mirror_stamp) {
+    tc::grid_launch_dependents();                       // the next kernel may be made resident; it waits for this one
     tc::grid_dependency_wait();                         // the streaming kernel's records are complete and visible
     // (the streaming kernel of this call has read the counter; the next call sees it advanced)
     if (step_bump != nullptr && blockIdx.x == 0 && threadIdx.x == 0) *step_bump += 1u;
@@ -725,7 +726,9 @@ unmask_finalize_kernel(const UnmaskPartial* __restrict__ partial, int32_t* __res
         const int nc = (n_masked == 0) ? 0 : (n_pass > 0 ? n_pass : 1);
         n_committed[fork] = nc;
         n_left[fork] = n_masked - nc;
-        if (left_mirror != nullptr) left_mirror[fork] = n_masked - nc;     // host memory the GPU can write: no copy needed
+        // host memory the GPU can write: count and stamp go out as one 8-byte store, so a host that
+        // sees the stamp of this call sees its count
+        if (left_mirror != nullptr) left_mirror[fork] = make_int2(n_masked - nc, mirror_stamp);
     }
 }
 
@@ -901,7 +904,7 @@ cudaError_t launch_unmask_kernels(const UnmaskProblem& p, UnmaskPartial* partial
         cudaLaunchKernelEx(&cfg, unmask_finalize_kernel, static_cast<const UnmaskPartial*>(partial), p.tokens, p.state,
                            p.n_committed, p.n_left, p.conf, p.sets, items_per_row, p.threshold,
                            mode == 1 ? static_cast<int>(FDD_DRAFT) : static_cast<int>(FDD_COMMITTED),
-                           p.bump_counter ? p.step_counter : static_cast<uint32_t*>(nullptr), p.left_mirror);
+                           p.bump_counter ? p.step_counter : static_cast<uint32_t*>(nullptr), p.left_mirror, p.mirror_stamp);
     }
     return cudaGetLastError();
 }
