@@ -179,19 +179,22 @@ constexpr float kPoly2 = 0.2426108568906784f * kPolyScale;
 constexpr float kPoly3 = 0.055171459913253784f * kPolyScale;
 constexpr float kRoundMagic = 12582912.0f;                    // 1.5 * 2^23: adding it rounds to an integer
 
-// Merge of a unit cut between CTAs:  out = sum_k w_k O_k,  w_k = 2^(lse_k - M) / sum_j 2^(lse_j - M).
+// Merge of a unit cut between CTAs:  out = sum_k w_k O_k / sum_k w_k,  w_k = 2^(lse_k - M), M = max_k lse_k.
 // Every CTA that holds a piece merges an equal share of the unit's rows.  A thread takes CT float4
-// columns of one row: 32 / CT pieces are read per round trip, 32 independent 16-byte reads in flight.
+// columns of one row: 32 / CT pieces are read per round trip, 32 independent 16-byte reads (and the
+// pieces' log-sum-exps) in flight.  M is not known in advance: the sums are kept relative to the
+// largest log-sum-exp seen so far and rescaled when a chunk raises it, so the pieces are read once.
 // Partials lie column-major in their slots ([D / 4][256 rows] float4).
 template <int D, int CT>
 __device__ __forceinline__ void merge_columns(const float* part_o, const float* part_lse, const int* slot_s, int n_pieces,
-                                              int row, int col0, float M, float inv_wsum, __nv_bfloat16* op) {
+                                              int row, int col0, __nv_bfloat16* op) {
     constexpr int NC4 = D / 4;
     constexpr int PC = 32 / CT;                     // pieces per chunk
     const float4* po4 = reinterpret_cast<const float4*>(part_o);
     float4 acc[CT];
 #pragma unroll
     for (int c = 0; c < CT; ++c) acc[c] = make_float4(0.f, 0.f, 0.f, 0.f);
+    float M = -CUDART_INF_F, wsum = 0.0f;
     for (int k0 = 0; k0 < n_pieces; k0 += PC) {
         float ls[PC];
         float4 ov[PC][CT];
@@ -204,9 +207,20 @@ __device__ __forceinline__ void merge_columns(const float* part_o, const float* 
             for (int c = 0; c < CT; ++c)
                 ov[k][c] = live ? __ldcg(po4 + (slot * NC4 + col0 + c) * 256 + row) : make_float4(0.f, 0.f, 0.f, 0.f);
         }
+        float mc = ls[0];
+#pragma unroll
+        for (int k = 1; k < PC; ++k) mc = fmaxf(mc, ls[k]);
+        const float mn = fmaxf(M, mc);
+        if (!(mn > -CUDART_INF_F)) continue;                        // nothing but empty pieces so far
+        const float back = exp2f(M - mn);                           // 0 the first time (M = -inf), 1 while M stands
+        wsum *= back;
+#pragma unroll
+        for (int c = 0; c < CT; ++c) { acc[c].x *= back; acc[c].y *= back; acc[c].z *= back; acc[c].w *= back; }
+        M = mn;
 #pragma unroll
         for (int k = 0; k < PC; ++k) {
-            const float wgt = exp2f(ls[k] - M) * inv_wsum;          // 0 for a piece that is not there
+            const float wgt = exp2f(ls[k] - M);                     // 0 for a piece that is not there
+            wsum += wgt;
 #pragma unroll
             for (int c = 0; c < CT; ++c) {
                 acc[c].x = fmaf(wgt, ov[k][c].x, acc[c].x); acc[c].y = fmaf(wgt, ov[k][c].y, acc[c].y);
@@ -214,9 +228,10 @@ __device__ __forceinline__ void merge_columns(const float* part_o, const float* 
             }
         }
     }
+    const float iw = wsum > 0.0f ? 1.0f / wsum : 0.0f;
 #pragma unroll
     for (int c = 0; c < CT; ++c) {
-        const __nv_bfloat162 b0 = __floats2bfloat162_rn(acc[c].x, acc[c].y), b1 = __floats2bfloat162_rn(acc[c].z, acc[c].w);
+        const __nv_bfloat162 b0 = __floats2bfloat162_rn(acc[c].x * iw, acc[c].y * iw), b1 = __floats2bfloat162_rn(acc[c].z * iw, acc[c].w * iw);
         *reinterpret_cast<uint2*>(op + (col0 + c) * 4) =
             make_uint2(*reinterpret_cast<const uint32_t*>(&b0), *reinterpret_cast<const uint32_t*>(&b1));
     }
@@ -768,16 +783,10 @@ attn_ptc_kernel(const __grid_constant__ TcArgs<MAXSETS> a) {
                     if (last_s) {
                         __threadfence();
                         if (row_ok) {                            // thread = row
-                            const float l0 = __ldcg(a.part_lse + static_cast<size_t>(slot_s[0]) * 256 + tid);
-                            const float l1 = __ldcg(a.part_lse + static_cast<size_t>(slot_s[1]) * 256 + tid);
-                            float M = fmaxf(l0, l1);
-                            if (!(M > -CUDART_INF_F)) M = 0.0f;
-                            const float wsum = exp2f(l0 - M) + exp2f(l1 - M);
-                            const float iw = wsum > 0.0f ? 1.0f / wsum : 0.0f;
                             __nv_bfloat16* op = p.out + ((static_cast<size_t>(f) * p.d + qi) * p.n_q_heads + h * p.G + qg) * D;
 #pragma unroll
                             for (int col0 = 0; col0 < D / 4; col0 += 16)
-                                merge_columns<D, 16>(a.part_o, a.part_lse, slot_s, 2, tid, col0, M, iw, op);
+                                merge_columns<D, 16>(a.part_o, a.part_lse, slot_s, 2, tid, col0, op);
                         }
                     }
                     tc::named_barrier(1, 256);                   // slot_s is free again
@@ -849,37 +858,17 @@ attn_ptc_kernel(const __grid_constant__ TcArgs<MAXSETS> a) {
                 const int row_in_share = lt / col_groups, cg = lt - row_in_share * col_groups;
                 if (share > 0 && row_in_share < share) {
                     const int rowu = row_lo + row_in_share;
-                    float M = -CUDART_INF_F, wsum = 0.0f;
-                    for (int k0 = 0; k0 < n_pieces; k0 += 8) {
-                        float ls[8];
-#pragma unroll
-                        for (int k = 0; k < 8; ++k)
-                            ls[k] = k0 + k < n_pieces ? __ldcg(a.part_lse + static_cast<size_t>(slots[min(k0 + k, n_pieces - 1)]) * 256 + rowu)
-                                                      : -CUDART_INF_F;
-                        float mc = ls[0];
-#pragma unroll
-                        for (int k = 1; k < 8; ++k) mc = fmaxf(mc, ls[k]);
-                        const float mn = fmaxf(M, mc);
-                        if (mn > -CUDART_INF_F) {
-                            wsum *= exp2f(M - mn);                  // 0 the first time (M = -inf)
-#pragma unroll
-                            for (int k = 0; k < 8; ++k) wsum += exp2f(ls[k] - mn);
-                            M = mn;
-                        }
-                    }
-                    if (!(M > -CUDART_INF_F)) M = 0.0f;
-                    const float iw = wsum > 0.0f ? 1.0f / wsum : 0.0f;
                     const int r = dfr.rp * 256 + rowu;
                     const int qi2 = r / p.G, qg2 = r - qi2 * p.G;
                     __nv_bfloat16* op = p.out + ((static_cast<size_t>(dfr.f) * p.d + qi2) * p.n_q_heads + dfr.h * p.G + qg2) * D;
                     const int col0 = cg * ct;
                     switch (ct) {
-                        case 1: merge_columns<D, 1>(a.part_o, a.part_lse, slots, n_pieces, rowu, col0, M, iw, op); break;
-                        case 2: merge_columns<D, 2>(a.part_o, a.part_lse, slots, n_pieces, rowu, col0, M, iw, op); break;
-                        case 4: merge_columns<D, 4>(a.part_o, a.part_lse, slots, n_pieces, rowu, col0, M, iw, op); break;
-                        case 8: merge_columns<D, 8>(a.part_o, a.part_lse, slots, n_pieces, rowu, col0, M, iw, op); break;
-                        case 16: merge_columns<D, 16>(a.part_o, a.part_lse, slots, n_pieces, rowu, col0, M, iw, op); break;
-                        default: merge_columns<D, 32>(a.part_o, a.part_lse, slots, n_pieces, rowu, col0, M, iw, op); break;
+                        case 1: merge_columns<D, 1>(a.part_o, a.part_lse, slots, n_pieces, rowu, col0, op); break;
+                        case 2: merge_columns<D, 2>(a.part_o, a.part_lse, slots, n_pieces, rowu, col0, op); break;
+                        case 4: merge_columns<D, 4>(a.part_o, a.part_lse, slots, n_pieces, rowu, col0, op); break;
+                        case 8: merge_columns<D, 8>(a.part_o, a.part_lse, slots, n_pieces, rowu, col0, op); break;
+                        case 16: merge_columns<D, 16>(a.part_o, a.part_lse, slots, n_pieces, rowu, col0, op); break;
+                        default: merge_columns<D, 32>(a.part_o, a.part_lse, slots, n_pieces, rowu, col0, op); break;
                     }
                 }
                 tc::named_barrier(1, 256);
