@@ -878,6 +878,8 @@ def test_step_recorded_as_a_cuda_graph_replays_the_block_loop():
     # One denoising step (gated attention, unmask with the step counted on the device, copy of the
     # counts) is recorded once as a CUDA graph and replayed until the block is complete; the result
     # must be what the same calls give when issued one by one with the step passed by value.
+    # (This test holds the replay against the CUDA path itself; that the calls issued one by one
+    # agree with the oracle is what test_pipelined_block_loop_* and test_block_loop_* check.)
     w = synth.small_variant(synth.workload("tts"), prefix_len=300, vocab=4096, n_forks=5)
     sc = w.scenes[0]
     N, d = sc.n_forks, sc.block_len
