@@ -728,7 +728,9 @@ unmask_finalize_kernel(const UnmaskPartial* __restrict__ partial, int32_t* __res
         n_left[fork] = n_masked - nc;
         // host memory the GPU can write: count and stamp go out as one 8-byte store, so a host that
         // sees the stamp of this call sees its count
-        if (left_mirror != nullptr) left_mirror[fork] = make_int2(n_masked - nc, mirror_stamp);
+        if (left_mirror != nullptr)
+            *reinterpret_cast<unsigned long long*>(left_mirror + fork) =
+                (static_cast<unsigned long long>(static_cast<uint32_t>(mirror_stamp)) << 32) | static_cast<uint32_t>(n_masked - nc);
     }
 }
 

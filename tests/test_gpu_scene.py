@@ -297,5 +297,13 @@ def test_library_block_loop_matches_the_oracle_loop():
         fdd.fdd_poll_status(ctx)
         assert steps == 1 and left == int((state.cpu().numpy() == MASKED).sum()) > 0
         assert fdd.fdd_forkset_suffix_len(scene.forkset) == before
+        # argument errors come back before anything is issued
+        launches = fdd.fdd_launch_count(ctx)
+        for bad in (dict(n_layers=L + 1), dict(max_steps=0)):
+            with pytest.raises(fdd.FddError) as ei:
+                fdd.fdd_decode_block(ctx, [scene.forkset], bad.get("n_layers", L), bad.get("max_steps", 1), dq[:1], dk[:1], dv[:1],
+                                     dout[:1], dlg[:1], tokens, state, [d], scale, 0, w.threshold, w.temperature, 0, 1, n_c, n_l)
+            assert ei.value.status == fdd.FDD_ERR_INVALID_ARG
+        assert fdd.fdd_launch_count(ctx) == launches
     finally:
         fdd.fdd_destroy(ctx)
