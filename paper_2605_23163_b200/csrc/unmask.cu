@@ -46,6 +46,7 @@ constexpr int kLaneIds = 64;                          // consecutive ids a lane 
 constexpr int kTile = kUnmaskTile;                    // ids per tile (one bulk copy, one warp)
 constexpr int kStages = 3;                            // tiles a warp holds in shared memory (two in flight while one is reduced)
 constexpr int kMaxRows = kUnmaskMaxRows;              // rows of one launch (32 per thread in the set-up)
+constexpr int kMinPiecesPerRow = 8;                   // rows are cut on their own when each can have this many warps
 constexpr int kMaxList = 224;                         // blocks in reach of the running lower bound kept per piece (a few dozen expected)
 constexpr long long kCopyWaitLimit = 4000000000LL;    // SM clocks a warp waits for one of its own copies (about two seconds)
 static_assert(kTile == 32 * kLaneIds, "a tile is 64 ids for each of 32 lanes");
@@ -317,14 +318,31 @@ unmask_stream_kernel(const T* __restrict__ logits, const uint8_t* __restrict__ s
 
     // ---- this warp's range of work items.  An item is tiles_per_item consecutive tiles of a row
     // (the last item of a row may be shorter); a row has items_per_row of them and as many record
-    // slots.  Warp c (of the G that get work) owns items [W c / G, W (c + 1) / G).
+    // slots.  Two ways to hand them out:
+    //  - few rows (at least kMinPiecesPerRow warps for each): a row is cut into ppr equal pieces, warp c
+    //    takes piece c % ppr of row c / ppr.  No warp then works on two rows, which would cost it two
+    //    rounds of the per-piece work (reductions, exact re-scoring, a record) while the others wait;
+    //  - otherwise the items of all rows, laid end to end, are cut into equal contiguous ranges, warp
+    //    c (of the G that get work) owns items [W c / G, W (c + 1) / G): tail of a row, whole rows, head
+    //    of the next.
     const int tiles_per_row = (vocab + kTile - 1) / kTile;
     const int ipr = (tiles_per_row + tiles_per_item - 1) / tiles_per_item;
     const long long W = static_cast<long long>(n_rows) * ipr;
-    const long long G = min(static_cast<long long>(gridDim.x) * kWarps, W);
+    const long long warps_all = static_cast<long long>(gridDim.x) * kWarps;
     const long long gw = static_cast<long long>(warp) * gridDim.x + blockIdx.x;   // warps of a CTA lie a grid apart: few items spread over all SMs
+    const int ppr = static_cast<int>(min(static_cast<long long>(ipr), warps_all / n_rows));   // pieces per row if rows are cut on their own
+    const bool by_row = ppr == ipr || ppr >= kMinPiecesPerRow;                   // (few pieces per row would leave too many warps without work)
+    const long long G = by_row ? static_cast<long long>(n_rows) * ppr : min(warps_all, W);
     if (gw >= G) return;
-    const long long range_begin = W * gw / G, range_end = W * (gw + 1) / G;
+    long long range_begin, range_end;
+    if (by_row) {
+        const int ri = static_cast<int>(gw / ppr), pc = static_cast<int>(gw - static_cast<long long>(ri) * ppr);
+        range_begin = static_cast<long long>(ri) * ipr + ipr * pc / ppr;
+        range_end = static_cast<long long>(ri) * ipr + ipr * (pc + 1) / ppr;
+    } else {
+        range_begin = W * gw / G;
+        range_end = W * (gw + 1) / G;
+    }
 
     const uint32_t full = 0xFFFFFFFFu;
     const int sw = lane & 7;                            // rotation of the chunk order (bank conflicts)
@@ -374,11 +392,17 @@ unmask_stream_kernel(const T* __restrict__ logits, const uint8_t* __restrict__ s
         const int row = nth_selected_row(s_before, s_mask, per, ri);
         const int seg_end = min(vocab, tile1 * kTile);
         // which of the row's records this is, and how many there are
-        const long long row_first = static_cast<long long>(ri) * ipr;
-        const int w_first = static_cast<int>(((row_first + 1) * G + W - 1) / W) - 1;
-        const int w_last = static_cast<int>(((row_first + ipr) * G + W - 1) / W) - 1;
-        const int seg = static_cast<int>(gw) - w_first;
-        const int segs = w_last - w_first + 1;
+        int seg, segs;
+        if (by_row) {
+            seg = static_cast<int>(gw - static_cast<long long>(ri) * ppr);
+            segs = ppr;
+        } else {
+            const long long row_first = static_cast<long long>(ri) * ipr;
+            const int w_first = static_cast<int>(((row_first + 1) * G + W - 1) / W) - 1;
+            const int w_last = static_cast<int>(((row_first + ipr) * G + W - 1) / W) - 1;
+            seg = static_cast<int>(gw) - w_first;
+            segs = w_last - w_first + 1;
+        }
         const T* row_ptr = logits + static_cast<size_t>(row) * vocab;
         int set = 0;
         while (set + 1 < sets.n_sets && row >= sets.row_off[set + 1]) ++set;
@@ -553,14 +577,71 @@ unmask_stream_kernel(const T* __restrict__ logits, const uint8_t* __restrict__ s
                     __syncwarp();
                 }
             }
-            for (int b0 = 0; b0 < n_blocks; b0 += 32 / kLaneGroups) {
-                const int blk = b0 + lane / kLaneGroups;
+            // Up to eight listed blocks (the usual case): one turn, a group of 16 ids per lane.
+            if (n_blocks <= 32 / kLaneGroups) {
+                const int blk = lane / kLaneGroups;
                 if (blk < n_blocks) {
                     const int tl = every ? blk / 32 : list[blk].tile, fl = every ? blk % 32 : list[blk].lane;
                     const int v0 = (tile0 + tl) * kTile + fl * kLaneIds + (lane % kLaneGroups) * kGroup;
                     if (v0 < seg_end) best = better(best, score_group<T>(row_ptr, v0, sargs, noise));
                 }
                 __syncwarp();
+                n_blocks = 0;
+            }
+            // More: thirty-two listed blocks at a time, in two stages.  Stage one, a block per lane: the
+            // block's four words (one Philox block) and the largest logit of each of its four groups give a
+            // bound per group, which is tighter than the block's (about one group in three of a listed
+            // block still reaches).  Stage two, a group per lane: the groups that reach are dealt out over
+            // the lanes and scored exactly, so that no lane idles behind a group that was ruled out.  The
+            // best exact score so far raises the bar for the next thirty-two.
+            ScoreArgs turn_args = sargs;
+            for (int c0 = 0; c0 < n_blocks; c0 += 32) {
+                const int c = c0 + lane;
+                int vb0 = seg_end;                              // first id of this lane's block (none: seg_end)
+                if (c < n_blocks) {
+                    const int tl = every ? c / 32 : list[c].tile, fl = every ? c % 32 : list[c].lane;
+                    vb0 = (tile0 + tl) * kTile + fl * kLaneIds;
+                }
+                uint32_t reach = 0;                             // bit g: group g of the block can reach the bar
+                if (vb0 < seg_end) {
+                    // (a listed block lies inside the piece as a whole; only the row's end can cut it short,
+                    // and ids beyond the vocabulary read as -inf)
+                    const uint4 rq4 = philox4x32_10(make_uint4(static_cast<uint32_t>(vb0 >> 6), static_cast<uint32_t>(pos), step, block_idx), keys);
+                    float val[kLaneGroups][kGroup];
+#pragma unroll
+                    for (int g = 0; g < kLaneGroups; ++g) load_group(row_ptr, vb0 + g * kGroup, vocab, bulk_ok, val[g]);
+#pragma unroll
+                    for (int g = 0; g < kLaneGroups; ++g) {
+                        float gmax = val[g][0];
+#pragma unroll
+                        for (int i = 1; i < kGroup; ++i) gmax = fmaxf(gmax, val[g][i]);
+                        if (fmaf(temperature, word_gumbel_bound(pick_word(rq4, g)), gmax) >= turn_args.lb - 1e-3f) reach |= 1u << g;
+                    }
+                }
+                uint32_t mg[kLaneGroups];
+                int total = 0;
+#pragma unroll
+                for (int g = 0; g < kLaneGroups; ++g) {
+                    mg[g] = __ballot_sync(full, (reach >> g) & 1u);
+                    total += __popc(mg[g]);
+                }
+                for (int j0 = 0; j0 < total; j0 += 32) {
+                    int r = j0 + lane, g = 0, src = 0;
+                    const bool act = r < total;
+                    if (act) {
+                        while (r >= __popc(mg[g])) { r -= __popc(mg[g]); ++g; }
+                        src = nth_set_bit(mg[g], r);
+                    }
+                    const int v_src = __shfl_sync(full, vb0, src);
+                    if (act) best = better(best, score_group<T>(row_ptr, v_src + g * kGroup, turn_args, noise));
+                    __syncwarp();
+                }
+                if (c0 + 32 < n_blocks) {
+                    float seen = best.score;
+#pragma unroll
+                    for (int off = 16; off > 0; off >>= 1) seen = fmaxf(seen, __shfl_xor_sync(full, seen, off));
+                    turn_args.lb = fmaxf(turn_args.lb, seen);
+                }
             }
             if (lane == 0) s_n_list[warp] = 0;          // the list is empty again for the next piece
         } else {
