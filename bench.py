@@ -235,7 +235,7 @@ def run_ours(args):
         pending = [None, None]      # the event records of a step, completed once its entry counts are known
 
         def enqueue(t):
-            q, k, v, lg = inputs(t)
+            q, k, v, lg, *after = inputs(t)       # (after: an event the logits are ready behind, if they come by another stream)
             kv_of[t % 2] = (k, v)
             gate = n_left0_d if t == 0 else n_left_d[(t - 1) % 2]     # who still decodes: the counts of the step before
             recs = []
@@ -251,6 +251,8 @@ def run_ours(args):
             if timed_attn:
                 u0, u1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
                 u0.record(stream)
+            if after:
+                stream.wait_event(after[0])
             fdd.fdd_unmask(ctx, fs, lg, tokens, state, ds_c, w.threshold, w.temperature, 0, t, n_comm, n_left_d[t % 2])
             if timed_attn:
                 u1.record(stream)
@@ -482,20 +484,20 @@ def run_ours(args):
         stage = [torch.empty_like(x) for x in dev_steps[0]]
         tok_host = torch.zeros_like(tokens0_d, device="cpu").pin_memory()
         traj_host = torch.zeros((n_scenes, w.waypoints, 2), dtype=torch.float32).pin_memory()
-        state_host = torch.zeros_like(state0_d, device="cpu").pin_memory()
-        d2h_step = n_left_host.numel() * 4 + state_host.numel()
-        h2d_total = [0]
+        d2h_step = n_left_host.numel() * 4
+
+        pulled = torch.zeros(1, dtype=torch.int64, device="cuda")
+        qkv_bytes = [0]
 
         def from_host(t):
-            """q, k, v in full; of the logits only the rows the method reads (MASKED positions), which
-            the host learns from the state array it reads back first."""
+            """q, k, v in full (copies); of the logits only the rows the method reads (MASKED positions),
+            which a kernel pulls out of the pinned host buffer after reading the state on the device:
+            nothing is read back and nothing waits on the host."""
             src = pinned[t % PRE_STEPS]
-            state_host.copy_(state, non_blocking=True)
             for dst, s_ in zip(stage[:3], src[:3]):
                 dst.view(torch.int16).copy_(s_, non_blocking=True)
-                h2d_total[0] += s_.numel() * s_.element_size()
-            stream.synchronize()
-            h2d_total[0] += fdd.fdd_upload_masked_rows(ctx, src[3], stage[3], state_host)
+                qkv_bytes[0] += s_.numel() * s_.element_size()
+            fdd.fdd_pull_masked_rows(ctx, src[3], stage[3], state, pulled)
             return tuple(stage)
 
         e2e_steps = max(1, min(args.steps, args.e2e_steps))
@@ -504,9 +506,10 @@ def run_ours(args):
         ee0, ee1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         ee0.record(stream)
         e2e_denoise = 0
-        h2d_total[0] = 0
+        qkv_bytes[0] = 0
+        pulled.zero_()
         for _ in range(e2e_steps):
-            e2e_denoise += decode_block(from_host, False, False)
+            e2e_denoise += decode_block(from_host, False, False)     # (no step ahead: its q, k, v would cross the link for nothing)
             tok_host.copy_(tokens, non_blocking=True)
             traj_host.copy_(traj_out, non_blocking=True)
             stream.synchronize()
@@ -516,7 +519,7 @@ def run_ours(args):
         e_ms = replicas.max_over_ranks(e_ms, dist, "cuda")
         per_block_denoise = e2e_denoise / e2e_steps
         e2e = {"value": world * value_tokens * e2e_steps / (e_ms * 1e-3), "unit": UNIT,
-               "h2d_bytes_per_step": int(h2d_total[0] / e2e_steps),
+               "h2d_bytes_per_step": int((qkv_bytes[0] + int(pulled.item())) / e2e_steps),
                "d2h_bytes_per_step": int(d2h_step * per_block_denoise + tok_host.numel() * 4 + traj_host.numel() * 4),
                "steps": e2e_steps, "ms_per_step": e_ms / e2e_steps}
 

@@ -425,6 +425,23 @@ fdd_status fdd_upload_masked_rows(fdd_ctx* ctx, const void* host_logits, void* d
                                   const uint8_t* host_state, int rows, size_t* bytes_copied, void* stream);
 
 /*
+ * fdd_pull_masked_rows -- the same rows (Sec. 3.3: only MASKED value positions are decoded), fetched
+ * by a kernel that reads the state array on the device and pulls the rows out of host memory
+ * itself.  Nothing goes back to the host and nothing is synchronised, so the call can be issued
+ * ahead of the counts of the step before, like the other calls of a step.
+ *   host_logits   pinned host memory that the device can address (cudaHostAlloc / cudaHostRegister;
+ *                 FDD_ERR_INVALID_ARG otherwise) [rows][V], dtype per cfg.logits_dtype
+ *   dev_logits    device buffer of the same shape; rows that are not MASKED keep their old bytes
+ *   dev_state     device uint8 [rows], read when the kernel runs (stream order)
+ *   bytes_pulled  device counter or NULL: the bytes of every pulled row are added to it
+ * One launch of 32 CTAs on `stream` (a link of 55 GB/s is filled by 16); rows whose pitch is a
+ * multiple of 16 bytes move in 16-byte pieces, others two bytes at a time.
+ */
+fdd_status fdd_pull_masked_rows(fdd_ctx* ctx, const void* host_logits, void* dev_logits,
+                                const uint8_t* dev_state, int rows, unsigned long long* bytes_pulled,
+                                void* stream);
+
+/*
  * fdd_set_merge_wait_limit -- how long a CTA of fdd_block_attn waits for the partial results of the
  * other CTAs that share a unit of work with it, in SM clocks (default 4e9, about two seconds).  When
  * the limit runs out the CTA records FDD_ERR_DEVICE_TIMEOUT in the device status word and returns

@@ -22,7 +22,7 @@ EXPORTS = (
     "fdd_create", "fdd_destroy", "fdd_last_error", "fdd_launch_count", "fdd_fork",
     "fdd_forkset_free", "fdd_forkset_suffix_len", "fdd_forkset_reset", "fdd_block_attn", "fdd_block_attn_gated", "fdd_average_rollouts_jmt", "fdd_unmask_counted",
     "fdd_unmask", "fdd_ss_draft", "fdd_ss_accept", "fdd_kv_commit", "fdd_average_rollouts", "fdd_poll_status", "fdd_unmask_static", "fdd_plan_blocks", "fdd_upload_masked_rows",
-    "fdd_prefix_extend", "fdd_forkset_prefix_len", "fdd_set_merge_wait_limit", "fdd_decode_block",
+    "fdd_prefix_extend", "fdd_forkset_prefix_len", "fdd_set_merge_wait_limit", "fdd_decode_block", "fdd_pull_masked_rows",
 )
 FDD_UNMASK_STATIC_MAX_RECORDS = 65536
 
@@ -328,6 +328,17 @@ def fdd_plan_blocks(editable, section_end, d, capacity=4096):
     if st < 0:
         raise FddError(st, "fdd_plan_blocks failed")
     return [(int(bb[i]), int(be[i]), int(bs[i])) for i in range(n.value)]
+
+
+def fdd_pull_masked_rows(ctx, host_logits, dev_logits, dev_state, bytes_pulled=None, stream=None):
+    """host_logits: pinned CPU tensor [rows, V]; dev_logits: CUDA tensor of the same shape; dev_state: CUDA
+    uint8 tensor [rows]; bytes_pulled: CUDA int64 tensor of one element or None."""
+    L = lib()
+    L.fdd_pull_masked_rows.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int,
+                                       ctypes.c_void_p, ctypes.c_void_p]
+    L.fdd_pull_masked_rows.restype = ctypes.c_int
+    return _check(ctx, L.fdd_pull_masked_rows(ctx, _ptr(host_logits), _ptr(dev_logits), _ptr(dev_state),
+                                              int(dev_state.numel()), _ptr(bytes_pulled), _stream(stream)))
 
 
 def fdd_upload_masked_rows(ctx, host_logits, dev_logits, host_state, stream=None):

@@ -1054,6 +1054,43 @@ def test_upload_masked_rows_copies_exactly_the_rows_that_are_read():
         fdd.fdd_destroy(ctx)
 
 
+@pytest.mark.parametrize("vocab", [4096, 1001])
+def test_pull_masked_rows_fetches_exactly_the_rows_that_are_read(vocab):
+    # The same contract as the copy above, but a kernel reads the state on the device and pulls the
+    # rows out of pinned host memory itself; an odd vocabulary takes the path for rows that are not
+    # 16 bytes apart.
+    w = synth.small_variant(synth.workload("tts"), prefix_len=64, vocab=vocab, n_forks=3, n_blocks=1)
+    sc = w.scenes[0]
+    ctx = harness.create_context(w)
+    try:
+        rows = sc.n_forks * sc.block_len
+        g = np.random.default_rng(4)
+        host = torch.from_numpy(g.integers(-30000, 30000, size=(rows, w.vocab), dtype=np.int16)).pin_memory()
+        dev = torch.full((rows, w.vocab), 77, dtype=torch.int16, device="cuda")
+        _, state = synth.make_block_template(w, 0, 0)
+        state = state.reshape(-1).copy()
+        state[5] = COMMITTED
+        st = torch.from_numpy(state).cuda()
+        count = torch.zeros(1, dtype=torch.int64, device="cuda")
+        fdd.fdd_pull_masked_rows(ctx, host, dev, st, count)
+        torch.cuda.synchronize()
+        masked = state == MASKED
+        assert int(count.item()) == int(masked.sum()) * w.vocab * 2
+        got = dev.cpu().numpy()
+        assert np.array_equal(got[masked], host.numpy()[masked])
+        assert np.all(got[~masked] == 77)
+        fdd.fdd_pull_masked_rows(ctx, host, dev, torch.full((rows,), COMMITTED, dtype=torch.uint8, device="cuda"), count)
+        torch.cuda.synchronize()
+        assert int(count.item()) == int(masked.sum()) * w.vocab * 2          # nothing MASKED: nothing pulled
+        pageable = torch.zeros((rows, w.vocab), dtype=torch.int16)           # not pinned: the device cannot address it
+        with pytest.raises(fdd.FddError) as ei:
+            fdd.fdd_pull_masked_rows(ctx, pageable, dev, st, None)
+        assert ei.value.status == fdd.FDD_ERR_INVALID_ARG
+        fdd.fdd_poll_status(ctx)
+    finally:
+        fdd.fdd_destroy(ctx)
+
+
 # ---------------------------------------------------------------------------------------------
 # host-side error paths (nothing is launched)
 # ---------------------------------------------------------------------------------------------
