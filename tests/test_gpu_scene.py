@@ -307,3 +307,61 @@ def test_library_block_loop_matches_the_oracle_loop():
         assert fdd.fdd_launch_count(ctx) == launches
     finally:
         fdd.fdd_destroy(ctx)
+
+
+def test_library_block_loop_with_more_scenes_than_one_unmask_launch_takes():
+    # Eighteen small scenes (different rollouts, block lengths and prefix lengths) in one
+    # fdd_decode_block call: the unmasking step splits them into two launches, whose counts must all
+    # reach the loop's host buffer at the right place.  Every scene against the oracle's own loop.
+    from oracle.decode import decode_block
+    base = synth.workload("serving_mix")
+    rng = np.random.default_rng(7)
+    scenes = tuple(synth.Scene(int(rng.integers(1, 200)), int(rng.integers(1, 4)), int(rng.choice([16, 32])),
+                               int(rng.integers(3, 9)), 1) for _ in range(18))
+    w = synth.Workload("mix_loop", base.n_q_heads, base.n_kv_heads, base.head_dim, 512, "bf16", "peaked", 0.9, 1.0,
+                       scenes, page_tokens=64, seed=23)
+    scale = 1.0 / np.sqrt(w.head_dim)
+    d_max = max(sc.block_len for sc in scenes)
+    ctx = harness.create_context(w)
+    try:
+        gs = [harness.GpuScene(ctx, w, i, suffix_capacity=sc.block_len) for i, sc in enumerate(scenes)]
+        refs, host_steps = [], [[] for _ in range(d_max)]
+        tokens0, state0 = [], []
+        for i, sc in enumerate(scenes):
+            pk, pv = synth.make_prefix(w, i)
+            ofs = ForkSet([pk], [pv], sc.n_forks, gs[i].seeds)
+            t0, s0 = synth.make_block_template(w, i, 0)
+            per_step = [dict(qkv=synth.make_qkv(w, i, 0, 0, t), logits=synth.make_logits(w, i, 0, t, rows="all"))
+                        for t in range(d_max)]
+            inputs = lambda t, ps=per_step: dict(q=[ps[t]["qkv"][0]], k=[ps[t]["qkv"][1]], v=[ps[t]["qkv"][2]],
+                                                 logits=ps[t]["logits"])
+            refs.append(decode_block(ofs, inputs, t0, s0, w.threshold, w.temperature, 0, scale, want_attention=False))
+            for t in range(d_max):
+                host_steps[t].append(per_step[t])
+            tokens0.append(t0.reshape(-1)); state0.append(s0.reshape(-1))
+        pack = lambda xs: np.concatenate([np.asarray(x).reshape(-1) for x in xs])
+        dq = [[harness.bf16_tensor(pack([p["qkv"][0] for p in host_steps[t]]))] for t in range(d_max)]
+        dk = [[harness.bf16_tensor(pack([p["qkv"][1] for p in host_steps[t]]))] for t in range(d_max)]
+        dv = [[harness.bf16_tensor(pack([p["qkv"][2] for p in host_steps[t]]))] for t in range(d_max)]
+        dout = [[torch.empty_like(x[0])] for x in dq]
+        dlg = [harness.logits_tensor(w, pack([p["logits"] for p in host_steps[t]])) for t in range(d_max)]
+        tokens = torch.from_numpy(np.concatenate(tokens0)).cuda()
+        state = torch.from_numpy(np.concatenate(state0)).cuda()
+        N = sum(sc.n_forks for sc in scenes)
+        n_c = torch.zeros(N, dtype=torch.int32, device="cuda")
+        n_l = torch.zeros(N, dtype=torch.int32, device="cuda")
+        steps, left = fdd.fdd_decode_block(ctx, [g.forkset for g in gs], 1, d_max, dq, dk, dv, dout, dlg, tokens, state,
+                                           [sc.block_len for sc in scenes], scale, 0, w.threshold, w.temperature, 0, 1,
+                                           n_c, n_l)
+        fdd.fdd_poll_status(ctx)
+        assert left == 0 and steps == max(r["steps"] for r in refs)
+        got_tok, got_st = tokens.cpu().numpy(), state.cpu().numpy()
+        off = 0
+        for sc, ref, g in zip(scenes, refs, gs):
+            n = sc.n_forks * sc.block_len
+            assert np.array_equal(got_st[off:off + n].reshape(ref["state"].shape), ref["state"])
+            assert np.array_equal(got_tok[off:off + n].reshape(ref["tokens"].shape), ref["tokens"])
+            assert fdd.fdd_forkset_suffix_len(g.forkset) == sc.block_len
+            off += n
+    finally:
+        fdd.fdd_destroy(ctx)
