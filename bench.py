@@ -181,8 +181,12 @@ def run_ours(args):
     state0 = np.concatenate([s_.reshape(-1) for _, s_ in templates])
     tokens0_d = torch.from_numpy(tokens0).cuda()
     state0_d = torch.from_numpy(state0).cuda()
-    tokens = torch.empty_like(tokens0_d)
-    state = torch.empty_like(state0_d)
+    # tokens and state of the block live in one buffer (and their templates in another of the same
+    # layout), so that a block starts with one copy
+    blk0 = torch.cat([tokens0_d.view(torch.uint8), state0_d])
+    blk = torch.empty_like(blk0)
+    tokens = blk[:tokens0_d.numel() * 4].view(torch.int32)
+    state = blk[tokens0_d.numel() * 4:]
     out = torch.empty_like(dev_steps[0][0])
     n_comm = torch.zeros(N, dtype=torch.int32, device="cuda")
     n_left = torch.zeros(N, dtype=torch.int32, device="cuda")
@@ -373,7 +377,7 @@ def run_ours(args):
     # ---- the same loop run by the library (fdd_decode_block): the calls of a step are issued from
     # native code, one step ahead of the counts, and the block's K/V are committed by the same call.
     # The fork sets are made once and start every block with fdd_forkset_reset.
-    nat = {"list": None, "arr": None}
+    nat = {"list": None, "arr": None, "call": None}
     nat_q = fdd.ptr_array([dev_steps[t][0] for t in range(PRE_STEPS) for _ in range(L)])
     nat_k = fdd.ptr_array([dev_steps[t][1] for t in range(PRE_STEPS) for _ in range(L)])
     nat_v = fdd.ptr_array([dev_steps[t][2] for t in range(PRE_STEPS) for _ in range(L)])
@@ -384,13 +388,15 @@ def run_ours(args):
         if nat["list"] is None:
             nat["list"] = [fdd.fdd_fork(ctx, *fa) for fa in fork_args]
             nat["arr"] = fdd.ptr_array(nat["list"])
+            # (the same call block after block: its arguments are marshalled once)
+            nat["call"] = fdd.decode_block_call(ctx, nat["arr"], L, d, nat_q, nat_k, nat_v, nat_out, nat_lg, tokens, state,
+                                                ds_c, scale, 0, w.threshold, w.temperature, 0, 1, n_comm, n_left,
+                                                stream=stream_c)
         else:
             for f_ in nat["list"]:
                 fdd.fdd_forkset_reset(ctx, f_)
-        tokens.copy_(tokens0_d, non_blocking=True)
-        state.copy_(state0_d, non_blocking=True)
-        steps, left = fdd.fdd_decode_block(ctx, nat["arr"], L, d, nat_q, nat_k, nat_v, nat_out, nat_lg, tokens, state, ds_c,
-                                           scale, 0, w.threshold, w.temperature, 0, 1, n_comm, n_left, stream=stream_c)
+        blk.copy_(blk0, non_blocking=True)
+        steps, left = nat["call"]()
         assert left == 0
         for i in range(n_scenes):
             fdd.fdd_average_rollouts(ctx, trajs[i], Ns[i], w.waypoints, traj_out[i])

@@ -259,6 +259,33 @@ def fdd_decode_block(ctx, sets, n_layers, max_steps, q, k_blk, v_blk, out, logit
     return steps.value, left.value
 
 
+def decode_block_call(ctx, sets, n_layers, max_steps, q, k_blk, v_blk, out, logits, tokens, state, block_len, scale,
+                      causal_in_block, threshold, temperature, block_idx, commit_kv, n_committed, n_left, stream=None):
+    """The arguments of fdd_decode_block marshalled once: returns call() -> (steps_taken, masked_left) for a
+    caller that repeats the same call block after block (the conversion costs more than a short block's
+    first launch)."""
+    n_inputs = len(logits)
+
+    def flat(x):
+        return x if isinstance(x, ctypes.Array) else _ptr_array([t for per_set in x for t in per_set])
+
+    steps, left = ctypes.c_int(0), ctypes.c_int(0)
+    fn = lib().fdd_decode_block
+    args = (ctx, _ptr_array(sets), len(sets), int(n_layers), int(max_steps), int(n_inputs),
+            flat(q), flat(k_blk), flat(v_blk), flat(out), _ptr_array(logits), _ptr(tokens), _ptr(state),
+            _i32_array(block_len), float(scale), int(causal_in_block), float(threshold), float(temperature),
+            int(block_idx), int(commit_kv), _ptr(n_committed), _ptr(n_left), ctypes.byref(steps), ctypes.byref(left),
+            None, None, _stream(stream))
+
+    def call():
+        status = fn(*args)
+        if status < 0:
+            _check(ctx, status)
+        return steps.value, left.value
+
+    return call
+
+
 def fdd_unmask_counted(ctx, sets, logits, tokens, state, block_len, threshold, temperature, block_idx,
                        step_counter, n_committed, n_left, conf=None, stream=None):
     return _check(ctx, lib().fdd_unmask_counted(
