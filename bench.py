@@ -377,7 +377,7 @@ def run_ours(args):
     # ---- the same loop run by the library (fdd_decode_block): the calls of a step are issued from
     # native code, one step ahead of the counts, and the block's K/V are committed by the same call.
     # The fork sets are made once and start every block with fdd_forkset_reset.
-    nat = {"list": None, "arr": None, "call": None}
+    nat = {"list": None, "arr": None, "call": None, "avg": None}
     nat_q = fdd.ptr_array([dev_steps[t][0] for t in range(PRE_STEPS) for _ in range(L)])
     nat_k = fdd.ptr_array([dev_steps[t][1] for t in range(PRE_STEPS) for _ in range(L)])
     nat_v = fdd.ptr_array([dev_steps[t][2] for t in range(PRE_STEPS) for _ in range(L)])
@@ -392,14 +392,16 @@ def run_ours(args):
             nat["call"] = fdd.decode_block_call(ctx, nat["arr"], L, d, nat_q, nat_k, nat_v, nat_out, nat_lg, tokens, state,
                                                 ds_c, scale, 0, w.threshold, w.temperature, 0, 1, n_comm, n_left,
                                                 stream=stream_c)
+            nat["avg"] = [fdd.average_rollouts_call(ctx, trajs[i], Ns[i], w.waypoints, traj_out[i], stream=stream_c)
+                          for i in range(n_scenes)]
         else:
             for f_ in nat["list"]:
                 fdd.fdd_forkset_reset(ctx, f_)
         blk.copy_(blk0, non_blocking=True)
         steps, left = nat["call"]()
         assert left == 0
-        for i in range(n_scenes):
-            fdd.fdd_average_rollouts(ctx, trajs[i], Ns[i], w.waypoints, traj_out[i])
+        for avg in nat["avg"]:
+            avg()
         return steps
 
     def barrier():
@@ -431,7 +433,7 @@ def run_ours(args):
         denoise_steps = 0
         timed_blocks = 0
         for b_ in range(args.steps):
-            per_kernel = b_ % TIME_EVERY == 0
+            per_kernel = TIME_EVERY > 0 and b_ % TIME_EVERY == 0
             timed_blocks += per_kernel
             if GRAPH and not per_kernel:
                 denoise_steps += decode_block_graph()
@@ -570,6 +572,7 @@ def run_ours(args):
                                      if LOOKAHEAD else "attention gated by n_left; one step in flight"),
                    "steps_from_cuda_graph": bool(GRAPH),
                    "block_loop": ("library (fdd_decode_block)" if NATIVE_LOOP and not GRAPH else "bench.py"),
+                   "blocks_timed_kernel_by_kernel": (f"one in {TIME_EVERY}" if TIME_EVERY else "none"),
                    "count_copy": "own stream" if use_count_stream else "compute stream",
                    "rollouts_decoding_per_attention_call": float(np.mean([n for _, n in attn_all])) if attn_all else None,
                    "replicas": "independent scene per GPU, no collective"},
@@ -784,7 +787,7 @@ def run_replica_selftest(args):
 
 
 def main():
-    global PRE_STEPS, LOOKAHEAD, COUNT_STREAM, GRAPH, NATIVE_LOOP
+    global PRE_STEPS, LOOKAHEAD, COUNT_STREAM, GRAPH, NATIVE_LOOP, TIME_EVERY
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=40)
@@ -803,6 +806,9 @@ def main():
                     help="where the per-rollout counts are copied to the host: on the compute stream or on a stream of their own")
     ap.add_argument("--loop", choices=["library", "python"], default="library",
                     help="who runs the block loop of the blocks that are not timed kernel by kernel: the library's fdd_decode_block or this file")
+    ap.add_argument("--time-every", type=int, default=TIME_EVERY,
+                    help="every N-th block runs through the loop in this file with CUDA events around each kernel (the "
+                         "per-kernel figures of the roofline objects); 0: none, every block runs as a user would run it")
     ap.add_argument("--graph", action="store_true",
                     help="replay every denoising step from a CUDA graph (blocks whose kernels are timed one by one still run call by call)")
     ap.add_argument("--selftest-replicas", action="store_true",
@@ -813,6 +819,7 @@ def main():
     PRE_STEPS = max(1, args.pre_steps)
     LOOKAHEAD = not args.no_lookahead
     GRAPH = args.graph
+    TIME_EVERY = max(0, args.time_every)
     NATIVE_LOOP = args.loop == "library" and not args.no_lookahead
     COUNT_STREAM = {"auto": None, "in-line": False, "own-stream": True}[args.counts]
     if args.impl == "reference":

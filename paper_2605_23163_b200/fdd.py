@@ -338,6 +338,19 @@ def fdd_average_rollouts(ctx, traj, n, w, out, stream=None):
                                                   _stream(stream)))
 
 
+def average_rollouts_call(ctx, traj, n, w, out, stream=None):
+    """The arguments of fdd_average_rollouts marshalled once: returns call() for a caller that repeats it."""
+    fn = lib().fdd_average_rollouts
+    args = (ctx, _ptr(traj), int(n), int(w), _ptr(out), _stream(stream))
+
+    def call():
+        status = fn(*args)
+        if status < 0:
+            _check(ctx, status)
+
+    return call
+
+
 def fdd_plan_blocks(editable, section_end, d, capacity=4096):
     """Host-side block planner; returns a list of (begin, end, section)."""
     import numpy as np
