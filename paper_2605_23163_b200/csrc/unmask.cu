@@ -46,6 +46,7 @@ constexpr int kLaneIds = 64;                          // consecutive ids a lane 
 constexpr int kTile = kUnmaskTile;                    // ids per tile (one bulk copy, one warp)
 constexpr int kStages = 3;                            // tiles a warp holds in shared memory (two in flight while one is reduced)
 constexpr int kMaxRows = kUnmaskMaxRows;              // rows of one launch (32 per thread in the set-up)
+constexpr int kPiecePadNoisy = 5, kPiecePadGreedy = 3;   // the per-piece work of a warp, in tiles of streaming
 constexpr int kMinPiecesPerRow = 8;                   // rows are cut on their own when each can have this many warps
 constexpr int kMaxList = 224;                         // blocks in reach of the running lower bound kept per piece (a few dozen expected)
 constexpr long long kCopyWaitLimit = 4000000000LL;    // SM clocks a warp waits for one of its own copies (about two seconds)
@@ -236,6 +237,13 @@ __device__ __forceinline__ int nth_selected_row(const int* s_before, const uint3
     return lo * per + nth_set_bit(s_mask[lo], ri - s_before[lo]);
 }
 
+// Item index of position v on the axis that has `pad` extra items in front of every row's ipr items.
+__device__ __forceinline__ long long padded_to_item(long long v, int ipr, int pad) {
+    const long long r = v / (ipr + pad);
+    const long long off = v - r * (ipr + pad);
+    return r * ipr + (off > pad ? off - pad : 0);
+}
+
 // A block (the 64 ids of one lane in one tile) whose upper bound reached the running lower bound.
 struct Reach {
     float ub;            // upper bound of the block's scores
@@ -334,14 +342,22 @@ unmask_stream_kernel(const T* __restrict__ logits, const uint8_t* __restrict__ s
     const bool by_row = ppr == ipr || ppr >= kMinPiecesPerRow;                   // (few pieces per row would leave too many warps without work)
     const long long G = by_row ? static_cast<long long>(n_rows) * ppr : min(warps_all, W);
     if (gw >= G) return;
+    // (in items; only where a range is much longer than it)
+    const int pad = (W >= 16 * G) ? ((NOISY ? kPiecePadNoisy : kPiecePadGreedy) + tiles_per_item - 1) / tiles_per_item : 0;
+    const long long Vp = static_cast<long long>(n_rows) * (ipr + pad);
     long long range_begin, range_end;
     if (by_row) {
         const int ri = static_cast<int>(gw / ppr), pc = static_cast<int>(gw - static_cast<long long>(ri) * ppr);
         range_begin = static_cast<long long>(ri) * ipr + ipr * pc / ppr;
         range_end = static_cast<long long>(ri) * ipr + ipr * (pc + 1) / ppr;
     } else {
-        range_begin = W * gw / G;
-        range_end = W * (gw + 1) / G;
+        // A warp whose range takes in a row's start works on two rows and pays the per-piece work
+        // twice.  That work is counted as `pad` items at the start of every row: the ranges are equal on
+        // the axis with those items put in, and are then mapped back (a range that falls inside the
+        // padding alone, which needs a range shorter than pad, is empty).
+        range_begin = padded_to_item(Vp * gw / G, ipr, pad);
+        range_end = padded_to_item(Vp * (gw + 1) / G, ipr, pad);
+        if (range_begin >= range_end) return;
     }
 
     const uint32_t full = 0xFFFFFFFFu;
@@ -397,9 +413,10 @@ unmask_stream_kernel(const T* __restrict__ logits, const uint8_t* __restrict__ s
             seg = static_cast<int>(gw - static_cast<long long>(ri) * ppr);
             segs = ppr;
         } else {
-            const long long row_first = static_cast<long long>(ri) * ipr;
-            const int w_first = static_cast<int>(((row_first + 1) * G + W - 1) / W) - 1;
-            const int w_last = static_cast<int>(((row_first + ipr) * G + W - 1) / W) - 1;
+            // the warps that hold the row's first and last item, on the padded axis
+            const long long v_first = static_cast<long long>(ri) * (ipr + pad) + pad;
+            const int w_first = static_cast<int>(((v_first + 1) * G + Vp - 1) / Vp) - 1;
+            const int w_last = static_cast<int>(((v_first + ipr) * G + Vp - 1) / Vp) - 1;
             seg = static_cast<int>(gw) - w_first;
             segs = w_last - w_first + 1;
         }
