@@ -749,6 +749,65 @@ attn_ptc_kernel(const __grid_constant__ TcArgs<MAXSETS> a) {
                 // A piece that starts at the CTA's range start uses the CTA's slot 0, a later one
                 // (necessarily the CTA's last item) slot 1.
                 const int own_slot = blockIdx.x * 2 + (pos == range_begin ? 0 : 1);
+                // Two pieces, and the other one is there already (the usual case for a CTA's last item: its
+                // neighbour wrote the unit's other piece as its first item, long ago): this piece does not
+                // go through scratch at all, it is merged straight out of TMEM with the other one's partials.
+                bool direct = false;
+                if (n_pieces == 2) {
+                    if (tid == 0) {
+                        const int gu = unit_base_s[it.s] + it.unit;
+                        const int there = *reinterpret_cast<volatile int*>(a.unit_count + gu) == 1;
+                        if (there) a.unit_count[gu] = 0;         // (nobody else counts on this unit any more: ready for the next launch)
+                        last_s = there;
+                        slot_s[0] = c_first * 2 + (it.unit_begin <= T * c_first / C ? 0 : 1);
+                        slot_s[1] = (c_first + 1) * 2;           // the second piece starts its CTA's range
+                    }
+                    tc::named_barrier(1, 256);
+                    direct = last_s != 0;
+                }
+                if (direct) {
+                    __threadfence();                             // the other piece was published before its count
+                    if (active && ok) {                          // (warp-uniform: the TMEM loads below are warp-wide)
+                        const int other = slot_s[0] == own_slot ? slot_s[1] : slot_s[0];
+                        const float l_own = m_used + log2f(l);
+                        const float l_oth = row_ok ? __ldcg(a.part_lse + static_cast<size_t>(other) * 256 + tid) : -CUDART_INF_F;
+                        float M = fmaxf(l_own, l_oth);
+                        if (!(M > -CUDART_INF_F)) M = 0.0f;
+                        const float w_own = exp2f(l_own - M), w_oth = exp2f(l_oth - M);
+                        const float wsum = w_own + w_oth;
+                        const float iw = wsum > 0.0f ? 1.0f / wsum : 0.0f;
+                        const float a_own = w_own * iw * inv, a_oth = w_oth * iw;     // (the other piece is stored normalised)
+                        const float4* po4 = reinterpret_cast<const float4*>(a.part_o) + static_cast<size_t>(other) * (D / 4) * 256 + tid;
+                        __nv_bfloat16* op = p.out + ((static_cast<size_t>(f) * p.d + qi) * p.n_q_heads + h * p.G + qg) * D;
+#pragma unroll
+                        for (int cc = 0; cc < D / 32; ++cc) {
+                            float4 ov[8];
+#pragma unroll
+                            for (int v4 = 0; v4 < 8; ++v4)
+                                ov[v4] = row_ok ? __ldcg(po4 + (cc * 8 + v4) * 256) : make_float4(0.f, 0.f, 0.f, 0.f);
+                            uint32_t o[32];
+                            tc::tmem_ld32(tm_o[q] + lane_base + cc * 32, o);
+                            tc::wait_ld();
+                            if (row_ok) {
+#pragma unroll
+                                for (int v4 = 0; v4 < 4; ++v4) {
+                                    uint32_t wv[4];
+#pragma unroll
+                                    for (int x = 0; x < 4; ++x) {
+                                        const int e0 = v4 * 8 + 2 * x;       // element inside the 32 columns
+                                        const float4& src = ov[e0 / 4];
+                                        const float s0 = (e0 % 4 == 0) ? src.x : src.z, s1 = (e0 % 4 == 0) ? src.y : src.w;
+                                        const __nv_bfloat162 pk = __floats2bfloat162_rn(fmaf(a_own, __uint_as_float(o[e0]), a_oth * s0),
+                                                                                          fmaf(a_own, __uint_as_float(o[e0 + 1]), a_oth * s1));
+                                        wv[x] = *reinterpret_cast<const uint32_t*>(&pk);
+                                    }
+                                    *reinterpret_cast<uint4*>(op + cc * 32 + v4 * 8) = make_uint4(wv[0], wv[1], wv[2], wv[3]);
+                                }
+                            }
+                        }
+                    }
+                    tc::named_barrier(1, 256);                   // slot_s is free again
+                } else {
                 if (active && ok) {
                     // column-major inside the slot ([D / 4 float4 columns][256 rows]): the 32 rows of a
                     // warp make one contiguous 512-byte store, and the merge reads them back the same way
@@ -801,6 +860,7 @@ attn_ptc_kernel(const __grid_constant__ TcArgs<MAXSETS> a) {
                     dfr.c_first = c_first; dfr.n_pieces = n_pieces; dfr.gu = gu;
                     dfr.unit_begin = it.unit_begin;
                 }
+                }   // not direct
             }
             if (!ok) {
                 if (*abort_flag == 0) atomicCAS(a.status, 0, FDD_ERR_DEVICE_TIMEOUT);
