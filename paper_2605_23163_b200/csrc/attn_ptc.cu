@@ -769,22 +769,25 @@ attn_ptc_kernel(const __grid_constant__ TcArgs<MAXSETS> a) {
                     __threadfence();                             // the other piece was published before its count
                     if (active && ok) {                          // (warp-uniform: the TMEM loads below are warp-wide)
                         const int other = slot_s[0] == own_slot ? slot_s[1] : slot_s[0];
-                        const float l_own = m_used + log2f(l);
+                        // every read of the other piece goes out at once: the merge costs one round trip
+                        const float4* po4 = reinterpret_cast<const float4*>(a.part_o) + static_cast<size_t>(other) * (D / 4) * 256 + tid;
+                        float4 ov[D / 32][8];
+#pragma unroll
+                        for (int cc = 0; cc < D / 32; ++cc)
+#pragma unroll
+                            for (int v4 = 0; v4 < 8; ++v4)
+                                ov[cc][v4] = row_ok ? __ldcg(po4 + (cc * 8 + v4) * 256) : make_float4(0.f, 0.f, 0.f, 0.f);
                         const float l_oth = row_ok ? __ldcg(a.part_lse + static_cast<size_t>(other) * 256 + tid) : -CUDART_INF_F;
+                        const float l_own = m_used + log2f(l);
                         float M = fmaxf(l_own, l_oth);
                         if (!(M > -CUDART_INF_F)) M = 0.0f;
                         const float w_own = exp2f(l_own - M), w_oth = exp2f(l_oth - M);
                         const float wsum = w_own + w_oth;
                         const float iw = wsum > 0.0f ? 1.0f / wsum : 0.0f;
                         const float a_own = w_own * iw * inv, a_oth = w_oth * iw;     // (the other piece is stored normalised)
-                        const float4* po4 = reinterpret_cast<const float4*>(a.part_o) + static_cast<size_t>(other) * (D / 4) * 256 + tid;
                         __nv_bfloat16* op = p.out + ((static_cast<size_t>(f) * p.d + qi) * p.n_q_heads + h * p.G + qg) * D;
 #pragma unroll
                         for (int cc = 0; cc < D / 32; ++cc) {
-                            float4 ov[8];
-#pragma unroll
-                            for (int v4 = 0; v4 < 8; ++v4)
-                                ov[v4] = row_ok ? __ldcg(po4 + (cc * 8 + v4) * 256) : make_float4(0.f, 0.f, 0.f, 0.f);
                             uint32_t o[32];
                             tc::tmem_ld32(tm_o[q] + lane_base + cc * 32, o);
                             tc::wait_ld();
@@ -795,7 +798,7 @@ attn_ptc_kernel(const __grid_constant__ TcArgs<MAXSETS> a) {
 #pragma unroll
                                     for (int x = 0; x < 4; ++x) {
                                         const int e0 = v4 * 8 + 2 * x;       // element inside the 32 columns
-                                        const float4& src = ov[e0 / 4];
+                                        const float4& src = ov[cc][e0 / 4];
                                         const float s0 = (e0 % 4 == 0) ? src.x : src.z, s1 = (e0 % 4 == 0) ? src.y : src.w;
                                         const __nv_bfloat162 pk = __floats2bfloat162_rn(fmaf(a_own, __uint_as_float(o[e0]), a_oth * s0),
                                                                                           fmaf(a_own, __uint_as_float(o[e0 + 1]), a_oth * s1));
