@@ -459,7 +459,9 @@ unmask_stream_kernel(const T* __restrict__ logits, const uint8_t* __restrict__ s
             const uint4* sp = reinterpret_cast<const uint4*>(buf) + lane * kLaneChunks;
             const T* lp = reinterpret_cast<const T*>(buf) + lane * kLaneIds;
             float bm64 = -CUDART_INF_F;
-            const bool whole = tile_base + kTile <= seg_end;
+            // (per lane: in a row's last tile the lanes whose 64 ids all exist take the fast path too, the
+            // lanes beyond the row's end have nothing to do, and at most one lane straddles the end)
+            const bool whole = vb + kLaneIds <= seg_end;
             uint4 rq = make_uint4(0u, 0u, 0u, 0u);      // the words of the block's four groups
             if (NOISY) rq = philox4x32_10(make_uint4(static_cast<uint32_t>(vb >> 6), pos, step, block_idx), keys);
             if (whole) {
@@ -498,8 +500,8 @@ unmask_stream_kernel(const T* __restrict__ logits, const uint8_t* __restrict__ s
                     tc::unpack2(tc::add2(acc[0], acc[1]), a0, a1);
                     s += a0 + a1;
                 }
-            } else {
-                // the row's last tile: ids from seg_end on do not exist
+            } else if (vb < seg_end) {
+                // the lane that straddles the row's end: ids from seg_end on do not exist
                 for (int e = 0; e < kLaneIds; ++e)
                     if (vb + e < seg_end) bm64 = fmaxf(bm64, Logit<T>::load1(lp + e));
                 if (bm64 > m) {
