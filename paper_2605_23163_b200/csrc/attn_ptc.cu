@@ -612,14 +612,20 @@ attn_ptc_kernel(const __grid_constant__ TcArgs<MAXSETS> a) {
                         for (int i = 0; i < 128; ++i)
                             if (i >= limit) sr[i] = 0xFF800000u;        // -inf
                     }
-                    float mx[4] = {-CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F};
+                    // the row's maximum: sixteen short chains, then a tree (the maximum sits on the path from
+                    // the scores to the probabilities, so its depth counts, not its instruction count)
+                    float mx[16];
 #pragma unroll
-                    for (int i = 0; i < 128; i += 8) {
+                    for (int u = 0; u < 16; ++u) mx[u] = fmaxf(__uint_as_float(sr[2 * u]), __uint_as_float(sr[2 * u + 1]));
 #pragma unroll
-                        for (int u = 0; u < 4; ++u)
+                    for (int i = 32; i < 128; i += 32) {
+#pragma unroll
+                        for (int u = 0; u < 16; ++u)
                             mx[u] = tc::max3(mx[u], __uint_as_float(sr[i + 2 * u]), __uint_as_float(sr[i + 2 * u + 1]));
                     }
-                    const float tmax = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
+#pragma unroll
+                    for (int u = 0; u < 5; ++u) mx[u] = tc::max3(mx[3 * u], mx[3 * u + 1], mx[3 * u + 2]);   // 15 -> 5
+                    const float tmax = fmaxf(tc::max3(mx[0], mx[1], mx[2]), tc::max3(mx[3], mx[4], mx[15]));
                     float m_tile = tmax * c;
                     if (!(m_tile > -CUDART_INF_F)) m_tile = m_used > -CUDART_INF_F ? m_used : 0.0f;
                     // The previous PV of this query tile must be complete before P is overwritten and
