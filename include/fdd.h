@@ -136,7 +136,8 @@ fdd_status fdd_forkset_reset(fdd_ctx* ctx, fdd_forkset* set);
  *   layer          which per-layer cache to read, 0 <= layer < L.
  *   q              device bf16, rollouts of all sets packed in set order:
  *                  set s contributes [N_s][d_s][Hq][D]; k_blk, v_blk likewise [N_s][d_s][Hkv][D].
- *   out            device bf16, same packing and shape as q.
+ *   out            device bf16, same packing and shape as q; 32-byte aligned (rows are written in
+ *                  32-byte pieces).
  *   block_len      host int32 [n_sets]: d_s, 1 <= d_s <= cfg.max_block.
  *   scale          soft-max scale (1/sqrt(D) by convention), the same for every set of the call.
  * The tensor-core kernel is launched cooperatively (its CTAs wait, with a bound, for one another's

@@ -28,6 +28,9 @@
 //   by more than 2^8), P = exp2(S * c - m) -> TMEM  ->  O += P V (TMEM x smem, V keys-major).
 // The MMA warp issues QK(1, j), PV(1, j - 1), QK(0, j + 1), PV(0, j) in that order, which keeps the
 // tensor pipe fed while each soft-max group spends a whole period on one tile.
+// Items follow one another without a meeting of the whole CTA: Q of the next item is staged as soon as
+// the last score product of the current one has completed, its first scores are computed while
+// the soft-max groups still write the current item's output, and each group moves on by itself.
 // The exponentials can be split between the special-function unit (ex2.approx) and a cubic
 // polynomial on the FMA pipe (one ex2 per score needs as many cycles as the MMAs).
 // Every mbarrier wait is bounded; on a timeout the CTA records FDD_ERR_DEVICE_TIMEOUT, drains
@@ -256,7 +259,7 @@ attn_ptc_kernel(const __grid_constant__ TcArgs<MAXSETS> a) {
     const uint32_t v_s = k_s + kStages * Shape::kTileBytes;
 
     __shared__ __align__(8) unsigned long long bar_q_full, bar_k_full[kStages], bar_k_empty[kStages],
-        bar_v_full[kStages], bar_v_empty[kStages], bar_s_full[2], bar_s_free[2], bar_p_full[2], bar_o_done[2], bar_item_done;
+        bar_v_full[kStages], bar_v_empty[kStages], bar_s_full[2], bar_s_free[2], bar_p_full[2], bar_o_done[2], bar_o_final[2], bar_q_empty;
     __shared__ uint32_t tmem_base_s;
     __shared__ int abort_s, n_deferred_s, last_s;
     __shared__ Deferred deferred_s[2];                  // a range starts and ends inside at most one cut unit each
@@ -318,7 +321,7 @@ attn_ptc_kernel(const __grid_constant__ TcArgs<MAXSETS> a) {
         abort_s = 0;
         n_deferred_s = 0;
         tc::mbar_init(tc::smem_u32(&bar_q_full), 1);
-        tc::mbar_init(tc::smem_u32(&bar_item_done), 1);
+        tc::mbar_init(tc::smem_u32(&bar_q_empty), 1);      // every QK^T product of an item has completed: Q may be overwritten
         for (int s = 0; s < kStages; ++s) {
             tc::mbar_init(tc::smem_u32(&bar_k_full[s]), 1);
             tc::mbar_init(tc::smem_u32(&bar_k_empty[s]), 1);
@@ -330,6 +333,7 @@ attn_ptc_kernel(const __grid_constant__ TcArgs<MAXSETS> a) {
             tc::mbar_init(tc::smem_u32(&bar_s_free[q]), 128);   // group q has copied them out of S
             tc::mbar_init(tc::smem_u32(&bar_p_full[q]), 128);   // group q has written P[q]
             tc::mbar_init(tc::smem_u32(&bar_o_done[q]), 1);     // a PV product of query tile q has completed
+            tc::mbar_init(tc::smem_u32(&bar_o_final[q]), 1);    // the last PV product of query tile q in an item has completed
         }
         tc::fence_barrier_init();
     }
@@ -345,7 +349,11 @@ attn_ptc_kernel(const __grid_constant__ TcArgs<MAXSETS> a) {
     const uint32_t tm_p[2] = {tmem + 128, tmem + 192};
     const uint32_t tm_o[2] = {tmem + 256, tmem + 256 + D};
 
-    // Each role runs its own copy of the item loop; all of them meet at the end of every item.
+    // Each role runs its own copy of the item loop.  Nothing brings all of them together between two
+    // items: the producer stages the next item's Q as soon as the last QK^T product of this one has
+    // completed and its K/V tiles as ring stages come free, the first scores of the next item are
+    // computed while the soft-max groups still read this item's output out of TMEM, and a group's
+    // first P of the next item (written after its epilogue) is what lets the PV issuer overwrite O.
     struct ItemView {
         Item it;
         int f, rp, h, nt, rows_here, NQ;
@@ -365,14 +373,6 @@ attn_ptc_kernel(const __grid_constant__ TcArgs<MAXSETS> a) {
         v.NQ = v.rows_here > 128 ? 2 : 1;
         return v;
     };
-    // End of an item: every MMA of the item has completed (the soft-max groups waited for the
-    // last PV), O has been read out, Q may be overwritten.  Returns false after an abort.
-    auto end_of_item = [&]() {
-        tc::fence_before_sync();
-        tc::named_barrier(2, kTcThreads);
-        tc::fence_after_sync();
-        return *abort_flag == 0;
-    };
 
     if (warp >= 8) {
         // The soft-max warps hold a 128-wide score row in registers; this warpgroup gives most of
@@ -381,14 +381,21 @@ attn_ptc_kernel(const __grid_constant__ TcArgs<MAXSETS> a) {
         if (warp == 8) {
             // ------------------------------------------------------------------ TMA producer
             uint32_t kv_cnt = 0;            // K/V tiles staged so far: ring stage and phase carry over between items
-            for (long long pos = range_begin; pos < range_end;) {
+            uint32_t item_cnt = 0;
+            bool ok = true;
+            for (long long pos = range_begin; pos < range_end && ok;) {
                 const ItemView v = view_item(pos);
                 {
                     // warp-uniform loop, one elected lane issues the copies
                     const SetParams& p = a.sets[v.it.s];
                     const TcSetMaps& maps = a.maps[v.it.s];
                     const uint32_t bq = tc::smem_u32(&bar_q_full);
-                    if (tc::elect_one()) {
+                    if (item_cnt > 0) {
+                        // Q of the item before is still being read until its last QK^T product has completed
+                        ok = tc::mbar_wait(tc::smem_u32(&bar_q_empty), (item_cnt - 1) & 1, abort_flag, kWaitLimit);
+                        ok = __shfl_sync(0xFFFFFFFFu, ok ? 1 : 0, 0) != 0;
+                    }
+                    if (ok && tc::elect_one()) {
                         tc::prefetch_tmap(&maps.q);
                         tc::mbar_arrive_expect_tx(bq, v.NQ * Shape::kTileBytes);
                         for (int q = 0; q < v.NQ; ++q)
@@ -397,7 +404,6 @@ attn_ptc_kernel(const __grid_constant__ TcArgs<MAXSETS> a) {
                                                 v.h * p.G, (v.rp * 2 + q) * (128 / p.G), v.f);
                     }
                     __syncwarp();
-                    bool ok = true;
                     for (int jl = 0; jl < v.nt && ok; ++jl) {
                         const TileInfo t = tile_info(p, v.it.t0 + jl);
                         const uint32_t n = kv_cnt + jl;
@@ -436,15 +442,18 @@ attn_ptc_kernel(const __grid_constant__ TcArgs<MAXSETS> a) {
                     if (!ok && lane == 0) {
                         if (*abort_flag == 0) atomicCAS(a.status, 0, FDD_ERR_DEVICE_TIMEOUT);
                         *abort_flag = 1;
-                        const long long t0 = clock64();          // let copies already in flight land
-                        while (clock64() - t0 < 2000000) {}
                     }
                 }
                 __syncwarp();
                 kv_cnt += v.nt;
+                ++item_cnt;
                 pos += v.nt;
-                if (!end_of_item()) break;
             }
+            if (*abort_flag != 0 && lane == 0) {
+                const long long t0 = clock64();                  // let copies already in flight land
+                while (clock64() - t0 < 2000000) {}
+            }
+            __syncwarp();
         } else if (warp == 9 || warp == 10) {
             // ------------------------------------------------------------------ MMA issuers
             // Warp 9 issues every QK^T, warp 10 every PV: while one of them checks the barriers of its
@@ -453,7 +462,13 @@ attn_ptc_kernel(const __grid_constant__ TcArgs<MAXSETS> a) {
             const bool qk_role = warp == 9;
             uint32_t kv_cnt = 0, item_cnt = 0;
             uint32_t sp_cnt[2] = {0, 0};    // key tiles handled so far per query tile
-            for (long long pos = range_begin; pos < range_end;) {
+            // the soft-max group that read S last, and which of its tiles that was: S is not written
+            // again before that group has copied its scores out, across items as well as inside one
+            int s_prev_q = 0;
+            uint32_t s_prev_idx = 0;
+            bool s_has_prev = false;
+            bool ok = true;
+            for (long long pos = range_begin; pos < range_end && ok;) {
                 const ItemView v = view_item(pos);
                 const int nt = v.nt, NQ = v.NQ;
                 {
@@ -496,6 +511,8 @@ attn_ptc_kernel(const __grid_constant__ TcArgs<MAXSETS> a) {
                         const int s = stage_of(jl);
                         bool good = true;
                         if (first_user_of_v) good = wait(&bar_v_full[s], phase_of(jl));
+                        // (the first P of an item is written after the group has read the output of the
+                        // item before out of TMEM: O[q] may be overwritten once that P is there)
                         good = good && wait(&bar_p_full[q], sp_cnt[q] + jl);
                         good = __shfl_sync(0xFFFFFFFFu, good ? 1 : 0, 0) != 0;
                         if (!good) return false;
@@ -504,17 +521,19 @@ attn_ptc_kernel(const __grid_constant__ TcArgs<MAXSETS> a) {
                             issue_pv(q, s, jl > 0);
                             tc::mma_commit(tc::smem_u32(&bar_o_done[q]));
                             if (last_user_of_v) tc::mma_commit(tc::smem_u32(&bar_v_empty[s]));
+                            // the item's output for query tile q is complete (the products of one
+                            // issuing thread complete in order)
+                            if (jl == nt - 1) tc::mma_commit(tc::smem_u32(&bar_o_final[q]));
                         }
                         __syncwarp();
                         return true;
                     };
                     // QK(q, jl) into S: needs K tile jl and S handed back by its previous reader
-                    auto do_qk = [&](int q, int jl, bool first_user_of_k, bool last_user_of_k, int prev_q, uint32_t prev_idx,
-                                     bool has_prev) {
+                    auto do_qk = [&](int q, int jl, bool first_user_of_k, bool last_user_of_k) {
                         const int s = stage_of(jl);
                         bool good = true;
                         if (first_user_of_k) good = wait(&bar_k_full[s], phase_of(jl));
-                        if (has_prev) good = good && wait(&bar_s_free[prev_q], prev_idx);
+                        if (s_has_prev) good = good && wait(&bar_s_free[s_prev_q], s_prev_idx);
                         good = __shfl_sync(0xFFFFFFFFu, good ? 1 : 0, 0) != 0;
                         if (!good) return false;
                         tc::fence_after_sync();
@@ -522,19 +541,23 @@ attn_ptc_kernel(const __grid_constant__ TcArgs<MAXSETS> a) {
                             issue_qk(q, s);
                             tc::mma_commit(tc::smem_u32(&bar_s_full[q]));
                             if (last_user_of_k) tc::mma_commit(tc::smem_u32(&bar_k_empty[s]));
+                            // the item's last score product: once it has completed nothing reads Q any more
+                            if (jl == nt - 1 && q == NQ - 1) tc::mma_commit(tc::smem_u32(&bar_q_empty));
                         }
                         __syncwarp();
+                        s_prev_q = q;
+                        s_prev_idx = sp_cnt[q] + jl;
+                        s_has_prev = true;
                         return true;
                     };
-                    bool ok = true;
                     if (qk_role) {
                         // scores: QK(0,0) | QK(1,j) QK(0,j+1) | ...   (S is one buffer: each product waits
                         // until the group that owned the previous scores has copied them out)
                         ok = __shfl_sync(0xFFFFFFFFu, wait(&bar_q_full, item_cnt) ? 1 : 0, 0) != 0;
-                        ok = ok && do_qk(0, 0, true, NQ == 1, 0, 0, false);
+                        ok = ok && do_qk(0, 0, true, NQ == 1);
                         for (int jl = 0; jl < nt && ok; ++jl) {
-                            if (NQ == 2) ok = do_qk(1, jl, false, true, 0, sp_cnt[0] + jl, true);
-                            if (ok && jl + 1 < nt) ok = do_qk(0, jl + 1, true, NQ == 1, NQ - 1, sp_cnt[NQ - 1] + jl, true);
+                            if (NQ == 2) ok = do_qk(1, jl, false, true);
+                            if (ok && jl + 1 < nt) ok = do_qk(0, jl + 1, true, NQ == 1);
                         }
                     } else {
                         // outputs: PV(1,j-1) PV(0,j) | ... | PV(1,nt-1), in the order the P tiles appear
@@ -543,9 +566,6 @@ attn_ptc_kernel(const __grid_constant__ TcArgs<MAXSETS> a) {
                             if (ok) ok = do_pv(0, jl, true, NQ == 1);
                         }
                         if (ok && NQ == 2) ok = do_pv(1, nt - 1, false, true);
-                        // One arrival per item once every PV (hence every MMA) of the item has completed.
-                        // (bar_o_done cannot serve here: a waiter could be two of its phases behind.)
-                        if (ok && tc::elect_one()) tc::mma_commit(tc::smem_u32(&bar_item_done));
                     }
                     if (!ok && lane == 0) {
                         if (*abort_flag == 0) atomicCAS(a.status, 0, FDD_ERR_DEVICE_TIMEOUT);
@@ -557,16 +577,9 @@ attn_ptc_kernel(const __grid_constant__ TcArgs<MAXSETS> a) {
                 for (int q = 0; q < NQ; ++q) sp_cnt[q] += nt;
                 ++item_cnt;
                 pos += nt;
-                if (!end_of_item()) break;
-            }
-        } else {
-            // idle warps of the donor warpgroup: only keep the item barriers company
-            for (long long pos = range_begin; pos < range_end;) {
-                const ItemView v = view_item(pos);
-                pos += v.nt;
-                if (!end_of_item()) break;
             }
         }
+        // (warp 11 has nothing to do but to have given up its registers)
     } else {
         tc::reg_alloc<kRegsSoftmax>();
         // ---------------------------------------------------------------------- soft-max groups
@@ -575,7 +588,9 @@ attn_ptc_kernel(const __grid_constant__ TcArgs<MAXSETS> a) {
         const uint32_t lane_base = (static_cast<uint32_t>(warp & 3) * 32u) << 16;
         const uint32_t bo = tc::smem_u32(&bar_o_done[q]);
         uint32_t sp0 = 0;                   // key tiles this group has handled so far
-        uint32_t item_cnt = 0;
+        uint32_t items_mine = 0;            // items this group has taken part in so far
+        // After a wait has given up, the groups still walk the rest of the range (without computing):
+        // both of them must meet at the same named barriers of the epilogues.
         for (long long pos = range_begin; pos < range_end;) {
             const ItemView v = view_item(pos);
             const Item& it = v.it;
@@ -587,8 +602,8 @@ attn_ptc_kernel(const __grid_constant__ TcArgs<MAXSETS> a) {
             const int qi = row_ok ? r / p.G : 0;
             const int qg = row_ok ? r - qi * p.G : 0;
             float m_used = -CUDART_INF_F, l = 0.0f;
-            bool ok = true;
-            if (active) {
+            bool ok = *abort_flag == 0;
+            if (active && ok) {
                 const float c = a.scale_log2;
                 const uint64_t c2 = tc::pack2(c, c);
                 const float c_emu = c * (1.0f / 128.0f);
@@ -718,7 +733,8 @@ attn_ptc_kernel(const __grid_constant__ TcArgs<MAXSETS> a) {
                     tc::fence_before_sync();
                     tc::mbar_arrive(bp);
                 }
-                if (ok) ok = tc::mbar_wait(tc::smem_u32(&bar_item_done), item_cnt & 1, abort_flag, kWaitLimit);
+                // the item's last PV product of this query tile (and with it every product before it)
+                if (ok) ok = tc::mbar_wait(tc::smem_u32(&bar_o_final[q]), items_mine & 1, abort_flag, kWaitLimit);
                 if (ok) tc::fence_after_sync();
             }
 
@@ -737,16 +753,17 @@ attn_ptc_kernel(const __grid_constant__ TcArgs<MAXSETS> a) {
                         tc::tmem_ld32(tm_o[q] + lane_base + cc * 32, o);
                         tc::wait_ld();
                         if (row_ok) {
+                            // (a row is D * 2 bytes and starts on a multiple of that: 32-byte stores are aligned)
 #pragma unroll
-                            for (int v4 = 0; v4 < 4; ++v4) {
-                                uint32_t w[4];
+                            for (int v8 = 0; v8 < 2; ++v8) {
+                                uint32_t w[8];
 #pragma unroll
-                                for (int x = 0; x < 4; ++x) {
-                                    const __nv_bfloat162 pk = __floats2bfloat162_rn(__uint_as_float(o[v4 * 8 + 2 * x]) * inv,
-                                                                                      __uint_as_float(o[v4 * 8 + 2 * x + 1]) * inv);
+                                for (int x = 0; x < 8; ++x) {
+                                    const __nv_bfloat162 pk = __floats2bfloat162_rn(__uint_as_float(o[v8 * 16 + 2 * x]) * inv,
+                                                                                      __uint_as_float(o[v8 * 16 + 2 * x + 1]) * inv);
                                     w[x] = *reinterpret_cast<const uint32_t*>(&pk);
                                 }
-                                *reinterpret_cast<uint4*>(op + cc * 32 + v4 * 8) = make_uint4(w[0], w[1], w[2], w[3]);
+                                tc::st_global_32B(op + cc * 32 + v8 * 16, w);
                             }
                         }
                     }
@@ -764,6 +781,9 @@ attn_ptc_kernel(const __grid_constant__ TcArgs<MAXSETS> a) {
                         const int gu = unit_base_s[it.s] + it.unit;
                         const int there = *reinterpret_cast<volatile int*>(a.unit_count + gu) == 1;
                         if (there) a.unit_count[gu] = 0;         // (nobody else counts on this unit any more: ready for the next launch)
+                        // the other piece was published before its count: one fence by the thread that read the
+                        // count, ahead of the barrier behind which the others read the piece
+                        if (there) __threadfence();
                         last_s = there;
                         slot_s[0] = c_first * 2 + (it.unit_begin <= T * c_first / C ? 0 : 1);
                         slot_s[1] = (c_first + 1) * 2;           // the second piece starts its CTA's range
@@ -772,7 +792,6 @@ attn_ptc_kernel(const __grid_constant__ TcArgs<MAXSETS> a) {
                     direct = last_s != 0;
                 }
                 if (direct) {
-                    __threadfence();                             // the other piece was published before its count
                     if (active && ok) {                          // (warp-uniform: the TMEM loads below are warp-wide)
                         const int other = slot_s[0] == own_slot ? slot_s[1] : slot_s[0];
                         // every read of the other piece goes out at once: the merge costs one round trip
@@ -799,18 +818,18 @@ attn_ptc_kernel(const __grid_constant__ TcArgs<MAXSETS> a) {
                             tc::wait_ld();
                             if (row_ok) {
 #pragma unroll
-                                for (int v4 = 0; v4 < 4; ++v4) {
-                                    uint32_t wv[4];
+                                for (int v8 = 0; v8 < 2; ++v8) {
+                                    uint32_t wv[8];
 #pragma unroll
-                                    for (int x = 0; x < 4; ++x) {
-                                        const int e0 = v4 * 8 + 2 * x;       // element inside the 32 columns
+                                    for (int x = 0; x < 8; ++x) {
+                                        const int e0 = v8 * 16 + 2 * x;      // element inside the 32 columns
                                         const float4& src = ov[cc][e0 / 4];
                                         const float s0 = (e0 % 4 == 0) ? src.x : src.z, s1 = (e0 % 4 == 0) ? src.y : src.w;
                                         const __nv_bfloat162 pk = __floats2bfloat162_rn(fmaf(a_own, __uint_as_float(o[e0]), a_oth * s0),
                                                                                           fmaf(a_own, __uint_as_float(o[e0 + 1]), a_oth * s1));
                                         wv[x] = *reinterpret_cast<const uint32_t*>(&pk);
                                     }
-                                    *reinterpret_cast<uint4*>(op + cc * 32 + v4 * 8) = make_uint4(wv[0], wv[1], wv[2], wv[3]);
+                                    tc::st_global_32B(op + cc * 32 + v8 * 16, wv);
                                 }
                             }
                         }
@@ -834,22 +853,27 @@ attn_ptc_kernel(const __grid_constant__ TcArgs<MAXSETS> a) {
                     }
                     __stcg(a.part_lse + static_cast<size_t>(own_slot) * 256 + q * 128 + row_local, m_used + log2f(l));
                 }
-                __threadfence();
+                // Publishing the piece: every thread's stores are ordered before the barrier, the one thread
+                // that counts the piece fences between the barrier and the count (and again after it, on
+                // behalf of the threads that read the other pieces behind the next barrier).
                 tc::named_barrier(1, 256);
                 if (n_pieces == 2) {
                     // Two pieces: whichever of the two CTAs writes its piece second merges the unit
                     // at once; nobody waits.
                     if (tid == 0) {
                         const int gu = unit_base_s[it.s] + it.unit;
+                        __threadfence();
                         const int last = atomicAdd(a.unit_count + gu, 1) == 1;
-                        if (last) a.unit_count[gu] = 0;          // both pieces are there: ready for the next launch
+                        if (last) {
+                            a.unit_count[gu] = 0;                // both pieces are there: ready for the next launch
+                            __threadfence();
+                        }
                         last_s = last;
                         slot_s[0] = c_first * 2 + (it.unit_begin <= T * c_first / C ? 0 : 1);
                         slot_s[1] = (c_first + 1) * 2;           // the second piece starts its CTA's range
                     }
                     tc::named_barrier(1, 256);
                     if (last_s) {
-                        __threadfence();
                         if (row_ok) {                            // thread = row
                             __nv_bfloat16* op = p.out + ((static_cast<size_t>(f) * p.d + qi) * p.n_q_heads + h * p.G + qg) * D;
 #pragma unroll
@@ -863,6 +887,7 @@ attn_ptc_kernel(const __grid_constant__ TcArgs<MAXSETS> a) {
                     // which follows once the whole range is done (waiting here, in the middle of the
                     // range, would chain every CTA behind its neighbour).
                     const int gu = unit_base_s[it.s] + it.unit;
+                    __threadfence();
                     atomicAdd(a.unit_count + gu, 1);
                     Deferred& dfr = deferred_s[n_deferred_s++];
                     dfr.s = it.s; dfr.unit = it.unit; dfr.f = f; dfr.rp = rp; dfr.h = h;
@@ -875,10 +900,11 @@ attn_ptc_kernel(const __grid_constant__ TcArgs<MAXSETS> a) {
                 if (*abort_flag == 0) atomicCAS(a.status, 0, FDD_ERR_DEVICE_TIMEOUT);
                 *abort_flag = 1;
             }
-            if (active) sp0 += nt;
-            ++item_cnt;
+            if (active) {
+                sp0 += nt;
+                ++items_mine;
+            }
             pos += nt;
-            if (!end_of_item()) break;
         }
 
         // ------------------------------------------------------------ merges of the cut units
@@ -901,6 +927,7 @@ attn_ptc_kernel(const __grid_constant__ TcArgs<MAXSETS> a) {
                         }
                     }
                 }
+                __threadfence();                                      // the pieces were published before their counts
             }
             for (int e = 0; e < n_deferred; ++e)
                 if (tid < deferred_s[e].n_pieces && tid < kMaxPieces) {
@@ -909,7 +936,6 @@ attn_ptc_kernel(const __grid_constant__ TcArgs<MAXSETS> a) {
                 }
             tc::named_barrier(1, 256);
             if (*abort_flag == 0) {
-                __threadfence();
                 const int threads_e = 256 / n_deferred;               // threads per unit
                 const int e = tid / threads_e, lt = tid - e * threads_e;
                 const Deferred dfr = deferred_s[e];

@@ -297,8 +297,8 @@ fdd_status fdd_block_attn_gated(fdd_ctx* ctx, fdd_forkset* const* sets, int n_se
     fdd_status st = check_sets(ctx, sets, n_sets, block_len, &total);
     if (st != FDD_OK) return st;
     if (!q || !k_blk || !v_blk || !out) return fail(ctx, FDD_ERR_INVALID_ARG, "q/k_blk/v_blk/out is NULL");
-    if (!aligned16(q) || !aligned16(k_blk) || !aligned16(v_blk) || !aligned16(out))
-        return fail(ctx, FDD_ERR_INVALID_ARG, "q/k_blk/v_blk/out must be 16-byte aligned");
+    if (!aligned16(q) || !aligned16(k_blk) || !aligned16(v_blk) || (reinterpret_cast<uintptr_t>(out) & 31u) != 0)
+        return fail(ctx, FDD_ERR_INVALID_ARG, "q/k_blk/v_blk must be 16-byte aligned, out 32-byte aligned");
     if (layer < 0 || layer >= ctx->cfg.n_layers) return fail(ctx, FDD_ERR_SHAPE, "layer %d outside [0, %d)", layer, ctx->cfg.n_layers);
     if (!(scale > 0.0f)) return fail(ctx, FDD_ERR_INVALID_ARG, "scale must be positive");
     if (gate && total > kAttnMaxGatedForks)

@@ -69,6 +69,13 @@ __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* m, 
         : "memory");
 }
 
+// One 32-byte store (a whole sector of a row); the address is 32-byte aligned.
+__device__ __forceinline__ void st_global_32B(void* dst, const uint32_t (&w)[8]) {
+    asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
+                 ::"l"(dst), "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3]), "r"(w[4]), "r"(w[5]), "r"(w[6]), "r"(w[7])
+                 : "memory");
+}
+
 // ----------------------------------------------------------------------------- tcgen05: TMEM
 // Allocate `ncols` (power of two, 32..512) TMEM columns; the base address lands in *dst_smem.
 // Must be executed by one full warp.

@@ -81,9 +81,17 @@ __device__ __forceinline__ uint32_t pick_word(const uint4& r, int k) {
 
 // One bulk asynchronous copy global -> shared of this CTA; `bytes` and both addresses are multiples
 // of 16.  Completion is counted in bytes on the mbarrier.
-__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar)
+// The logits are read once: the copy marks their lines as the first to leave L2, so that a step's
+// hundreds of MB do not push out what the attention kernel of the next step reads again (the
+// shared prefix and the caches).
+__device__ __forceinline__ uint64_t read_once_policy() {
+    uint64_t policy;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(policy));
+    return policy;
+}
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar, uint64_t policy) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;"
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar), "l"(policy)
                  : "memory");
 }
 
@@ -371,6 +379,7 @@ unmask_stream_kernel(const T* __restrict__ logits, const uint8_t* __restrict__ s
     int p_tile = 0, p_tile_end = 0;
     const T* p_row_ptr = nullptr;
     uint32_t p_k = 0;
+    const uint64_t l2_policy = read_once_policy();
     auto produce_one = [&](int stage) {
         if (!bulk_ok) return;
         if (p_tile == p_tile_end) {
@@ -388,7 +397,7 @@ unmask_stream_kernel(const T* __restrict__ logits, const uint8_t* __restrict__ s
             const uint32_t bytes = static_cast<uint32_t>(min(kTile, vocab - v0)) * sizeof(T);
             const uint32_t bar = bars_u32 + stage * 8;
             tc::mbar_arrive_expect_tx(bar, bytes);
-            bulk_load(ring_u32 + stage * kStageBytes, p_row_ptr + v0, bytes, bar);
+            bulk_load(ring_u32 + stage * kStageBytes, p_row_ptr + v0, bytes, bar, l2_policy);
         }
         ++p_tile;
         ++p_k;
