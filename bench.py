@@ -30,7 +30,7 @@ UNIT = "tokens/s"
 TIMED_PASSES = 3    # the timed region (exactly --steps blocks) is run this often; the median pass is reported
 COUNT_STREAM = None  # copy the per-rollout counts to the host on a stream of their own (None: for large steps only)
 GRAPH = False       # replay every denoising step from a CUDA graph (--graph)
-TIME_EVERY = 10     # blocks between two blocks whose kernels are timed one by one
+TIME_EVERY = 20     # blocks between two blocks whose kernels are timed one by one
 NATIVE_LOOP = True  # the block loop is run by the library (fdd_decode_block); --loop python keeps it in this file
 LOOKAHEAD = True   # enqueue step t + 1 before the host has read the counts of step t (--no-lookahead)
 PRE_STEPS = 6      # distinct per-step input sets kept resident; later steps cycle through them (--pre-steps)

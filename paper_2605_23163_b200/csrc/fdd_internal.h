@@ -183,6 +183,17 @@ struct CommitArgs {
     int n_kv_heads, vec_per_row;
     int* status;             // device status word
 };
+// Launch attribute that lets a kernel be made resident while the kernel ahead of it on the stream
+// drains (such a kernel waits for that kernel's completion, griddepcontrol.wait, before it reads or
+// writes anything).  Not used while the stream is being captured into a graph.  Returns the number
+// of attributes written.
+inline int overlap_launch_attribute(cudaStream_t st, cudaLaunchAttribute* attr) {
+    cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+    if (cudaStreamIsCapturing(st, &cap) != cudaSuccess || cap != cudaStreamCaptureStatusNone) return 0;
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    return 1;
+}
 cudaError_t launch_kv_commit(const CommitArgs& a, int sm_count, cudaStream_t st);
 cudaError_t launch_average(const float* traj, int n, int w, float* out, cudaStream_t st);
 bool jmt_weights(int w, int w_out, std::vector<double>* weights);

@@ -7,9 +7,11 @@
 //   paged prefix      [pages][Hkv][64][D], logical page -> physical page through the page table.
 // 16-byte copies; all scenes of a call go into one launch.
 #include "fdd_internal.h"
+#include "tc_ptx.cuh"
 
 namespace {
 __global__ void kv_commit_kernel(const __grid_constant__ CommitArgs a) {
+    tc::grid_dependency_wait();          // (launched for an early start behind the kernel ahead of it)
     for (long long idx = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x; idx < a.total;
          idx += static_cast<long long>(gridDim.x) * blockDim.x) {
         int s = 0;
@@ -47,6 +49,12 @@ cudaError_t launch_kv_commit(const CommitArgs& a, int sm_count, cudaStream_t st)
     const long long most = static_cast<long long>(sm_count > 0 ? sm_count : 148) * 8;
     if (blocks > most) blocks = most;
     if (blocks < 1) blocks = 1;
-    kv_commit_kernel<<<static_cast<unsigned>(blocks), threads, 0, st>>>(a);
-    return cudaGetLastError();
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(static_cast<unsigned>(blocks));
+    cfg.blockDim = dim3(threads);
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    cfg.numAttrs = overlap_launch_attribute(st, attr);
+    cfg.attrs = attr;
+    return cudaLaunchKernelEx(&cfg, kv_commit_kernel, a);
 }

@@ -938,17 +938,6 @@ cudaError_t device_setup(int dev, int* sm_count, const int** ctas_per_sm) {
     return cudaSuccess;
 }
 
-// Launch attribute that lets a kernel be made resident while the kernel ahead of it on the stream
-// drains (the kernels here wait with grid_dependency_wait before they read anything).  Not used
-// while the stream is being captured into a graph.  Returns the number of attributes written.
-int overlap_launch_attribute(cudaStream_t st, cudaLaunchAttribute* attr) {
-    cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
-    if (cudaStreamIsCapturing(st, &cap) != cudaSuccess || cap != cudaStreamCaptureStatusNone) return 0;
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
-    return 1;
-}
-
 template <typename T, bool NOISY>
 void launch_stream(const UnmaskProblem& p, UnmaskPartial* partial, int tiles_per_item, int bulk_ok, int select_state,
                    int* status, int resident_ctas, cudaStream_t st) {
