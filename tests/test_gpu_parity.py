@@ -173,6 +173,45 @@ def test_attention_many_scenes_one_call():
         fdd.fdd_destroy(ctx)
 
 
+def test_attention_many_short_units_per_cta():
+    # Hundreds of units of two to four key tiles each, so that every CTA's range holds half a dozen
+    # items: whole units, pieces at both ends, and, at the borders between the scenes, the change
+    # between units with two query tiles (256 stacked rows) and units with one.  The items of a range
+    # follow one another without a barrier of the whole CTA; every output row is compared.
+    base = synth.workload("long_prefix")
+    scenes = (synth.Scene(130, 48, 64, 19, 1), synth.Scene(70, 40, 16, 5, 1), synth.Scene(300, 24, 32, 10, 1),
+              synth.Scene(129, 9, 64, 19, 1))
+    w = synth.Workload("short_units", base.n_q_heads, base.n_kv_heads, base.head_dim, 1024, "bf16", "peaked", 0.9, 1.0,
+                       scenes, seed=23)
+    ctx = harness.create_context(w)
+    try:
+        gs, refs, qs, ks, vs = [], [], [], [], []
+        for i, sc in enumerate(scenes):
+            gs.append(harness.GpuScene(ctx, w, i))
+            pk, pv = synth.make_prefix(w, i)
+            q, k, v = synth.make_qkv(w, i, 0, 0, 0)
+            empty = ([np.zeros((0, w.n_kv_heads, w.head_dim), dtype=np.uint16)] * sc.n_forks,) * 2
+            refs.append(pu.attention_oracle(w, (pk, pv), empty, q, k, v))
+            qs.append(q); ks.append(k); vs.append(v)
+        pack = lambda xs: harness.bf16_tensor(np.concatenate([x.reshape(-1) for x in xs]))
+        qd, kd, vd = pack(qs), pack(ks), pack(vs)
+        for rep in range(2):                 # (the second call finds the counters of the cut units as the first left them)
+            out = torch.full_like(qd, float("nan"))
+            n0 = fdd.fdd_launch_count(ctx)
+            fdd.fdd_block_attn(ctx, [g.forkset for g in gs], 0, qd, kd, vd, out, [sc.block_len for sc in scenes],
+                               1.0 / np.sqrt(w.head_dim), 0)
+            fdd.fdd_poll_status(ctx)
+            assert fdd.fdd_launch_count(ctx) - n0 == 1
+            got = out.float().cpu().numpy().astype(np.float64)
+            off = 0
+            for ref in refs:
+                pu.assert_attention_close(got[off:off + ref.size].reshape(ref.shape), ref)
+                off += ref.size
+            assert off == got.size
+    finally:
+        fdd.fdd_destroy(ctx)
+
+
 def test_attention_gated_rollouts_are_skipped_and_the_rest_is_unchanged():
     # fdd_block_attn_gated: rollouts whose gate entry is 0 sit the call out (their rows of out keep
     # what was there), every other rollout gets what the ungated call gives, whatever the mix:
