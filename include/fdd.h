@@ -23,6 +23,8 @@
  *   - Calls enqueue work on `stream` (a cudaStream_t passed as void*; NULL = default
  *     stream) and return without synchronising unless stated.  Argument errors are
  *     detected on the host before anything is launched and returned synchronously.
+ *   - Every call that enqueues work (and fdd_plan_blocks) is wrapped in an NVTX range that
+ *     carries its name, for profilers that follow NVTX; without one attached this costs nothing.
  *   - No call aborts, throws or prints.  A negative fdd_status is an error; the text
  *     is available from fdd_last_error().
  *   - A context and its fork sets must be used from one host thread at a time.  The calls

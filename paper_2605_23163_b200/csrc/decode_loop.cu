@@ -69,6 +69,7 @@ fdd_status fdd_decode_block(fdd_ctx* ctx, fdd_forkset* const* sets, int n_sets, 
                             int32_t* n_committed, int32_t* n_left,
                             int* steps_taken, int* masked_left,
                             fdd_step_fn before_step, void* user, void* stream) {
+    CallRange range("fdd_decode_block");
     if (!ctx) return FDD_ERR_INVALID_ARG;
     if (!q || !k_blk || !v_blk || !out || !logits || !steps_taken || !n_left || !n_committed) {
         ctx->last_error = "fdd_decode_block: a required pointer is NULL";

@@ -292,6 +292,7 @@ fdd_status fdd_block_attn_gated(fdd_ctx* ctx, fdd_forkset* const* sets, int n_se
                                 const void* q, const void* k_blk, const void* v_blk, void* out,
                                 const int32_t* block_len, float scale, int causal_in_block,
                                 const int32_t* gate, void* stream) {
+    CallRange range("fdd_block_attn");
     if (!ctx) return FDD_ERR_INVALID_ARG;
     int total = 0;
     fdd_status st = check_sets(ctx, sets, n_sets, block_len, &total);
@@ -431,6 +432,7 @@ fdd_status fdd_unmask(fdd_ctx* ctx, fdd_forkset* const* sets, int n_sets, const 
                       int32_t* tokens, uint8_t* state, const int32_t* block_len,
                       float threshold, float temperature, uint32_t block_idx, uint32_t step,
                       int32_t* n_committed, int32_t* n_left, float* conf, void* stream) {
+    CallRange range("fdd_unmask");
     return unmask_like(ctx, sets, n_sets, logits, tokens, state, block_len, threshold, temperature, block_idx, step,
                        n_committed, n_left, conf, stream, 0);
 }
@@ -439,6 +441,7 @@ fdd_status fdd_unmask_counted(fdd_ctx* ctx, fdd_forkset* const* sets, int n_sets
                               int32_t* tokens, uint8_t* state, const int32_t* block_len,
                               float threshold, float temperature, uint32_t block_idx, uint32_t* step_counter,
                               int32_t* n_committed, int32_t* n_left, float* conf, void* stream) {
+    CallRange range("fdd_unmask_counted");
     if (ctx && !step_counter) return fail(ctx, FDD_ERR_INVALID_ARG, "step_counter is NULL");
     return unmask_like(ctx, sets, n_sets, logits, tokens, state, block_len, threshold, temperature, block_idx, 0u,
                        n_committed, n_left, conf, stream, 0, step_counter);
@@ -448,6 +451,7 @@ fdd_status fdd_ss_draft(fdd_ctx* ctx, fdd_forkset* const* sets, int n_sets, cons
                         int32_t* tokens, uint8_t* state, const int32_t* block_len,
                         float temperature, uint32_t block_idx, uint32_t step,
                         int32_t* n_drafted, int32_t* n_left, void* stream) {
+    CallRange range("fdd_ss_draft");
     // every MASKED position passes a threshold below any probability
     return unmask_like(ctx, sets, n_sets, logits, tokens, state, block_len, -1.0f, temperature, block_idx, step,
                        n_drafted, n_left, nullptr, stream, 1);
@@ -457,6 +461,7 @@ fdd_status fdd_ss_accept(fdd_ctx* ctx, fdd_forkset* const* sets, int n_sets, con
                          int32_t* tokens, uint8_t* state, const int32_t* block_len,
                          float temperature, uint32_t block_idx, uint32_t step,
                          int32_t* n_accepted, int32_t* n_left, void* stream) {
+    CallRange range("fdd_ss_accept");
     return unmask_like(ctx, sets, n_sets, ar_logits, tokens, state, block_len, 0.0f, temperature, block_idx, step,
                        n_accepted, n_left, nullptr, stream, 2);
 }
@@ -545,18 +550,21 @@ static fdd_status commit_like(fdd_ctx* ctx, fdd_forkset* const* sets, int n_sets
 fdd_status fdd_kv_commit(fdd_ctx* ctx, fdd_forkset* const* sets, int n_sets, int layer,
                          const void* k_blk, const void* v_blk, const int32_t* block_len,
                          int advance, void* stream) {
+    CallRange range("fdd_kv_commit");
     return commit_like(ctx, sets, n_sets, layer, k_blk, v_blk, block_len, advance, stream, false);
 }
 
 fdd_status fdd_prefix_extend(fdd_ctx* ctx, fdd_forkset* const* sets, int n_sets, int layer,
                              const void* k_blk, const void* v_blk, const int32_t* block_len,
                              int advance, void* stream) {
+    CallRange range("fdd_prefix_extend");
     return commit_like(ctx, sets, n_sets, layer, k_blk, v_blk, block_len, advance, stream, true);
 }
 
 int fdd_forkset_prefix_len(const fdd_forkset* set) { return set ? set->prefix_len : FDD_ERR_INVALID_ARG; }
 
 fdd_status fdd_average_rollouts(fdd_ctx* ctx, const float* traj, int n, int w, float* out, void* stream) {
+    CallRange range("fdd_average_rollouts");
     if (!ctx) return FDD_ERR_INVALID_ARG;
     if (!traj || !out) return fail(ctx, FDD_ERR_INVALID_ARG, "traj/out is NULL");
     if (n < 1 || w < 1) return fail(ctx, FDD_ERR_INVALID_ARG, "n and w must be >= 1");
@@ -568,6 +576,7 @@ fdd_status fdd_average_rollouts(fdd_ctx* ctx, const float* traj, int n, int w, f
 
 fdd_status fdd_average_rollouts_jmt(fdd_ctx* ctx, const float* traj, int n, int w, int w_out, float* out,
                                     void* stream) {
+    CallRange range("fdd_average_rollouts_jmt");
     if (!ctx) return FDD_ERR_INVALID_ARG;
     if (!traj || !out) return fail(ctx, FDD_ERR_INVALID_ARG, "traj/out is NULL");
     if (n < 1 || w < 1 || w_out < 1) return fail(ctx, FDD_ERR_INVALID_ARG, "n, w and w_out must be >= 1");
@@ -599,6 +608,7 @@ fdd_status fdd_average_rollouts_jmt(fdd_ctx* ctx, const float* traj, int n, int 
 
 fdd_status fdd_upload_masked_rows(fdd_ctx* ctx, const void* host_logits, void* dev_logits,
                                   const uint8_t* host_state, int rows, size_t* bytes_copied, void* stream) {
+    CallRange range("fdd_upload_masked_rows");
     if (!ctx) return FDD_ERR_INVALID_ARG;
     if (bytes_copied) *bytes_copied = 0;
     if (!host_logits || !dev_logits || !host_state || rows < 0)

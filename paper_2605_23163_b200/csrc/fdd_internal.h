@@ -7,7 +7,18 @@
 #include <string>
 #include <vector>
 
+#include <nvtx3/nvToolsExt.h>
+
 #include "fdd.h"
+
+// A named NVTX range around one library call: profilers that follow NVTX show which call a kernel
+// belongs to; without one attached the two calls return at once.
+struct CallRange {
+    explicit CallRange(const char* name) { nvtxRangePushA(name); }
+    ~CallRange() { nvtxRangePop(); }
+    CallRange(const CallRange&) = delete;
+    CallRange& operator=(const CallRange&) = delete;
+};
 
 // TMA tensor maps of one scene for the persistent tensor-core attention kernel.
 struct TcSetMaps {

@@ -2,11 +2,12 @@
 // block.  Section s, with E_s editable positions, is cut into ceil(E_s / d) blocks filled from the
 // left; a block ends right after its last editable position, the last block of a section at the
 // section's end; a section without editable positions is one block that needs no decoding.
-#include "fdd.h"
+#include "fdd_internal.h"
 
 extern "C" fdd_status fdd_plan_blocks(const uint8_t* editable, const int32_t* section_end, int n_sections,
                                       int length, int d, int32_t* block_begin, int32_t* block_end,
                                       int32_t* block_section, int capacity, int* n_blocks) {
+    CallRange range("fdd_plan_blocks");
     if (n_blocks) *n_blocks = 0;
     if (!editable || !section_end || !block_begin || !block_end || !block_section || !n_blocks) return FDD_ERR_INVALID_ARG;
     if (n_sections < 1 || length < 0 || d < 1 || capacity < 0) return FDD_ERR_INVALID_ARG;

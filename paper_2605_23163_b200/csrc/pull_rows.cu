@@ -46,6 +46,7 @@ pull_rows_kernel(const unsigned char* __restrict__ src, unsigned char* __restric
 
 fdd_status fdd_pull_masked_rows(fdd_ctx* ctx, const void* host_logits, void* dev_logits, const uint8_t* dev_state,
                                 int rows, unsigned long long* bytes_pulled, void* stream) {
+    CallRange range("fdd_pull_masked_rows");
     if (!ctx) return FDD_ERR_INVALID_ARG;
     if (!host_logits || !dev_logits || !dev_state || rows < 0) {
         ctx->last_error = "fdd_pull_masked_rows: host_logits/dev_logits/dev_state is NULL or rows < 0";

@@ -1051,6 +1051,7 @@ extern "C" fdd_status fdd_unmask_static(const void* logits, int logits_dtype, in
                                         float threshold, float temperature, uint32_t block_idx,
                                         uint32_t step, int32_t* n_committed, int32_t* n_left, float* conf,
                                         void* stream, char* err, size_t err_len) {
+    CallRange range("fdd_unmask_static");
     if (!logits || !tokens || !state || !seeds || !n_committed || !n_left) {
         put_error(err, err_len, "fdd_unmask_static: a required pointer is NULL");
         return FDD_ERR_INVALID_ARG;
